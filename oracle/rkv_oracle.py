@@ -1,0 +1,145 @@
+"""ctypes front end of ``rkv_oracle.c`` (TEST INFRASTRUCTURE, not a product path).
+
+Marshals numpy arrays into the C oracle and back; it holds no arithmetic of the
+method.  Keys and queries are handed over as float32 (bf16 widens to float32
+exactly); the C side computes in double (Eq. 1-7, Algorithm 1).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from dataclasses import dataclass
+from typing import Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "rkv_oracle.c")
+_LIB = os.path.join(_HERE, "librkv_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle with gcc (OpenMP over head-problems) if it is stale."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared", "-Wall", "-Wextra",
+               "-o", _LIB, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        dp, fp, ip = (ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_float),
+                      ctypes.POINTER(ctypes.c_int32))
+        lib.rkv_oracle_head.restype = ctypes.c_int
+        lib.rkv_oracle_head.argtypes = [fp, fp] + [ctypes.c_int] * 7 + [ctypes.c_double] * 3 + \
+            [ip] + [dp] * 7
+        lib.rkv_oracle_batch.restype = ctypes.c_int
+        lib.rkv_oracle_batch.argtypes = [fp, fp, ip] + [ctypes.c_int] * 9 + [ctypes.c_double] * 3 + \
+            [ip, dp, ip]
+        lib.rkv_oracle_gather.restype = None
+        lib.rkv_oracle_gather.argtypes = [ctypes.c_void_p, ip, ctypes.c_int, ctypes.c_size_t,
+                                          ctypes.c_void_p]
+        _lib = lib
+    return _lib
+
+
+def _f32(a) -> np.ndarray:
+    return np.ascontiguousarray(np.asarray(a, dtype=np.float32))
+
+
+def _ptr(a: Optional[np.ndarray], ctype):
+    return None if a is None else a.ctypes.data_as(ctypes.POINTER(ctype))
+
+
+@dataclass
+class HeadResult:
+    compressed: bool
+    idx: np.ndarray            # [budget] int32
+    A: Optional[np.ndarray]    # [alpha, n]
+    I: Optional[np.ndarray]    # [n]
+    Sbar: Optional[np.ndarray]
+    R: Optional[np.ndarray]
+    Z: Optional[np.ndarray]
+    S_raw: Optional[np.ndarray]  # [n, n], Eq. 5 with zero diagonal
+    S_mod: Optional[np.ndarray]  # [n, n], after the retention rule
+
+
+def oracle_head(K, Q, *, budget: int, alpha: int, lam: float, W: int, beta: int, T: float,
+                eps: float = 1e-8, L: Optional[int] = None, want_S: bool = False) -> HeadResult:
+    """One (sequence, KV head): K [>=L, d], Q [G, alpha, d]."""
+    lib = _load()
+    K = _f32(K)
+    Q = _f32(Q)
+    L = K.shape[0] if L is None else int(L)
+    d = K.shape[1]
+    G = Q.shape[0]
+    assert Q.shape == (G, alpha, d) and K.shape[0] >= L
+    idx = np.empty(budget, dtype=np.int32)
+    n = max(L - alpha, 0)
+    live = L > budget
+    A = np.zeros((alpha, n)) if live else None
+    I, Sbar, R, Z = (np.zeros(n) if live else None for _ in range(4))
+    S_raw = np.zeros((n, n)) if (live and want_S) else None
+    S_mod = np.zeros((n, n)) if (live and want_S) else None
+    r = lib.rkv_oracle_head(_ptr(K, ctypes.c_float), _ptr(Q, ctypes.c_float), L, d, G, alpha, budget,
+                            W, beta, float(T), float(eps), float(lam), _ptr(idx, ctypes.c_int32),
+                            _ptr(A, ctypes.c_double), _ptr(I, ctypes.c_double),
+                            _ptr(Sbar, ctypes.c_double), _ptr(R, ctypes.c_double),
+                            _ptr(Z, ctypes.c_double), _ptr(S_raw, ctypes.c_double),
+                            _ptr(S_mod, ctypes.c_double))
+    if r < 0:
+        raise ValueError("rkv_oracle_head: bad arguments")
+    return HeadResult(bool(r), idx, A, I, Sbar, R, Z, S_raw, S_mod)
+
+
+@dataclass
+class BatchResult:
+    idx: np.ndarray         # [B, Hkv, budget] int32
+    compressed: np.ndarray  # [B] bool
+    I: Optional[np.ndarray]     # [B, Hkv, cap] (first n = L - alpha entries meaningful)
+    Sbar: Optional[np.ndarray]
+    R: Optional[np.ndarray]
+    Z: Optional[np.ndarray]
+    threads: int
+
+
+def oracle_batch(K, Q, seq_lens, *, budget: int, alpha: int, lam: float, W: int, beta: int,
+                 T: float, eps: float = 1e-8, want_scores: bool = True) -> BatchResult:
+    """K [B, Hkv, cap, d], Q [B, Hq, alpha, d], seq_lens [B]."""
+    lib = _load()
+    K = _f32(K)
+    Q = _f32(Q)
+    seq = np.ascontiguousarray(np.asarray(seq_lens, dtype=np.int32))
+    B, Hkv, cap, d = K.shape
+    Hq = Q.shape[1]
+    assert Q.shape == (B, Hq, alpha, d) and seq.shape == (B,)
+    idx = np.empty((B, Hkv, budget), dtype=np.int32)
+    scores = np.zeros((4, B, Hkv, cap)) if want_scores else None
+    comp = np.zeros(B, dtype=np.int32)
+    t = lib.rkv_oracle_batch(_ptr(K, ctypes.c_float), _ptr(Q, ctypes.c_float),
+                             _ptr(seq, ctypes.c_int32), B, Hkv, Hq, cap, d, alpha, budget, W, beta,
+                             float(T), float(eps), float(lam), _ptr(idx, ctypes.c_int32),
+                             _ptr(scores, ctypes.c_double), _ptr(comp, ctypes.c_int32))
+    if t < 0:
+        raise ValueError("rkv_oracle_batch: bad arguments (seq_len > cap, or sizes)")
+    if scores is None:
+        return BatchResult(idx, comp.astype(bool), None, None, None, None, t)
+    return BatchResult(idx, comp.astype(bool), scores[0], scores[1], scores[2], scores[3], t)
+
+
+def oracle_gather(rows: np.ndarray, idx: np.ndarray) -> np.ndarray:
+    """Algorithm 1's gather for one head: rows [L, ...] of any dtype, idx [count] (-1 = skip).
+    Returns out [count, ...] with out[j] = rows[idx[j]], copied byte for byte."""
+    lib = _load()
+    rows = np.ascontiguousarray(rows)
+    idx = np.ascontiguousarray(idx, dtype=np.int32)
+    out = np.zeros((idx.shape[0],) + rows.shape[1:], dtype=rows.dtype)
+    row_bytes = rows.dtype.itemsize * int(np.prod(rows.shape[1:], dtype=np.int64))
+    lib.rkv_oracle_gather(rows.ctypes.data, _ptr(idx, ctypes.c_int32), idx.shape[0], row_bytes,
+                          out.ctypes.data)
+    return out
