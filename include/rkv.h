@@ -1,0 +1,167 @@
+/*
+ * rkv.h -- C ABI of the B200 (sm_100a) implementation of R-KV's periodic decode-time
+ * KV-cache compression step.
+ *
+ * What one call computes, per (sequence b, KV head h), with L = seq_lens[b],
+ * n = L - alpha candidate tokens (the last alpha cached tokens are the observation
+ * tokens and are always kept; Section 3.1) and k = budget - alpha:
+ *
+ *   importance   I_i    Eq. 2-4: scaled logits of the alpha observation queries of each of
+ *                       the G query heads of the group against the n candidate keys, max
+ *                       over the group, ONE softmax over the keys, sliding max over the
+ *                       window {i-W .. i+W-1}, mean over the alpha queries.
+ *   redundancy   R_i    Eq. 5-6 and the retention rule of Section 3.3: cosine similarity
+ *                       of all candidate keys, zero diagonal; per token the entries of the
+ *                       (up to) beta largest positions j with S[j][i] > T are zeroed;
+ *                       column mean (divided by n); softmax over the n tokens.
+ *   joint score  Z_i    Eq. 7: lambda * I_i - (1 - lambda) * R_i.
+ *   selection           the k candidates with the largest Z, per KV head (Section 3.4);
+ *                       equal scores: the later position is kept.
+ *   compaction          Algorithm 1's gather + concatenate, in place: rows [0, budget) of
+ *                       K and V become the kept rows in ascending original position (the
+ *                       k selected candidates, then the alpha observation tokens).
+ *
+ * All pointers in the signatures are DEVICE pointers unless the name starts with
+ * "host_".  The library never allocates or frees device memory; scratch comes from
+ * the caller through rkv_desc_t.workspace.  Calls enqueue
+ * work on the given stream and do not synchronise.  Errors are return codes; nothing
+ * throws or aborts.
+ */
+#ifndef RKV_H_
+#define RKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define RKV_API __attribute__((visibility("default")))
+#else
+#define RKV_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    RKV_OK = 0,
+    RKV_ERR_INVALID_ARG = 1, /* null / misaligned pointer, size out of range */
+    RKV_ERR_UNSUPPORTED = 2, /* head_dim != 128, unknown dtype, cap too large, device is not sm_100 */
+    RKV_ERR_WORKSPACE = 3,   /* workspace missing or too small */
+    RKV_ERR_CUDA = 4,        /* a CUDA runtime / driver call failed */
+    RKV_ERR_TIMEOUT = 5      /* device status only: a bounded wait inside a kernel ran out */
+} rkv_status_t;
+
+typedef enum { RKV_BF16 = 0, RKV_F32 = 1 } rkv_dtype_t;
+
+/* rkv_desc_t.flags */
+#define RKV_FLAG_SIMT_SCORES 1u /* score with the plain fp32 CUDA-core kernel instead of the tcgen05
+                                   kernel (always used for RKV_F32; a debugging aid for RKV_BF16) */
+
+/* stage bits for rkv_compress_stages */
+#define RKV_STAGE_PREP 1u    /* key inverse norms and per-tile sums of normalised keys */
+#define RKV_STAGE_SCORES 2u  /* Eq. 2-3 pooled logits; Eq. 5 matrix + retention rule + Eq. 6 column means */
+#define RKV_STAGE_SELECT 4u  /* Eq. 3 softmax, Eq. 4, Eq. 6 softmax, Eq. 7, top-k, index list */
+#define RKV_STAGE_GATHER 8u  /* in-place compaction of K and V, seq_lens update */
+#define RKV_STAGE_ALL 15u
+
+#define RKV_MAX_CAP 8192     /* largest supported budget + buffer */
+#define RKV_MAX_GROUP_ROWS 128 /* largest supported (n_q_heads / n_kv_heads) * alpha */
+
+/*
+ * Problem descriptor.  Plain data, owned by the caller, copied on use.
+ * Fill it with rkv_desc_default() first, then set the shape fields.
+ */
+typedef struct rkv_desc {
+    int32_t batch;       /* sequences; layers that fire together are folded into this dimension */
+    int32_t n_kv_heads;  /* KV heads per sequence */
+    int32_t n_q_heads;   /* query heads; G = n_q_heads / n_kv_heads must be integral (G = 1: Eq. 1) */
+    int32_t head_dim;    /* d; only 128 */
+    int32_t dtype;       /* rkv_dtype_t of k_cache, v_cache and q_window */
+    int32_t pool_w;      /* W of Eq. 4; 0 = no pooling.  Range [0, 64].  Default 4 (the paper prints no value) */
+    int32_t beta;        /* beta of Section 3.3; 0 = rule off.  Default 1 (the paper prints no value) */
+    float sim_threshold; /* T of Section 3.3, in [0, 1].  Default 0.5 (the paper prints no value) */
+    float eps;           /* epsilon of Eq. 5, >= 0.  Default 1e-8 */
+    uint32_t flags;      /* RKV_FLAG_* */
+    void *workspace;     /* device scratch, 256-byte aligned, >= rkv_workspace_bytes(); contents are
+                            undefined between calls; two calls that overlap on the GPU need two workspaces */
+    size_t workspace_bytes;
+    int32_t *device_status; /* optional device int32; kernels store the first error they meet
+                               (RKV_ERR_INVALID_ARG for seq_lens[b] > cap or < 0, RKV_ERR_TIMEOUT).  The caller
+                               zeroes it and reads it after synchronising the stream */
+    /* optional device dumps of the scores, each [batch][n_kv_heads][cap] float, first n entries written */
+    float *dbg_I, *dbg_Sbar, *dbg_R, *dbg_Z;
+    /* optional: 5 cudaEvent_t handles; event s is recorded before stage s (prep, scores, select, gather)
+       and event 4 after the last stage, on the call's stream */
+    void *const *stage_events;
+} rkv_desc_t;
+
+/* Fill *desc with the defaults above (pool_w 4, beta 1, T 0.5, eps 1e-8, head_dim 128, bf16), zero elsewhere. */
+RKV_API void rkv_desc_default(rkv_desc_t *desc);
+
+/* Bytes of device scratch a call with this descriptor and these sizes needs (0 if the arguments are invalid). */
+RKV_API size_t rkv_workspace_bytes(const rkv_desc_t *desc, int32_t budget, int32_t buffer, int32_t alpha);
+
+/* Install *desc (copied) as the calling thread's current descriptor, used by rkv_compress(). */
+RKV_API int rkv_set_desc(const rkv_desc_t *desc);
+
+/*
+ * One firing of the compression step (Section 3.1; Algorithm 1) for every sequence in the batch.
+ *
+ *   k_cache, v_cache  [batch][n_kv_heads][cap][head_dim], cap = budget + buffer, contiguous, 16-byte aligned;
+ *                     modified in place
+ *   q_window          [batch][n_q_heads][alpha][head_dim]: the query states of the last alpha tokens (the
+ *                     paper's query cache); query head q belongs to KV head q / G
+ *   seq_lens          [batch] int32, in/out: cached length L of each sequence
+ *   out_idx           [batch][n_kv_heads][budget] int32, out
+ *   stream            cudaStream_t (NULL = the legacy default stream)
+ *
+ * For each b with budget < seq_lens[b] <= cap: rows [0, budget) of every head hold the kept rows in ascending
+ * original position, rows [budget, cap) are unspecified, out_idx[b][h] lists the kept original positions
+ * (ascending; the last alpha are L-alpha .. L-1) and seq_lens[b] becomes budget.
+ * For seq_lens[b] <= budget (Algorithm 1's guard) nothing changes; out_idx[b][h][j] = j for j < L, -1 after.
+ * seq_lens[b] > cap or < 0 cannot be seen without a sync: that sequence is skipped, out_idx[b] = -1 and
+ * RKV_ERR_INVALID_ARG is stored to device_status.
+ * Requires 1 <= alpha < budget, buffer >= 1, cap <= RKV_MAX_CAP, G * alpha <= RKV_MAX_GROUP_ROWS,
+ * lambda in [0, 1].  Host-detectable errors return before anything is launched.
+ * Uses the thread's current descriptor (rkv_set_desc).
+ */
+RKV_API int rkv_compress(void *k_cache, void *v_cache, const void *q_window, int32_t *seq_lens, int32_t budget,
+                 int32_t buffer, int32_t alpha, float lambda, int32_t *out_idx, void *stream);
+
+/* The same with an explicit descriptor. */
+RKV_API int rkv_compress_ex(const rkv_desc_t *desc, void *k_cache, void *v_cache, const void *q_window,
+                    int32_t *seq_lens, int32_t budget, int32_t buffer, int32_t alpha, float lambda,
+                    int32_t *out_idx, void *stream);
+
+/* The same, running only the stages in stage_mask (RKV_STAGE_*); stages hand their results on through the
+ * workspace, so running them one by one in order equals one full call.  For per-stage timing and tests. */
+RKV_API int rkv_compress_stages(const rkv_desc_t *desc, void *k_cache, void *v_cache, const void *q_window,
+                        int32_t *seq_lens, int32_t budget, int32_t buffer, int32_t alpha, float lambda,
+                        int32_t *out_idx, void *stream, uint32_t stage_mask);
+
+/*
+ * End-to-end form with HOST buffers (pinned memory recommended): copies host_k_cache, host_v_cache,
+ * host_q_window and host_seq_lens to device staging inside desc->workspace, runs the step, and copies back
+ * rows [0, budget) of K and V of every head, seq_lens and out_idx -- all asynchronously on `stream`; the
+ * results are valid once the stream is synchronised.  desc->workspace must hold rkv_host_workspace_bytes().
+ * Shapes and semantics as rkv_compress.
+ */
+RKV_API size_t rkv_host_workspace_bytes(const rkv_desc_t *desc, int32_t budget, int32_t buffer, int32_t alpha);
+RKV_API int rkv_compress_host(const rkv_desc_t *desc, void *host_k_cache, void *host_v_cache, const void *host_q_window,
+                      int32_t *host_seq_lens, int32_t budget, int32_t buffer, int32_t alpha, float lambda,
+                      int32_t *host_out_idx, void *stream);
+
+/* Number of kernels a call with this descriptor and stage mask launches (for launch accounting). */
+RKV_API int rkv_launch_count(const rkv_desc_t *desc, uint32_t stage_mask);
+
+/* Human-readable name of a status code. */
+RKV_API const char *rkv_status_string(int status);
+
+/* Text of the last CUDA error seen by the calling thread inside the library ("" if none). */
+RKV_API const char *rkv_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RKV_H_ */

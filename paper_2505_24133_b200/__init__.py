@@ -1,0 +1,11 @@
+"""B200-native R-KV decode-time KV-cache compression step (C-ABI CUDA library + thin ctypes binding).
+
+Every step of the path runs in the CUDA kernels of ``librkv_b200.so``; this package only marshals
+arguments.  There is no CPU fallback: loading fails loudly if the library has not been built.
+"""
+from .binding import (  # noqa: F401
+    RKV_BF16, RKV_F32, RKV_FLAG_SIMT_SCORES, RKV_STAGE_ALL, RKV_STAGE_GATHER, RKV_STAGE_PREP,
+    RKV_STAGE_SCORES, RKV_STAGE_SELECT, RKV_OK, RkvDesc, RkvError, Compressor, lib, lib_path,
+    rkv_compress, rkv_compress_ex, rkv_compress_stages, rkv_compress_host, rkv_desc_default,
+    rkv_host_workspace_bytes, rkv_launch_count, rkv_set_desc, rkv_status_string, rkv_workspace_bytes,
+)

@@ -1,0 +1,292 @@
+// C ABI of the R-KV compression library: argument checks, workspace carve-up, stage launches.
+// See include/rkv.h for the contract of every entry point.
+#include <cstdio>
+#include <cstring>
+
+#include "rkv_common.cuh"
+
+namespace rkv {
+
+namespace {
+
+thread_local rkv_desc_t g_desc;
+thread_local bool g_desc_set = false;
+thread_local char g_cuda_error[256] = "";
+
+int cuda_fail(cudaError_t e, const char *where)
+{
+    snprintf(g_cuda_error, sizeof(g_cuda_error), "%s: %s", where, cudaGetErrorString(e));
+    return RKV_ERR_CUDA;
+}
+
+struct Layout {
+    size_t inv_norm, tile_sum, logits, sbar, meta, counters, total;
+    int cap, cap_pad, tiles;
+};
+
+// Returns RKV_OK and fills *lay when the shape arguments are usable.
+int check_shapes(const rkv_desc_t *d, int budget, int buffer, int alpha, Layout *lay)
+{
+    if (!d) return RKV_ERR_INVALID_ARG;
+    if (d->batch < 1 || d->n_kv_heads < 1 || d->n_q_heads < 1) return RKV_ERR_INVALID_ARG;
+    if (d->n_q_heads % d->n_kv_heads != 0) return RKV_ERR_INVALID_ARG;
+    if (alpha < 1 || budget <= alpha || buffer < 1) return RKV_ERR_INVALID_ARG;
+    if (d->pool_w < 0 || d->pool_w > 64 || d->beta < 0) return RKV_ERR_INVALID_ARG;
+    if (!(d->sim_threshold >= 0.f && d->sim_threshold <= 1.f) || !(d->eps >= 0.f)) return RKV_ERR_INVALID_ARG;
+    if (d->head_dim != kHeadDim) return RKV_ERR_UNSUPPORTED;
+    if (d->dtype != RKV_BF16 && d->dtype != RKV_F32) return RKV_ERR_UNSUPPORTED;
+    const long long cap = (long long)budget + buffer;
+    if (cap > RKV_MAX_CAP) return RKV_ERR_UNSUPPORTED;
+    if ((long long)(d->n_q_heads / d->n_kv_heads) * alpha > RKV_MAX_GROUP_ROWS) return RKV_ERR_UNSUPPORTED;
+    if ((long long)d->batch * d->n_kv_heads > (1ll << 24)) return RKV_ERR_UNSUPPORTED;
+    if (lay) {
+        const size_t P = (size_t)d->batch * d->n_kv_heads;
+        lay->cap = (int)cap;
+        lay->tiles = (int)((cap + kTile - 1) / kTile);
+        lay->cap_pad = lay->tiles * kTile;
+        size_t off = 0;
+        lay->inv_norm = off;  off = align_up(off + P * lay->cap_pad * sizeof(float), 256);
+        lay->tile_sum = off;  off = align_up(off + P * lay->tiles * kHeadDim * sizeof(float), 256);
+        lay->logits = off;    off = align_up(off + P * alpha * lay->cap_pad * sizeof(float), 256);
+        lay->sbar = off;      off = align_up(off + P * lay->cap_pad * sizeof(float), 256);
+        lay->meta = off;      off = align_up(off + (size_t)d->batch * sizeof(int32_t), 256);
+        lay->counters = off;  off = align_up(off + 4 * sizeof(unsigned long long), 256);
+        lay->total = off;
+    }
+    return RKV_OK;
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+bool use_simt(const rkv_desc_t *d) { return d->dtype == RKV_F32 || (d->flags & RKV_FLAG_SIMT_SCORES); }
+
+int run(const rkv_desc_t *d, void *k_cache, void *v_cache, const void *q_window, int32_t *seq_lens, int budget,
+        int buffer, int alpha, float lambda, int32_t *out_idx, void *stream, uint32_t stages)
+{
+    Layout lay;
+    int rc = check_shapes(d, budget, buffer, alpha, &lay);
+    if (rc != RKV_OK) return rc;
+    if (!k_cache || !v_cache || !q_window || !seq_lens || !out_idx) return RKV_ERR_INVALID_ARG;
+    if (!aligned16(k_cache) || !aligned16(v_cache) || !aligned16(q_window)) return RKV_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(seq_lens) & 3u) || (reinterpret_cast<uintptr_t>(out_idx) & 3u))
+        return RKV_ERR_INVALID_ARG;
+    if (!(lambda >= 0.f && lambda <= 1.f)) return RKV_ERR_INVALID_ARG;
+    if ((stages & ~RKV_STAGE_ALL) != 0u || stages == 0u) return RKV_ERR_INVALID_ARG;
+    if (!d->workspace || d->workspace_bytes < lay.total) return RKV_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(d->workspace) & 255u) return RKV_ERR_WORKSPACE;
+    if (!use_simt(d) && !scores_sm100_available()) return RKV_ERR_UNSUPPORTED;
+
+    Params p;
+    memset(&p, 0, sizeof(p));
+    p.k_cache = k_cache;
+    p.v_cache = v_cache;
+    p.q_window = q_window;
+    p.seq_lens = seq_lens;
+    p.out_idx = out_idx;
+    p.batch = d->batch;
+    p.hkv = d->n_kv_heads;
+    p.hq = d->n_q_heads;
+    p.group = d->n_q_heads / d->n_kv_heads;
+    p.cap = lay.cap;
+    p.cap_pad = lay.cap_pad;
+    p.tiles = lay.tiles;
+    p.budget = budget;
+    p.buffer = buffer;
+    p.alpha = alpha;
+    p.dtype = d->dtype;
+    p.pool_w = d->pool_w;
+    p.beta = d->beta;
+    p.sim_threshold = d->sim_threshold;
+    p.eps = d->eps;
+    p.lambda = lambda;
+    char *ws = static_cast<char *>(d->workspace);
+    p.inv_norm = reinterpret_cast<float *>(ws + lay.inv_norm);
+    p.tile_sum = reinterpret_cast<float *>(ws + lay.tile_sum);
+    p.logits = reinterpret_cast<float *>(ws + lay.logits);
+    p.sbar = reinterpret_cast<float *>(ws + lay.sbar);
+    p.meta = reinterpret_cast<int32_t *>(ws + lay.meta);
+    p.counters = reinterpret_cast<unsigned long long *>(ws + lay.counters);
+    p.status = d->device_status;
+    p.dbg_I = d->dbg_I;
+    p.dbg_Sbar = d->dbg_Sbar;
+    p.dbg_R = d->dbg_R;
+    p.dbg_Z = d->dbg_Z;
+
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    void *const *ev = d->stage_events;
+    cudaError_t e;
+    auto mark = [&](int i) -> cudaError_t {
+        return ev && ev[i] ? cudaEventRecord(static_cast<cudaEvent_t>(ev[i]), s) : cudaSuccess;
+    };
+    if ((e = mark(0)) != cudaSuccess) return cuda_fail(e, "cudaEventRecord");
+    if (stages & RKV_STAGE_PREP)
+        if ((e = launch_prep(p, s)) != cudaSuccess) return cuda_fail(e, "prep launch");
+    if ((e = mark(1)) != cudaSuccess) return cuda_fail(e, "cudaEventRecord");
+    if (stages & RKV_STAGE_SCORES) {
+        e = use_simt(d) ? launch_scores_simt(p, s) : launch_scores_sm100(p, s);
+        if (e != cudaSuccess) return cuda_fail(e, "scores launch");
+    }
+    if ((e = mark(2)) != cudaSuccess) return cuda_fail(e, "cudaEventRecord");
+    if (stages & RKV_STAGE_SELECT)
+        if ((e = launch_select(p, s)) != cudaSuccess) return cuda_fail(e, "select launch");
+    if ((e = mark(3)) != cudaSuccess) return cuda_fail(e, "cudaEventRecord");
+    if (stages & RKV_STAGE_GATHER)
+        if ((e = launch_gather(p, s)) != cudaSuccess) return cuda_fail(e, "gather launch");
+    if ((e = mark(4)) != cudaSuccess) return cuda_fail(e, "cudaEventRecord");
+    return RKV_OK;
+}
+
+struct HostLayout {
+    size_t k, v, q, seq, idx, inner, total;
+    size_t kv_bytes, q_bytes, seq_bytes, idx_bytes, row_bytes;
+};
+
+int host_layout(const rkv_desc_t *d, int budget, int buffer, int alpha, HostLayout *h)
+{
+    Layout lay;
+    int rc = check_shapes(d, budget, buffer, alpha, &lay);
+    if (rc != RKV_OK) return rc;
+    const size_t esz = d->dtype == RKV_BF16 ? 2 : 4;
+    const size_t P = (size_t)d->batch * d->n_kv_heads;
+    h->row_bytes = kHeadDim * esz;
+    h->kv_bytes = P * lay.cap * h->row_bytes;
+    h->q_bytes = (size_t)d->batch * d->n_q_heads * alpha * h->row_bytes;
+    h->seq_bytes = (size_t)d->batch * sizeof(int32_t);
+    h->idx_bytes = P * budget * sizeof(int32_t);
+    size_t off = 0;
+    h->k = off;      off = align_up(off + h->kv_bytes, 256);
+    h->v = off;      off = align_up(off + h->kv_bytes, 256);
+    h->q = off;      off = align_up(off + h->q_bytes, 256);
+    h->seq = off;    off = align_up(off + h->seq_bytes, 256);
+    h->idx = off;    off = align_up(off + h->idx_bytes, 256);
+    h->inner = off;  off = off + lay.total;
+    h->total = off;
+    return RKV_OK;
+}
+
+}  // namespace
+}  // namespace rkv
+
+using namespace rkv;
+
+extern "C" {
+
+void rkv_desc_default(rkv_desc_t *desc)
+{
+    if (!desc) return;
+    memset(desc, 0, sizeof(*desc));
+    desc->head_dim = kHeadDim;
+    desc->dtype = RKV_BF16;
+    desc->pool_w = 4;
+    desc->beta = 1;
+    desc->sim_threshold = 0.5f;
+    desc->eps = 1e-8f;
+}
+
+size_t rkv_workspace_bytes(const rkv_desc_t *desc, int32_t budget, int32_t buffer, int32_t alpha)
+{
+    Layout lay;
+    return check_shapes(desc, budget, buffer, alpha, &lay) == RKV_OK ? lay.total : 0;
+}
+
+int rkv_set_desc(const rkv_desc_t *desc)
+{
+    if (!desc) return RKV_ERR_INVALID_ARG;
+    g_desc = *desc;
+    g_desc_set = true;
+    return RKV_OK;
+}
+
+int rkv_compress(void *k_cache, void *v_cache, const void *q_window, int32_t *seq_lens, int32_t budget,
+                 int32_t buffer, int32_t alpha, float lambda, int32_t *out_idx, void *stream)
+{
+    if (!g_desc_set) return RKV_ERR_INVALID_ARG;
+    return run(&g_desc, k_cache, v_cache, q_window, seq_lens, budget, buffer, alpha, lambda, out_idx, stream,
+               RKV_STAGE_ALL);
+}
+
+int rkv_compress_ex(const rkv_desc_t *desc, void *k_cache, void *v_cache, const void *q_window,
+                    int32_t *seq_lens, int32_t budget, int32_t buffer, int32_t alpha, float lambda,
+                    int32_t *out_idx, void *stream)
+{
+    return run(desc, k_cache, v_cache, q_window, seq_lens, budget, buffer, alpha, lambda, out_idx, stream,
+               RKV_STAGE_ALL);
+}
+
+int rkv_compress_stages(const rkv_desc_t *desc, void *k_cache, void *v_cache, const void *q_window,
+                        int32_t *seq_lens, int32_t budget, int32_t buffer, int32_t alpha, float lambda,
+                        int32_t *out_idx, void *stream, uint32_t stage_mask)
+{
+    return run(desc, k_cache, v_cache, q_window, seq_lens, budget, buffer, alpha, lambda, out_idx, stream,
+               stage_mask);
+}
+
+size_t rkv_host_workspace_bytes(const rkv_desc_t *desc, int32_t budget, int32_t buffer, int32_t alpha)
+{
+    HostLayout h;
+    return host_layout(desc, budget, buffer, alpha, &h) == RKV_OK ? h.total : 0;
+}
+
+int rkv_compress_host(const rkv_desc_t *desc, void *host_k_cache, void *host_v_cache, const void *host_q_window,
+                      int32_t *host_seq_lens, int32_t budget, int32_t buffer, int32_t alpha, float lambda,
+                      int32_t *host_out_idx, void *stream)
+{
+    HostLayout h;
+    int rc = host_layout(desc, budget, buffer, alpha, &h);
+    if (rc != RKV_OK) return rc;
+    if (!host_k_cache || !host_v_cache || !host_q_window || !host_seq_lens || !host_out_idx)
+        return RKV_ERR_INVALID_ARG;
+    if (!desc->workspace || desc->workspace_bytes < h.total) return RKV_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(desc->workspace) & 255u) return RKV_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    char *ws = static_cast<char *>(desc->workspace);
+    cudaError_t e;
+    if ((e = cudaMemcpyAsync(ws + h.k, host_k_cache, h.kv_bytes, cudaMemcpyHostToDevice, s)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(ws + h.v, host_v_cache, h.kv_bytes, cudaMemcpyHostToDevice, s)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(ws + h.q, host_q_window, h.q_bytes, cudaMemcpyHostToDevice, s)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(ws + h.seq, host_seq_lens, h.seq_bytes, cudaMemcpyHostToDevice, s)) != cudaSuccess)
+        return cuda_fail(e, "host to device copy");
+    rkv_desc_t inner = *desc;
+    inner.workspace = ws + h.inner;
+    inner.workspace_bytes = desc->workspace_bytes - h.inner;
+    rc = run(&inner, ws + h.k, ws + h.v, ws + h.q, reinterpret_cast<int32_t *>(ws + h.seq), budget, buffer, alpha,
+             lambda, reinterpret_cast<int32_t *>(ws + h.idx), stream, RKV_STAGE_ALL);
+    if (rc != RKV_OK) return rc;
+    // rows [0, budget) of every head come back; rows beyond are unspecified after a compression and are left
+    // as the host has them
+    const size_t P = (size_t)desc->batch * desc->n_kv_heads;
+    const size_t cap = (size_t)budget + buffer;
+    if ((e = cudaMemcpy2DAsync(host_k_cache, cap * h.row_bytes, ws + h.k, cap * h.row_bytes, budget * h.row_bytes, P,
+                               cudaMemcpyDeviceToHost, s)) != cudaSuccess ||
+        (e = cudaMemcpy2DAsync(host_v_cache, cap * h.row_bytes, ws + h.v, cap * h.row_bytes, budget * h.row_bytes, P,
+                               cudaMemcpyDeviceToHost, s)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(host_seq_lens, ws + h.seq, h.seq_bytes, cudaMemcpyDeviceToHost, s)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(host_out_idx, ws + h.idx, h.idx_bytes, cudaMemcpyDeviceToHost, s)) != cudaSuccess)
+        return cuda_fail(e, "device to host copy");
+    return RKV_OK;
+}
+
+int rkv_launch_count(const rkv_desc_t *desc, uint32_t stage_mask)
+{
+    (void)desc;
+    int c = 0;
+    for (uint32_t bit = 1; bit <= RKV_STAGE_GATHER; bit <<= 1) c += (stage_mask & bit) ? 1 : 0;
+    return c;
+}
+
+const char *rkv_status_string(int status)
+{
+    switch (status) {
+        case RKV_OK: return "RKV_OK";
+        case RKV_ERR_INVALID_ARG: return "RKV_ERR_INVALID_ARG";
+        case RKV_ERR_UNSUPPORTED: return "RKV_ERR_UNSUPPORTED";
+        case RKV_ERR_WORKSPACE: return "RKV_ERR_WORKSPACE";
+        case RKV_ERR_CUDA: return "RKV_ERR_CUDA";
+        case RKV_ERR_TIMEOUT: return "RKV_ERR_TIMEOUT";
+        default: return "RKV_ERR_UNKNOWN";
+    }
+}
+
+const char *rkv_last_cuda_error(void) { return g_cuda_error; }
+
+}  // extern "C"

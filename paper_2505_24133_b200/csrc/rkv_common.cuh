@@ -1,0 +1,93 @@
+// Internal declarations shared by the kernels of the R-KV compression library (sm_100a).
+// Nothing here is part of the public ABI (see include/rkv.h).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "rkv.h"
+
+namespace rkv {
+
+constexpr int kHeadDim = 128;   // d
+constexpr int kTile = 128;      // keys per tile (rows of one tensor-core operand tile)
+
+// meta[b] values
+constexpr int kMetaInvalid = -1;
+
+// Everything a kernel needs; passed by value.
+struct Params {
+    // caller tensors
+    void *k_cache;
+    void *v_cache;
+    const void *q_window;
+    int32_t *seq_lens;
+    int32_t *out_idx;
+    // shapes
+    int batch, hkv, hq, group;      // group = G
+    int cap, cap_pad, tiles;        // cap_pad = tiles * kTile
+    int budget, buffer, alpha;
+    int dtype;
+    // hyper-parameters
+    int pool_w, beta;
+    float sim_threshold, eps, lambda;
+    // workspace carve-up
+    float *inv_norm;     // [P][cap_pad]         r_i = 1 / (||k_i|| + eps); 0 for i >= n
+    float *tile_sum;     // [P][tiles][128]      sum over the tile's candidate rows of r_i * k_i
+    float *logits;       // [P][alpha][cap_pad]  Eq. 2-3: group-max of scaled logits
+    float *sbar;         // [P][cap_pad]         Eq. 6 column means after the retention rule
+    int32_t *meta;       // [batch]              snapshot of seq_lens (kMetaInvalid if out of range)
+    unsigned long long *counters;   // [4]       [0] = similarity tiles computed by the tcgen05 kernel
+    // optional outputs
+    int32_t *status;
+    float *dbg_I, *dbg_Sbar, *dbg_R, *dbg_Z;
+};
+
+__host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+__device__ __forceinline__ void report(int32_t *status, int code)
+{
+    if (status) atomicCAS(status, 0, code);
+}
+
+// Number of candidates of sequence b as every stage after prep sees it: 0 = nothing to compress.
+__device__ __forceinline__ int candidates_from_meta(int L, int budget, int alpha)
+{
+    return (L > budget) ? (L - alpha) : 0;
+}
+
+template <typename T> struct Elem;
+template <> struct Elem<__nv_bfloat16> {
+    static constexpr int kPerVec = 8;   // elements per 16-byte vector
+    __device__ static void unpack(const uint4 &v, float *f)
+    {
+        const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&v);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float2 t = __bfloat1622float2(h[i]);
+            f[2 * i] = t.x;
+            f[2 * i + 1] = t.y;
+        }
+    }
+};
+template <> struct Elem<float> {
+    static constexpr int kPerVec = 4;
+    __device__ static void unpack(const uint4 &v, float *f)
+    {
+        f[0] = __uint_as_float(v.x);
+        f[1] = __uint_as_float(v.y);
+        f[2] = __uint_as_float(v.z);
+        f[3] = __uint_as_float(v.w);
+    }
+};
+
+// launchers (one per stage); each returns cudaGetLastError() of its launch
+cudaError_t launch_prep(const Params &p, cudaStream_t s);
+cudaError_t launch_scores_simt(const Params &p, cudaStream_t s);
+cudaError_t launch_scores_sm100(const Params &p, cudaStream_t s);
+cudaError_t launch_select(const Params &p, cudaStream_t s);
+cudaError_t launch_gather(const Params &p, cudaStream_t s);
+bool scores_sm100_available();
+
+}  // namespace rkv

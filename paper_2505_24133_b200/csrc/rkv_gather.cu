@@ -1,0 +1,68 @@
+// Stage "gather": Algorithm 1's gather + concatenate, done in place.
+//
+// For every head, row j of K and of V becomes row idx[j] (j < budget).  idx is strictly ascending, so
+// idx[j] >= j: rows only move towards lower positions and the untouched prefix (idx[j] == j) is free.
+// One thread block owns one (head, K|V) stream and walks it in chunks of 64 rows: load the chunk's source
+// rows into registers, barrier, store.  A later chunk reads only rows at or beyond its own first row, which
+// no earlier chunk writes, so one barrier per chunk is all the ordering in-place compaction needs.
+// No scratch copy, no reallocation.  HBM-bound: 16-byte loads and stores, a row is 16 (bf16) or 32 (fp32) lanes wide.
+// The block of (KV head 0, K) also stores the new length, seq_lens[b] = budget.
+#include "rkv_common.cuh"
+
+namespace rkv {
+
+namespace {
+
+constexpr int kGatherThreads = 256;
+constexpr int kChunkRows = 64;
+
+template <int kVecPerRow>   // 16-byte vectors per row
+__global__ void __launch_bounds__(kGatherThreads) gather_kernel(Params p)
+{
+    constexpr int kVecPerThread = kChunkRows * kVecPerRow / kGatherThreads;   // 4 or 8
+    constexpr int kRowsPerStep = kGatherThreads / kVecPerRow;                  // 16 or 8
+    const int head = blockIdx.x >> 1;
+    const int which = blockIdx.x & 1;
+    const int b = head / p.hkv;
+    const int L = p.meta[b];
+    if (L <= p.budget) return;                      // nothing was selected for this sequence
+    if (which == 0 && head % p.hkv == 0 && threadIdx.x == 0) p.seq_lens[b] = p.budget;
+
+    uint4 *base = reinterpret_cast<uint4 *>(which ? p.v_cache : p.k_cache) + (size_t)head * p.cap * kVecPerRow;
+    const int32_t *idx = p.out_idx + (size_t)head * p.budget;
+    const int lane_vec = threadIdx.x % kVecPerRow;
+    const int lane_row = threadIdx.x / kVecPerRow;
+
+    for (int j0 = 0; j0 < p.budget; j0 += kChunkRows) {
+        const int j_end = min(j0 + kChunkRows, p.budget);
+        if (idx[j_end - 1] == j_end - 1) continue;   // ascending and idx[j] >= j: the whole chunk is in place
+        uint4 held[kVecPerThread];
+        int src[kVecPerThread];
+#pragma unroll
+        for (int q = 0; q < kVecPerThread; ++q) {
+            const int j = j0 + q * kRowsPerStep + lane_row;
+            src[q] = (j < j_end) ? idx[j] : -1;
+            if (src[q] >= 0 && src[q] != j) held[q] = base[(size_t)src[q] * kVecPerRow + lane_vec];
+        }
+        __syncthreads();                             // every source row of the chunk is in registers
+#pragma unroll
+        for (int q = 0; q < kVecPerThread; ++q) {
+            const int j = j0 + q * kRowsPerStep + lane_row;
+            if (src[q] >= 0 && src[q] != j) base[(size_t)j * kVecPerRow + lane_vec] = held[q];
+        }
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_gather(const Params &p, cudaStream_t s)
+{
+    const unsigned grid = 2u * (unsigned)(p.batch * p.hkv);
+    if (p.dtype == RKV_BF16)
+        gather_kernel<16><<<grid, kGatherThreads, 0, s>>>(p);
+    else
+        gather_kernel<32><<<grid, kGatherThreads, 0, s>>>(p);
+    return cudaGetLastError();
+}
+
+}  // namespace rkv

@@ -1,0 +1,109 @@
+// Stage "prep": one streaming pass over the candidate keys.
+//
+// For every key row i of every head it produces r_i = 1 / (||k_i||_2 + eps), the normalisation
+// factor of Eq. 5, and per 128-row tile the vector sum_i r_i * k_i.  The tile sums let the
+// scoring stage obtain sum_j S[j][i] = Kbar_i . (sum_j Kbar_j) - Kbar_i . Kbar_i (Eq. 6 before the
+// retention rule) without accumulating the n x n matrix element by element.
+// Rows i >= n (observation tokens, unused capacity) get r_i = 0 and contribute nothing.
+//
+// HBM-bound: K is read once with 16-byte loads, rows coalesced across the lanes of a warp; the row
+// norm is reduced with warp shuffles.  Outputs are 4 bytes per 256-byte row.
+#include "rkv_common.cuh"
+
+namespace rkv {
+
+namespace {
+
+constexpr int kPrepThreads = 256;
+constexpr int kPrepWarps = kPrepThreads / 32;
+
+template <typename T>
+__global__ void __launch_bounds__(kPrepThreads) prep_kernel(Params p)
+{
+    constexpr int kPerVec = Elem<T>::kPerVec;            // elements per 16-byte vector
+    constexpr int kLanesPerRow = kHeadDim / kPerVec;     // 16 (bf16) or 32 (fp32)
+    constexpr int kRowsPerPass = 32 / kLanesPerRow;      // rows a warp covers with one load
+    constexpr int kRowsPerWarp = kTile / kPrepWarps;     // 16
+    constexpr int kPasses = kRowsPerWarp / kRowsPerPass;
+
+    const int tile = blockIdx.x % p.tiles;
+    const int head = blockIdx.x / p.tiles;               // head-problem index b * hkv + h
+    const int b = head / p.hkv;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    int L = p.seq_lens[b];
+    if (L < 0 || L > p.cap) {
+        report(p.status, RKV_ERR_INVALID_ARG);
+        L = kMetaInvalid;
+    }
+    if (tile == 0 && head % p.hkv == 0 && threadIdx.x == 0) p.meta[b] = L;
+    const int n = candidates_from_meta(L, p.budget, p.alpha);
+
+    const T *K = static_cast<const T *>(p.k_cache) + (size_t)head * p.cap * kHeadDim;
+    float *inv_norm = p.inv_norm + (size_t)head * p.cap_pad;
+
+    const int sub = lane / kLanesPerRow;                 // which of the rows of this pass
+    const int col = (lane % kLanesPerRow) * kPerVec;     // first column this lane holds
+    const int row0 = tile * kTile + warp * kRowsPerWarp;
+
+    // issue every load of this warp's 16 rows first (all independent), then reduce
+    uint4 vec[kPasses];
+#pragma unroll
+    for (int q = 0; q < kPasses; ++q) {
+        const int row = row0 + q * kRowsPerPass + sub;
+        vec[q] = make_uint4(0u, 0u, 0u, 0u);
+        if (row < n) vec[q] = __ldg(reinterpret_cast<const uint4 *>(K + (size_t)row * kHeadDim + col));
+    }
+
+    float acc[kPerVec];
+#pragma unroll
+    for (int e = 0; e < kPerVec; ++e) acc[e] = 0.f;
+
+#pragma unroll
+    for (int q = 0; q < kPasses; ++q) {
+        const int row = row0 + q * kRowsPerPass + sub;
+        float f[kPerVec];
+        Elem<T>::unpack(vec[q], f);
+        float sq = 0.f;
+#pragma unroll
+        for (int e = 0; e < kPerVec; ++e) sq = fmaf(f[e], f[e], sq);
+#pragma unroll
+        for (int off = kLanesPerRow / 2; off > 0; off >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, off);
+        const float r = (row < n) ? __fdiv_rn(1.0f, __fsqrt_rn(sq) + p.eps) : 0.f;
+        if (lane % kLanesPerRow == 0 && row < p.cap_pad) inv_norm[row] = r;
+#pragma unroll
+        for (int e = 0; e < kPerVec; ++e) acc[e] = fmaf(r, f[e], acc[e]);
+    }
+
+    // fold the row groups of a warp, then the warps, in a fixed order (deterministic sums)
+    if (kRowsPerPass == 2) {
+#pragma unroll
+        for (int e = 0; e < kPerVec; ++e) acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], 16);
+    }
+    __shared__ float part[kPrepWarps][kHeadDim];
+    if (sub == 0) {
+#pragma unroll
+        for (int e = 0; e < kPerVec; ++e) part[warp][col + e] = acc[e];
+    }
+    __syncthreads();
+    if (threadIdx.x < kHeadDim) {
+        float s = 0.f;
+#pragma unroll
+        for (int w = 0; w < kPrepWarps; ++w) s += part[w][threadIdx.x];
+        p.tile_sum[((size_t)head * p.tiles + tile) * kHeadDim + threadIdx.x] = s;
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_prep(const Params &p, cudaStream_t s)
+{
+    const unsigned grid = (unsigned)p.tiles * (unsigned)(p.batch * p.hkv);
+    if (p.dtype == RKV_BF16)
+        prep_kernel<__nv_bfloat16><<<grid, kPrepThreads, 0, s>>>(p);
+    else
+        prep_kernel<float><<<grid, kPrepThreads, 0, s>>>(p);
+    return cudaGetLastError();
+}
+
+}  // namespace rkv

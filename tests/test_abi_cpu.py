@@ -1,0 +1,126 @@
+"""Host-side checks of the C-ABI library that need no GPU: it loads, exports every declared symbol, and
+rejects host-detectable errors before any launch."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def rkv():
+    from paper_2505_24133_b200 import build as b
+    b.build()
+    import paper_2505_24133_b200 as r
+    return r
+
+
+def test_library_exports_every_declared_symbol(rkv):
+    header = open(os.path.join(ROOT, "include", "rkv.h")).read()
+    names = re.findall(r"RKV_API\s+[\w\s\*]+?\b(rkv_\w+)\s*\(", header)
+    assert len(names) >= 11
+    lib = ctypes.CDLL(rkv.lib_path())
+    for name in names:
+        assert hasattr(lib, name), f"{name} is declared in include/rkv.h but not exported"
+
+
+def test_desc_mirror_matches_the_c_struct(rkv):
+    d = rkv.rkv_desc_default()
+    assert (d.head_dim, d.dtype, d.pool_w, d.beta) == (128, rkv.RKV_BF16, 4, 1)
+    assert abs(d.sim_threshold - 0.5) < 1e-7 and abs(d.eps - 1e-8) < 1e-15
+    assert d.workspace is None and d.stage_events is None and d.flags == 0
+
+
+def _desc(rkv, **kw):
+    d = rkv.rkv_desc_default()
+    d.batch, d.n_kv_heads, d.n_q_heads = 2, 8, 32
+    for k, v in kw.items():
+        setattr(d, k, v)
+    return d
+
+
+def test_workspace_size_rules(rkv):
+    d = _desc(rkv)
+    a = rkv.rkv_workspace_bytes(d, 1024, 128, 8)
+    assert a > 0 and a % 256 == 0
+    d2 = _desc(rkv, batch=4)
+    assert rkv.rkv_workspace_bytes(d2, 1024, 128, 8) > a
+    assert rkv.rkv_host_workspace_bytes(d, 1024, 128, 8) > a + 2 * 2 * 8 * 1152 * 256
+    # invalid shapes give 0
+    assert rkv.rkv_workspace_bytes(_desc(rkv, n_q_heads=30), 1024, 128, 8) == 0      # G not integral
+    assert rkv.rkv_workspace_bytes(_desc(rkv, head_dim=64), 1024, 128, 8) == 0
+    assert rkv.rkv_workspace_bytes(d, 8, 128, 8) == 0                                # budget <= alpha
+    assert rkv.rkv_workspace_bytes(d, 8192, 128, 8) == 0                             # cap > RKV_MAX_CAP
+    assert rkv.rkv_workspace_bytes(_desc(rkv, n_q_heads=8 * 17), 1024, 128, 8) == 0  # G * alpha > 128
+
+
+@pytest.mark.parametrize("case,want", [
+    ("null_k", 1), ("misaligned_q", 1), ("lambda", 1), ("alpha0", 1), ("budget_le_alpha", 1), ("buffer0", 1),
+    ("threshold", 1), ("group", 1), ("head_dim", 2), ("dtype", 2), ("no_workspace", 3), ("small_workspace", 3),
+    ("stage_mask", 1),
+])
+def test_host_detectable_errors_return_before_any_launch(rkv, case, want):
+    """No CUDA call is made on these paths, so they run without a GPU; fake non-null pointers are never
+    dereferenced."""
+    d = _desc(rkv)
+    d.workspace, d.workspace_bytes = 0x10000, 1 << 40
+    k = v = q = 0x20000
+    seq = idx = 0x30000
+    budget, buffer, alpha, lam, mask = 1024, 128, 8, 0.1, rkv.RKV_STAGE_ALL
+    if case == "null_k":
+        k = None
+    elif case == "misaligned_q":
+        q = 0x20008
+    elif case == "lambda":
+        lam = 1.5
+    elif case == "alpha0":
+        alpha = 0
+    elif case == "budget_le_alpha":
+        budget = 8
+    elif case == "buffer0":
+        buffer = 0
+    elif case == "threshold":
+        d.sim_threshold = -0.1
+    elif case == "group":
+        d.n_q_heads = 30
+    elif case == "head_dim":
+        d.head_dim = 256
+    elif case == "dtype":
+        d.dtype = 7
+    elif case == "no_workspace":
+        d.workspace = None
+    elif case == "small_workspace":
+        d.workspace_bytes = 1024
+    elif case == "stage_mask":
+        mask = 32
+    rc = rkv.rkv_compress_stages(d, k, v, q, seq, budget, buffer, alpha, lam, idx, 0, mask)
+    assert rc == want, rkv.rkv_status_string(rc)
+
+
+def test_rkv_compress_needs_a_current_descriptor(rkv):
+    import threading
+    out = {}
+
+    def fresh_thread():     # the current descriptor is per thread
+        out["rc"] = rkv.rkv_compress(0x20000, 0x20000, 0x20000, 0x30000, 1024, 128, 8, 0.1, 0x30000, 0)
+    t = threading.Thread(target=fresh_thread)
+    t.start()
+    t.join()
+    assert out["rc"] == 1
+    assert rkv.rkv_status_string(5) == "RKV_ERR_TIMEOUT"
+    assert rkv.rkv_launch_count(_desc(rkv), rkv.RKV_STAGE_ALL) == 4
+
+
+def test_product_package_does_not_touch_the_oracle():
+    pkg = os.path.join(ROOT, "paper_2505_24133_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                text = open(os.path.join(dirpath, f)).read()
+                assert "oracle" not in text.lower(), f"{f} mentions the oracle"
+    for f in os.listdir(os.path.join(ROOT, "oracle")):
+        if f.endswith((".py", ".c")):
+            text = open(os.path.join(ROOT, "oracle", f)).read()
+            assert "paper_2505_24133_b200" not in text and "librkv_b200" not in text
