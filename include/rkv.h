@@ -88,7 +88,8 @@ typedef struct rkv_desc {
     size_t workspace_bytes;
     int32_t *device_status; /* optional device int32; kernels store the first error they meet
                                (RKV_ERR_INVALID_ARG for seq_lens[b] > cap or < 0, RKV_ERR_TIMEOUT).  The caller
-                               zeroes it and reads it after synchronising the stream */
+                               zeroes it and reads it after synchronising the stream; while it is non-zero the
+                               scoring stage does no work (after an error the results are invalid anyway) */
     /* optional device dumps of the scores, each [batch][n_kv_heads][cap] float, first n entries written */
     float *dbg_I, *dbg_Sbar, *dbg_R, *dbg_Z;
     /* optional: 5 cudaEvent_t handles; event s is recorded before stage s (prep, scores, select, gather)

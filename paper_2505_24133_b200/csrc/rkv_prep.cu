@@ -37,6 +37,7 @@ __global__ void __launch_bounds__(kPrepThreads) prep_kernel(Params p)
         L = kMetaInvalid;
     }
     if (tile == 0 && head % p.hkv == 0 && threadIdx.x == 0) p.meta[b] = L;
+    if (blockIdx.x == 0 && threadIdx.x < 4) p.counters[threadIdx.x] = 0ull;
     const int n = candidates_from_meta(L, p.budget, p.alpha);
 
     const T *K = static_cast<const T *>(p.k_cache) + (size_t)head * p.cap * kHeadDim;
