@@ -23,7 +23,8 @@
  *
  * All pointers in the signatures are DEVICE pointers unless the name starts with
  * "host_".  The library never allocates or frees device memory; scratch comes from
- * the caller through rkv_desc_t.workspace.  Calls enqueue
+ * the caller through rkv_desc_t.workspace (rkv_compress_static alone uses an array
+ * built into the library instead).  Calls enqueue
  * work on the given stream and do not synchronise.  Errors are return codes; nothing
  * throws or aborts.
  */
@@ -152,6 +153,36 @@ RKV_API size_t rkv_host_workspace_bytes(const rkv_desc_t *desc, int32_t budget, 
 RKV_API int rkv_compress_host(const rkv_desc_t *desc, void *host_k_cache, void *host_v_cache, const void *host_q_window,
                       int32_t *host_seq_lens, int32_t budget, int32_t buffer, int32_t alpha, float lambda,
                       int32_t *host_out_idx, void *stream);
+
+/*
+ * rkv_compress_ex for callers that cannot provide a workspace.  (The paper has no counterpart: this is a
+ * deployment convenience, not a step of the method.)
+ *
+ * Who needs it: code that may not call cudaMalloc, or any allocator built on it, at the point where the
+ * buffer fills -- an inference server whose memory pool already owns all of the GPU's memory and hands out
+ * nothing beyond KV blocks, a plug-in running inside another framework's callback where allocation is
+ * forbidden, a real-time loop that must not take the driver's allocation lock.  For them the scratch lives in
+ * a fixed array inside the library's device image, RKV_STATIC_SCRATCH_BYTES (16 MiB) large.  Every GPU that
+ * loads the library carries that array until the process ends, used or not.
+ *
+ * Arguments, layouts, results and error codes are those of rkv_compress_ex; desc->workspace and
+ * desc->workspace_bytes are ignored.  In addition:
+ *   - a shape whose rkv_workspace_bytes() exceeds RKV_STATIC_SCRATCH_BYTES is refused with RKV_ERR_WORKSPACE
+ *     before anything is launched (rkv_workspace_bytes() tells what a shape needs).  16 MiB covers, for example, 256 head-problems at budget 1024 + buffer 128 (all 32 layers of an 8-KV-head model, batch 1);
+ *     larger batches are split into several calls over sub-ranges of the batch dimension, one after the other.
+ *   - the call makes no cudaMalloc / cudaFree and calls no allocating library routine.
+ *   - the FIRST call on each device looks up the array's device address (with that device current) and caches
+ *     it; make that first call outside any stream capture.
+ *   - all calls on a device share the one array, which still holds the previous call's contents.  Nothing in
+ *     it has to start at zero -- every stage writes what the next one reads, and the prep stage clears the
+ *     counters -- but two calls that overlap on the GPU (different streams, no dependency between them) race on
+ *     it and corrupt each other's scores.  Serialise them, or give one of them a workspace of its own through
+ *     rkv_compress_ex.
+ */
+#define RKV_STATIC_SCRATCH_BYTES (16u << 20)
+RKV_API int rkv_compress_static(const rkv_desc_t *desc, void *k_cache, void *v_cache, const void *q_window,
+                        int32_t *seq_lens, int32_t budget, int32_t buffer, int32_t alpha, float lambda,
+                        int32_t *out_idx, void *stream);
 
 /* Number of kernels a call with this descriptor and stage mask launches (for launch accounting). */
 RKV_API int rkv_launch_count(const rkv_desc_t *desc, uint32_t stage_mask);

@@ -62,6 +62,7 @@ def lib():
         L.rkv_compress_ex.restype, L.rkv_compress_ex.argtypes = ctypes.c_int, [P] + ten
         L.rkv_compress_stages.restype, L.rkv_compress_stages.argtypes = ctypes.c_int, [P] + ten + [U32]
         L.rkv_compress_host.restype, L.rkv_compress_host.argtypes = ctypes.c_int, [P] + ten
+        L.rkv_compress_static.restype, L.rkv_compress_static.argtypes = ctypes.c_int, [P] + ten
         L.rkv_launch_count.restype, L.rkv_launch_count.argtypes = ctypes.c_int, [P, U32]
         L.rkv_status_string.restype, L.rkv_status_string.argtypes = ctypes.c_char_p, [ctypes.c_int]
         L.rkv_last_cuda_error.restype, L.rkv_last_cuda_error.argtypes = ctypes.c_char_p, []
@@ -133,6 +134,19 @@ def rkv_compress_host(desc, host_k, host_v, host_q, host_seq_lens, budget, buffe
     return lib().rkv_compress_host(ctypes.byref(desc), _ptr(host_k), _ptr(host_v), _ptr(host_q),
                                    _ptr(host_seq_lens), budget, buffer, alpha, float(lam), _ptr(host_out_idx),
                                    _stream(stream))
+
+
+RKV_STATIC_SCRATCH_BYTES = 16 << 20
+
+
+def rkv_compress_static(desc, k_cache, v_cache, q_window, seq_lens, budget, buffer, alpha, lam, out_idx,
+                        stream=None) -> int:
+    """rkv_compress_ex with the scratch taken from the library's built-in 16 MiB device array, for callers that
+    cannot allocate a workspace; desc.workspace is ignored.  Calls on one device share that array: do not let
+    two of them overlap on the GPU."""
+    return lib().rkv_compress_static(ctypes.byref(desc), _ptr(k_cache), _ptr(v_cache), _ptr(q_window),
+                                     _ptr(seq_lens), budget, buffer, alpha, float(lam), _ptr(out_idx),
+                                     _stream(stream))
 
 
 class Compressor:
