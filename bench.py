@@ -44,6 +44,8 @@ def parse_args():
     ap.add_argument("--pool-w", type=int, default=None)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--batch", type=int, default=None, help="fewer sequences than the workload names (ncu captures)")
+    ap.add_argument("--layers", type=int, default=None, help="fewer layers than the workload names (ncu captures)")
     ap.add_argument("--mem-gb", type=float, default=60.0, help="device memory the input replicas may take")
     return ap.parse_args()
 
@@ -180,11 +182,13 @@ def main():
     dev = torch.device("cuda", local_rank)
     rank, local_rank, world = rd.init("nccl")
     spec = ri.SPECS[args.workload]
+    if args.batch is not None or args.layers is not None:
+        spec = ri.scaled(spec, layers=args.layers, batch=args.batch)
     K, W = args.steps, max(args.warmup, 3)
     peaks = measured_peaks()
 
     # ---- inputs: one pristine workload per rank, replicated so that every step compresses fresh caches
-    wl = ri.make_workload(spec, device=dev, seed=ri.BASE_SEED + 1000 * rank + ri.CONFIG_ORDER.index(spec.name))
+    wl = ri.make_workload(spec, device=dev, seed=ri.BASE_SEED + 1000 * rank + ri.CONFIG_ORDER.index(args.workload))
     bytes_per_replica = 2 * wl.k_cache.numel() * wl.k_cache.element_size()
     budget_bytes = int(args.mem_gb * 2 ** 30)
     n_rep = max(1, min(K + W, budget_bytes // bytes_per_replica))

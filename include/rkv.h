@@ -57,7 +57,11 @@ typedef enum { RKV_BF16 = 0, RKV_F32 = 1 } rkv_dtype_t;
 
 /* rkv_desc_t.flags */
 #define RKV_FLAG_SIMT_SCORES 1u /* score with the plain fp32 CUDA-core kernel instead of the tcgen05
-                                   kernel (always used for RKV_F32; a debugging aid for RKV_BF16) */
+                                   kernels (always used for RKV_F32; a debugging aid for RKV_BF16) */
+#define RKV_FLAG_ROWBLOCK_SCORES 2u /* bf16: score with the row-block tcgen05 kernel (forms the full similarity
+                                   matrix) instead of the default triangle kernels (upper-triangular tiles, then
+                                   only the tokens still short of partners against the tiles to their left);
+                                   a cross-check */
 
 /* stage bits for rkv_compress_stages */
 #define RKV_STAGE_PREP 1u    /* key inverse norms and per-tile sums of normalised keys */
@@ -67,7 +71,7 @@ typedef enum { RKV_BF16 = 0, RKV_F32 = 1 } rkv_dtype_t;
 #define RKV_STAGE_ALL 15u
 
 #define RKV_MAX_CAP 8192     /* largest supported budget + buffer */
-#define RKV_MAX_GROUP_ROWS 128 /* largest supported (n_q_heads / n_kv_heads) * alpha */
+#define RKV_MAX_GROUP_ROWS 112 /* largest supported (n_q_heads / n_kv_heads) * alpha */
 
 /*
  * Problem descriptor.  Plain data, owned by the caller, copied on use.
@@ -184,7 +188,8 @@ RKV_API int rkv_compress_static(const rkv_desc_t *desc, void *k_cache, void *v_c
                         int32_t *seq_lens, int32_t budget, int32_t buffer, int32_t alpha, float lambda,
                         int32_t *out_idx, void *stream);
 
-/* Number of kernels a call with this descriptor and stage mask launches (for launch accounting). */
+/* Number of kernels a call with this descriptor and stage mask launches (for launch accounting; the memset that
+ * precedes the prep kernel is not counted). */
 RKV_API int rkv_launch_count(const rkv_desc_t *desc, uint32_t stage_mask);
 
 /* Human-readable name of a status code. */

@@ -20,9 +20,15 @@ int cuda_fail(cudaError_t e, const char *where)
 }
 
 struct Layout {
-    size_t inv_norm, tile_sum, logits, sbar, meta, counters, total;
-    int cap, cap_pad, tiles;
+    size_t inv_norm, tile_sum, head_sum, logits, sbar, left, strag, strag_count, strag_items, self_dot, head_sum_bf16, meta, counters,
+        tile_done, zero_bytes, total;
+    int cap, cap_pad, tiles, tri;
 };
+
+bool use_simt(const rkv_desc_t *d) { return d->dtype == RKV_F32 || (d->flags & RKV_FLAG_SIMT_SCORES); }
+
+// 1 when the triangle tensor-core kernels score (bf16 caches, unless a cross-check kernel is asked for).
+int use_tri(const rkv_desc_t *d) { return !(use_simt(d) || (d->flags & RKV_FLAG_ROWBLOCK_SCORES)); }
 
 // Returns RKV_OK and fills *lay when the shape arguments are usable.
 int check_shapes(const rkv_desc_t *d, int budget, int buffer, int alpha, Layout *lay)
@@ -47,18 +53,28 @@ int check_shapes(const rkv_desc_t *d, int budget, int buffer, int alpha, Layout 
         size_t off = 0;
         lay->inv_norm = off;  off = align_up(off + P * lay->cap_pad * sizeof(float), 256);
         lay->tile_sum = off;  off = align_up(off + P * lay->tiles * kHeadDim * sizeof(float), 256);
+        lay->head_sum = off;  off = align_up(off + P * kHeadDim * sizeof(float), 256);
         lay->logits = off;    off = align_up(off + P * alpha * lay->cap_pad * sizeof(float), 256);
         lay->sbar = off;      off = align_up(off + P * lay->cap_pad * sizeof(float), 256);
-        lay->meta = off;      off = align_up(off + (size_t)d->batch * sizeof(int32_t), 256);
-        lay->counters = off;  off = align_up(off + 4 * sizeof(unsigned long long), 256);
+        lay->tri = use_tri(d);
+        const size_t tri = (size_t)lay->tri;
+        lay->left = off;        off = align_up(off + tri * P * lay->cap_pad * sizeof(int32_t), 256);
+        lay->strag = off;       off = align_up(off + tri * P * lay->cap_pad * sizeof(int32_t), 256);
+        lay->strag_count = off; off = align_up(off + tri * P * sizeof(int32_t), 256);
+        lay->strag_items = off; off = align_up(off + tri * P * (lay->cap_pad / 256 + 1) * sizeof(int2), 256);
+        lay->self_dot = off;    off = align_up(off + P * lay->cap_pad * sizeof(float), 256);
+        lay->head_sum_bf16 = off; off = align_up(off + P * 16 * kHeadDim * sizeof(__nv_bfloat16), 256);
+        lay->meta = off;        off = align_up(off + (size_t)d->batch * sizeof(int32_t), 256);
+        // the region the prep stage zeroes: counters and per-head tile tickets
+        lay->counters = off;    off = align_up(off + 4 * sizeof(unsigned long long), 256);
+        lay->tile_done = off;   off = align_up(off + P * sizeof(uint32_t), 256);
+        lay->zero_bytes = off - lay->counters;
         lay->total = off;
     }
     return RKV_OK;
 }
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
-
-bool use_simt(const rkv_desc_t *d) { return d->dtype == RKV_F32 || (d->flags & RKV_FLAG_SIMT_SCORES); }
 
 int run(const rkv_desc_t *d, void *k_cache, void *v_cache, const void *q_window, int32_t *seq_lens, int budget,
         int buffer, int alpha, float lambda, int32_t *out_idx, void *stream, uint32_t stages)
@@ -102,10 +118,20 @@ int run(const rkv_desc_t *d, void *k_cache, void *v_cache, const void *q_window,
     char *ws = static_cast<char *>(d->workspace);
     p.inv_norm = reinterpret_cast<float *>(ws + lay.inv_norm);
     p.tile_sum = reinterpret_cast<float *>(ws + lay.tile_sum);
+    p.head_sum = reinterpret_cast<float *>(ws + lay.head_sum);
     p.logits = reinterpret_cast<float *>(ws + lay.logits);
     p.sbar = reinterpret_cast<float *>(ws + lay.sbar);
+    p.left = reinterpret_cast<int32_t *>(ws + lay.left);
+    p.strag = reinterpret_cast<int32_t *>(ws + lay.strag);
+    p.strag_count = reinterpret_cast<int32_t *>(ws + lay.strag_count);
+    p.strag_items = reinterpret_cast<int2 *>(ws + lay.strag_items);
+    p.self_dot = reinterpret_cast<float *>(ws + lay.self_dot);
+    p.head_sum_bf16 = reinterpret_cast<__nv_bfloat16 *>(ws + lay.head_sum_bf16);
     p.meta = reinterpret_cast<int32_t *>(ws + lay.meta);
     p.counters = reinterpret_cast<unsigned long long *>(ws + lay.counters);
+    p.tile_done = reinterpret_cast<uint32_t *>(ws + lay.tile_done);
+    p.zero_bytes = lay.zero_bytes;
+    p.tri = lay.tri;
     p.status = d->device_status;
     p.dbg_I = d->dbg_I;
     p.dbg_Sbar = d->dbg_Sbar;
@@ -119,11 +145,14 @@ int run(const rkv_desc_t *d, void *k_cache, void *v_cache, const void *q_window,
         return ev && ev[i] ? cudaEventRecord(static_cast<cudaEvent_t>(ev[i]), s) : cudaSuccess;
     };
     if ((e = mark(0)) != cudaSuccess) return cuda_fail(e, "cudaEventRecord");
-    if (stages & RKV_STAGE_PREP)
+    if (stages & RKV_STAGE_PREP) {
+        if ((e = cudaMemsetAsync(p.counters, 0, p.zero_bytes, s)) != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
         if ((e = launch_prep(p, s)) != cudaSuccess) return cuda_fail(e, "prep launch");
+    }
     if ((e = mark(1)) != cudaSuccess) return cuda_fail(e, "cudaEventRecord");
     if (stages & RKV_STAGE_SCORES) {
-        e = use_simt(d) ? launch_scores_simt(p, s) : launch_scores_sm100(p, s);
+        e = use_simt(d) ? launch_scores_simt(p, s)
+                        : (p.tri ? launch_scores_tri_sm100(p, s) : launch_scores_sm100(p, s));
         if (e != cudaSuccess) return cuda_fail(e, "scores launch");
     }
     if ((e = mark(2)) != cudaSuccess) return cuda_fail(e, "cudaEventRecord");
@@ -268,9 +297,10 @@ int rkv_compress_host(const rkv_desc_t *desc, void *host_k_cache, void *host_v_c
 
 int rkv_launch_count(const rkv_desc_t *desc, uint32_t stage_mask)
 {
-    (void)desc;
     int c = 0;
     for (uint32_t bit = 1; bit <= RKV_STAGE_GATHER; bit <<= 1) c += (stage_mask & bit) ? 1 : 0;
+    // the triangle scoring path is three kernels (pass 1, listing, pass 2) while the retention rule is on
+    if (desc && (stage_mask & RKV_STAGE_SCORES) && use_tri(desc) && desc->beta > 0 && desc->sim_threshold < 1.0f) c += 2;
     return c;
 }
 

@@ -35,10 +35,25 @@ struct Params {
     // workspace carve-up
     float *inv_norm;     // [P][cap_pad]         r_i = 1 / (||k_i|| + eps); 0 for i >= n
     float *tile_sum;     // [P][tiles][128]      sum over the tile's candidate rows of r_i * k_i
+    float *head_sum;     // [P][128]             sum over all candidate rows of r_i * k_i (the tile sums added up)
     float *logits;       // [P][alpha][cap_pad]  Eq. 2-3: group-max of scaled logits
-    float *sbar;         // [P][cap_pad]         Eq. 6 column means after the retention rule
+    float *sbar;         // [P][cap_pad]         Eq. 6 column means after the retention rule.  With `tri` set the scoring
+                         //                      kernels leave column SUMS minus the removed entries (the select stage
+                         //                      divides by n)
+    int32_t *left;       // [P][cap_pad]         tri: partners a token still lacks after the scan of its own line
+    int32_t *strag;      // [P][cap_pad]         tri: positions of the head's tokens with left > 0, ascending
+    int32_t *strag_count;// [P]                  tri: how many
+    int2 *strag_items;   // [P * cap_pad / 256]  tri: work list of the second scoring pass, {head, chunk of 256}
+    float *self_dot;     // [P][cap_pad]         Kbar_i . Kbar_i (1 up to rounding and eps; 0 for a zero key)
+    __nv_bfloat16 *head_sum_bf16;   // [P][16][128] head_sum split into three bf16 rows (hi, mid, lo), 13 zero rows
     int32_t *meta;       // [batch]              snapshot of seq_lens (kMetaInvalid if out of range)
-    unsigned long long *counters;   // [4]       [0] = similarity tiles computed by the tcgen05 kernel
+    // zeroed by the prep stage's memset, in this order, contiguous:
+    unsigned long long *counters;   // [4]       [0] = similarity tiles computed by the tcgen05 kernels, [1] = item
+                                    //           ticket of the first scoring pass, [2] = entries in strag_items,
+                                    //           [3] = item ticket of the second pass
+    uint32_t *tile_done;            // [P]       tiles of the head finished by the prep stage
+    size_t zero_bytes;              // bytes from `counters` to the end of `tile_done`
+    int tri;                        // 1: the triangle kernels score (bf16 default); 0: another kernel does
     // optional outputs
     int32_t *status;
     float *dbg_I, *dbg_Sbar, *dbg_R, *dbg_Z;
@@ -86,6 +101,7 @@ template <> struct Elem<float> {
 cudaError_t launch_prep(const Params &p, cudaStream_t s);
 cudaError_t launch_scores_simt(const Params &p, cudaStream_t s);
 cudaError_t launch_scores_sm100(const Params &p, cudaStream_t s);
+cudaError_t launch_scores_tri_sm100(const Params &p, cudaStream_t s);
 cudaError_t launch_select(const Params &p, cudaStream_t s);
 cudaError_t launch_gather(const Params &p, cudaStream_t s);
 bool scores_sm100_available();

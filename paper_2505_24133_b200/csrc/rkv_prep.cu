@@ -5,6 +5,8 @@
 // scoring stage obtain sum_j S[j][i] = Kbar_i . (sum_j Kbar_j) - Kbar_i . Kbar_i (Eq. 6 before the
 // retention rule) without accumulating the n x n matrix element by element.
 // Rows i >= n (observation tokens, unused capacity) get r_i = 0 and contribute nothing.
+// The last block to finish a head also leaves sum_i r_i * k_i over the whole head (head_sum).
+// Kbar_i . Kbar_i is kept per row as well (self_dot).
 //
 // HBM-bound: K is read once with 16-byte loads, rows coalesced across the lanes of a warp; the row
 // norm is reduced with warp shuffles.  Outputs are 4 bytes per 256-byte row.
@@ -37,7 +39,6 @@ __global__ void __launch_bounds__(kPrepThreads) prep_kernel(Params p)
         L = kMetaInvalid;
     }
     if (tile == 0 && head % p.hkv == 0 && threadIdx.x == 0) p.meta[b] = L;
-    if (blockIdx.x == 0 && threadIdx.x < 4) p.counters[threadIdx.x] = 0ull;
     const int n = candidates_from_meta(L, p.budget, p.alpha);
 
     const T *K = static_cast<const T *>(p.k_cache) + (size_t)head * p.cap * kHeadDim;
@@ -71,7 +72,10 @@ __global__ void __launch_bounds__(kPrepThreads) prep_kernel(Params p)
 #pragma unroll
         for (int off = kLanesPerRow / 2; off > 0; off >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, off);
         const float r = (row < n) ? __fdiv_rn(1.0f, __fsqrt_rn(sq) + p.eps) : 0.f;
-        if (lane % kLanesPerRow == 0 && row < p.cap_pad) inv_norm[row] = r;
+        if (lane % kLanesPerRow == 0) {
+            inv_norm[row] = r;                       // row < cap_pad: the grid covers exactly cap_pad rows per head
+            p.self_dot[(size_t)head * p.cap_pad + row] = (r * r) * sq;     // Kbar_i . Kbar_i
+        }
 #pragma unroll
         for (int e = 0; e < kPerVec; ++e) acc[e] = fmaf(r, f[e], acc[e]);
     }
@@ -92,6 +96,32 @@ __global__ void __launch_bounds__(kPrepThreads) prep_kernel(Params p)
 #pragma unroll
         for (int w = 0; w < kPrepWarps; ++w) s += part[w][threadIdx.x];
         p.tile_sum[((size_t)head * p.tiles + tile) * kHeadDim + threadIdx.x] = s;
+    }
+
+    // The block that finishes a head's last tile adds the tile sums up, always in tile order, so the result does
+    // not depend on which block that is.  (tile_done is zeroed by the memset that precedes this kernel.)
+    __shared__ bool last_block;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) last_block = (atomicAdd(&p.tile_done[head], 1u) == (unsigned)p.tiles - 1u);
+    __syncthreads();
+    if (last_block && threadIdx.x < kHeadDim) {
+        __threadfence();
+        const float *ts = p.tile_sum + (size_t)head * p.tiles * kHeadDim + threadIdx.x;
+        float s = 0.f;
+        for (int t = 0; t < p.tiles; ++t) s += __ldcg(ts + (size_t)t * kHeadDim);
+        p.head_sum[(size_t)head * kHeadDim + threadIdx.x] = s;
+        // the same vector as three bf16 rows whose sum is s to fp32 accuracy (rows 3..15 of the 16-row block are
+        // zero): appended to the query rows, it lets the tensor cores form Kbar_i . s along with the logits
+        __nv_bfloat16 *hs = p.head_sum_bf16 + (size_t)head * 16 * kHeadDim + threadIdx.x;
+        float rest = s;
+#pragma unroll
+        for (int part_i = 0; part_i < 3; ++part_i) {
+            const __nv_bfloat16 h16 = __float2bfloat16_rn(rest);
+            hs[part_i * kHeadDim] = h16;
+            rest -= __bfloat162float(h16);
+        }
+        for (int z = 3; z < 16; ++z) hs[z * kHeadDim] = __float2bfloat16_rn(0.f);
     }
 }
 

@@ -1,0 +1,661 @@
+// Stage "scores", tensor-core version for bf16 caches (the default): tcgen05.mma with TMEM accumulators, fed by
+// TMA, one persistent block per SM.  Two passes over Eq. 5's similarity matrix that form only the part of it the
+// result can depend on.
+//
+// Section 3.3's rule needs, per token i, the beta LARGEST positions j with S[j][i] > T.  S is symmetric before the
+// rule, so token i's line can be read as row i.
+//
+//   pass 1  Every token against the LAST positions.  Work item = (head, pair of row tiles p): rows
+//           [256 p, 256 p + 256) stay resident in shared memory as two 128 x 128 bf16 operand tiles
+//           (double-buffered across items); the last kPass1Depth key tiles (for the last row tiles: down to their
+//           own, diagonal tile) stream through a 3-stage ring.  One thread owns one token and scans its line from
+//           the last position downwards, so the rule is "the first beta hits", kept in registers.  Before the key
+//           tiles, the item multiplies its resident tiles with the head's G * alpha query rows (Eq. 2-3: a thread
+//           ends up with all logits of its key and takes the max over the group).  Out: logits, the column sum
+//           minus the removed entries, and `left` = partners still lacking.
+//   compact The tokens with left > 0 (a few per cent when similar keys are common; all of them when nothing
+//           exceeds T) are listed per head, ascending, in chunks of 256.
+//   pass 2  Work item = (head, chunk of 256 listed tokens): their key rows are gathered into the resident tiles
+//           by the epilogue warps; the key tiles from where pass 1 stopped down to tile 0 stream through the same
+//           ring.  The removed entries are subtracted from what pass 1 stored.
+//
+// So the tensor cores form (tokens) x (the last positions) plus (listed tokens) x (the rest) entries per head
+// instead of n^2; the n x n matrix never leaves TMEM, and no atomics or global flags are involved.
+//
+// Per element the epilogue costs one multiply (g r_j) and half a max; only a 32-column chunk whose maximum
+// exceeds the token's threshold T / r_i is looked at entry by entry, last first.
+// The plain column sum of Eq. 6 is not accumulated element by element:
+// sum_j S[j][i] = Kbar_i . (sum_j Kbar_j) - Kbar_i . Kbar_i, with sum_j Kbar_j from the prep stage.
+//
+// Items are handed out by a global ticket counter, longest first within a head, so neighbouring blocks work on
+// the same head while its keys are in L2.
+// Warp roles (320 threads): warp 0 = ticket + TMA producer, warp 1 = MMA issuer and TMEM owner, warps 2..9 =
+// epilogue (warp w may touch TMEM lanes 32 (w % 4) .. +31; warps 2-5 serve row tile 0, warps 6-9 row tile 1).
+// TMEM: four 128-column fp32 accumulators, two per row tile, so the tensor pipe fills one while the epilogue
+// drains the other.  Every wait on an mbarrier is bounded; on expiry the block records RKV_ERR_TIMEOUT, stops
+// issuing work and leaves through the common exit that frees TMEM.  No TMA multicast and no cluster launch.
+#include "rkv_sm100.cuh"
+
+namespace rkv {
+
+namespace {
+
+using namespace sm100;
+
+constexpr int kThreads = 320;
+constexpr int kStagesB = 3;                      // ring depth of streamed tiles
+constexpr int kItemSlots = 4;                    // ring depth of item descriptors
+constexpr int kHalfBytes = kTile * 64 * 2;       // one TMA box: 128 rows x 64 bf16 (128-byte swizzled rows)
+constexpr int kTileBytes = 2 * kHalfBytes;       // 32 KB: a 128 x 128 bf16 operand tile
+constexpr int kRowsPerItem = 2 * kTile;
+constexpr uint32_t kTmemCols = 512;
+constexpr int kPass1Depth = 2;                   // key tiles every token is scanned against in pass 1
+
+// shared memory carve-up (offsets from a 1024-byte aligned base)
+constexpr int kOffA = 0;                                   // 2 buffers x 2 resident tiles
+constexpr int kOffB = kOffA + 2 * 2 * kTileBytes;          // kStagesB streamed tiles
+constexpr int kOffBar = kOffB + kStagesB * kTileBytes;     // mbarriers
+enum {
+    kBarQFull = 0,                          // [kItemSlots] item descriptor written
+    kBarQEmpty = kBarQFull + kItemSlots,    // [kItemSlots] read by the MMA thread and the 8 epilogue warps
+    kBarAFull = kBarQEmpty + kItemSlots,    // [2] resident tiles in place
+    kBarAEmpty = kBarAFull + 2,             // [2] resident tiles no longer read
+    kBarBFull = kBarAEmpty + 2,             // [kStagesB]
+    kBarBEmpty = kBarBFull + kStagesB,      // [kStagesB]
+    kBarAccFull = kBarBEmpty + kStagesB,    // [2 buffers][2 row tiles]
+    kBarAccEmpty = kBarAccFull + 4,         // [2][2], 4 warps each
+    kNumBars = kBarAccEmpty + 4
+};
+constexpr int kOffItems = kOffBar + kNumBars * 8;          // kItemSlots x int4
+constexpr int kOffMisc = kOffItems + kItemSlots * 16;      // tmem base, abort flag, bail flag
+constexpr int kOffRj = kOffMisc + 16;                      // [2 row tiles][128] r_j of the key tile being drained
+constexpr int kSmemBytes = kOffRj + 2 * kTile * 4 + 1024;  // + slack for the manual 1024-byte alignment
+static_assert(kOffItems % 16 == 0 && kOffRj % 16 == 0, "item descriptors are read as int4, r_j as float4");
+static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
+
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&r)[8])
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_ld1(uint32_t taddr, uint32_t &r)
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(r) : "r"(taddr) : "memory");
+}
+// Wait for the thread's TMEM loads; the loaded registers pass through the statement so that nothing that uses
+// them can be scheduled ahead of it.
+__device__ __forceinline__ void tmem_wait8(uint32_t (&r)[8])
+{
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7])
+                 :: "memory");
+}
+__device__ __forceinline__ void tmem_wait32(uint32_t (&r)[32])
+{
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                   "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+                   "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
+                   "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+                 :: "memory");
+}
+
+// max(a, b, c), NaN operands ignored
+__device__ __forceinline__ float max3(float a, float b, float c)
+{
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
+struct Bars {
+    uint32_t bar0;
+    __device__ __forceinline__ uint32_t at(int idx) const { return bar0 + 8 * idx; }
+};
+
+// Item descriptor (int4).  Pass 1: {head, pair p, n, -}.  Pass 2: {head, first listed token k0, tokens in the item
+// (1..256), first streamed tile}.  x < 0: no more items.
+//
+// kPass2 = false: pass 1; true: pass 2 (see the top of the file).
+template <bool kPass2>
+__global__ void __launch_bounds__(kThreads, 1)
+scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_q,
+                        const __grid_constant__ CUtensorMap map_hs, int items_per_head,
+                        unsigned long long total_items_host, int q_rows_pad)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const uint32_t sbase = smem_u32(smem);
+    int4 *items = reinterpret_cast<int4 *>(smem + kOffItems);
+    uint32_t *tmem_holder = reinterpret_cast<uint32_t *>(smem + kOffMisc);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + kOffMisc + 4);
+    volatile int *bail = reinterpret_cast<volatile int *>(smem + kOffMisc + 8);
+    const Bars bar{sbase + kOffBar};
+
+    // Once any block has recorded an error, the blocks still to start return at once.  Pass 2 has nothing to do
+    // when the list is empty.
+    if (threadIdx.x == 0) {
+        int b = (p.status != nullptr && *reinterpret_cast<volatile int32_t *>(p.status) != 0);
+        if (kPass2 && p.counters[2] == 0ull) b = 1;
+        *bail = b;
+    }
+    __syncthreads();
+    if (*bail) return;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const bool rule_on = p.beta > 0 && p.sim_threshold < 1.0f;
+    const unsigned long long total_items = kPass2 ? p.counters[2] : total_items_host;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kItemSlots; ++s) {
+            mbar_init(bar.at(kBarQFull + s), 1);
+            mbar_init(bar.at(kBarQEmpty + s), 9);
+        }
+        for (int s = 0; s < 2; ++s) {
+            // pass 1: TMA fills the resident tiles; pass 2: the 8 epilogue warps do; the MMA thread reads them
+            mbar_init(bar.at(kBarAFull + s), kPass2 ? 8 : 1);
+            mbar_init(bar.at(kBarAEmpty + s), 1);
+        }
+        for (int s = 0; s < kStagesB; ++s) {
+            mbar_init(bar.at(kBarBFull + s), 1);
+            mbar_init(bar.at(kBarBEmpty + s), 1);
+        }
+        for (int s = 0; s < 4; ++s) {
+            mbar_init(bar.at(kBarAccFull + s), 1);
+            mbar_init(bar.at(kBarAccEmpty + s), 4);
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(tmem_holder)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_holder;
+    unsigned long long tiles_done = 0ull;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ tickets + TMA producer
+        if (lane == 0) {
+            uint32_t k_item = 0, bcount = 0;
+            bool ok = true;
+            // the next ticket is drawn while the current item is set up (a block draws one ticket too many)
+            unsigned long long next_ticket = atomicAdd(&p.counters[kPass2 ? 3 : 1], 1ull);
+            while (ok) {
+                const unsigned long long ticket = next_ticket;
+                if (ticket >= total_items) break;
+                next_ticket = atomicAdd(&p.counters[kPass2 ? 3 : 1], 1ull);
+                int4 desc;
+                int n_iter, first_tile, head;
+                if (!kPass2) {
+                    head = (int)(ticket / (unsigned)items_per_head);
+                    const int pi = (int)(ticket % (unsigned)items_per_head);
+                    const int n = candidates_from_meta(p.meta[head / p.hkv], p.budget, p.alpha);
+                    if (n == 0 || pi * kRowsPerItem >= n) continue;             // nothing to score in this item
+                    const int n_tiles = (n + kTile - 1) / kTile;
+                    desc = make_int4(head, pi, n, 0);
+                    first_tile = n_tiles - 1;                  // streamed tiles: first_tile .. max(2 pi, n_tiles - depth)
+                    n_iter = 1 + (rule_on ? n_tiles - max(2 * pi, n_tiles - kPass1Depth) : 0);   // + the query rows
+                } else {
+                    const int2 e = p.strag_items[ticket];
+                    head = e.x;
+                    const int k0 = e.y * kRowsPerItem;
+                    const int rows = min(p.strag_count[head] - k0, kRowsPerItem);
+                    const int last = p.strag[(size_t)head * p.cap_pad + k0 + rows - 1];
+                    const int n = candidates_from_meta(p.meta[head / p.hkv], p.budget, p.alpha);
+                    // pass 1 took the last listed token down to tile max(its own, n_tiles - depth)
+                    first_tile = max(last / kTile, (n + kTile - 1) / kTile - kPass1Depth) - 1;   // streamed: first_tile .. 0
+                    if (rows <= 0 || first_tile < 0) continue;                  // (the list holds no such item)
+                    desc = make_int4(head, k0, rows, first_tile);
+                    n_iter = first_tile + 1;
+                }
+                const int key_row_base = head * p.cap;                         // first row of the head in the 2-D key view
+
+                const uint32_t qs = k_item % kItemSlots;
+                if (!mbar_wait(bar.at(kBarQEmpty + qs), ((k_item / kItemSlots) & 1) ^ 1, abort_flag, p.status)) break;
+                items[qs] = desc;
+                mbar_arrive(bar.at(kBarQFull + qs));
+
+                if (!kPass2) {
+                    const int row0 = desc.y * kRowsPerItem;
+                    const int num_m = (desc.z - row0 > kTile) ? 2 : 1;
+                    const uint32_t ab = k_item & 1;
+                    if (!mbar_wait(bar.at(kBarAEmpty + ab), ((k_item >> 1) & 1) ^ 1, abort_flag, p.status)) break;
+                    mbar_expect_tx(bar.at(kBarAFull + ab), (uint32_t)(num_m * kTileBytes));
+                    for (int m = 0; m < num_m; ++m) {
+                        const uint32_t dst = sbase + kOffA + (ab * 2 + m) * kTileBytes;
+                        const int y = key_row_base + row0 + m * kTile;
+                        tma_load_2d(dst, &map_k, 0, y, bar.at(kBarAFull + ab));
+                        tma_load_2d(dst + kHalfBytes, &map_k, 64, y, bar.at(kBarAFull + ab));
+                    }
+                }
+                for (int it = 0; it < n_iter; ++it) {
+                    const uint32_t s = bcount % kStagesB;
+                    if (!mbar_wait(bar.at(kBarBEmpty + s), ((bcount / kStagesB) & 1) ^ 1, abort_flag, p.status)) {
+                        ok = false;
+                        break;
+                    }
+                    const uint32_t dst = sbase + kOffB + s * kTileBytes;
+                    if (!kPass2 && it == 0) {
+                        const int b = head / p.hkv, h = head % p.hkv;
+                        const int q_row = (b * p.hq + h * p.group) * p.alpha;
+                        // the query rows, then 16 rows holding sum_j Kbar_j split into bf16 parts
+                        mbar_expect_tx(bar.at(kBarBFull + s), (uint32_t)(2 * (q_rows_pad + 16) * 128));
+                        tma_load_2d(dst, &map_q, 0, q_row, bar.at(kBarBFull + s));
+                        tma_load_2d(dst + kHalfBytes, &map_q, 64, q_row, bar.at(kBarBFull + s));
+                        tma_load_2d(dst + q_rows_pad * 128, &map_hs, 0, head * 16, bar.at(kBarBFull + s));
+                        tma_load_2d(dst + kHalfBytes + q_rows_pad * 128, &map_hs, 64, head * 16, bar.at(kBarBFull + s));
+                    } else {
+                        const int jt = first_tile - (kPass2 ? it : it - 1);
+                        const int y = key_row_base + jt * kTile;
+                        mbar_expect_tx(bar.at(kBarBFull + s), kTileBytes);
+                        tma_load_2d(dst, &map_k, 0, y, bar.at(kBarBFull + s));
+                        tma_load_2d(dst + kHalfBytes, &map_k, 64, y, bar.at(kBarBFull + s));
+                    }
+                    ++bcount;
+                }
+                ++k_item;
+            }
+            // terminator: tells the other roles that no item follows (skipped when the block is aborting)
+            if (!*abort_flag) {
+                const uint32_t qs = k_item % kItemSlots;
+                if (mbar_wait(bar.at(kBarQEmpty + qs), ((k_item / kItemSlots) & 1) ^ 1, abort_flag, p.status)) {
+                    items[qs] = make_int4(-1, 0, 0, 0);
+                    mbar_arrive(bar.at(kBarQFull + qs));
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc_k = instr_desc(kTile, kTile), idesc_q = instr_desc(kTile, q_rows_pad + 16);
+            uint32_t k_item = 0, bcount = 0, cnt[2] = {0u, 0u};
+            bool ok = true;
+            while (ok) {
+                const uint32_t qs = k_item % kItemSlots;
+                if (!mbar_wait(bar.at(kBarQFull + qs), (k_item / kItemSlots) & 1, abort_flag, p.status)) break;
+                const int4 d = items[qs];
+                mbar_arrive(bar.at(kBarQEmpty + qs));
+                if (d.x < 0) break;
+                int num_m, n_iter, skip_it;       // skip_it: the iteration whose row tile 1 would mirror row tile 0's
+                if (!kPass2) {
+                    const int n_tiles = (d.z + kTile - 1) / kTile;
+                    num_m = (d.z - d.y * kRowsPerItem > kTile) ? 2 : 1;
+                    n_iter = 1 + (rule_on ? n_tiles - max(2 * d.y, n_tiles - kPass1Depth) : 0);
+                    // row tile 2p + 1 stops at its diagonal tile: it skips tile 2p if the item gets that far
+                    skip_it = (2 * d.y >= n_tiles - kPass1Depth) ? n_iter - 1 : -1;
+                } else {
+                    num_m = d.z > kTile ? 2 : 1;
+                    n_iter = d.w + 1;
+                    skip_it = -1;
+                }
+                const uint32_t ab = k_item & 1;
+                if (!mbar_wait(bar.at(kBarAFull + ab), (k_item >> 1) & 1, abort_flag, p.status)) break;
+                if (kPass2) asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                for (int it = 0; it < n_iter; ++it) {
+                    const uint32_t s = bcount % kStagesB;
+                    if (!mbar_wait(bar.at(kBarBFull + s), (bcount / kStagesB) & 1, abort_flag, p.status)) {
+                        ok = false;
+                        break;
+                    }
+                    const uint32_t stage = sbase + kOffB + s * kTileBytes;
+                    const bool is_q = !kPass2 && it == 0;
+                    for (int m = 0; m < num_m; ++m) {
+                        if (m == 1 && it == skip_it && it > 0) continue;
+                        const uint32_t a = cnt[m] & 1;
+                        if (!mbar_wait(bar.at(kBarAccEmpty + a * 2 + m), ((cnt[m] >> 1) & 1) ^ 1, abort_flag, p.status)) {
+                            ok = false;
+                            break;
+                        }
+                        tc_fence_after();
+                        const uint32_t resident = sbase + kOffA + (ab * 2 + m) * kTileBytes;
+                        const uint32_t d_tmem = tmem_base + a * 256 + m * 128;
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) {
+                            // K = 16 per instruction: 32 bytes along the swizzled row; k >= 4 is the second box
+                            const uint32_t koff = (k >> 2) * kHalfBytes + (k & 3) * 32;
+                            umma(d_tmem, smem_desc(resident + koff), smem_desc(stage + koff), is_q ? idesc_q : idesc_k,
+                                 k > 0);
+                        }
+                        umma_commit(bar.at(kBarAccFull + a * 2 + m));
+                        ++cnt[m];
+                        if (!is_q) ++tiles_done;
+                    }
+                    if (!ok) break;
+                    umma_commit(bar.at(kBarBEmpty + s));          // the stage may be refilled once these MMAs have read it
+                    ++bcount;
+                }
+                if (!ok) break;
+                umma_commit(bar.at(kBarAEmpty + ab));             // so may the resident tiles
+                ++k_item;
+            }
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------------ epilogue warps
+        const int ew = warp - 2;                 // 0..7
+        const int m = ew >> 2;                   // row tile of the item this warp serves
+        const int quad = warp & 3;               // TMEM lane quadrant this warp may access
+        const int lrow = quad * 32 + lane;       // row within the 128-row tile
+        const uint32_t lane_base = tmem_base + ((uint32_t)(quad * 32) << 16);
+        const float kInf = __int_as_float(0x7f800000);
+        const float scale = 0.08838834764831845f;             // 1 / sqrt(128)
+        const int G = p.group;
+        uint32_t k_item = 0, cnt = 0;
+
+        while (true) {
+            const uint32_t qs = k_item % kItemSlots;
+            if (!mbar_wait(bar.at(kBarQFull + qs), (k_item / kItemSlots) & 1, abort_flag, p.status)) break;
+            const int4 d = items[qs];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar.at(kBarQEmpty + qs));
+            if (d.x < 0) break;
+            const int head = d.x;
+            const float *inv_norm = p.inv_norm + (size_t)head * p.cap_pad;
+            const uint32_t ab = k_item & 1;
+
+            // ---- per item: which token this thread owns, its threshold, where its scan starts and ends
+            // (a failed wait does not leave the item at once: the warps of a row tile meet at named barriers in the
+            // tile loop below, so all of them have to reach it)
+            bool active, row_ok, item_ok = true;
+            int i, first_tile, my_last_tile, own_tile;
+            float ri, self = 0.f, total = 0.f;
+            int left = 0;
+            if (!kPass2) {
+                const int pi = d.y, n = d.z;
+                const int row0 = pi * kRowsPerItem;
+                active = (m == 0) || (n - row0 > kTile);
+                i = row0 + m * kTile + lrow;
+                row_ok = active && i < n;
+                ri = row_ok ? __ldg(inv_norm + i) : 0.f;
+                self = row_ok ? __ldg(p.self_dot + (size_t)head * p.cap_pad + i) : 0.f;
+                first_tile = (n + kTile - 1) / kTile - 1;                 // first streamed tile
+                my_last_tile = max(2 * pi + m, first_tile + 1 - kPass1Depth);   // where this row tile's scan stops
+                own_tile = 0x7fffffff;                                    // pass 1: every streamed tile takes part
+                left = row_ok ? p.beta : 0;
+            } else {
+                const int k0 = d.y, rows = d.z;
+                active = (m == 0) || (rows > kTile);
+                const int k = k0 + m * kTile + lrow;
+                row_ok = active && (m * kTile + lrow) < rows;
+                i = row_ok ? p.strag[(size_t)head * p.cap_pad + k] : 0;
+                ri = row_ok ? __ldg(inv_norm + i) : 0.f;
+                {
+                    const int n = candidates_from_meta(p.meta[head / p.hkv], p.budget, p.alpha);
+                    // pass 1 scanned the token down to tile max(its own, n_tiles - depth): it takes part below that
+                    own_tile = row_ok ? max(i / kTile, (n + kTile - 1) / kTile - kPass1Depth) : 0;
+                }
+                first_tile = d.w;
+                my_last_tile = 0;
+                left = row_ok ? p.left[(size_t)head * p.cap_pad + i] : 0;
+
+                // gather this thread's key row into the resident tile (same swizzled layout as a TMA load); every
+                // warp waits and arrives, also one without rows of its own, so that no arrival runs ahead
+                item_ok = mbar_wait(bar.at(kBarAEmpty + ab), ((k_item >> 1) & 1) ^ 1, abort_flag, p.status);
+                if (active && item_ok) {
+                    uint8_t *tile = smem + kOffA + (ab * 2 + m) * kTileBytes;
+                    const uint4 *src = reinterpret_cast<const uint4 *>(
+                        static_cast<const __nv_bfloat16 *>(p.k_cache) + ((size_t)head * p.cap + i) * kHeadDim);
+#pragma unroll
+                    for (int hb = 0; hb < 2; ++hb) {
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) {
+                            const uint4 v = row_ok ? __ldg(src + hb * 8 + c) : make_uint4(0u, 0u, 0u, 0u);
+                            *reinterpret_cast<uint4 *>(tile + hb * kHalfBytes + lrow * 128 + ((c ^ (lrow & 7)) << 4)) = v;
+                        }
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> tensor-core reads
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar.at(kBarAFull + ab));
+            }
+
+            const bool scan = active && (kPass2 || rule_on);
+            // r_j of the first key tile of the scan: loaded now, staged in shared memory when the tile is drained
+            float rj_next = scan ? __ldg(inv_norm + first_tile * kTile + lrow) : 0.f;
+
+            if (!kPass2 && active) {
+                const uint32_t a = cnt & 1;
+                item_ok = mbar_wait(bar.at(kBarAccFull + a * 2 + m), (cnt >> 1) & 1, abort_flag, p.status);
+            }
+            if (!kPass2 && active && item_ok) {
+                // ---- iteration 0, Eq. 2-3: thread = key, all G * alpha logits of that key in its accumulator row,
+                // followed by k_i . s in three parts
+                const uint32_t a = cnt & 1;
+                tc_fence_after();
+                const uint32_t qbase = lane_base + a * 256 + m * 128;
+                float *logits = p.logits + (size_t)head * p.alpha * p.cap_pad;
+                uint32_t sp[8];
+                tmem_ld8(qbase + q_rows_pad, sp);
+                if (p.alpha == 8) {
+                    float best[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) best[j] = -kInf;
+                    for (int g0 = 0; g0 < G; g0 += 2) {
+                        uint32_t t0[8], t1[8];
+                        tmem_ld8(qbase + g0 * 8, t0);
+                        tmem_ld8(qbase + min(g0 + 1, G - 1) * 8, t1);     // an odd G reads its last head twice
+                        tmem_wait8(t0);
+                        tmem_wait8(t1);
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+                            best[j] = fmaxf(best[j], fmaxf(__uint_as_float(t0[j]), __uint_as_float(t1[j])));
+                    }
+                    tmem_wait8(sp);
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar.at(kBarAccEmpty + a * 2 + m));
+                    if (row_ok) {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) logits[(size_t)j * p.cap_pad + i] = best[j] * scale;
+                    }
+                } else {
+                    for (int j = 0; j < p.alpha; ++j) {
+                        float best = -kInf;
+                        for (int g0 = 0; g0 < G; g0 += 4) {
+                            uint32_t t[4];
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) tmem_ld1(qbase + min(g0 + u, G - 1) * p.alpha + j, t[u]);
+                            asm volatile("tcgen05.wait::ld.sync.aligned;"
+                                         : "+r"(t[0]), "+r"(t[1]), "+r"(t[2]), "+r"(t[3]) :: "memory");
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) best = fmaxf(best, __uint_as_float(t[u]));
+                        }
+                        if (row_ok) logits[(size_t)j * p.cap_pad + i] = best * scale;
+                    }
+                    tmem_wait8(sp);
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar.at(kBarAccEmpty + a * 2 + m));
+                }
+                // sum_j S[j][i] before the retention rule: Kbar_i . s - Kbar_i . Kbar_i
+                total = ri * ((__uint_as_float(sp[0]) + __uint_as_float(sp[1])) + __uint_as_float(sp[2])) - self;
+                ++cnt;
+            }
+
+            float removed = 0.f;
+            if (scan) {
+                // ---- key tiles, last to first.  The four warps of a row tile share the tile's r_j through shared
+                // memory; they run this loop in step (two named barriers per tile), so even a warp that has seen a
+                // wait fail keeps going through the loop, without touching TMEM, until the item's last tile.
+                const float thr = (row_ok && ri > 0.f) ? __fdiv_rn(p.sim_threshold, ri) : kInf;   // g r_j vs T / r_i
+                float *rj_s = reinterpret_cast<float *>(smem + kOffRj) + m * kTile;
+                const float4 *rj4 = reinterpret_cast<const float4 *>(rj_s);
+                bool ok = item_ok;
+                for (int jt = first_tile; jt >= my_last_tile; --jt) {
+                    const int jbase = jt * kTile;
+                    asm volatile("bar.sync %0, 128;" ::"r"(1 + m) : "memory");      // the previous tile's r_j are done with
+                    rj_s[lrow] = rj_next;
+                    asm volatile("bar.sync %0, 128;" ::"r"(1 + m) : "memory");
+                    if (jt > my_last_tile) rj_next = __ldg(inv_norm + jbase - kTile + lrow);
+                    const uint32_t a = cnt & 1;
+                    if (ok) ok = mbar_wait(bar.at(kBarAccFull + a * 2 + m), (cnt >> 1) & 1, abort_flag, p.status);
+                    ++cnt;
+                    if (!ok) continue;
+                    tc_fence_after();
+                    const uint32_t base = lane_base + a * 256 + m * 128;
+                    // +inf once the token has its beta partners, and (pass 2) while the scan is still in pass 1's part
+                    float thr_row = (left > 0 && jt < own_tile) ? thr : kInf;
+                    if (__any_sync(0xffffffffu, thr_row < kInf)) {
+                        uint32_t g0[32], g1[32];
+#define RKV_CHUNK(G_, C0_)                                                                                     \
+    {                                                                                                          \
+        float4 R_[8];                                                                                          \
+        _Pragma("unroll") for (int q = 0; q < 8; ++q) R_[q] = rj4[(C0_) / 4 + q];                              \
+        float mx = 0.f;                                                                                        \
+        _Pragma("unroll") for (int q = 0; q < 8; ++q) {                                                        \
+            mx = max3(mx, __uint_as_float(G_[4 * q]) * R_[q].x, __uint_as_float(G_[4 * q + 1]) * R_[q].y);     \
+            mx = max3(mx, __uint_as_float(G_[4 * q + 2]) * R_[q].z, __uint_as_float(G_[4 * q + 3]) * R_[q].w); \
+        }                                                                                                      \
+        if (__any_sync(0xffffffffu, mx > thr_row)) {                                                           \
+            _Pragma("unroll") for (int q = 7; q >= 0; --q) {                                                   \
+                const float rr[4] = {R_[q].x, R_[q].y, R_[q].z, R_[q].w};                                      \
+                _Pragma("unroll") for (int e = 3; e >= 0; --e) {                                               \
+                    const float v = __uint_as_float(G_[4 * q + e]) * rr[e];                                    \
+                    if (v > thr_row && jbase + (C0_) + 4 * q + e != i) {      /* zero diagonal (Eq. 5) */      \
+                        removed += v;                                                                          \
+                        if (--left == 0) thr_row = kInf;                                                       \
+                    }                                                                                          \
+                }                                                                                              \
+            }                                                                                                  \
+        }                                                                                                      \
+    }
+                        tmem_ld32(base + 96, g0);
+                        tmem_wait32(g0);
+                        tmem_ld32(base + 64, g1);
+                        RKV_CHUNK(g0, 96)
+                        tmem_wait32(g1);
+                        tmem_ld32(base + 32, g0);
+                        RKV_CHUNK(g1, 64)
+                        tmem_wait32(g0);
+                        tmem_ld32(base, g1);
+                        RKV_CHUNK(g0, 32)
+                        tmem_wait32(g1);
+                        // the accumulator has been read completely: hand it back before the last chunk's arithmetic
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar.at(kBarAccEmpty + a * 2 + m));
+                        RKV_CHUNK(g1, 0)
+#undef RKV_CHUNK
+                    } else {
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar.at(kBarAccEmpty + a * 2 + m));
+                    }
+                }
+                item_ok = ok;
+            }
+            if (!item_ok) break;
+            if (row_ok) {
+                float *out = p.sbar + (size_t)head * p.cap_pad + i;
+                if (!kPass2) {
+                    *out = total - removed * ri;
+                    p.left[(size_t)head * p.cap_pad + i] = rule_on ? left : 0;
+                } else {
+                    *out -= removed * ri;
+                }
+            }
+            ++k_item;
+        }
+    }
+
+    // ---------------------------------------------------------------------- common exit
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        if (*abort_flag) __nanosleep(200000);      // error path only: let copies and MMAs in flight land
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+        if (lane == 0 && !*abort_flag && tiles_done) atomicAdd(p.counters, tiles_done);
+    }
+}
+
+// ---- between the passes: list, per head, the tokens still short of partners with positions not yet looked at -----
+constexpr int kCompactThreads = 256;
+
+__global__ void __launch_bounds__(kCompactThreads) strag_compact_kernel(Params p)
+{
+    __shared__ int warp_tot[kCompactThreads / 32];
+    __shared__ int running;
+    const int head = blockIdx.x;
+    const int n = candidates_from_meta(p.meta[head / p.hkv], p.budget, p.alpha);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int32_t *left = p.left + (size_t)head * p.cap_pad;
+    int32_t *list = p.strag + (size_t)head * p.cap_pad;
+    if (threadIdx.x == 0) running = 0;
+    __syncthreads();
+    const int low = (n + kTile - 1) / kTile - kPass1Depth;    // pass 1 scanned every token down to this tile at least
+    for (int i0 = 0; i0 < n; i0 += kCompactThreads) {
+        const int i = i0 + threadIdx.x;
+        const bool want = i < n && left[i] > 0 && max(i / kTile, low) >= 1;   // something is left below pass 1's part
+        const unsigned bal = __ballot_sync(0xffffffffu, want);
+        if (lane == 0) warp_tot[warp] = __popc(bal);
+        __syncthreads();
+        int before = running;
+        for (int w = 0; w < warp; ++w) before += warp_tot[w];
+        if (want) list[before + __popc(bal & ((1u << lane) - 1u))] = i;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            int t = 0;
+            for (int w = 0; w < kCompactThreads / 32; ++w) t += warp_tot[w];
+            running += t;
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        const int count = running;
+        p.strag_count[head] = count;
+        const int chunks = (count + kRowsPerItem - 1) / kRowsPerItem;
+        if (chunks > 0) {
+            const unsigned long long at = atomicAdd(&p.counters[2], (unsigned long long)chunks);
+            // longest scans (largest positions) first
+            for (int q = 0; q < chunks; ++q) p.strag_items[at + q] = make_int2(head, chunks - 1 - q);
+        }
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_scores_tri_sm100(const Params &p, cudaStream_t s)
+{
+    const int q_rows = p.group * p.alpha;
+    const int q_rows_pad = (q_rows + 15) / 16 * 16;
+    CUtensorMap map_k, map_q, map_hs;
+    if (!make_map(&map_k, p.k_cache, (uint64_t)p.batch * p.hkv * p.cap, kTile) ||
+        !make_map(&map_q, p.q_window, (uint64_t)p.batch * p.hq * p.alpha, (uint32_t)q_rows_pad) ||
+        !make_map(&map_hs, p.head_sum_bf16, (uint64_t)p.batch * p.hkv * 16, 16u))
+        return cudaErrorInvalidValue;
+    cudaError_t e;
+    if ((e = cudaFuncSetAttribute(scores_tri_sm100_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  kSmemBytes)) != cudaSuccess ||
+        (e = cudaFuncSetAttribute(scores_tri_sm100_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  kSmemBytes)) != cudaSuccess)
+        return e;
+    int dev = 0, sms = 0;
+    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+    if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+    const int heads = p.batch * p.hkv;
+    const int items_per_head = (p.tiles + 1) / 2;
+    const unsigned long long total_items = (unsigned long long)items_per_head * (unsigned long long)heads;
+    const unsigned grid1 = (unsigned)(total_items < (unsigned long long)sms ? total_items : (unsigned long long)sms);
+    scores_tri_sm100_kernel<false><<<grid1, kThreads, kSmemBytes, s>>>(p, map_k, map_q, map_hs, items_per_head,
+                                                                       total_items, q_rows_pad);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    const bool rule_on = p.beta > 0 && p.sim_threshold < 1.0f;
+    if (!rule_on || p.tiles < 2) return cudaSuccess;       // nobody can lack partners / pass 1 has seen everything
+    strag_compact_kernel<<<(unsigned)heads, kCompactThreads, 0, s>>>(p);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    const unsigned long long max_items2 = (unsigned long long)heads * (unsigned long long)(p.cap_pad / kRowsPerItem + 1);
+    const unsigned grid2 = (unsigned)(max_items2 < (unsigned long long)sms ? max_items2 : (unsigned long long)sms);
+    scores_tri_sm100_kernel<true><<<grid2, kThreads, kSmemBytes, s>>>(p, map_k, map_q, map_hs, 0, 0ull, q_rows_pad);
+    return cudaGetLastError();
+}
+
+}  // namespace rkv

@@ -111,7 +111,8 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(Params p)
     const float *sbar = p.sbar + (size_t)head * p.cap_pad;
     float m = -INFINITY;
     for (int i = tid; i < n; i += kSelThreads) {
-        const float v = sbar[i];
+        float v = sbar[i];
+        if (p.tri) v = v / (float)n;        // the triangle kernels leave the column sum minus the removed entries
         row[i] = v;
         m = fmaxf(m, v);
     }

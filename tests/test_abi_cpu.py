@@ -53,7 +53,7 @@ def test_workspace_size_rules(rkv):
     assert rkv.rkv_workspace_bytes(_desc(rkv, head_dim=64), 1024, 128, 8) == 0
     assert rkv.rkv_workspace_bytes(d, 8, 128, 8) == 0                                # budget <= alpha
     assert rkv.rkv_workspace_bytes(d, 8192, 128, 8) == 0                             # cap > RKV_MAX_CAP
-    assert rkv.rkv_workspace_bytes(_desc(rkv, n_q_heads=8 * 17), 1024, 128, 8) == 0  # G * alpha > 128
+    assert rkv.rkv_workspace_bytes(_desc(rkv, n_q_heads=8 * 17), 1024, 128, 8) == 0  # G * alpha = 136 > 112
 
 
 @pytest.mark.parametrize("case,want", [
@@ -110,7 +110,8 @@ def test_rkv_compress_needs_a_current_descriptor(rkv):
     t.join()
     assert out["rc"] == 1
     assert rkv.rkv_status_string(5) == "RKV_ERR_TIMEOUT"
-    assert rkv.rkv_launch_count(_desc(rkv), rkv.RKV_STAGE_ALL) == 4
+    assert rkv.rkv_launch_count(_desc(rkv), rkv.RKV_STAGE_ALL) == 6      # prep, 3 scoring kernels, select, gather
+    assert rkv.rkv_launch_count(_desc(rkv, flags=rkv.RKV_FLAG_SIMT_SCORES), rkv.RKV_STAGE_ALL) == 4
 
 
 def test_product_package_does_not_touch_the_oracle():

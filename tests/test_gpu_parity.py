@@ -74,7 +74,9 @@ def test_tiny_shape_other_seeds_and_margin(rkv, seed):
 
 
 # ----------------------------------------------------------------------------- small shapes, both score kernels
-SCORE_FLAGS = [pytest.param(1, id="simt"), pytest.param(0, id="tcgen05")]
+# the three scoring kernels: fp32 CUDA cores; symmetric tcgen05 (default; beta > 4 falls back to the row-block
+# kernel by itself); row-block tcgen05 forced
+SCORE_FLAGS = [pytest.param(1, id="simt"), pytest.param(0, id="sym"), pytest.param(2, id="rowblock")]
 
 
 @pytest.mark.parametrize("flags", SCORE_FLAGS)
