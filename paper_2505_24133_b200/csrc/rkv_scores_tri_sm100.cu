@@ -504,46 +504,56 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
                     // +inf once the token has its beta partners, and (pass 2) while the scan is still in pass 1's part
                     float thr_row = (left > 0 && jt < own_tile) ? thr : kInf;
                     if (__any_sync(0xffffffffu, thr_row < kInf)) {
-                        uint32_t g0[32], g1[32];
-#define RKV_CHUNK(G_, C0_)                                                                                     \
-    {                                                                                                          \
-        float4 R_[8];                                                                                          \
-        _Pragma("unroll") for (int q = 0; q < 8; ++q) R_[q] = rj4[(C0_) / 4 + q];                              \
-        float mx = 0.f;                                                                                        \
-        _Pragma("unroll") for (int q = 0; q < 8; ++q) {                                                        \
-            mx = max3(mx, __uint_as_float(G_[4 * q]) * R_[q].x, __uint_as_float(G_[4 * q + 1]) * R_[q].y);     \
-            mx = max3(mx, __uint_as_float(G_[4 * q + 2]) * R_[q].z, __uint_as_float(G_[4 * q + 3]) * R_[q].w); \
-        }                                                                                                      \
-        if (__any_sync(0xffffffffu, mx > thr_row)) {                                                           \
-            _Pragma("unroll") for (int q = 7; q >= 0; --q) {                                                   \
-                const float rr[4] = {R_[q].x, R_[q].y, R_[q].z, R_[q].w};                                      \
-                _Pragma("unroll") for (int e = 3; e >= 0; --e) {                                               \
-                    const float v = __uint_as_float(G_[4 * q + e]) * rr[e];                                    \
-                    if (v > thr_row && jbase + (C0_) + 4 * q + e != i) {      /* zero diagonal (Eq. 5) */      \
-                        removed += v;                                                                          \
-                        if (--left == 0) thr_row = kInf;                                                       \
-                    }                                                                                          \
-                }                                                                                              \
-            }                                                                                                  \
-        }                                                                                                      \
-    }
-                        tmem_ld32(base + 96, g0);
-                        tmem_wait32(g0);
-                        tmem_ld32(base + 64, g1);
-                        RKV_CHUNK(g0, 96)
-                        tmem_wait32(g1);
-                        tmem_ld32(base + 32, g0);
-                        RKV_CHUNK(g1, 64)
-                        tmem_wait32(g0);
-                        tmem_ld32(base, g1);
-                        RKV_CHUNK(g0, 32)
-                        tmem_wait32(g1);
-                        // the accumulator has been read completely: hand it back before the last chunk's arithmetic
+                        // 32-column chunks, last first.  The loop is kept rolled on purpose: ten warps in three roles
+                        // share the instruction cache, and one copy of this body is what fits.
+#pragma unroll 1
+                        for (int ch = 3; ch >= 0; --ch) {
+                            uint32_t g[32];
+                            tmem_ld32(base + ch * 32, g);
+                            float4 R[8];
+#pragma unroll
+                            for (int q = 0; q < 8; ++q) R[q] = rj4[ch * 8 + q];
+                            tmem_wait32(g);
+                            float v[32];
+#pragma unroll
+                            for (int q = 0; q < 8; ++q) {
+                                v[4 * q] = __uint_as_float(g[4 * q]) * R[q].x;
+                                v[4 * q + 1] = __uint_as_float(g[4 * q + 1]) * R[q].y;
+                                v[4 * q + 2] = __uint_as_float(g[4 * q + 2]) * R[q].z;
+                                v[4 * q + 3] = __uint_as_float(g[4 * q + 3]) * R[q].w;
+                            }
+                            float m0 = 0.f, m1 = 0.f;
+#pragma unroll
+                            for (int c = 0; c < 32; c += 4) {
+                                m0 = max3(m0, v[c], v[c + 1]);
+                                m1 = max3(m1, v[c + 2], v[c + 3]);
+                            }
+                            if (!__any_sync(0xffffffffu, fmaxf(m0, m1) > thr_row)) continue;
+                            // some token of the warp has partners in this chunk: a bit mask of the entries above the
+                            // threshold (no entry depends on another), cut down to the highest positions if they are
+                            // more than the token still lacks, then their sum
+                            uint32_t hits = 0u;
+#pragma unroll
+                            for (int c = 0; c < 32; ++c) hits |= (v[c] > thr_row) ? (1u << c) : 0u;
+                            const unsigned own = (unsigned)(i - (jbase + ch * 32));           // zero diagonal (Eq. 5)
+                            if (own < 32u) hits &= ~(1u << own);
+                            int taken = __popc(hits);
+                            for (; taken > left; --taken) hits &= hits - 1u;                   // drop the lowest positions
+                            float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+                            for (int c = 0; c < 32; c += 4) {
+                                s0 += (hits >> c & 1u) ? v[c] : 0.f;
+                                s1 += (hits >> (c + 1) & 1u) ? v[c + 1] : 0.f;
+                                s2 += (hits >> (c + 2) & 1u) ? v[c + 2] : 0.f;
+                                s3 += (hits >> (c + 3) & 1u) ? v[c + 3] : 0.f;
+                            }
+                            removed += (s0 + s1) + (s2 + s3);
+                            left -= taken;
+                            if (left == 0) thr_row = kInf;
+                        }
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) mbar_arrive(bar.at(kBarAccEmpty + a * 2 + m));
-                        RKV_CHUNK(g1, 0)
-#undef RKV_CHUNK
                     } else {
                         tc_fence_before();
                         __syncwarp();
