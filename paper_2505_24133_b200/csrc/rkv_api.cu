@@ -20,7 +20,7 @@ int cuda_fail(cudaError_t e, const char *where)
 }
 
 struct Layout {
-    size_t inv_norm, tile_sum, head_sum, logits, sbar, left, strag, strag_count, strag_items, self_dot, head_sum_bf16, meta, counters,
+    size_t inv_norm, tile_sum, head_sum, logits, row_stat, imp, sbar, left, strag, strag_count, strag_items, self_dot, head_sum_bf16, meta, counters,
         tile_done, zero_bytes, total;
     int cap, cap_pad, tiles, tri;
 };
@@ -55,6 +55,8 @@ int check_shapes(const rkv_desc_t *d, int budget, int buffer, int alpha, Layout 
         lay->tile_sum = off;  off = align_up(off + P * lay->tiles * kHeadDim * sizeof(float), 256);
         lay->head_sum = off;  off = align_up(off + P * kHeadDim * sizeof(float), 256);
         lay->logits = off;    off = align_up(off + P * alpha * lay->cap_pad * sizeof(float), 256);
+        lay->row_stat = off;  off = align_up(off + P * alpha * 2 * sizeof(float), 256);
+        lay->imp = off;       off = align_up(off + P * lay->cap_pad * sizeof(float), 256);
         lay->sbar = off;      off = align_up(off + P * lay->cap_pad * sizeof(float), 256);
         lay->tri = use_tri(d);
         const size_t tri = (size_t)lay->tri;
@@ -120,6 +122,8 @@ int run(const rkv_desc_t *d, void *k_cache, void *v_cache, const void *q_window,
     p.tile_sum = reinterpret_cast<float *>(ws + lay.tile_sum);
     p.head_sum = reinterpret_cast<float *>(ws + lay.head_sum);
     p.logits = reinterpret_cast<float *>(ws + lay.logits);
+    p.row_stat = reinterpret_cast<float *>(ws + lay.row_stat);
+    p.imp = reinterpret_cast<float *>(ws + lay.imp);
     p.sbar = reinterpret_cast<float *>(ws + lay.sbar);
     p.left = reinterpret_cast<int32_t *>(ws + lay.left);
     p.strag = reinterpret_cast<int32_t *>(ws + lay.strag);
@@ -299,6 +303,7 @@ int rkv_launch_count(const rkv_desc_t *desc, uint32_t stage_mask)
 {
     int c = 0;
     for (uint32_t bit = 1; bit <= RKV_STAGE_GATHER; bit <<= 1) c += (stage_mask & bit) ? 1 : 0;
+    if (stage_mask & RKV_STAGE_SELECT) c += 2;      // row statistics and importance run ahead of the selection kernel
     // the triangle scoring path is three kernels (pass 1, listing, pass 2) while the retention rule is on
     if (desc && (stage_mask & RKV_STAGE_SCORES) && use_tri(desc) && desc->beta > 0 && desc->sim_threshold < 1.0f) c += 2;
     return c;

@@ -37,6 +37,8 @@ struct Params {
     float *tile_sum;     // [P][tiles][128]      sum over the tile's candidate rows of r_i * k_i
     float *head_sum;     // [P][128]             sum over all candidate rows of r_i * k_i (the tile sums added up)
     float *logits;       // [P][alpha][cap_pad]  Eq. 2-3: group-max of scaled logits
+    float *row_stat;     // [P][alpha][2]        Eq. 3 per row: max logit, 1 / sum of exp(logit - max)
+    float *imp;          // [P][cap_pad]         Eq. 4: importance I
     float *sbar;         // [P][cap_pad]         Eq. 6 column means after the retention rule.  With `tri` set the scoring
                          //                      kernels leave column SUMS minus the removed entries (the select stage
                          //                      divides by n)

@@ -20,7 +20,7 @@ constexpr int kPrepThreads = 256;
 constexpr int kPrepWarps = kPrepThreads / 32;
 
 template <typename T>
-__global__ void __launch_bounds__(kPrepThreads) prep_kernel(Params p)
+__global__ void __launch_bounds__(kPrepThreads, 4) prep_kernel(Params p)
 {
     constexpr int kPerVec = Elem<T>::kPerVec;            // elements per 16-byte vector
     constexpr int kLanesPerRow = kHeadDim / kPerVec;     // 16 (bf16) or 32 (fp32)
@@ -101,9 +101,11 @@ __global__ void __launch_bounds__(kPrepThreads) prep_kernel(Params p)
     // The block that finishes a head's last tile adds the tile sums up, always in tile order, so the result does
     // not depend on which block that is.  (tile_done is zeroed by the memset that precedes this kernel.)
     __shared__ bool last_block;
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) last_block = (atomicAdd(&p.tile_done[head], 1u) == (unsigned)p.tiles - 1u);
+    __syncthreads();                       // the block's tile sums are written ...
+    if (threadIdx.x == 0) {
+        __threadfence();                   // ... and made visible device-wide before the ticket is drawn
+        last_block = (atomicAdd(&p.tile_done[head], 1u) == (unsigned)p.tiles - 1u);
+    }
     __syncthreads();
     if (last_block && threadIdx.x < kHeadDim) {
         __threadfence();

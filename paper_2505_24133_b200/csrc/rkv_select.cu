@@ -1,24 +1,26 @@
-// Stage "select": one thread block per head-problem finishes the scores and picks the kept tokens.
+// Stage "select": three kernels finish the scores and pick the kept tokens.
 //
-//   Eq. 3  softmax over the candidate keys of each of the alpha pooled-logit rows
-//   Eq. 4  sliding max over {i-W .. i+W-1} per row (taken on the logits: exp is monotone, so the
-//          max of the weights is the weight of the max), mean over the alpha rows  -> I
-//   Eq. 6  R = softmax over tokens of the column means left by the scoring stage
-//   Eq. 7  Z = lambda I - (1 - lambda) R
-//   top-k  exact k-th largest Z by a 4 x 8-bit radix select over order-preserving integer keys in shared
-//          memory; among equal scores the later position is kept; the kept candidate positions are written
-//          in ascending order, then the alpha observation positions.
+//   row_stats   one block per (head, query row): the maximum and the sum of exponentials of the row's n pooled
+//               logits, i.e. the softmax of Eq. 3 in two numbers
+//   importance  one block per (head, 1024 tokens): Eq. 4's sliding max over {i-W .. i+W-1} per row (taken on the
+//               logits: exp is monotone, so the max of the weights is the weight of the max), the softmax weight of
+//               that maximum, mean over the alpha rows  -> I
+//   select      one block per head:
+//     Eq. 6  R = softmax over tokens of the column means left by the scoring stage
+//     Eq. 7  Z = lambda I - (1 - lambda) R
+//     top-k  exact k-th largest Z by a 4 x 8-bit radix select over order-preserving integer keys in shared
+//            memory; among equal scores the later position is kept; the kept candidate positions are written
+//            in ascending order, then the alpha observation positions.
 //
-// Latency-bound (about 40 bytes per token, all of it L2-resident scratch).
+// All three read scratch that the scoring stage has just written (L2-resident for small batches).
 #include "rkv_common.cuh"
 
 namespace rkv {
 
 namespace {
 
-constexpr int kSelThreads = 1024;
+constexpr int kSelThreads = 512;
 constexpr int kSelWarps = kSelThreads / 32;
-constexpr int kMaxItems = RKV_MAX_CAP / kSelThreads;   // tokens per thread, upper bound
 
 __device__ __forceinline__ uint32_t order_key(float z)
 {
@@ -34,7 +36,7 @@ __device__ __forceinline__ float block_max(float v, float *scratch)
     __syncthreads();
     if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = v;
     __syncthreads();
-    float r = scratch[threadIdx.x & 31];    // kSelWarps == 32
+    float r = (threadIdx.x & 31) < kSelWarps ? scratch[threadIdx.x & 31] : -INFINITY;
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) r = fmaxf(r, __shfl_xor_sync(0xffffffffu, r, off));
     return r;
@@ -48,13 +50,74 @@ __device__ __forceinline__ float block_sum(float v, float *scratch)
     __syncthreads();
     if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = v;
     __syncthreads();
-    float r = scratch[threadIdx.x & 31];
+    float r = (threadIdx.x & 31) < kSelWarps ? scratch[threadIdx.x & 31] : 0.f;
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) r += __shfl_xor_sync(0xffffffffu, r, off);
     return r;
 }
 
-__global__ void __launch_bounds__(kSelThreads) select_kernel(Params p)
+constexpr int kStatThreads = 256;
+constexpr int kImpThreads = 256;
+constexpr int kImpTokens = 1024;     // tokens per importance block
+
+// Eq. 3 in two numbers per (head, query row): row_stat[..][0] = max_i logit, [1] = 1 / sum_i exp(logit - max).
+__global__ void __launch_bounds__(kStatThreads) row_stats_kernel(Params p)
+{
+    __shared__ float scratch[kStatThreads / 32];
+    const int head = blockIdx.x / p.alpha, j = blockIdx.x % p.alpha;
+    const int n = candidates_from_meta(p.meta[head / p.hkv], p.budget, p.alpha);
+    if (n == 0) return;
+    const float *row = p.logits + ((size_t)head * p.alpha + j) * p.cap_pad;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    float m = -INFINITY;
+    for (int i = tid; i < n; i += kStatThreads) m = fmaxf(m, row[i]);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+    if (lane == 0) scratch[warp] = m;
+    __syncthreads();
+    m = scratch[0];
+#pragma unroll
+    for (int w = 1; w < kStatThreads / 32; ++w) m = fmaxf(m, scratch[w]);
+    __syncthreads();
+    float s = 0.f;
+    for (int i = tid; i < n; i += kStatThreads) s += expf(row[i] - m);      // second read: the row is in L1/L2
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+    if (lane == 0) scratch[warp] = s;
+    __syncthreads();
+    if (tid == 0) {
+        float t = 0.f;
+        for (int w = 0; w < kStatThreads / 32; ++w) t += scratch[w];            // fixed order
+        p.row_stat[((size_t)head * p.alpha + j) * 2] = m;
+        p.row_stat[((size_t)head * p.alpha + j) * 2 + 1] = 1.0f / t;
+    }
+}
+
+// Eq. 4 for kImpTokens tokens of one head.
+__global__ void __launch_bounds__(kImpThreads) importance_kernel(Params p)
+{
+    const int chunks = (p.cap + kImpTokens - 1) / kImpTokens;
+    const int head = blockIdx.x / chunks, i0 = (blockIdx.x % chunks) * kImpTokens;
+    const int n = candidates_from_meta(p.meta[head / p.hkv], p.budget, p.alpha);
+    if (i0 >= n) return;
+    const int W = p.pool_w;
+    const float *logits = p.logits + (size_t)head * p.alpha * p.cap_pad;
+    const float *stat = p.row_stat + (size_t)head * p.alpha * 2;
+    const float inv_alpha = 1.0f / (float)p.alpha;
+    for (int i = i0 + threadIdx.x; i < min(i0 + kImpTokens, n); i += kImpThreads) {
+        const int lo = max(i - W, 0), hi = min(i + W - 1, n - 1);
+        float acc = 0.f;
+        for (int j = 0; j < p.alpha; ++j) {
+            const float *row = logits + (size_t)j * p.cap_pad;
+            float best = row[i];
+            for (int u = lo; u <= hi; ++u) best = fmaxf(best, row[u]);
+            acc += expf(best - stat[2 * j]) * stat[2 * j + 1];
+        }
+        p.imp[(size_t)head * p.cap_pad + i] = acc * inv_alpha;
+    }
+}
+
+__global__ void __launch_bounds__(kSelThreads, 2) select_kernel(Params p)
 {
     extern __shared__ float row[];                 // [cap_pad] one logits row / the Sbar row, then the keys
     __shared__ float scratch[kSelWarps];
@@ -74,37 +137,6 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(Params p)
     }
     const int n = L - p.alpha;
     const int k = p.budget - p.alpha;
-    const int W = p.pool_w;
-
-    // ---- Eq. 3-4: importance
-    float I_acc[kMaxItems];
-#pragma unroll
-    for (int t = 0; t < kMaxItems; ++t) I_acc[t] = 0.f;
-    const float *logits = p.logits + (size_t)head * p.alpha * p.cap_pad;
-    for (int j = 0; j < p.alpha; ++j) {
-        __syncthreads();
-        float m = -INFINITY;
-        for (int i = tid; i < n; i += kSelThreads) {
-            const float l = logits[(size_t)j * p.cap_pad + i];
-            row[i] = l;
-            m = fmaxf(m, l);
-        }
-        m = block_max(m, scratch);
-        float s = 0.f;
-        for (int i = tid; i < n; i += kSelThreads) s += expf(row[i] - m);
-        s = block_sum(s, scratch);
-        const float inv = 1.0f / s;
-#pragma unroll
-        for (int t = 0; t < kMaxItems; ++t) {
-            const int i = tid + t * kSelThreads;
-            if (i < n) {
-                float best = row[i];
-                const int lo = max(i - W, 0), hi = min(i + W - 1, n - 1);
-                for (int u = lo; u <= hi; ++u) best = fmaxf(best, row[u]);
-                I_acc[t] += expf(best - m) * inv;
-            }
-        }
-    }
 
     // ---- Eq. 6: R = softmax(Sbar)
     __syncthreads();
@@ -121,16 +153,14 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(Params p)
     for (int i = tid; i < n; i += kSelThreads) s += expf(row[i] - m);
     s = block_sum(s, scratch);
     const float inv = 1.0f / s;
-    const float inv_alpha = 1.0f / (float)p.alpha;
+    const float *imp = p.imp + (size_t)head * p.cap_pad;
 
     // ---- Eq. 7 and the integer keys (kept in the same shared row, one owner per slot)
     uint32_t *keys = reinterpret_cast<uint32_t *>(row);
     const size_t dbg = (size_t)head * p.cap;
-#pragma unroll
-    for (int t = 0; t < kMaxItems; ++t) {
-        const int i = tid + t * kSelThreads;
-        if (i < n) {
-            const float I = I_acc[t] * inv_alpha;
+    for (int i = tid; i < n; i += kSelThreads) {
+        {
+            const float I = imp[i];
             const float sb = row[i];
             const float R = expf(sb - m) * inv;
             const float Z = p.lambda * I - (1.0f - p.lambda) * R;
@@ -207,7 +237,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(Params p)
     }
     if (lane == 31) warp_tot[warp] = incl;
     __syncthreads();
-    uint32_t wsum = warp_tot[lane], wincl = wsum;
+    uint32_t wsum = lane < kSelWarps ? warp_tot[lane] : 0u, wincl = wsum;
 #pragma unroll
     for (int off = 1; off < 32; off <<= 1) {
         const uint32_t o = __shfl_up_sync(0xffffffffu, wincl, off);
@@ -237,6 +267,12 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(Params p)
 
 cudaError_t launch_select(const Params &p, cudaStream_t s)
 {
+    const unsigned heads = (unsigned)(p.batch * p.hkv);
+    row_stats_kernel<<<heads * (unsigned)p.alpha, kStatThreads, 0, s>>>(p);
+    cudaError_t e0 = cudaGetLastError();
+    if (e0 != cudaSuccess) return e0;
+    importance_kernel<<<heads * (unsigned)((p.cap + kImpTokens - 1) / kImpTokens), kImpThreads, 0, s>>>(p);
+    if ((e0 = cudaGetLastError()) != cudaSuccess) return e0;
     const size_t smem = (size_t)p.cap_pad * sizeof(float);
     cudaError_t e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;

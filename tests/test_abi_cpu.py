@@ -110,8 +110,8 @@ def test_rkv_compress_needs_a_current_descriptor(rkv):
     t.join()
     assert out["rc"] == 1
     assert rkv.rkv_status_string(5) == "RKV_ERR_TIMEOUT"
-    assert rkv.rkv_launch_count(_desc(rkv), rkv.RKV_STAGE_ALL) == 6      # prep, 3 scoring kernels, select, gather
-    assert rkv.rkv_launch_count(_desc(rkv, flags=rkv.RKV_FLAG_SIMT_SCORES), rkv.RKV_STAGE_ALL) == 4
+    assert rkv.rkv_launch_count(_desc(rkv), rkv.RKV_STAGE_ALL) == 8      # prep, 3 scoring kernels, 3 select kernels, gather
+    assert rkv.rkv_launch_count(_desc(rkv, flags=rkv.RKV_FLAG_SIMT_SCORES), rkv.RKV_STAGE_ALL) == 6
 
 
 def test_product_package_does_not_touch_the_oracle():
