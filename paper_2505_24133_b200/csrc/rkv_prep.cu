@@ -8,9 +8,10 @@
 // The last block to finish a head also leaves sum_i r_i * k_i over the whole head (head_sum).
 // Kbar_i . Kbar_i is kept per row as well (self_dot).
 //
-// HBM-bound: K is read once with 16-byte loads, rows coalesced across the lanes of a warp; the row
-// norm is reduced with warp shuffles.  Outputs are 4 bytes per 256-byte row.
-#include "rkv_common.cuh"
+// HBM-bound: each block brings its tile of K into shared memory with one bulk copy (cp.async.bulk, bounded wait
+// on its mbarrier) and reads it from there; the row norm is reduced with warp shuffles.  Outputs are 8 bytes per
+// 256-byte row.
+#include "rkv_sm100.cuh"
 
 namespace rkv {
 
@@ -20,8 +21,12 @@ constexpr int kPrepThreads = 256;
 constexpr int kPrepWarps = kPrepThreads / 32;
 
 template <typename T>
-__global__ void __launch_bounds__(kPrepThreads, 4) prep_kernel(Params p)
+__global__ void __launch_bounds__(kPrepThreads, 6) prep_kernel(Params p)
 {
+    using namespace sm100;
+    extern __shared__ __align__(128) uint8_t prep_smem[];       // the tile's candidate rows, then one mbarrier
+    constexpr int kTileBytesT = kTile * kHeadDim * (int)sizeof(T);
+    __shared__ int abort_flag;
     constexpr int kPerVec = Elem<T>::kPerVec;            // elements per 16-byte vector
     constexpr int kLanesPerRow = kHeadDim / kPerVec;     // 16 (bf16) or 32 (fp32)
     constexpr int kRowsPerPass = 32 / kLanesPerRow;      // rows a warp covers with one load
@@ -46,26 +51,41 @@ __global__ void __launch_bounds__(kPrepThreads, 4) prep_kernel(Params p)
 
     const int sub = lane / kLanesPerRow;                 // which of the rows of this pass
     const int col = (lane % kLanesPerRow) * kPerVec;     // first column this lane holds
-    const int row0 = tile * kTile + warp * kRowsPerWarp;
 
-    // issue every load of this warp's 16 rows first (all independent), then reduce
-    uint4 vec[kPasses];
-#pragma unroll
-    for (int q = 0; q < kPasses; ++q) {
-        const int row = row0 + q * kRowsPerPass + sub;
-        vec[q] = make_uint4(0u, 0u, 0u, 0u);
-        if (row < n) vec[q] = __ldg(reinterpret_cast<const uint4 *>(K + (size_t)row * kHeadDim + col));
+    // One bulk copy brings the tile's candidate rows (contiguous in memory) into shared memory: the bytes in
+    // flight cost no registers, so several blocks per SM keep HBM busy.
+    const int rows_here = min(max(n - tile * kTile, 0), kTile);
+    const uint32_t bar = smem_u32(prep_smem + kTileBytesT);
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        mbar_init(bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        if (rows_here > 0) {
+            const uint32_t bytes = (uint32_t)rows_here * kHeadDim * (uint32_t)sizeof(T);
+            mbar_expect_tx(bar, bytes);
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         ::"r"(smem_u32(prep_smem)), "l"(K + (size_t)tile * kTile * kHeadDim), "r"(bytes), "r"(bar)
+                         : "memory");
+        }
     }
-
+    __syncthreads();
+    if (rows_here > 0 && !mbar_wait(bar, 0, &abort_flag, p.status)) {
+        __nanosleep(200000);        // error path only: let the copy land before the block's memory is reused
+        return;
+    }
+    const uint4 *tile_s = reinterpret_cast<const uint4 *>(prep_smem);
     float acc[kPerVec];
 #pragma unroll
     for (int e = 0; e < kPerVec; ++e) acc[e] = 0.f;
 
-#pragma unroll
+#pragma unroll 2
     for (int q = 0; q < kPasses; ++q) {
-        const int row = row0 + q * kRowsPerPass + sub;
+        const int lr = warp * kRowsPerWarp + q * kRowsPerPass + sub;       // row within the tile
+        const int row = tile * kTile + lr;
+        uint4 vec = make_uint4(0u, 0u, 0u, 0u);
+        if (lr < rows_here) vec = tile_s[lr * kLanesPerRow + (lane % kLanesPerRow)];
         float f[kPerVec];
-        Elem<T>::unpack(vec[q], f);
+        Elem<T>::unpack(vec, f);
         float sq = 0.f;
 #pragma unroll
         for (int e = 0; e < kPerVec; ++e) sq = fmaf(f[e], f[e], sq);
@@ -132,10 +152,19 @@ __global__ void __launch_bounds__(kPrepThreads, 4) prep_kernel(Params p)
 cudaError_t launch_prep(const Params &p, cudaStream_t s)
 {
     const unsigned grid = (unsigned)p.tiles * (unsigned)(p.batch * p.hkv);
-    if (p.dtype == RKV_BF16)
-        prep_kernel<__nv_bfloat16><<<grid, kPrepThreads, 0, s>>>(p);
-    else
-        prep_kernel<float><<<grid, kPrepThreads, 0, s>>>(p);
+    cudaError_t e;
+    if (p.dtype == RKV_BF16) {
+        const int smem = kTile * kHeadDim * 2 + 16;
+        if ((e = cudaFuncSetAttribute(prep_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)) !=
+            cudaSuccess)
+            return e;
+        prep_kernel<__nv_bfloat16><<<grid, kPrepThreads, smem, s>>>(p);
+    } else {
+        const int smem = kTile * kHeadDim * 4 + 16;
+        if ((e = cudaFuncSetAttribute(prep_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)) != cudaSuccess)
+            return e;
+        prep_kernel<float><<<grid, kPrepThreads, smem, s>>>(p);
+    }
     return cudaGetLastError();
 }
 
