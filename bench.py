@@ -28,7 +28,8 @@ import rkv_inputs as ri  # noqa: E402
 
 METRIC = "cached tokens scored/s (KV compressions/s alongside)"
 UNIT = "tokens/s"
-# DRAM traffic of one launch of the dominant kernel from the committed ncu captures (bytes), per workload
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch, from the ncu captures summarised
+# under profiles/: {workload: {kernel: bytes}}
 NCU_TRAFFIC = {}
 
 
@@ -254,46 +255,70 @@ def main():
     value, ms_slowest = rd.whole_job_rate(toks * K, ms_total, dev)
     ms_per_step = ms_slowest / K
 
-    # ---- pass B: the same steps with per-stage events, for the roofline of the dominant kernel
+    # ---- pass B: the same steps with per-kernel events, for the roofline of the dominant kernel
     comp_ev = rkv.Compressor(spec.folded_batch, spec.n_kv_heads, spec.n_q_heads, spec.budget, spec.buffer, spec.alpha,
                              spec.lam, dtype=spec.torch_dtype, device=dev, stage_events=True, **kw)
-    stage_ms = [0.0] * 4
+    names = list(comp_ev.KERNEL_NAMES)
+    kernel_ms = [0.0] * len(names)
     KB = min(K, 20)
+    tiles_executed = moved_rows = 0
     for i in range(KB):
         restore(i % n_rep)
         flush.fill_(i & 255)
         step(i, comp_ev)
         torch.cuda.synchronize()
-        for s_i, t in enumerate(comp_ev.stage_ms()):
-            stage_ms[s_i] += t / KB
-    names = ["prep", "scores_tcgen05", "select", "gather"]
-    dom = max(range(4), key=lambda s_i: stage_ms[s_i])
+        for s_i, t in enumerate(comp_ev.kernel_ms()):
+            kernel_ms[s_i] += t / KB
+        if i == 0:
+            tiles_executed = int(comp_ev.counters[0].item())
+            idx = comp_ev.out_idx
+            moved_rows = int((idx != torch.arange(spec.budget, device=dev, dtype=idx.dtype)).sum().item())
     n = spec.cap - spec.alpha
     esz = wl.k_cache.element_size()
     row = spec.head_dim * esz
-    algo_bytes = {
-        "prep": spec.head_problems * (n * row + spec.cap * 4),
-        "select": spec.head_problems * (n * 4 * (spec.alpha + 1) + spec.budget * 4),
-        "gather": spec.head_problems * 2 * 2 * spec.budget * row,       # K and V, read + write, upper bound
+    P = spec.head_problems
+    T = (n + 127) // 128
+    depth = 2                                          # key tiles every token meets in the first scoring pass
+    q_cols = -(-(spec.n_q_heads // spec.n_kv_heads) * spec.alpha // 16) * 16 + 16
+    tile_flops = 2.0 * 128 ** 3
+    pass1_tiles = P * sum(min(T - I, depth) for I in range(T))
+    pass1_flops = pass1_tiles * tile_flops + P * T * 2.0 * 128 * q_cols * 128
+    pass2_flops = max(tiles_executed - pass1_tiles, 0) * tile_flops
+    # algorithmic work per launch: bytes a kernel has to move / flops it has to execute, nothing it merely could
+    work = {
+        "prep": ("hbm", P * (n * row + spec.cap * 8)),                          # K once; r_i and Kbar_i.Kbar_i out
+        "scores_pass1": ("tensor", pass1_flops),
+        "scores_list": ("hbm", P * n * 8),
+        "scores_pass2": ("tensor", pass2_flops),
+        "row_stats": ("hbm", P * spec.alpha * n * 4),
+        "importance": ("hbm", P * (spec.alpha + 1) * n * 4),
+        "select": ("hbm", P * (2 * n * 4 + spec.budget * 4)),
+        "gather": ("hbm", moved_rows * row * 2 * 2 + P * spec.budget * 4),      # K and V rows that move: read + write
     }
-    stages = {}
-    for s_i, nm in enumerate(names):
-        t = stage_ms[s_i] * 1e-3
-        if nm == "scores_tcgen05":
-            stages[nm] = {"ms": stage_ms[s_i], "tflops": sim_flops_per_step(spec) / t / 1e12 if t > 0 else None}
-        else:
-            stages[nm] = {"ms": stage_ms[s_i], "gbs": algo_bytes[nm] / t / 1e9 if t > 0 else None}
-    if names[dom] == "scores_tcgen05":
-        ach = stages[names[dom]]["tflops"]
-        roofline = {"kernel": "scores_sm100_kernel", "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"],
+    kernels = {}
+    for nm, ms in zip(names, kernel_ms):
+        bound, amount = work[nm]
+        rate = amount / (ms * 1e-3) if ms > 0 else 0.0
+        kernels[nm] = {"ms": ms, ("tflops" if bound == "tensor" else "gbs"): rate / (1e12 if bound == "tensor" else 1e9)}
+    dom = max(range(len(names)), key=lambda s_i: kernel_ms[s_i])
+    dom_name = names[dom]
+    bound, amount = work[dom_name]
+    full_matrix_tflops = sim_flops_per_step(spec) / ((kernel_ms[1] + kernel_ms[2] + kernel_ms[3]) * 1e-3) / 1e12
+    if bound == "tensor":
+        ach = kernels[dom_name]["tflops"]
+        roofline = {"kernel": dom_name, "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"],
                     "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops"],
-                    "peak_source": f"{peaks['source']} burst cuBLAS bf16", "traffic": NCU_TRAFFIC.get(spec.name),
-                    "flops_per_launch": sim_flops_per_step(spec)}
+                    "peak_source": f"{peaks['source']} burst cuBLAS bf16",
+                    "traffic": NCU_TRAFFIC.get(spec.name, {}).get(dom_name),
+                    "flops_per_launch": amount}
     else:
-        ach = stages[names[dom]]["gbs"]
-        roofline = {"kernel": names[dom], "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+        ach = kernels[dom_name]["gbs"]
+        roofline = {"kernel": dom_name, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                     "frac": ach / peaks["hbm_gbs"], "peak_source": f"{peaks['source']} copy",
-                    "traffic": NCU_TRAFFIC.get(spec.name), "bytes_per_launch": algo_bytes[names[dom]]}
+                    "traffic": NCU_TRAFFIC.get(spec.name, {}).get(dom_name), "bytes_per_launch": amount}
+    scoring = {"tiles_executed": tiles_executed, "tiles_full_matrix": P * T * T,
+               "executed_tflops": (pass1_flops + pass2_flops) / ((kernel_ms[1] + kernel_ms[2] + kernel_ms[3]) * 1e-3) / 1e12,
+               "full_matrix_equivalent_tflops": full_matrix_tflops}
 
     # ---- e2e: the host-buffer entry point, copies inside the timed region
     e2e = None
@@ -367,7 +392,8 @@ def main():
             "compressions_per_s": value / toks * spec.folded_batch,
             "head_problems_per_s": value / n,
             "gpu_launches": launches_per_step * K,
-            "stages": stages,
+            "kernels": kernels,
+            "scoring": scoring,
             "roofline": roofline,
             "clocks": clocks,
         }

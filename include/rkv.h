@@ -100,6 +100,13 @@ typedef struct rkv_desc {
     /* optional: 5 cudaEvent_t handles; event s is recorded before stage s (prep, scores, select, gather)
        and event 4 after the last stage, on the call's stream */
     void *const *stage_events;
+    /* optional: 4 more cudaEvent_t handles that split the multi-kernel stages: recorded after the first scoring
+       pass, after the listing kernel between the passes, after the row statistics and after the importance
+       kernel (with a scoring kernel that is a single launch the first two coincide with the stage's start) */
+    void *const *kernel_events;
+    /* optional device uint64[4], written at the end of the scoring stage: [0] = 128 x 128 x 128 tile products the
+       tensor-core kernels executed in this call, [2] = work items of the second scoring pass */
+    unsigned long long *dbg_counters;
 } rkv_desc_t;
 
 /* Fill *desc with the defaults above (pool_w 4, beta 1, T 0.5, eps 1e-8, head_dim 128, bf16), zero elsewhere. */

@@ -37,6 +37,7 @@ class RkvDesc(ctypes.Structure):
         ("flags", ctypes.c_uint32), ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
         ("device_status", ctypes.c_void_p), ("dbg_I", ctypes.c_void_p), ("dbg_Sbar", ctypes.c_void_p),
         ("dbg_R", ctypes.c_void_p), ("dbg_Z", ctypes.c_void_p), ("stage_events", ctypes.c_void_p),
+        ("kernel_events", ctypes.c_void_p), ("dbg_counters", ctypes.c_void_p),
     ]
 
 
@@ -190,13 +191,18 @@ class Compressor:
         if dump_scores:
             self.scores = torch.zeros(4, batch, n_kv_heads, self.cap, dtype=torch.float32, device=self.device)
             d.dbg_I, d.dbg_Sbar, d.dbg_R, d.dbg_Z = (self.scores[i].data_ptr() for i in range(4))
-        self.events = None
+        self.events = self.kevents = self.counters = None
         if stage_events:
             self.events = [torch.cuda.Event(enable_timing=True) for _ in range(5)]
-            for ev in self.events:      # torch creates the handle lazily, on first record
+            self.kevents = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+            for ev in self.events + self.kevents:      # torch creates the handle lazily, on first record
                 ev.record()
             self._event_array = (ctypes.c_void_p * 5)(*[ev.cuda_event for ev in self.events])
+            self._kevent_array = (ctypes.c_void_p * 4)(*[ev.cuda_event for ev in self.kevents])
             d.stage_events = ctypes.cast(self._event_array, ctypes.c_void_p)
+            d.kernel_events = ctypes.cast(self._kevent_array, ctypes.c_void_p)
+            self.counters = torch.zeros(4, dtype=torch.int64, device=self.device)
+            d.dbg_counters = self.counters.data_ptr()
         self.desc = d
         self.out_idx = torch.empty(batch, n_kv_heads, budget, dtype=torch.int32, device=self.device)
 
@@ -217,6 +223,15 @@ class Compressor:
     def stage_ms(self) -> Sequence[float]:
         """Milliseconds of prep, scores, select, gather of the last call (after a synchronise)."""
         return [self.events[i].elapsed_time(self.events[i + 1]) for i in range(4)]
+
+    KERNEL_NAMES = ("prep", "scores_pass1", "scores_list", "scores_pass2", "row_stats", "importance", "select", "gather")
+
+    def kernel_ms(self) -> Sequence[float]:
+        """Milliseconds of the eight kernels of the last call (KERNEL_NAMES), after a synchronise.  With a
+        single-launch scoring kernel its time is under scores_pass2."""
+        s, k = self.events, self.kevents
+        order = [s[0], s[1], k[0], k[1], s[2], k[2], k[3], s[3], s[4]]
+        return [order[i].elapsed_time(order[i + 1]) for i in range(8)]
 
     def check_status(self):
         s = int(self.status.item())

@@ -137,6 +137,8 @@ int run(const rkv_desc_t *d, void *k_cache, void *v_cache, const void *q_window,
     p.zero_bytes = lay.zero_bytes;
     p.tri = lay.tri;
     p.status = d->device_status;
+    p.kernel_events = d->kernel_events;
+    p.dbg_counters = d->dbg_counters;
     p.dbg_I = d->dbg_I;
     p.dbg_Sbar = d->dbg_Sbar;
     p.dbg_R = d->dbg_R;
@@ -158,6 +160,12 @@ int run(const rkv_desc_t *d, void *k_cache, void *v_cache, const void *q_window,
         e = use_simt(d) ? launch_scores_simt(p, s)
                         : (p.tri ? launch_scores_tri_sm100(p, s) : launch_scores_sm100(p, s));
         if (e != cudaSuccess) return cuda_fail(e, "scores launch");
+        if (!p.tri && ((e = mark_kernel(p, 0, s)) != cudaSuccess || (e = mark_kernel(p, 1, s)) != cudaSuccess))
+            return cuda_fail(e, "cudaEventRecord");
+        if (p.dbg_counters &&
+            (e = cudaMemcpyAsync(p.dbg_counters, p.counters, 4 * sizeof(unsigned long long), cudaMemcpyDeviceToDevice, s)) !=
+                cudaSuccess)
+            return cuda_fail(e, "cudaMemcpyAsync");
     }
     if ((e = mark(2)) != cudaSuccess) return cuda_fail(e, "cudaEventRecord");
     if (stages & RKV_STAGE_SELECT)

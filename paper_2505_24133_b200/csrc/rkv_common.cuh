@@ -57,11 +57,20 @@ struct Params {
     size_t zero_bytes;              // bytes from `counters` to the end of `tile_done`
     int tri;                        // 1: the triangle kernels score (bf16 default); 0: another kernel does
     // optional outputs
+    void *const *kernel_events;     // see rkv_desc_t
+    unsigned long long *dbg_counters;
     int32_t *status;
     float *dbg_I, *dbg_Sbar, *dbg_R, *dbg_Z;
 };
 
 __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Record optional event i of p.kernel_events on the stream.
+inline cudaError_t mark_kernel(const Params &p, int i, cudaStream_t s)
+{
+    return (p.kernel_events && p.kernel_events[i]) ? cudaEventRecord(static_cast<cudaEvent_t>(p.kernel_events[i]), s)
+                                                   : cudaSuccess;
+}
 
 __device__ __forceinline__ void report(int32_t *status, int code)
 {

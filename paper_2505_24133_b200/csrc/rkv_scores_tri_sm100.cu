@@ -317,13 +317,7 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
                         tc_fence_after();
                         const uint32_t resident = sbase + kOffA + (ab * 2 + m) * kTileBytes;
                         const uint32_t d_tmem = tmem_base + a * 256 + m * 128;
-#pragma unroll
-                        for (int k = 0; k < 8; ++k) {
-                            // K = 16 per instruction: 32 bytes along the swizzled row; k >= 4 is the second box
-                            const uint32_t koff = (k >> 2) * kHalfBytes + (k & 3) * 32;
-                            umma(d_tmem, smem_desc(resident + koff), smem_desc(stage + koff), is_q ? idesc_q : idesc_k,
-                                 k > 0);
-                        }
+                        umma_tile_k128(d_tmem, resident, stage, is_q ? idesc_q : idesc_k);
                         umma_commit(bar.at(kBarAccFull + a * 2 + m));
                         ++cnt[m];
                         if (!is_q) ++tiles_done;
@@ -658,10 +652,12 @@ cudaError_t launch_scores_tri_sm100(const Params &p, cudaStream_t s)
     scores_tri_sm100_kernel<false><<<grid1, kThreads, kSmemBytes, s>>>(p, map_k, map_q, map_hs, items_per_head,
                                                                        total_items, q_rows_pad);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    if ((e = mark_kernel(p, 0, s)) != cudaSuccess) return e;
     const bool rule_on = p.beta > 0 && p.sim_threshold < 1.0f;
-    if (!rule_on || p.tiles < 2) return cudaSuccess;       // nobody can lack partners / pass 1 has seen everything
+    if (!rule_on || p.tiles < 2) return mark_kernel(p, 1, s);       // nobody can lack partners / pass 1 has seen everything
     strag_compact_kernel<<<(unsigned)heads, kCompactThreads, 0, s>>>(p);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    if ((e = mark_kernel(p, 1, s)) != cudaSuccess) return e;
     const unsigned long long max_items2 = (unsigned long long)heads * (unsigned long long)(p.cap_pad / kRowsPerItem + 1);
     const unsigned grid2 = (unsigned)(max_items2 < (unsigned long long)sms ? max_items2 : (unsigned long long)sms);
     scores_tri_sm100_kernel<true><<<grid2, kThreads, kSmemBytes, s>>>(p, map_k, map_q, map_hs, 0, 0ull, q_rows_pad);

@@ -271,8 +271,10 @@ cudaError_t launch_select(const Params &p, cudaStream_t s)
     row_stats_kernel<<<heads * (unsigned)p.alpha, kStatThreads, 0, s>>>(p);
     cudaError_t e0 = cudaGetLastError();
     if (e0 != cudaSuccess) return e0;
+    if ((e0 = mark_kernel(p, 2, s)) != cudaSuccess) return e0;
     importance_kernel<<<heads * (unsigned)((p.cap + kImpTokens - 1) / kImpTokens), kImpThreads, 0, s>>>(p);
     if ((e0 = cudaGetLastError()) != cudaSuccess) return e0;
+    if ((e0 = mark_kernel(p, 3, s)) != cudaSuccess) return e0;
     const size_t smem = (size_t)p.cap_pad * sizeof(float);
     cudaError_t e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;

@@ -91,6 +91,38 @@ __device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t a_desc, uint64_t 
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accum)
         : "memory");
 }
+// One 128 x N x 128 product: the eight K = 16 steps of two K-major, 128-byte swizzled bf16 operand tiles (each two
+// 16 KB boxes of 64 columns, 1024-byte aligned) into the accumulator at d_tmem, overwriting it.  Everything is in
+// one statement so that the issuing thread spends a handful of instructions per step: the descriptors differ
+// only in their start-address field (16-byte units; +2 per step, +1024 for the second box).
+__device__ __forceinline__ void umma_tile_k128(uint32_t d_tmem, uint32_t a_addr, uint32_t b_addr, uint32_t idesc)
+{
+    const uint32_t a_lo = ((a_addr & 0x3FFFFu) >> 4) | (1u << 16);
+    const uint32_t b_lo = ((b_addr & 0x3FFFFu) >> 4) | (1u << 16);
+    const uint32_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);      // stride 1024 B, descriptor version, 128-byte swizzle
+    asm volatile(
+        "{\n\t.reg .pred p0, p1;\n\t.reg .b64 da, db;\n\t.reg .b32 ta, tb;\n\t"
+        "setp.ne.u32 p0, %3, %3;\n\tsetp.eq.u32 p1, %3, %3;\n\t"
+        "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p0;\n\t"
+        "add.u32 ta, %1, 2;\n\tadd.u32 tb, %2, 2;\n\tmov.b64 da, {ta, %3};\n\tmov.b64 db, {tb, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p1;\n\t"
+        "add.u32 ta, %1, 4;\n\tadd.u32 tb, %2, 4;\n\tmov.b64 da, {ta, %3};\n\tmov.b64 db, {tb, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p1;\n\t"
+        "add.u32 ta, %1, 6;\n\tadd.u32 tb, %2, 6;\n\tmov.b64 da, {ta, %3};\n\tmov.b64 db, {tb, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p1;\n\t"
+        "add.u32 ta, %1, 1024;\n\tadd.u32 tb, %2, 1024;\n\tmov.b64 da, {ta, %3};\n\tmov.b64 db, {tb, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p1;\n\t"
+        "add.u32 ta, %1, 1026;\n\tadd.u32 tb, %2, 1026;\n\tmov.b64 da, {ta, %3};\n\tmov.b64 db, {tb, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p1;\n\t"
+        "add.u32 ta, %1, 1028;\n\tadd.u32 tb, %2, 1028;\n\tmov.b64 da, {ta, %3};\n\tmov.b64 db, {tb, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p1;\n\t"
+        "add.u32 ta, %1, 1030;\n\tadd.u32 tb, %2, 1030;\n\tmov.b64 da, {ta, %3};\n\tmov.b64 db, {tb, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p1;\n\t"
+        "}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc)
+        : "memory");
+}
 __device__ __forceinline__ void umma_commit(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
