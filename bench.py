@@ -30,7 +30,11 @@ METRIC = "cached tokens scored/s (KV compressions/s alongside)"
 UNIT = "tokens/s"
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch, from the ncu captures summarised
 # under profiles/: {workload: {kernel: bytes}}
-NCU_TRAFFIC = {}
+NCU_TRAFFIC = {
+    # profiles/all_kernels_llama8b_b1.md (cold caches: the scoring passes read K from DRAM there)
+    "llama8b_b1": {"prep": 76.97e6, "scores_pass1": 85.33e6, "scores_list": 1.19e6, "scores_pass2": 72.29e6,
+                   "row_stats": 9.45e6, "importance": 9.46e6, "select": 2.39e6, "gather": 209.74e6},
+}
 
 
 def parse_args():
