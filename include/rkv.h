@@ -173,24 +173,26 @@ RKV_API int rkv_compress_host(const rkv_desc_t *desc, void *host_k_cache, void *
  * buffer fills -- an inference server whose memory pool already owns all of the GPU's memory and hands out
  * nothing beyond KV blocks, a plug-in running inside another framework's callback where allocation is
  * forbidden, a real-time loop that must not take the driver's allocation lock.  For them the scratch lives in
- * a fixed array inside the library's device image, RKV_STATIC_SCRATCH_BYTES (16 MiB) large.  Every GPU that
+ * a fixed array inside the library's device image, RKV_STATIC_SCRATCH_BYTES (24 MiB) large.  Every GPU that
  * loads the library carries that array until the process ends, used or not.
  *
  * Arguments, layouts, results and error codes are those of rkv_compress_ex; desc->workspace and
  * desc->workspace_bytes are ignored.  In addition:
  *   - a shape whose rkv_workspace_bytes() exceeds RKV_STATIC_SCRATCH_BYTES is refused with RKV_ERR_WORKSPACE
- *     before anything is launched (rkv_workspace_bytes() tells what a shape needs).  16 MiB covers, for example, 256 head-problems at budget 1024 + buffer 128 (all 32 layers of an 8-KV-head model, batch 1);
+ *     before anything is launched (rkv_workspace_bytes() tells what a shape needs).  24 MiB covers, for example,
+ *     256 head-problems at budget 1024 + buffer 128 (all 32 layers of an 8-KV-head model, batch 1);
  *     larger batches are split into several calls over sub-ranges of the batch dimension, one after the other.
  *   - the call makes no cudaMalloc / cudaFree and calls no allocating library routine.
  *   - the FIRST call on each device looks up the array's device address (with that device current) and caches
  *     it; make that first call outside any stream capture.
- *   - all calls on a device share the one array, which still holds the previous call's contents.  Nothing in
- *     it has to start at zero -- every stage writes what the next one reads, and the prep stage clears the
- *     counters -- but two calls that overlap on the GPU (different streams, no dependency between them) race on
+ *   - all calls on a device share the one array, which still holds the previous call's contents.  The few
+ *     words that have to start at zero (work counters, per-head tickets) are cleared by the call itself, on the
+ *     stream, before its first kernel; everything else is written by one stage before the next reads it.  But
+ *     two calls that overlap on the GPU (different streams, no dependency between them) race on
  *     it and corrupt each other's scores.  Serialise them, or give one of them a workspace of its own through
  *     rkv_compress_ex.
  */
-#define RKV_STATIC_SCRATCH_BYTES (16u << 20)
+#define RKV_STATIC_SCRATCH_BYTES (24u << 20)
 RKV_API int rkv_compress_static(const rkv_desc_t *desc, void *k_cache, void *v_cache, const void *q_window,
                         int32_t *seq_lens, int32_t budget, int32_t buffer, int32_t alpha, float lambda,
                         int32_t *out_idx, void *stream);
