@@ -372,13 +372,15 @@ def main():
         Kh = wl.k_cache[:seqs].float().cpu().numpy()
         Qh = wl.q_window[:seqs].float().cpu().numpy()
         oracle.build()
-        t0 = time.perf_counter()
-        res = oracle.oracle_batch(Kh, Qh, wl.seq_lens[:seqs].cpu().numpy(), budget=spec.budget, alpha=spec.alpha,
-                                  lam=spec.lam, W=d.pool_w, beta=d.beta, T=d.sim_threshold, eps=d.eps,
-                                  want_scores=False)
+        seq_h = wl.seq_lens[:seqs].cpu().numpy()
+        passes, t0 = 0, time.perf_counter()
+        while passes < 1 or (time.perf_counter() - t0 < 12.0 and passes < 200):      # about 12 s of CPU work
+            res = oracle.oracle_batch(Kh, Qh, seq_h, budget=spec.budget, alpha=spec.alpha, lam=spec.lam, W=d.pool_w,
+                                      beta=d.beta, T=d.sim_threshold, eps=d.eps, want_scores=False)
+            passes += 1
         dt = time.perf_counter() - t0
-        cpu = {"value": seqs * spec.n_kv_heads * n / dt, "unit": UNIT, "cores": res.threads, "kind": "oracle",
-               "sample": f"first {seqs * spec.n_kv_heads} of {spec.head_problems} head-problems, one pass, {dt:.1f} s"}
+        cpu = {"value": passes * seqs * spec.n_kv_heads * n / dt, "unit": UNIT, "cores": res.threads, "kind": "oracle",
+               "sample": f"first {seqs * spec.n_kv_heads} of {spec.head_problems} head-problems, {passes} passes, {dt:.1f} s"}
 
     if rank == 0:
         line = {
