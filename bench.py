@@ -340,7 +340,7 @@ def main():
     row = spec.head_dim * esz
     P = spec.head_problems
     T = (n + 127) // 128
-    depth = 2                                          # key tiles every token meets in the first scoring pass
+    depth = 1                                          # key tiles every token meets in the first scoring pass
     q_cols = -(-(spec.n_q_heads // spec.n_kv_heads) * spec.alpha // 16) * 16 + 16
     tile_flops = 2.0 * 128 ** 3
     pass1_tiles = P * sum(min(T - I, depth) for I in range(T))
