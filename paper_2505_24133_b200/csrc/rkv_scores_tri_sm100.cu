@@ -516,13 +516,16 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
                                 v[4 * q + 2] = __uint_as_float(g[4 * q + 2]) * R[q].z;
                                 v[4 * q + 3] = __uint_as_float(g[4 * q + 3]) * R[q].w;
                             }
-                            float m0 = 0.f, m1 = 0.f;
+                            if (kPass2) {
+                                // screening: the listed tokens rarely have a partner in a given chunk
+                                float m0 = 0.f, m1 = 0.f;
 #pragma unroll
-                            for (int c = 0; c < 32; c += 4) {
-                                m0 = max3(m0, v[c], v[c + 1]);
-                                m1 = max3(m1, v[c + 2], v[c + 3]);
-                            }
-                            if (!__any_sync(0xffffffffu, fmaxf(m0, m1) > thr_row)) continue;
+                                for (int c = 0; c < 32; c += 4) {
+                                    m0 = max3(m0, v[c], v[c + 1]);
+                                    m1 = max3(m1, v[c + 2], v[c + 3]);
+                                }
+                                if (!__any_sync(0xffffffffu, fmaxf(m0, m1) > thr_row)) continue;
+                            }   // (pass 1 meets every token's first partners here: it goes straight to the mask)
                             // some token of the warp has partners in this chunk: a bit mask of the entries above the
                             // threshold (no entry depends on another), cut down to the highest positions if they are
                             // more than the token still lacks, then their sum
