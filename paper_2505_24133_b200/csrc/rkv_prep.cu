@@ -21,14 +21,16 @@ constexpr int kPrepThreads = 256;
 constexpr int kPrepWarps = kPrepThreads / 32;
 
 template <typename T>
-__global__ void __launch_bounds__(kPrepThreads, 6) prep_kernel(Params p)
+__global__ void __launch_bounds__(kPrepThreads, 5) prep_kernel(Params p)
 {
     using namespace sm100;
     extern __shared__ __align__(128) uint8_t prep_smem[];       // the tile's candidate rows, then one mbarrier
     constexpr int kTileBytesT = kTile * kHeadDim * (int)sizeof(T);
     __shared__ int abort_flag;
     constexpr int kPerVec = Elem<T>::kPerVec;            // elements per 16-byte vector
-    constexpr int kLanesPerRow = kHeadDim / kPerVec;     // 16 (bf16) or 32 (fp32)
+    constexpr int kVecPerLane = 2;                       // 16-byte vectors of a row held by one lane
+    constexpr int kLanesPerRow = kHeadDim / (kPerVec * kVecPerLane);     // 8 (bf16) or 16 (fp32)
+    constexpr int kVecPerRow = kHeadDim / kPerVec;
     constexpr int kRowsPerPass = 32 / kLanesPerRow;      // rows a warp covers with one load
     constexpr int kRowsPerWarp = kTile / kPrepWarps;     // 16
     constexpr int kPasses = kRowsPerWarp / kRowsPerPass;
@@ -50,7 +52,8 @@ __global__ void __launch_bounds__(kPrepThreads, 6) prep_kernel(Params p)
     float *inv_norm = p.inv_norm + (size_t)head * p.cap_pad;
 
     const int sub = lane / kLanesPerRow;                 // which of the rows of this pass
-    const int col = (lane % kLanesPerRow) * kPerVec;     // first column this lane holds
+    const int lane_in_row = lane % kLanesPerRow;         // vector u of the lane = vector lane_in_row + u * kLanesPerRow
+                                                         // of the row: a warp's load covers whole 128-byte lines
 
     // One bulk copy brings the tile's candidate rows (contiguous in memory) into shared memory: the bytes in
     // flight cost no registers, so several blocks per SM keep HBM busy.
@@ -74,41 +77,66 @@ __global__ void __launch_bounds__(kPrepThreads, 6) prep_kernel(Params p)
         return;
     }
     const uint4 *tile_s = reinterpret_cast<const uint4 *>(prep_smem);
-    float acc[kPerVec];
+    // packed fp32 arithmetic (two values per instruction), few lanes per row (short shuffle trees): this kernel is
+    // bound by its instruction count
+    constexpr int kHeld = kPerVec * kVecPerLane;         // elements of a row per lane
+    float2 acc2[kHeld / 2];
 #pragma unroll
-    for (int e = 0; e < kPerVec; ++e) acc[e] = 0.f;
+    for (int e = 0; e < kHeld / 2; ++e) acc2[e] = make_float2(0.f, 0.f);
 
 #pragma unroll 2
     for (int q = 0; q < kPasses; ++q) {
         const int lr = warp * kRowsPerWarp + q * kRowsPerPass + sub;       // row within the tile
         const int row = tile * kTile + lr;
-        uint4 vec = make_uint4(0u, 0u, 0u, 0u);
-        if (lr < rows_here) vec = tile_s[lr * kLanesPerRow + (lane % kLanesPerRow)];
-        float f[kPerVec];
-        Elem<T>::unpack(vec, f);
-        float sq = 0.f;
+        float f[kHeld];
 #pragma unroll
-        for (int e = 0; e < kPerVec; ++e) sq = fmaf(f[e], f[e], sq);
+        for (int u = 0; u < kVecPerLane; ++u) {
+            uint4 vec = make_uint4(0u, 0u, 0u, 0u);
+            if (lr < rows_here) vec = tile_s[lr * kVecPerRow + lane_in_row + u * kLanesPerRow];
+            Elem<T>::unpack(vec, f + u * kPerVec);
+        }
+        float2 sq2 = make_float2(0.f, 0.f);
+#pragma unroll
+        for (int e = 0; e < kHeld / 2; ++e) {
+            const float2 f2 = make_float2(f[2 * e], f[2 * e + 1]);
+            sq2 = __ffma2_rn(f2, f2, sq2);
+        }
+        float sq = sq2.x + sq2.y;
 #pragma unroll
         for (int off = kLanesPerRow / 2; off > 0; off >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, off);
-        const float r = (row < n) ? __fdiv_rn(1.0f, __fsqrt_rn(sq) + p.eps) : 0.f;
-        if (lane % kLanesPerRow == 0) {
+        // 1 / (sqrt(sq) + eps) from the hardware's approximate rsqrt and divide (a few ulp: far inside the score
+        // tolerances, and every scoring kernel uses these same r); sq = 0 (an all-zero key) gives 1 / eps
+        const float nrm = sq > 0.f ? sq * rsqrtf(sq) : 0.f;
+        const float r = (row < n) ? __fdividef(1.0f, nrm + p.eps) : 0.f;
+        if (lane_in_row == 0) {
             inv_norm[row] = r;                       // row < cap_pad: the grid covers exactly cap_pad rows per head
             p.self_dot[(size_t)head * p.cap_pad + row] = (r * r) * sq;     // Kbar_i . Kbar_i
         }
+        const float2 r2 = make_float2(r, r);
 #pragma unroll
-        for (int e = 0; e < kPerVec; ++e) acc[e] = fmaf(r, f[e], acc[e]);
+        for (int e = 0; e < kHeld / 2; ++e) acc2[e] = __ffma2_rn(r2, make_float2(f[2 * e], f[2 * e + 1]), acc2[e]);
     }
 
     // fold the row groups of a warp, then the warps, in a fixed order (deterministic sums)
-    if (kRowsPerPass == 2) {
 #pragma unroll
-        for (int e = 0; e < kPerVec; ++e) acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], 16);
+    for (int off = kLanesPerRow; off < 32; off <<= 1) {
+#pragma unroll
+        for (int e = 0; e < kHeld / 2; ++e) {
+            acc2[e].x += __shfl_xor_sync(0xffffffffu, acc2[e].x, off);
+            acc2[e].y += __shfl_xor_sync(0xffffffffu, acc2[e].y, off);
+        }
     }
     __shared__ float part[kPrepWarps][kHeadDim];
     if (sub == 0) {
 #pragma unroll
-        for (int e = 0; e < kPerVec; ++e) part[warp][col + e] = acc[e];
+        for (int u = 0; u < kVecPerLane; ++u) {
+            const int col = (lane_in_row + u * kLanesPerRow) * kPerVec;
+#pragma unroll
+            for (int e = 0; e < kPerVec / 2; ++e) {
+                part[warp][col + 2 * e] = acc2[u * kPerVec / 2 + e].x;
+                part[warp][col + 2 * e + 1] = acc2[u * kPerVec / 2 + e].y;
+            }
+        }
     }
     __syncthreads();
     if (threadIdx.x < kHeadDim) {
