@@ -343,10 +343,24 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
         const float scale = 0.08838834764831845f;             // 1 / sqrt(128)
         const int G = p.group;
         uint32_t k_item = 0, cnt = 0;
+        bool dead = false;                    // a wait of this warp has failed: it takes part in no further item
 
         while (true) {
             const uint32_t qs = k_item % kItemSlots;
-            if (!mbar_wait(bar.at(kBarQFull + qs), (k_item / kItemSlots) & 1, abort_flag, p.status)) break;
+            // The four warps of a row tile meet at named barriers inside an item, so they must leave the item loop
+            // together: each brings the outcome of its waits (the last item's and this item's first) to a vote,
+            // and a warp leaves only here, with its three mates, or at the terminator, which all of them see.
+            const bool have = !dead && mbar_wait(bar.at(kBarQFull + qs), (k_item / kItemSlots) & 1, abort_flag, p.status);
+            int all_have;
+            asm volatile(
+                "{\n\t.reg .pred p, q;\n\t"
+                "setp.ne.u32 p, %1, 0;\n\t"
+                "bar.red.and.pred q, %2, 128, p;\n\t"
+                "selp.u32 %0, 1, 0, q;\n\t}"
+                : "=r"(all_have)
+                : "r"((uint32_t)have), "r"(1 + m)
+                : "memory");
+            if (!all_have) break;
             const int4 d = items[qs];
             __syncwarp();
             if (lane == 0) mbar_arrive(bar.at(kBarQEmpty + qs));
@@ -559,7 +573,7 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
                 }
                 item_ok = ok;
             }
-            if (!item_ok) break;
+            if (!item_ok) dead = true;        // leaves at the next vote, together with the other warps of its row tile
             if (row_ok) {
                 float *out = p.sbar + (size_t)head * p.cap_pad + i;
                 if (!kPass2) {
