@@ -72,8 +72,9 @@ __global__ void __launch_bounds__(kPrepThreads, 5) prep_kernel(Params p)
         }
     }
     __syncthreads();
-    if (rows_here > 0 && !mbar_wait(bar, 0, &abort_flag, p.status)) {
-        __nanosleep(200000);        // error path only: let the copy land before the block's memory is reused
+    const bool landed = rows_here == 0 || mbar_wait(bar, 0, &abort_flag, p.status);
+    if (!__syncthreads_and(landed)) {      // the block leaves as a whole, or not at all
+        __nanosleep(200000);               // error path only: let the copy land before the block's memory is reused
         return;
     }
     const uint4 *tile_s = reinterpret_cast<const uint4 *>(prep_smem);
