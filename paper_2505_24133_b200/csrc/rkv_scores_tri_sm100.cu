@@ -552,6 +552,24 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
                             for (int c = 0; c < 32; ++c) hits |= (v[c] > thr_row) ? (1u << c) : 0u;
                             const unsigned own = (unsigned)(i - (jbase + ch * 32));           // zero diagonal (Eq. 5)
                             if (own < 32u) hits &= ~(1u << own);
+                            if (p.beta == 1) {
+                                // one partner at most: the entry at the highest set bit, picked by a select tree
+                                if (left > 0 && hits != 0u) {
+                                    const int top = 31 - __clz(hits);
+                                    float t16[16], t8[8], t4[4];
+#pragma unroll
+                                    for (int c = 0; c < 16; ++c) t16[c] = (top & 16) ? v[16 + c] : v[c];
+#pragma unroll
+                                    for (int c = 0; c < 8; ++c) t8[c] = (top & 8) ? t16[8 + c] : t16[c];
+#pragma unroll
+                                    for (int c = 0; c < 4; ++c) t4[c] = (top & 4) ? t8[4 + c] : t8[c];
+                                    const float u0 = (top & 2) ? t4[2] : t4[0], u1 = (top & 2) ? t4[3] : t4[1];
+                                    removed += (top & 1) ? u1 : u0;
+                                    left = 0;
+                                    thr_row = kInf;
+                                }
+                                continue;
+                            }
                             int taken = __popc(hits);
                             for (; taken > left; --taken) hits &= hits - 1u;                   // drop the lowest positions
                             float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
