@@ -2,7 +2,7 @@
 //
 // For every head, row j of K and of V becomes row idx[j] (j < budget).  idx is strictly ascending, so
 // idx[j] >= j: rows only move towards lower positions and the untouched prefix (idx[j] == j) is free.
-// One thread block owns one (head, K|V) stream and walks it in chunks of 64 rows: load the chunk's source
+// One thread block owns one (head, K|V) stream (or a column slice of it) and walks it in chunks of 64 rows or more: load the chunk's source
 // rows into registers, barrier, store.  A later chunk reads only rows at or beyond its own first row, which
 // no earlier chunk writes, so one barrier per chunk is all the ordering in-place compaction needs.
 // No scratch copy, no reallocation.  HBM-bound: 16-byte loads and stores, a row is 16 (bf16) or 32 (fp32) lanes wide.
@@ -16,25 +16,33 @@ namespace {
 constexpr int kGatherThreads = 256;
 constexpr int kChunkRows = 64;
 
-template <int kVecPerRow>   // 16-byte vectors per row
+// kVecPerRow: 16-byte vectors per row; kSplit: column slices a row is cut into, each moved by a block of its own
+// (slices are disjoint bytes, so they need no ordering among themselves; small batches need the extra blocks to
+// keep enough bytes in flight).
+template <int kVecPerRow, int kSplit>
 __global__ void __launch_bounds__(kGatherThreads) gather_kernel(Params p)
 {
-    constexpr int kVecPerThread = kChunkRows * kVecPerRow / kGatherThreads;   // 4 or 8
-    constexpr int kRowsPerStep = kGatherThreads / kVecPerRow;                  // 16 or 8
-    const int head = blockIdx.x >> 1;
-    const int which = blockIdx.x & 1;
+    constexpr int kVecPerSlice = kVecPerRow / kSplit;                           // vectors of a row this block moves
+    constexpr int kRows = kChunkRows * kSplit;                                  // rows per chunk: 16 KB in flight per block
+    constexpr int kVecPerThread = kRows * kVecPerSlice / kGatherThreads;       // 4 or 8
+    constexpr int kRowsPerStep = kGatherThreads / kVecPerSlice;
+    const int slice = blockIdx.x % kSplit;
+    const int stream = blockIdx.x / kSplit;
+    const int head = stream >> 1;
+    const int which = stream & 1;
     const int b = head / p.hkv;
     const int L = p.meta[b];
     if (L <= p.budget) return;                      // nothing was selected for this sequence
-    if (which == 0 && head % p.hkv == 0 && threadIdx.x == 0) p.seq_lens[b] = p.budget;
+    if (which == 0 && slice == 0 && head % p.hkv == 0 && threadIdx.x == 0) p.seq_lens[b] = p.budget;
 
-    uint4 *base = reinterpret_cast<uint4 *>(which ? p.v_cache : p.k_cache) + (size_t)head * p.cap * kVecPerRow;
+    uint4 *base = reinterpret_cast<uint4 *>(which ? p.v_cache : p.k_cache) + (size_t)head * p.cap * kVecPerRow +
+                  slice * kVecPerSlice;
     const int32_t *idx = p.out_idx + (size_t)head * p.budget;
-    const int lane_vec = threadIdx.x % kVecPerRow;
-    const int lane_row = threadIdx.x / kVecPerRow;
+    const int lane_vec = threadIdx.x % kVecPerSlice;
+    const int lane_row = threadIdx.x / kVecPerSlice;
 
-    for (int j0 = 0; j0 < p.budget; j0 += kChunkRows) {
-        const int j_end = min(j0 + kChunkRows, p.budget);
+    for (int j0 = 0; j0 < p.budget; j0 += kRows) {
+        const int j_end = min(j0 + kRows, p.budget);
         if (idx[j_end - 1] == j_end - 1) continue;   // ascending and idx[j] >= j: the whole chunk is in place
         uint4 held[kVecPerThread];
         int src[kVecPerThread];
@@ -57,11 +65,19 @@ __global__ void __launch_bounds__(kGatherThreads) gather_kernel(Params p)
 
 cudaError_t launch_gather(const Params &p, cudaStream_t s)
 {
-    const unsigned grid = 2u * (unsigned)(p.batch * p.hkv);
-    if (p.dtype == RKV_BF16)
-        gather_kernel<16><<<grid, kGatherThreads, 0, s>>>(p);
-    else
-        gather_kernel<32><<<grid, kGatherThreads, 0, s>>>(p);
+    const unsigned streams = 2u * (unsigned)(p.batch * p.hkv);
+    int dev = 0, sms = 0;
+    cudaError_t e;
+    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+    if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+    const bool small = streams < 8u * (unsigned)sms;        // fewer than 8 streams per SM: cut the rows in 4 slices
+    if (p.dtype == RKV_BF16) {
+        if (small) gather_kernel<16, 4><<<streams * 4u, kGatherThreads, 0, s>>>(p);
+        else gather_kernel<16, 1><<<streams, kGatherThreads, 0, s>>>(p);
+    } else {
+        if (small) gather_kernel<32, 4><<<streams * 4u, kGatherThreads, 0, s>>>(p);
+        else gather_kernel<32, 1><<<streams, kGatherThreads, 0, s>>>(p);
+    }
     return cudaGetLastError();
 }
 
