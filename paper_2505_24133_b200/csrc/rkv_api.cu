@@ -63,7 +63,7 @@ int check_shapes(const rkv_desc_t *d, int budget, int buffer, int alpha, Layout 
         lay->left = off;        off = align_up(off + tri * P * lay->cap_pad * sizeof(int32_t), 256);
         lay->strag = off;       off = align_up(off + tri * P * lay->cap_pad * sizeof(int32_t), 256);
         lay->strag_count = off; off = align_up(off + tri * P * sizeof(int32_t), 256);
-        lay->strag_items = off; off = align_up(off + tri * P * (lay->cap_pad / 256 + 1) * sizeof(int2), 256);
+        lay->strag_items = off; off = align_up(off + tri * P * (lay->cap_pad / 256 + 1) * sizeof(int4), 256);
         lay->self_dot = off;    off = align_up(off + P * lay->cap_pad * sizeof(float), 256);
         lay->head_sum_bf16 = off; off = align_up(off + P * 16 * kHeadDim * sizeof(__nv_bfloat16), 256);
         lay->meta = off;        off = align_up(off + (size_t)d->batch * sizeof(int32_t), 256);
@@ -128,7 +128,7 @@ int run(const rkv_desc_t *d, void *k_cache, void *v_cache, const void *q_window,
     p.left = reinterpret_cast<int32_t *>(ws + lay.left);
     p.strag = reinterpret_cast<int32_t *>(ws + lay.strag);
     p.strag_count = reinterpret_cast<int32_t *>(ws + lay.strag_count);
-    p.strag_items = reinterpret_cast<int2 *>(ws + lay.strag_items);
+    p.strag_items = reinterpret_cast<int4 *>(ws + lay.strag_items);
     p.self_dot = reinterpret_cast<float *>(ws + lay.self_dot);
     p.head_sum_bf16 = reinterpret_cast<__nv_bfloat16 *>(ws + lay.head_sum_bf16);
     p.meta = reinterpret_cast<int32_t *>(ws + lay.meta);

@@ -45,7 +45,8 @@ struct Params {
     int32_t *left;       // [P][cap_pad]         tri: partners a token still lacks after the scan of its own line
     int32_t *strag;      // [P][cap_pad]         tri: positions of the head's tokens with left > 0, ascending
     int32_t *strag_count;// [P]                  tri: how many
-    int2 *strag_items;   // [P * cap_pad / 256]  tri: work list of the second scoring pass, {head, chunk of 256}
+    int4 *strag_items;   // [P * cap_pad / 256]  tri: work list of the second scoring pass: {head, first listed
+                         //                      token, tokens (1..256), first streamed tile}
     float *self_dot;     // [P][cap_pad]         Kbar_i . Kbar_i (1 up to rounding and eps; 0 for a zero key)
     __nv_bfloat16 *head_sum_bf16;   // [P][16][128] head_sum split into three bf16 rows (hi, mid, lo), 13 zero rows
     int32_t *meta;       // [batch]              snapshot of seq_lens (kMetaInvalid if out of range)

@@ -203,16 +203,9 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
                     first_tile = n_tiles - 1;                  // streamed tiles: first_tile .. max(2 pi, n_tiles - depth)
                     n_iter = 1 + (rule_on ? n_tiles - max(2 * pi, n_tiles - kPass1Depth) : 0);   // + the query rows
                 } else {
-                    const int2 e = p.strag_items[ticket];
-                    head = e.x;
-                    const int k0 = e.y * kRowsPerItem;
-                    const int rows = min(p.strag_count[head] - k0, kRowsPerItem);
-                    const int last = p.strag[(size_t)head * p.cap_pad + k0 + rows - 1];
-                    const int n = candidates_from_meta(p.meta[head / p.hkv], p.budget, p.alpha);
-                    // pass 1 took the last listed token down to tile max(its own, n_tiles - depth)
-                    first_tile = max(last / kTile, (n + kTile - 1) / kTile - kPass1Depth) - 1;   // streamed: first_tile .. 0
-                    if (rows <= 0 || first_tile < 0) continue;                  // (the list holds no such item)
-                    desc = make_int4(head, k0, rows, first_tile);
+                    desc = p.strag_items[ticket];          // {head, first listed token, tokens, first streamed tile}
+                    head = desc.x;
+                    first_tile = desc.w;                   // streamed tiles: first_tile .. 0
                     n_iter = first_tile + 1;
                 }
                 const int key_row_base = head * p.cap;                         // first row of the head in the 2-D key view
@@ -658,8 +651,13 @@ __global__ void __launch_bounds__(kCompactThreads) strag_compact_kernel(Params p
         const int chunks = (count + kRowsPerItem - 1) / kRowsPerItem;
         if (chunks > 0) {
             const unsigned long long at = atomicAdd(&p.counters[2], (unsigned long long)chunks);
-            // longest scans (largest positions) first
-            for (int q = 0; q < chunks; ++q) p.strag_items[at + q] = make_int2(head, chunks - 1 - q);
+            // complete item descriptors, longest scans (largest positions) first: pass 1 took the chunk's last token
+            // down to tile max(its own, n_tiles - depth), so the chunk's scan starts one tile below that
+            for (int q = 0; q < chunks; ++q) {
+                const int c = chunks - 1 - q, k0 = c * kRowsPerItem, rows = min(count - k0, kRowsPerItem);
+                const int first_tile = max(list[k0 + rows - 1] / kTile, low) - 1;     // >= 0 for every listed token
+                p.strag_items[at + q] = make_int4(head, k0, rows, first_tile);
+            }
         }
     }
 }
