@@ -270,3 +270,21 @@ def test_thread_current_descriptor_entry_point(rkv):
     torch.cuda.synchronize()
     assert rc == 0 and torch.equal(out, ref)
     assert torch.equal(wl_a.k_cache.view(torch.int16), wl_b.k_cache.view(torch.int16))
+
+
+def test_kernel_events_and_executed_tile_counter(rkv):
+    """The profiling hooks of the descriptor: nine event boundaries give eight non-negative kernel times, and the
+    tensor-core kernels report how many 128 x 128 x 128 tile products they executed: at least one key tile per row
+    tile (pass 1), at most the full matrix."""
+    spec = small_spec("events", batch=4, budget=512, buffer=128)
+    wl = ri.make_workload(spec, device="cuda", seed=141)
+    comp = rkv.Compressor(spec.folded_batch, 2, 8, spec.budget, spec.buffer, spec.alpha, 0.1, stage_events=True)
+    comp.compress(wl.k_cache, wl.v_cache, wl.q_window, wl.seq_lens)
+    torch.cuda.synchronize()
+    comp.check_status()
+    ms = comp.kernel_ms()
+    assert len(ms) == len(comp.KERNEL_NAMES) == 8 and all(t >= 0.0 for t in ms) and sum(ms) > 0.0
+    heads, T = spec.head_problems, -(-(spec.cap - spec.alpha) // 128)
+    tiles = int(comp.counters[0].item())
+    assert heads * T <= tiles <= heads * T * T
+    assert rkv.rkv_launch_count(comp.desc, rkv.RKV_STAGE_ALL) == 8
