@@ -64,8 +64,14 @@ enum {
     kBarBEmpty = kBarBFull + kStagesB,      // [kStagesB]
     kBarAccFull = kBarBEmpty + kStagesB,    // [2 buffers][2 row tiles]
     kBarAccEmpty = kBarAccFull + 4,         // [2][2], 4 warps each
-    kNumBars = kBarAccEmpty + 4
+    kBarRFull = kBarAccEmpty + 4,           // [2] pass 2: the head's r_j are in shared memory
+    kBarREmpty = kBarRFull + 2,             // [2] pass 2: ... and no longer read (8 epilogue warps)
+    kNumBars = kBarREmpty + 2
 };
+// Pass 2 keeps one pair of resident tiles (its items are long) and uses the room of the second pair for the r_j of
+// the whole head, double-buffered across items, so its epilogue reads them in place.
+constexpr int kOffRHead = kOffA + 2 * kTileBytes;          // 2 x RKV_MAX_CAP floats
+static_assert(2 * RKV_MAX_CAP * 4 <= 2 * kTileBytes, "the head's r_j must fit the second resident pair");
 constexpr int kOffItems = kOffBar + kNumBars * 8;          // kItemSlots x int4
 constexpr int kOffMisc = kOffItems + kItemSlots * 16;      // tmem base, abort flag, bail flag
 constexpr int kOffRj = kOffMisc + 16;                      // [2 row tiles][128] r_j of the key tile being drained
@@ -166,6 +172,10 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
             mbar_init(bar.at(kBarAccFull + s), 1);
             mbar_init(bar.at(kBarAccEmpty + s), 4);
         }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(bar.at(kBarRFull + s), 1);
+            mbar_init(bar.at(kBarREmpty + s), 8);
+        }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -215,6 +225,17 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
                 items[qs] = desc;
                 mbar_arrive(bar.at(kBarQFull + qs));
 
+                if (kPass2) {
+                    // r_j of the tiles this item streams (0 .. first_tile), straight into shared memory
+                    const uint32_t rb = k_item & 1;
+                    if (!mbar_wait(bar.at(kBarREmpty + rb), ((k_item >> 1) & 1) ^ 1, abort_flag, p.status)) break;
+                    const uint32_t bytes = (uint32_t)(first_tile + 1) * kTile * 4u;
+                    mbar_expect_tx(bar.at(kBarRFull + rb), bytes);
+                    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                                 ::"r"(sbase + kOffRHead + rb * RKV_MAX_CAP * 4), "l"(p.inv_norm + (size_t)head * p.cap_pad),
+                                   "r"(bytes), "r"(bar.at(kBarRFull + rb))
+                                 : "memory");
+                }
                 if (!kPass2) {
                     const int row0 = desc.y * kRowsPerItem;
                     const int num_m = (desc.z - row0 > kTile) ? 2 : 1;
@@ -289,8 +310,9 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
                     n_iter = d.w + 1;
                     skip_it = -1;
                 }
-                const uint32_t ab = k_item & 1;
-                if (!mbar_wait(bar.at(kBarAFull + ab), (k_item >> 1) & 1, abort_flag, p.status)) break;
+                const uint32_t ab = kPass2 ? 0u : (k_item & 1);                          // pass 2: one pair of tiles
+                const uint32_t a_par = kPass2 ? (k_item & 1) : ((k_item >> 1) & 1);
+                if (!mbar_wait(bar.at(kBarAFull + ab), a_par, abort_flag, p.status)) break;
                 if (kPass2) asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 for (int it = 0; it < n_iter; ++it) {
                     const uint32_t s = bcount % kStagesB;
@@ -360,7 +382,8 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
             if (d.x < 0) break;
             const int head = d.x;
             const float *inv_norm = p.inv_norm + (size_t)head * p.cap_pad;
-            const uint32_t ab = k_item & 1;
+            const uint32_t ab = kPass2 ? 0u : (k_item & 1);
+            const uint32_t a_par = kPass2 ? (k_item & 1) : ((k_item >> 1) & 1);
 
             // ---- per item: which token this thread owns, its threshold, where its scan starts and ends
             // (a failed wait does not leave the item at once: the warps of a row tile meet at named barriers in the
@@ -399,7 +422,7 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
 
                 // gather this thread's key row into the resident tile (same swizzled layout as a TMA load); every
                 // warp waits and arrives, also one without rows of its own, so that no arrival runs ahead
-                item_ok = mbar_wait(bar.at(kBarAEmpty + ab), ((k_item >> 1) & 1) ^ 1, abort_flag, p.status);
+                item_ok = mbar_wait(bar.at(kBarAEmpty + ab), a_par ^ 1, abort_flag, p.status);
                 if (active && item_ok) {
                     uint8_t *tile = smem + kOffA + (ab * 2 + m) * kTileBytes;
                     const uint4 *src = reinterpret_cast<const uint4 *>(
@@ -420,7 +443,11 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
 
             const bool scan = active && (kPass2 || rule_on);
             // r_j of the first key tile of the scan: loaded now, staged in shared memory when the tile is drained
-            float rj_next = scan ? __ldg(inv_norm + first_tile * kTile + lrow) : 0.f;
+            float rj_next = (!kPass2 && scan) ? __ldg(inv_norm + first_tile * kTile + lrow) : 0.f;
+            if (kPass2) {       // every warp waits for the head's r_j, and hands them back at the item's end
+                const bool r_ok = mbar_wait(bar.at(kBarRFull + (k_item & 1)), (k_item >> 1) & 1, abort_flag, p.status);
+                item_ok = item_ok && r_ok;
+            }
 
             if (!kPass2 && active) {
                 const uint32_t a = cnt & 1;
@@ -488,14 +515,20 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
                 // wait fail keeps going through the loop, without touching TMEM, until the item's last tile.
                 const float thr = (row_ok && ri > 0.f) ? __fdiv_rn(p.sim_threshold, ri) : kInf;   // g r_j vs T / r_i
                 float *rj_s = reinterpret_cast<float *>(smem + kOffRj) + m * kTile;
-                const float4 *rj4 = reinterpret_cast<const float4 *>(rj_s);
+                const float *r_head = reinterpret_cast<const float *>(smem + kOffRHead) + (k_item & 1) * RKV_MAX_CAP;
                 bool ok = item_ok;
                 for (int jt = first_tile; jt >= my_last_tile; --jt) {
                     const int jbase = jt * kTile;
-                    asm volatile("bar.sync %0, 128;" ::"r"(1 + m) : "memory");      // the previous tile's r_j are done with
-                    rj_s[lrow] = rj_next;
-                    asm volatile("bar.sync %0, 128;" ::"r"(1 + m) : "memory");
-                    if (jt > my_last_tile) rj_next = __ldg(inv_norm + jbase - kTile + lrow);
+                    const float4 *rj4;
+                    if (kPass2) {
+                        rj4 = reinterpret_cast<const float4 *>(r_head + jbase);         // in place, nothing to stage
+                    } else {
+                        asm volatile("bar.sync %0, 128;" ::"r"(1 + m) : "memory");      // the previous tile's r_j are done with
+                        rj_s[lrow] = rj_next;
+                        asm volatile("bar.sync %0, 128;" ::"r"(1 + m) : "memory");
+                        if (jt > my_last_tile) rj_next = __ldg(inv_norm + jbase - kTile + lrow);
+                        rj4 = reinterpret_cast<const float4 *>(rj_s);
+                    }
                     const uint32_t a = cnt & 1;
                     if (ok) ok = mbar_wait(bar.at(kBarAccFull + a * 2 + m), (cnt >> 1) & 1, abort_flag, p.status);
                     ++cnt;
@@ -587,6 +620,10 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
                     }
                 }
                 item_ok = ok;
+            }
+            if (kPass2) {
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar.at(kBarREmpty + (k_item & 1)));
             }
             if (!item_ok) dead = true;        // leaves at the next vote, together with the other warps of its row tile
             if (row_ok) {
