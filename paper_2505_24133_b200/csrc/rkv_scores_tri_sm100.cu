@@ -64,8 +64,8 @@ enum {
     kBarBEmpty = kBarBFull + kStagesB,      // [kStagesB]
     kBarAccFull = kBarBEmpty + kStagesB,    // [2 buffers][2 row tiles]
     kBarAccEmpty = kBarAccFull + 4,         // [2][2], 4 warps each
-    kBarRFull = kBarAccEmpty + 4,           // [2] pass 2: the head's r_j are in shared memory
-    kBarREmpty = kBarRFull + 2,             // [2] pass 2: ... and no longer read (8 epilogue warps)
+    kBarRFull = kBarAccEmpty + 4,           // [2] the r_j of the item's key tiles are in shared memory
+    kBarREmpty = kBarRFull + 2,             // [2] ... and no longer read (8 epilogue warps)
     kNumBars = kBarREmpty + 2
 };
 // Pass 2 keeps one pair of resident tiles (its items are long) and uses the room of the second pair for the r_j of
@@ -74,8 +74,8 @@ constexpr int kOffRHead = kOffA + 2 * kTileBytes;          // 2 x RKV_MAX_CAP fl
 static_assert(2 * RKV_MAX_CAP * 4 <= 2 * kTileBytes, "the head's r_j must fit the second resident pair");
 constexpr int kOffItems = kOffBar + kNumBars * 8;          // kItemSlots x int4
 constexpr int kOffMisc = kOffItems + kItemSlots * 16;      // tmem base, abort flag, bail flag
-constexpr int kOffRj = kOffMisc + 16;                      // [2 row tiles][128] r_j of the key tile being drained
-constexpr int kSmemBytes = kOffRj + 2 * kTile * 4 + 1024;  // + slack for the manual 1024-byte alignment
+constexpr int kOffRj = kOffMisc + 16;                      // pass 1: [2 items][kPass1Depth * 128] r_j of the streamed tiles
+constexpr int kSmemBytes = kOffRj + 2 * kPass1Depth * kTile * 4 + 1024;  // + slack for the manual 1024-byte alignment
 static_assert(kOffItems % 16 == 0 && kOffRj % 16 == 0, "item descriptors are read as int4, r_j as float4");
 static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
 
@@ -236,6 +236,19 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
                                    "r"(bytes), "r"(bar.at(kBarRFull + rb))
                                  : "memory");
                 }
+                if (!kPass2 && rule_on) {
+                    // r_j of the key tiles this item streams (first_tile down to first_tile + 2 - n_iter)
+                    const uint32_t rb = k_item & 1;
+                    if (!mbar_wait(bar.at(kBarREmpty + rb), ((k_item >> 1) & 1) ^ 1, abort_flag, p.status)) break;
+                    const int low_tile = first_tile + 2 - n_iter;
+                    const uint32_t bytes = (uint32_t)(n_iter - 1) * kTile * 4u;
+                    mbar_expect_tx(bar.at(kBarRFull + rb), bytes);
+                    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                                 ::"r"(sbase + kOffRj + rb * kPass1Depth * kTile * 4),
+                                   "l"(p.inv_norm + (size_t)head * p.cap_pad + (size_t)low_tile * kTile), "r"(bytes),
+                                   "r"(bar.at(kBarRFull + rb))
+                                 : "memory");
+                }
                 if (!kPass2) {
                     const int row0 = desc.y * kRowsPerItem;
                     const int num_m = (desc.z - row0 > kTile) ? 2 : 1;
@@ -358,24 +371,10 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
         const float scale = 0.08838834764831845f;             // 1 / sqrt(128)
         const int G = p.group;
         uint32_t k_item = 0, cnt = 0;
-        bool dead = false;                    // a wait of this warp has failed: it takes part in no further item
 
         while (true) {
             const uint32_t qs = k_item % kItemSlots;
-            // The four warps of a row tile meet at named barriers inside an item, so they must leave the item loop
-            // together: each brings the outcome of its waits (the last item's and this item's first) to a vote,
-            // and a warp leaves only here, with its three mates, or at the terminator, which all of them see.
-            const bool have = !dead && mbar_wait(bar.at(kBarQFull + qs), (k_item / kItemSlots) & 1, abort_flag, p.status);
-            int all_have;
-            asm volatile(
-                "{\n\t.reg .pred p, q;\n\t"
-                "setp.ne.u32 p, %1, 0;\n\t"
-                "bar.red.and.pred q, %2, 128, p;\n\t"
-                "selp.u32 %0, 1, 0, q;\n\t}"
-                : "=r"(all_have)
-                : "r"((uint32_t)have), "r"(1 + m)
-                : "memory");
-            if (!all_have) break;
+            if (!mbar_wait(bar.at(kBarQFull + qs), (k_item / kItemSlots) & 1, abort_flag, p.status)) break;
             const int4 d = items[qs];
             __syncwarp();
             if (lane == 0) mbar_arrive(bar.at(kBarQEmpty + qs));
@@ -386,8 +385,6 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
             const uint32_t a_par = kPass2 ? (k_item & 1) : ((k_item >> 1) & 1);
 
             // ---- per item: which token this thread owns, its threshold, where its scan starts and ends
-            // (a failed wait does not leave the item at once: the warps of a row tile meet at named barriers in the
-            // tile loop below, so all of them have to reach it)
             bool active, row_ok, item_ok = true;
             int i, first_tile, my_last_tile, own_tile;
             float ri, self = 0.f, total = 0.f;
@@ -443,8 +440,8 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
 
             const bool scan = active && (kPass2 || rule_on);
             // r_j of the first key tile of the scan: loaded now, staged in shared memory when the tile is drained
-            float rj_next = (!kPass2 && scan) ? __ldg(inv_norm + first_tile * kTile + lrow) : 0.f;
-            if (kPass2) {       // every warp waits for the head's r_j, and hands them back at the item's end
+            const bool has_r = kPass2 || rule_on;
+            if (has_r) {        // every warp waits for the item's r_j, and hands them back at the item's end
                 const bool r_ok = mbar_wait(bar.at(kBarRFull + (k_item & 1)), (k_item >> 1) & 1, abort_flag, p.status);
                 item_ok = item_ok && r_ok;
             }
@@ -510,25 +507,16 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
 
             float removed = 0.f;
             if (scan) {
-                // ---- key tiles, last to first.  The four warps of a row tile share the tile's r_j through shared
-                // memory; they run this loop in step (two named barriers per tile), so even a warp that has seen a
-                // wait fail keeps going through the loop, without touching TMEM, until the item's last tile.
+                // ---- key tiles, last to first; their r_j lie in shared memory
                 const float thr = (row_ok && ri > 0.f) ? __fdiv_rn(p.sim_threshold, ri) : kInf;   // g r_j vs T / r_i
-                float *rj_s = reinterpret_cast<float *>(smem + kOffRj) + m * kTile;
-                const float *r_head = reinterpret_cast<const float *>(smem + kOffRHead) + (k_item & 1) * RKV_MAX_CAP;
+                // pass 2: the whole head from tile 0; pass 1: the item's tiles from its lowest one (that of row tile 0)
+                const float *r_base = kPass2 ? reinterpret_cast<const float *>(smem + kOffRHead) + (k_item & 1) * RKV_MAX_CAP
+                                             : reinterpret_cast<const float *>(smem + kOffRj) + (k_item & 1) * kPass1Depth * kTile -
+                                                   (size_t)max(2 * d.y, first_tile + 1 - kPass1Depth) * kTile;
                 bool ok = item_ok;
                 for (int jt = first_tile; jt >= my_last_tile; --jt) {
                     const int jbase = jt * kTile;
-                    const float4 *rj4;
-                    if (kPass2) {
-                        rj4 = reinterpret_cast<const float4 *>(r_head + jbase);         // in place, nothing to stage
-                    } else {
-                        asm volatile("bar.sync %0, 128;" ::"r"(1 + m) : "memory");      // the previous tile's r_j are done with
-                        rj_s[lrow] = rj_next;
-                        asm volatile("bar.sync %0, 128;" ::"r"(1 + m) : "memory");
-                        if (jt > my_last_tile) rj_next = __ldg(inv_norm + jbase - kTile + lrow);
-                        rj4 = reinterpret_cast<const float4 *>(rj_s);
-                    }
+                    const float4 *rj4 = reinterpret_cast<const float4 *>(r_base + jbase);
                     const uint32_t a = cnt & 1;
                     if (ok) ok = mbar_wait(bar.at(kBarAccFull + a * 2 + m), (cnt >> 1) & 1, abort_flag, p.status);
                     ++cnt;
@@ -621,11 +609,11 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
                 }
                 item_ok = ok;
             }
-            if (kPass2) {
+            if (has_r) {
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar.at(kBarREmpty + (k_item & 1)));
             }
-            if (!item_ok) dead = true;        // leaves at the next vote, together with the other warps of its row tile
+            if (!item_ok) break;              // (the epilogue warps meet at no barrier of their own: each may leave alone)
             if (row_ok) {
                 float *out = p.sbar + (size_t)head * p.cap_pad + i;
                 if (!kPass2) {
