@@ -220,7 +220,7 @@ def run_stream(args, rkv, rd, dev, rank, world, spec):
             "stream": {"firings": firings, "compressing_firings": real, "total_compression_ms": ms_slowest,
                        "ms_per_compressing_firing": real_ms / max(real, 1),
                        "compressions": real * spec.folded_batch},
-            "gpu_launches": firings * rkv.rkv_launch_count(comp.desc, rkv.RKV_STAGE_ALL),
+            "gpu_launches": firings * rkv.rkv_launch_count_for(comp.desc, spec.budget, spec.buffer, spec.alpha, rkv.RKV_STAGE_ALL),
             "clocks": clocks, "peaks": peaks["source"]}))
     if torch.distributed.is_initialized():
         torch.distributed.destroy_process_group()
@@ -273,7 +273,7 @@ def main():
         kw["pool_w"] = args.pool_w
     comp = rkv.Compressor(spec.folded_batch, spec.n_kv_heads, spec.n_q_heads, spec.budget, spec.buffer, spec.alpha,
                           spec.lam, dtype=spec.torch_dtype, device=dev, **kw)
-    launches_per_step = rkv.rkv_launch_count(comp.desc, rkv.RKV_STAGE_ALL)
+    launches_per_step = rkv.rkv_launch_count_for(comp.desc, spec.budget, spec.buffer, spec.alpha, rkv.RKV_STAGE_ALL)
     stream = torch.cuda.current_stream()
 
     def step(i, c=comp):

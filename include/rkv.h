@@ -197,9 +197,12 @@ RKV_API int rkv_compress_static(const rkv_desc_t *desc, void *k_cache, void *v_c
                         int32_t *seq_lens, int32_t budget, int32_t buffer, int32_t alpha, float lambda,
                         int32_t *out_idx, void *stream);
 
-/* Number of kernels a call with this descriptor and stage mask launches (for launch accounting; the memset that
- * precedes the prep kernel is not counted). */
+/* Number of kernels a call launches (for launch accounting; the memset that precedes the prep kernel is not
+ * counted).  rkv_launch_count_for() is exact for the given sizes; rkv_launch_count(), which does not know them, gives
+ * the count for large caches (small ones run the select stage as one kernel instead of three). */
 RKV_API int rkv_launch_count(const rkv_desc_t *desc, uint32_t stage_mask);
+RKV_API int rkv_launch_count_for(const rkv_desc_t *desc, int32_t budget, int32_t buffer, int32_t alpha,
+                         uint32_t stage_mask);
 
 /* Human-readable name of a status code. */
 RKV_API const char *rkv_status_string(int status);

@@ -8,5 +8,5 @@ from .binding import (  # noqa: F401
     RKV_STAGE_SCORES, RKV_STAGE_SELECT, RKV_OK, RkvDesc, RkvError, Compressor, lib, lib_path,
     rkv_compress, rkv_compress_ex, rkv_compress_stages, rkv_compress_host, rkv_compress_static,
     RKV_STATIC_SCRATCH_BYTES, rkv_desc_default,
-    rkv_host_workspace_bytes, rkv_launch_count, rkv_set_desc, rkv_status_string, rkv_workspace_bytes,
+    rkv_host_workspace_bytes, rkv_launch_count, rkv_launch_count_for, rkv_set_desc, rkv_status_string, rkv_workspace_bytes,
 )

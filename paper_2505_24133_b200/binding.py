@@ -66,6 +66,7 @@ def lib():
         L.rkv_compress_host.restype, L.rkv_compress_host.argtypes = ctypes.c_int, [P] + ten
         L.rkv_compress_static.restype, L.rkv_compress_static.argtypes = ctypes.c_int, [P] + ten
         L.rkv_launch_count.restype, L.rkv_launch_count.argtypes = ctypes.c_int, [P, U32]
+        L.rkv_launch_count_for.restype, L.rkv_launch_count_for.argtypes = ctypes.c_int, [P, I32, I32, I32, U32]
         L.rkv_status_string.restype, L.rkv_status_string.argtypes = ctypes.c_char_p, [ctypes.c_int]
         L.rkv_last_cuda_error.restype, L.rkv_last_cuda_error.argtypes = ctypes.c_char_p, []
         _lib = L
@@ -111,6 +112,10 @@ def rkv_set_desc(desc: RkvDesc) -> int:
 
 def rkv_launch_count(desc: RkvDesc, stage_mask: int = RKV_STAGE_ALL) -> int:
     return lib().rkv_launch_count(ctypes.byref(desc), stage_mask)
+
+
+def rkv_launch_count_for(desc: RkvDesc, budget: int, buffer: int, alpha: int, stage_mask: int = RKV_STAGE_ALL) -> int:
+    return lib().rkv_launch_count_for(ctypes.byref(desc), budget, buffer, alpha, stage_mask)
 
 
 def rkv_compress(k_cache, v_cache, q_window, seq_lens, budget, buffer, alpha, lam, out_idx, stream=None) -> int:

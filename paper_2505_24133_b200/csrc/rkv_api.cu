@@ -317,6 +317,17 @@ int rkv_launch_count(const rkv_desc_t *desc, uint32_t stage_mask)
     return c;
 }
 
+int rkv_launch_count_for(const rkv_desc_t *desc, int32_t budget, int32_t buffer, int32_t alpha, uint32_t stage_mask)
+{
+    Layout lay;
+    if (check_shapes(desc, budget, buffer, alpha, &lay) != RKV_OK) return 0;
+    int c = rkv_launch_count(desc, stage_mask);
+    if ((stage_mask & RKV_STAGE_SELECT) && select_is_fused(lay.cap_pad, alpha)) c -= 2;
+    if ((stage_mask & RKV_STAGE_SCORES) && use_tri(desc) && desc->beta > 0 && desc->sim_threshold < 1.0f && lay.tiles < 2)
+        c -= 2;                                     // one key tile: the first scoring pass has seen everything
+    return c;
+}
+
 const char *rkv_status_string(int status)
 {
     switch (status) {

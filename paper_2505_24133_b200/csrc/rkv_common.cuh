@@ -117,5 +117,6 @@ cudaError_t launch_scores_tri_sm100(const Params &p, cudaStream_t s);
 cudaError_t launch_select(const Params &p, cudaStream_t s);
 cudaError_t launch_gather(const Params &p, cudaStream_t s);
 bool scores_sm100_available();
+bool select_is_fused(int cap_pad, int alpha);   // the select stage is one kernel (small caches) instead of three
 
 }  // namespace rkv

@@ -56,6 +56,7 @@ __device__ __forceinline__ float block_sum(float v, float *scratch)
     return r;
 }
 
+constexpr size_t kFusedSmemLimit = 64 * 1024;   // largest shared-memory footprint for the single-kernel form
 constexpr int kStatThreads = 256;
 constexpr int kImpThreads = 256;
 constexpr int kImpTokens = 1024;     // tokens per importance block
@@ -117,9 +118,14 @@ __global__ void __launch_bounds__(kImpThreads) importance_kernel(Params p)
     }
 }
 
+// kFused: the block first does the work of row_stats_kernel and importance_kernel for its head, with the pooled
+// logits in shared memory (small caches only: one launch instead of three, all of them latency-bound there).
+template <bool kFused>
 __global__ void __launch_bounds__(kSelThreads, 2) select_kernel(Params p)
 {
-    extern __shared__ float row[];                 // [cap_pad] one logits row / the Sbar row, then the keys
+    extern __shared__ float row[];                 // [cap_pad] one logits row / the Sbar row, then the keys;
+                                                   // kFused: then [cap_pad] importance and [alpha][cap_pad] logits
+    __shared__ float stat_s[2 * RKV_MAX_GROUP_ROWS];
     __shared__ float scratch[kSelWarps];
     __shared__ uint32_t hist[256];
     __shared__ uint32_t sel_prefix, sel_want;
@@ -138,6 +144,46 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_kernel(Params p)
     const int n = L - p.alpha;
     const int k = p.budget - p.alpha;
 
+    const float *imp = p.imp + (size_t)head * p.cap_pad;
+    if (kFused) {
+        float *imp_s = row + p.cap_pad, *lg = row + 2 * p.cap_pad;
+        const float *logits = p.logits + (size_t)head * p.alpha * p.cap_pad;
+        const int lane = tid & 31, warp = tid >> 5;
+        for (int j = 0; j < p.alpha; ++j)
+            for (int i = tid; i < n; i += kSelThreads) lg[j * p.cap_pad + i] = logits[(size_t)j * p.cap_pad + i];
+        __syncthreads();
+        for (int j = warp; j < p.alpha; j += kSelWarps) {      // Eq. 3: one warp per query row
+            const float *r = lg + j * p.cap_pad;
+            float mj = -INFINITY;
+            for (int i = lane; i < n; i += 32) mj = fmaxf(mj, r[i]);
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) mj = fmaxf(mj, __shfl_xor_sync(0xffffffffu, mj, off));
+            float sj = 0.f;
+            for (int i = lane; i < n; i += 32) sj += expf(r[i] - mj);
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) sj += __shfl_xor_sync(0xffffffffu, sj, off);
+            if (lane == 0) {
+                stat_s[2 * j] = mj;
+                stat_s[2 * j + 1] = 1.0f / sj;
+            }
+        }
+        __syncthreads();
+        const int W = p.pool_w;
+        const float inv_alpha = 1.0f / (float)p.alpha;
+        for (int i = tid; i < n; i += kSelThreads) {            // Eq. 4
+            const int lo = max(i - W, 0), hi = min(i + W - 1, n - 1);
+            float acc = 0.f;
+            for (int j = 0; j < p.alpha; ++j) {
+                const float *r = lg + j * p.cap_pad;
+                float best = r[i];
+                for (int u = lo; u <= hi; ++u) best = fmaxf(best, r[u]);
+                acc += expf(best - stat_s[2 * j]) * stat_s[2 * j + 1];
+            }
+            imp_s[i] = acc * inv_alpha;
+        }
+        imp = imp_s;
+    }
+
     // ---- Eq. 6: R = softmax(Sbar)
     __syncthreads();
     const float *sbar = p.sbar + (size_t)head * p.cap_pad;
@@ -153,7 +199,6 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_kernel(Params p)
     for (int i = tid; i < n; i += kSelThreads) s += expf(row[i] - m);
     s = block_sum(s, scratch);
     const float inv = 1.0f / s;
-    const float *imp = p.imp + (size_t)head * p.cap_pad;
 
     // ---- Eq. 7 and the integer keys (kept in the same shared row, one owner per slot)
     uint32_t *keys = reinterpret_cast<uint32_t *>(row);
@@ -265,20 +310,33 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_kernel(Params p)
 
 }  // namespace
 
+bool select_is_fused(int cap_pad, int alpha) { return (size_t)(alpha + 2) * cap_pad * sizeof(float) <= kFusedSmemLimit; }
+
 cudaError_t launch_select(const Params &p, cudaStream_t s)
 {
     const unsigned heads = (unsigned)(p.batch * p.hkv);
+    cudaError_t e;
+    if (select_is_fused(p.cap_pad, p.alpha)) {
+        // small caches: one kernel does row statistics, importance and selection
+        if ((e = mark_kernel(p, 2, s)) != cudaSuccess || (e = mark_kernel(p, 3, s)) != cudaSuccess) return e;
+        const size_t smem = (size_t)(p.alpha + 2) * p.cap_pad * sizeof(float);
+        if ((e = cudaFuncSetAttribute(select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) !=
+            cudaSuccess)
+            return e;
+        select_kernel<true><<<heads, kSelThreads, smem, s>>>(p);
+        return cudaGetLastError();
+    }
     row_stats_kernel<<<heads * (unsigned)p.alpha, kStatThreads, 0, s>>>(p);
-    cudaError_t e0 = cudaGetLastError();
-    if (e0 != cudaSuccess) return e0;
-    if ((e0 = mark_kernel(p, 2, s)) != cudaSuccess) return e0;
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    if ((e = mark_kernel(p, 2, s)) != cudaSuccess) return e;
     importance_kernel<<<heads * (unsigned)((p.cap + kImpTokens - 1) / kImpTokens), kImpThreads, 0, s>>>(p);
-    if ((e0 = cudaGetLastError()) != cudaSuccess) return e0;
-    if ((e0 = mark_kernel(p, 3, s)) != cudaSuccess) return e0;
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    if ((e = mark_kernel(p, 3, s)) != cudaSuccess) return e;
     const size_t smem = (size_t)p.cap_pad * sizeof(float);
-    cudaError_t e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    select_kernel<<<(unsigned)(p.batch * p.hkv), kSelThreads, smem, s>>>(p);
+    if ((e = cudaFuncSetAttribute(select_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) !=
+        cudaSuccess)
+        return e;
+    select_kernel<false><<<heads, kSelThreads, smem, s>>>(p);
     return cudaGetLastError();
 }
 

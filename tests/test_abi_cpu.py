@@ -20,7 +20,7 @@ def rkv():
 def test_library_exports_every_declared_symbol(rkv):
     header = open(os.path.join(ROOT, "include", "rkv.h")).read()
     names = re.findall(r"RKV_API\s+[\w\s\*]+?\b(rkv_\w+)\s*\(", header)
-    assert len(names) >= 11
+    assert len(names) >= 13
     lib = ctypes.CDLL(rkv.lib_path())
     for name in names:
         assert hasattr(lib, name), f"{name} is declared in include/rkv.h but not exported"
@@ -112,6 +112,11 @@ def test_rkv_compress_needs_a_current_descriptor(rkv):
     assert rkv.rkv_status_string(5) == "RKV_ERR_TIMEOUT"
     assert rkv.rkv_launch_count(_desc(rkv), rkv.RKV_STAGE_ALL) == 8      # prep, 3 scoring kernels, 3 select kernels, gather
     assert rkv.rkv_launch_count(_desc(rkv, flags=rkv.RKV_FLAG_SIMT_SCORES), rkv.RKV_STAGE_ALL) == 6
+    # exact counts for given sizes: small caches run the select stage as one kernel
+    assert rkv.rkv_launch_count_for(_desc(rkv), 4096, 128, 8, rkv.RKV_STAGE_ALL) == 8
+    assert rkv.rkv_launch_count_for(_desc(rkv), 1024, 128, 8, rkv.RKV_STAGE_ALL) == 6
+    assert rkv.rkv_launch_count_for(_desc(rkv), 64, 32, 8, rkv.RKV_STAGE_ALL) == 4          # one key tile: no second pass
+    assert rkv.rkv_launch_count_for(_desc(rkv), 8, 128, 8, rkv.RKV_STAGE_ALL) == 0           # invalid sizes
 
 
 def test_product_package_does_not_touch_the_oracle():

@@ -287,4 +287,4 @@ def test_kernel_events_and_executed_tile_counter(rkv):
     heads, T = spec.head_problems, -(-(spec.cap - spec.alpha) // 128)
     tiles = int(comp.counters[0].item())
     assert heads * T <= tiles <= heads * T * T
-    assert rkv.rkv_launch_count(comp.desc, rkv.RKV_STAGE_ALL) == 8
+    assert rkv.rkv_launch_count_for(comp.desc, spec.budget, spec.buffer, spec.alpha, rkv.RKV_STAGE_ALL) == 6
