@@ -43,9 +43,11 @@ def test_config2_simt_and_tcgen05_agree(rkv):
     assert same > 0.5
 
 
-@pytest.mark.parametrize("name,rows", [("llama8b_b16", [0, 311]), ("qwen7b_b64", [0, 7, 1000, 1791])])
+@pytest.mark.parametrize("name,rows", [("llama8b_b16", [0, 311]), ("qwen7b_b64", [0, 7, 1000, 1791]),
+                                       ("qwen14b_b32", [5, 1535])])
 def test_full_size_configs_sampled(rkv, name, rows):
-    """Configs 3 and 4 at full size (about 9 and 8 GB of K+V), oracle on sampled sequences (all KV heads)."""
+    """Configs 3, 4 and (one firing of) 5 at full size (about 9, 8 and 27 GB of K+V), oracle on sampled sequences
+    (all KV heads)."""
     wl = ri.make_workload(ri.SPECS[name], device="cuda")
     rep, comp = run_and_check(rkv, wl, check_rows=rows)
     print(rep.summary())
