@@ -101,6 +101,37 @@ static void importance_scores(const double *A, int n, int alpha, int W,
     }
 }
 
+/* ---- Algorithm 1's ordering of the same two steps (a variant, off by default):
+ * mean over the alpha query rows first, then the 1-D pooling.  The algorithm box
+ * names neither the pooling's kind nor its size; it is read as the max pooling
+ * of Eq. 4 over the same window {i-W, ..., i+W-1}. ---------------------------- */
+static void importance_scores_mean_first(const double *A, int n, int alpha,
+                                         int W, double *I)
+{
+    double *mean = (double *)malloc((size_t)n * sizeof(double));
+    for (int i = 0; i < n; ++i) {
+        double acc = 0.0;
+        for (int j = 0; j < alpha; ++j)
+            acc += A[(size_t)j * n + i];
+        mean[i] = acc / (double)alpha;
+    }
+    for (int i = 0; i < n; ++i) {
+        double best = mean[i];
+        if (W > 0) {
+            int lo = i - W, hi = i + W - 1;
+            if (lo < 0)
+                lo = 0;
+            if (hi > n - 1)
+                hi = n - 1;
+            for (int t = lo; t <= hi; ++t)
+                if (mean[t] > best)
+                    best = mean[t];
+        }
+        I[i] = best;
+    }
+    free(mean);
+}
+
 /* ---- Eq. 5: S = Kbar Kbar^T with zero diagonal ---------------------------- */
 static void cosine_matrix(const float *K, int n, int d, double eps, double *S)
 {
@@ -190,6 +221,8 @@ static int ascending_int(const void *a, const void *b)
  *   A, I, Sbar, R, Z         optional outputs ([alpha][n] and [n]); may be NULL
  *   S_raw, S_mod             optional [n][n] dumps of Eq. 5's matrix before and
  *                            after the retention rule; may be NULL
+ *   variant                  0 = the method as the equations state it; bit 0 =
+ *                            Algorithm 1's order for the importance (mean, then pool)
  * Returns 1 if the head was compressed, 0 if L <= budget (nothing to do:
  * idx = 0..L-1 then -1), -1 on bad arguments.
  */
@@ -197,7 +230,7 @@ int rkv_oracle_head(const float *K, const float *Q, int L, int d, int G,
                     int alpha, int budget, int W, int beta, double T,
                     double eps, double lambda, int32_t *idx, double *A,
                     double *I, double *Sbar, double *R, double *Z,
-                    double *S_raw, double *S_mod)
+                    double *S_raw, double *S_mod, int variant)
 {
     if (L < 0 || d < 1 || G < 1 || alpha < 1 || budget <= alpha || W < 0 ||
         beta < 0)
@@ -222,7 +255,10 @@ int rkv_oracle_head(const float *K, const float *Q, int L, int d, int G,
     }
 
     attention_weights(K, Q, n, d, G, alpha, A_);
-    importance_scores(A_, n, alpha, W, I_);
+    if (variant & 1) /* RKV_ORACLE_MEAN_THEN_POOL */
+        importance_scores_mean_first(A_, n, alpha, W, I_);
+    else
+        importance_scores(A_, n, alpha, W, I_);
     cosine_matrix(K, n, d, eps, S_);
     if (S_raw)
         memcpy(S_raw, S_, (size_t)n * n * sizeof(double));
@@ -277,7 +313,7 @@ int rkv_oracle_batch(const float *K, const float *Q, const int32_t *seq_lens,
                      int B, int Hkv, int Hq, int cap, int d, int alpha,
                      int budget, int W, int beta, double T, double eps,
                      double lambda, int32_t *idx, double *scores,
-                     int32_t *compressed)
+                     int32_t *compressed, int variant)
 {
     if (Hkv < 1 || Hq % Hkv != 0)
         return -1;
@@ -305,7 +341,7 @@ int rkv_oracle_batch(const float *K, const float *Q, const int32_t *seq_lens,
                                 eps, lambda, idx + (size_t)p * budget, NULL,
                                 sc, sc ? sc + plane : NULL,
                                 sc ? sc + 2 * plane : NULL,
-                                sc ? sc + 3 * plane : NULL, NULL, NULL);
+                                sc ? sc + 3 * plane : NULL, NULL, NULL, variant);
         if (r < 0) {
 #ifdef _OPENMP
 #pragma omp atomic write

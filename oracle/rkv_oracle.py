@@ -37,10 +37,10 @@ def _load():
                       ctypes.POINTER(ctypes.c_int32))
         lib.rkv_oracle_head.restype = ctypes.c_int
         lib.rkv_oracle_head.argtypes = [fp, fp] + [ctypes.c_int] * 7 + [ctypes.c_double] * 3 + \
-            [ip] + [dp] * 7
+            [ip] + [dp] * 7 + [ctypes.c_int]
         lib.rkv_oracle_batch.restype = ctypes.c_int
         lib.rkv_oracle_batch.argtypes = [fp, fp, ip] + [ctypes.c_int] * 9 + [ctypes.c_double] * 3 + \
-            [ip, dp, ip]
+            [ip, dp, ip, ctypes.c_int]
         lib.rkv_oracle_gather.restype = None
         lib.rkv_oracle_gather.argtypes = [ctypes.c_void_p, ip, ctypes.c_int, ctypes.c_size_t,
                                           ctypes.c_void_p]
@@ -70,7 +70,8 @@ class HeadResult:
 
 
 def oracle_head(K, Q, *, budget: int, alpha: int, lam: float, W: int, beta: int, T: float,
-                eps: float = 1e-8, L: Optional[int] = None, want_S: bool = False) -> HeadResult:
+                eps: float = 1e-8, L: Optional[int] = None, want_S: bool = False,
+                mean_then_pool: bool = False) -> HeadResult:
     """One (sequence, KV head): K [>=L, d], Q [G, alpha, d]."""
     lib = _load()
     K = _f32(K)
@@ -91,7 +92,7 @@ def oracle_head(K, Q, *, budget: int, alpha: int, lam: float, W: int, beta: int,
                             _ptr(A, ctypes.c_double), _ptr(I, ctypes.c_double),
                             _ptr(Sbar, ctypes.c_double), _ptr(R, ctypes.c_double),
                             _ptr(Z, ctypes.c_double), _ptr(S_raw, ctypes.c_double),
-                            _ptr(S_mod, ctypes.c_double))
+                            _ptr(S_mod, ctypes.c_double), 1 if mean_then_pool else 0)
     if r < 0:
         raise ValueError("rkv_oracle_head: bad arguments")
     return HeadResult(bool(r), idx, A, I, Sbar, R, Z, S_raw, S_mod)
@@ -109,7 +110,8 @@ class BatchResult:
 
 
 def oracle_batch(K, Q, seq_lens, *, budget: int, alpha: int, lam: float, W: int, beta: int,
-                 T: float, eps: float = 1e-8, want_scores: bool = True) -> BatchResult:
+                 T: float, eps: float = 1e-8, want_scores: bool = True,
+                 mean_then_pool: bool = False) -> BatchResult:
     """K [B, Hkv, cap, d], Q [B, Hq, alpha, d], seq_lens [B]."""
     lib = _load()
     K = _f32(K)
@@ -124,7 +126,8 @@ def oracle_batch(K, Q, seq_lens, *, budget: int, alpha: int, lam: float, W: int,
     t = lib.rkv_oracle_batch(_ptr(K, ctypes.c_float), _ptr(Q, ctypes.c_float),
                              _ptr(seq, ctypes.c_int32), B, Hkv, Hq, cap, d, alpha, budget, W, beta,
                              float(T), float(eps), float(lam), _ptr(idx, ctypes.c_int32),
-                             _ptr(scores, ctypes.c_double), _ptr(comp, ctypes.c_int32))
+                             _ptr(scores, ctypes.c_double), _ptr(comp, ctypes.c_int32),
+                             1 if mean_then_pool else 0)
     if t < 0:
         raise ValueError("rkv_oracle_batch: bad arguments (seq_len > cap, or sizes)")
     if scores is None:

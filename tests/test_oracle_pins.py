@@ -445,3 +445,31 @@ def test_handworked_three_copies_fixture():
     np.testing.assert_allclose(r.R, g["R"], rtol=1e-6)
     np.testing.assert_allclose(r.Z, g["Z"], atol=2e-7)
     np.testing.assert_array_equal(r.idx, g["idx"])
+
+
+# ----------------------------------------------------------------------------- Algorithm 1's order (variant)
+@pytest.mark.parametrize("W", [0, 1, 3, 6])
+def test_mean_then_pool_variant_against_numpy_and_eq4(W):
+    """Algorithm 1 takes the mean over the alpha query rows first and pools afterwards (read as Eq. 4's max over
+    the same window).  Pinned by a numpy recomputation from the attention weights, by a library max filter, and by
+    max-of-means <= mean-of-maxes against the Eq. 4 order; with W = 0 the two orders coincide."""
+    rng = np.random.default_rng(40 + W)
+    L, alpha = 150, 8
+    K, Q = _rand(rng, L, D), _rand(rng, 4, alpha, D) * 2.5
+    eq4 = _run(K, Q, budget=60, alpha=alpha, W=W)
+    var = _run(K, Q, budget=60, alpha=alpha, W=W, mean_then_pool=True)
+    n = L - alpha
+    np.testing.assert_array_equal(var.A, eq4.A)                       # only the last two steps differ
+    mean = var.A.mean(axis=0)
+    if W == 0:
+        brute = mean
+        np.testing.assert_allclose(var.I, eq4.I, rtol=1e-13)
+    else:
+        brute = np.array([mean[max(0, i - W):min(n, i + W)].max() for i in range(n)])
+        lib = maximum_filter1d(mean, size=2 * W, mode="constant", cval=0.0, origin=0)
+        np.testing.assert_allclose(lib, brute, rtol=0, atol=0)
+    np.testing.assert_allclose(var.I, brute, rtol=1e-13)
+    assert np.all(var.I <= eq4.I + 1e-18)
+    # the scores downstream follow: Z = lambda I - (1 - lambda) R with the same R
+    np.testing.assert_array_equal(var.R, eq4.R)
+    np.testing.assert_allclose(var.Z, 0.1 * var.I - 0.9 * var.R, rtol=1e-12, atol=1e-18)
