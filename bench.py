@@ -47,6 +47,7 @@ def parse_args():
     ap.add_argument("--beta", type=int, default=None)
     ap.add_argument("--threshold", type=float, default=None)
     ap.add_argument("--pool-w", type=int, default=None)
+    ap.add_argument("--mean-then-pool", action="store_true", help="importance in Algorithm 1's order (a variant)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--batch", type=int, default=None, help="fewer sequences than the workload names (ncu captures)")
@@ -271,6 +272,8 @@ def main():
         kw["sim_threshold"] = args.threshold
     if args.pool_w is not None:
         kw["pool_w"] = args.pool_w
+    if args.mean_then_pool:
+        kw["flags"] = rkv.RKV_FLAG_MEAN_THEN_POOL
     comp = rkv.Compressor(spec.folded_batch, spec.n_kv_heads, spec.n_q_heads, spec.budget, spec.buffer, spec.alpha,
                           spec.lam, dtype=spec.torch_dtype, device=dev, **kw)
     launches_per_step = rkv.rkv_launch_count_for(comp.desc, spec.budget, spec.buffer, spec.alpha, rkv.RKV_STAGE_ALL)
@@ -434,7 +437,8 @@ def main():
         passes, t0 = 0, time.perf_counter()
         while passes < 1 or (time.perf_counter() - t0 < 12.0 and passes < 200):      # about 12 s of CPU work
             res = oracle.oracle_batch(Kh, Qh, seq_h, budget=spec.budget, alpha=spec.alpha, lam=spec.lam, W=d.pool_w,
-                                      beta=d.beta, T=d.sim_threshold, eps=d.eps, want_scores=False)
+                                      beta=d.beta, T=d.sim_threshold, eps=d.eps, want_scores=False,
+                                      mean_then_pool=args.mean_then_pool)
             passes += 1
         dt = time.perf_counter() - t0
         cpu = {"value": passes * seqs * spec.n_kv_heads * n / dt, "unit": UNIT, "cores": res.threads, "kind": "oracle",
@@ -449,7 +453,8 @@ def main():
                        "layers": spec.layers, "batch": spec.batch, "n_kv_heads": spec.n_kv_heads,
                        "n_q_heads": spec.n_q_heads, "budget": spec.budget, "buffer": spec.buffer, "alpha": spec.alpha,
                        "lambda": spec.lam, "pool_w": comp.desc.pool_w, "beta": comp.desc.beta,
-                       "sim_threshold": comp.desc.sim_threshold,
+                       "sim_threshold": comp.desc.sim_threshold, "importance_order": "mean, then pool (Algorithm 1)"
+                       if args.mean_then_pool else "pool, then mean (Eq. 4)",
                        "l2": (f"{n_rep} input replicas of {bytes_per_replica / 2**20:.0f} MiB cycled, each used once"
                               if contiguous else "inputs restored and a 256 MiB buffer written between timed steps"),
                        "parallelism": f"{world} independent replicas, no collective"},

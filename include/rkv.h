@@ -63,6 +63,9 @@ typedef enum { RKV_BF16 = 0, RKV_F32 = 1 } rkv_dtype_t;
                                    only the tokens still short of partners against the tiles to their left);
                                    a cross-check */
 
+#define RKV_FLAG_MEAN_THEN_POOL 4u /* importance in Algorithm 1's order: mean over the alpha query rows first, then the
+                                   pooling (read as Eq. 4's max over the same window); default is Eq. 4's order */
+
 /* stage bits for rkv_compress_stages */
 #define RKV_STAGE_PREP 1u    /* key inverse norms and per-tile sums of normalised keys */
 #define RKV_STAGE_SCORES 2u  /* Eq. 2-3 pooled logits; Eq. 5 matrix + retention rule + Eq. 6 column means */

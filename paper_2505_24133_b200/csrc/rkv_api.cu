@@ -114,6 +114,7 @@ int run(const rkv_desc_t *d, void *k_cache, void *v_cache, const void *q_window,
     p.dtype = d->dtype;
     p.pool_w = d->pool_w;
     p.beta = d->beta;
+    p.mean_then_pool = (d->flags & RKV_FLAG_MEAN_THEN_POOL) ? 1 : 0;
     p.sim_threshold = d->sim_threshold;
     p.eps = d->eps;
     p.lambda = lambda;

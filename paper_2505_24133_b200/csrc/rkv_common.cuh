@@ -31,6 +31,7 @@ struct Params {
     int dtype;
     // hyper-parameters
     int pool_w, beta;
+    int mean_then_pool;             // importance in Algorithm 1's order (mean over query rows, then pooling)
     float sim_threshold, eps, lambda;
     // workspace carve-up
     float *inv_norm;     // [P][cap_pad]         r_i = 1 / (||k_i|| + eps); 0 for i >= n

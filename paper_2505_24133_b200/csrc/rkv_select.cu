@@ -107,6 +107,18 @@ __global__ void __launch_bounds__(kImpThreads) importance_kernel(Params p)
     const float inv_alpha = 1.0f / (float)p.alpha;
     for (int i = i0 + threadIdx.x; i < min(i0 + kImpTokens, n); i += kImpThreads) {
         const int lo = max(i - W, 0), hi = min(i + W - 1, n - 1);
+        if (p.mean_then_pool) {
+            // Algorithm 1's order: the mean of the alpha softmax weights at each position of the window, then the max
+            float best = 0.f;
+            for (int u = min(lo, i); u <= max(hi, i); ++u) {
+                float mean = 0.f;
+                for (int j = 0; j < p.alpha; ++j)
+                    mean += expf(logits[(size_t)j * p.cap_pad + u] - stat[2 * j]) * stat[2 * j + 1];
+                best = fmaxf(best, mean * inv_alpha);
+            }
+            p.imp[(size_t)head * p.cap_pad + i] = best;
+            continue;
+        }
         float acc = 0.f;
         for (int j = 0; j < p.alpha; ++j) {
             const float *row = logits + (size_t)j * p.cap_pad;
@@ -170,6 +182,22 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_kernel(Params p)
         __syncthreads();
         const int W = p.pool_w;
         const float inv_alpha = 1.0f / (float)p.alpha;
+        if (p.mean_then_pool) {
+            // Algorithm 1's order: the mean of the alpha softmax weights per position (kept in `row`, free until
+            // Eq. 6), then the max over the window
+            for (int i = tid; i < n; i += kSelThreads) {
+                float mean = 0.f;
+                for (int j = 0; j < p.alpha; ++j) mean += expf(lg[j * p.cap_pad + i] - stat_s[2 * j]) * stat_s[2 * j + 1];
+                row[i] = mean * inv_alpha;
+            }
+            __syncthreads();
+            for (int i = tid; i < n; i += kSelThreads) {
+                float best = row[i];
+                for (int u = max(i - W, 0); u <= min(i + W - 1, n - 1); ++u) best = fmaxf(best, row[u]);
+                imp_s[i] = best;
+            }
+            __syncthreads();                                    // `row` is about to be reused
+        } else
         for (int i = tid; i < n; i += kSelThreads) {            // Eq. 4
             const int lo = max(i - W, 0), hi = min(i + W - 1, n - 1);
             float acc = 0.f;

@@ -40,7 +40,8 @@ def run_and_check(rkv, wl, *, flags=0, W=4, beta=1, T=0.5, eps=1e-8, lam=None, c
     sel = torch.tensor(rows, device=k0.device)
     rep = check_batch(k0[sel], v0[sel], q0[sel], s0[sel], budget=spec.budget, alpha=spec.alpha, lam=lam, W=W,
                       beta=beta, T=T, eps=eps, gpu_idx=idx[sel], gpu_k=wl.k_cache[sel], gpu_v=wl.v_cache[sel],
-                      gpu_seq=wl.seq_lens[sel], gpu_scores=comp.scores[:, sel])
+                      gpu_seq=wl.seq_lens[sel], gpu_scores=comp.scores[:, sel],
+                      mean_then_pool=bool(flags & 4))
     return rep, comp
 
 
@@ -130,6 +131,16 @@ def test_ragged_lengths_and_tile_edges(rkv, flags, budget, buffer, alpha, lens):
     rep, _ = run_and_check(rkv, wl, flags=flags)
     assert rep.ok(), rep.errors
     assert rep.compressed_heads == 2 * sum(L > budget for L in lens)
+
+
+@pytest.mark.parametrize("flags", [pytest.param(4 | 1, id="simt"), pytest.param(4, id="tri")])
+@pytest.mark.parametrize("W,budget,buffer", [(0, 256, 64), (4, 256, 64), (9, 256, 64), (4, 1800, 128)])
+def test_mean_then_pool_variant(rkv, flags, W, budget, buffer):
+    """Algorithm 1's order for the importance (flag RKV_FLAG_MEAN_THEN_POOL): both forms of the select stage (one
+    kernel for small caches, three for larger ones: budget 1800 + 128 is beyond the single-kernel limit)."""
+    wl = ri.make_workload(small_spec("mtp", budget=budget, buffer=buffer), device="cuda", seed=151)
+    rep, _ = run_and_check(rkv, wl, flags=flags, W=W)
+    assert rep.ok(), rep.errors
 
 
 def test_fp32_small_shapes(rkv):
