@@ -213,6 +213,27 @@ static int ascending_int(const void *a, const void *b)
     return (x > y) - (x < y);
 }
 
+/* the k candidates with the largest score (later position first among equals),
+ * ascending, then the alpha observation positions n .. n + alpha - 1 */
+static int select_kept(const double *z, int n, int k, int alpha, int32_t *idx)
+{
+    scored_t *order = (scored_t *)malloc((size_t)n * sizeof(scored_t));
+    if (!order)
+        return -1;
+    for (int i = 0; i < n; ++i) {
+        order[i].z = z[i];
+        order[i].pos = i;
+    }
+    qsort(order, (size_t)n, sizeof(scored_t), by_score_then_recency);
+    for (int j = 0; j < k; ++j)
+        idx[j] = order[j].pos;
+    qsort(idx, (size_t)k, sizeof(int32_t), ascending_int);
+    for (int j = 0; j < alpha; ++j) /* observation tokens, always kept */
+        idx[k + j] = n + j;
+    free(order);
+    return 0;
+}
+
 /*
  * One (sequence, KV head).
  *   K      [L][d]            keys as float
@@ -307,6 +328,8 @@ void rkv_oracle_gather(const uint8_t *in, const int32_t *idx, int count,
  *   belongs to KV head q / G), seq_lens [B], idx [B][Hkv][budget].
  *   scores: optional [4][B][Hkv][cap] doubles = I, Sbar, R, Z (first n used).
  *   compressed: optional [B] flags.
+ *   variant: bit 0 as in rkv_oracle_head; bit 1 = one kept set per sequence
+ *   from the head-averaged score (Algorithm 1) instead of one per KV head.
  * Returns the number of OpenMP threads used, or -1 on bad arguments.
  */
 int rkv_oracle_batch(const float *K, const float *Q, const int32_t *seq_lens,
@@ -320,6 +343,14 @@ int rkv_oracle_batch(const float *K, const float *Q, const int32_t *seq_lens,
     const int G = Hq / Hkv;
     int bad = 0, threads = 1;
     const size_t plane = (size_t)B * Hkv * cap;
+    /* variant bit 1: Algorithm 1's aggregated selection needs every head's Z */
+    double *zown = NULL;
+    if ((variant & 2) && !scores) {
+        zown = (double *)malloc(plane * sizeof(double));
+        if (!zown)
+            return -1;
+    }
+    double *zall = scores ? scores + 3 * plane : zown;
 #ifdef _OPENMP
     threads = omp_get_max_threads();
 #pragma omp parallel for schedule(dynamic, 1)
@@ -341,7 +372,8 @@ int rkv_oracle_batch(const float *K, const float *Q, const int32_t *seq_lens,
                                 eps, lambda, idx + (size_t)p * budget, NULL,
                                 sc, sc ? sc + plane : NULL,
                                 sc ? sc + 2 * plane : NULL,
-                                sc ? sc + 3 * plane : NULL, NULL, NULL, variant);
+                                zall ? zall + (size_t)p * cap : NULL, NULL, NULL,
+                                variant);
         if (r < 0) {
 #ifdef _OPENMP
 #pragma omp atomic write
@@ -351,5 +383,31 @@ int rkv_oracle_batch(const float *K, const float *Q, const int32_t *seq_lens,
         if (compressed && h == 0)
             compressed[b] = (r == 1);
     }
+    if ((variant & 2) && !bad) {
+        /* Algorithm 1's aggregated selection (a variant, off by default): the
+         * scores of a sequence's KV heads are averaged, AggScore_i = mean_h Z_i^h,
+         * and ONE set of positions is kept for all of its heads. */
+        for (int b = 0; b < B; ++b) {
+            const int L = seq_lens[b];
+            if (L <= budget)
+                continue;
+            const int n = L - alpha, k = budget - alpha;
+            double *zbar = (double *)malloc((size_t)n * sizeof(double));
+            for (int i = 0; i < n; ++i) {
+                double acc = 0.0;
+                for (int h = 0; h < Hkv; ++h)
+                    acc += zall[((size_t)b * Hkv + h) * cap + i];
+                zbar[i] = acc / (double)Hkv;
+            }
+            int32_t *first = idx + (size_t)b * Hkv * budget;
+            if (select_kept(zbar, n, k, alpha, first) < 0)
+                bad = 1;
+            for (int h = 1; h < Hkv; ++h)
+                memcpy(first + (size_t)h * budget, first,
+                       (size_t)budget * sizeof(int32_t));
+            free(zbar);
+        }
+    }
+    free(zown);
     return bad ? -1 : threads;
 }

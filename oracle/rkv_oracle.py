@@ -111,7 +111,7 @@ class BatchResult:
 
 def oracle_batch(K, Q, seq_lens, *, budget: int, alpha: int, lam: float, W: int, beta: int,
                  T: float, eps: float = 1e-8, want_scores: bool = True,
-                 mean_then_pool: bool = False) -> BatchResult:
+                 mean_then_pool: bool = False, head_mean: bool = False) -> BatchResult:
     """K [B, Hkv, cap, d], Q [B, Hq, alpha, d], seq_lens [B]."""
     lib = _load()
     K = _f32(K)
@@ -127,7 +127,7 @@ def oracle_batch(K, Q, seq_lens, *, budget: int, alpha: int, lam: float, W: int,
                              _ptr(seq, ctypes.c_int32), B, Hkv, Hq, cap, d, alpha, budget, W, beta,
                              float(T), float(eps), float(lam), _ptr(idx, ctypes.c_int32),
                              _ptr(scores, ctypes.c_double), _ptr(comp, ctypes.c_int32),
-                             1 if mean_then_pool else 0)
+                             (1 if mean_then_pool else 0) | (2 if head_mean else 0))
     if t < 0:
         raise ValueError("rkv_oracle_batch: bad arguments (seq_len > cap, or sizes)")
     if scores is None:

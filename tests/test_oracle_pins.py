@@ -473,3 +473,32 @@ def test_mean_then_pool_variant_against_numpy_and_eq4(W):
     # the scores downstream follow: Z = lambda I - (1 - lambda) R with the same R
     np.testing.assert_array_equal(var.R, eq4.R)
     np.testing.assert_allclose(var.Z, 0.1 * var.I - 0.9 * var.R, rtol=1e-12, atol=1e-18)
+
+
+def test_head_mean_aggregated_selection_variant():
+    """Algorithm 1 averages the heads' scores and keeps ONE set of positions per sequence.  Pinned by recomputing
+    the selection from the oracle's own per-head Z with numpy (stable sort: score descending, later position first
+    among equals), by H_kv = 1 reducing to the per-head selection, and by all heads sharing the set."""
+    rng = np.random.default_rng(77)
+    B, Hkv, Hq, cap, alpha, budget = 2, 3, 6, 90, 8, 50
+    K = _rand(rng, B, Hkv, cap, D)
+    K[:, :, 40:48] = K[:, :, 8:16] + 0.05 * _rand(rng, B, Hkv, 8, D)         # some redundancy
+    Q = _rand(rng, B, Hq, alpha, D) * 2.0
+    seq = np.array([90, 77], np.int32)
+    kw = dict(budget=budget, alpha=alpha, lam=0.1, W=4, beta=1, T=0.5)
+    per = oracle.oracle_batch(K, Q, seq, **kw)
+    agg = oracle.oracle_batch(K, Q, seq, head_mean=True, **kw)
+    np.testing.assert_array_equal(agg.Z, per.Z)                               # the scores themselves do not change
+    k = budget - alpha
+    for b in range(B):
+        n = int(seq[b]) - alpha
+        zbar = per.Z[b, :, :n].mean(axis=0)
+        order = sorted(range(n), key=lambda i: (-zbar[i], -i))
+        want = np.array(sorted(order[:k]) + list(range(n, n + alpha)), np.int32)
+        for h in range(Hkv):
+            np.testing.assert_array_equal(agg.idx[b, h], want)
+    # the per-head sets do differ on this input (otherwise the pin above would not tell the variants apart)
+    assert any(not np.array_equal(per.idx[b, 0], per.idx[b, 1]) for b in range(B))
+    one = oracle.oracle_batch(K[:, :1], Q[:, :2], seq, head_mean=True, **kw)
+    ref = oracle.oracle_batch(K[:, :1], Q[:, :2], seq, **kw)
+    np.testing.assert_array_equal(one.idx, ref.idx)
