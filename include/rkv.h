@@ -66,6 +66,10 @@ typedef enum { RKV_BF16 = 0, RKV_F32 = 1 } rkv_dtype_t;
 #define RKV_FLAG_MEAN_THEN_POOL 4u /* importance in Algorithm 1's order: mean over the alpha query rows first, then the
                                    pooling (read as Eq. 4's max over the same window); default is Eq. 4's order */
 
+#define RKV_FLAG_HEAD_MEAN 8u /* Algorithm 1's aggregated selection: the joint scores of a sequence's KV heads are
+                                   averaged and ONE set of positions is kept for all of them (every head's index
+                                   list is the same); default is one set per KV head.  One more launch. */
+
 /* stage bits for rkv_compress_stages */
 #define RKV_STAGE_PREP 1u    /* key inverse norms and per-tile sums of normalised keys */
 #define RKV_STAGE_SCORES 2u  /* Eq. 2-3 pooled logits; Eq. 5 matrix + retention rule + Eq. 6 column means */

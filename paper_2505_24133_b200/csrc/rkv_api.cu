@@ -115,6 +115,7 @@ int run(const rkv_desc_t *d, void *k_cache, void *v_cache, const void *q_window,
     p.pool_w = d->pool_w;
     p.beta = d->beta;
     p.mean_then_pool = (d->flags & RKV_FLAG_MEAN_THEN_POOL) ? 1 : 0;
+    p.head_mean = (d->flags & RKV_FLAG_HEAD_MEAN) ? 1 : 0;
     p.sim_threshold = d->sim_threshold;
     p.eps = d->eps;
     p.lambda = lambda;
@@ -313,6 +314,7 @@ int rkv_launch_count(const rkv_desc_t *desc, uint32_t stage_mask)
     int c = 0;
     for (uint32_t bit = 1; bit <= RKV_STAGE_GATHER; bit <<= 1) c += (stage_mask & bit) ? 1 : 0;
     if (stage_mask & RKV_STAGE_SELECT) c += 2;      // row statistics and importance run ahead of the selection kernel
+    if (desc && (stage_mask & RKV_STAGE_SELECT) && (desc->flags & RKV_FLAG_HEAD_MEAN)) c += 1;   // per-sequence selection
     // the triangle scoring path is three kernels (pass 1, listing, pass 2) while the retention rule is on
     if (desc && (stage_mask & RKV_STAGE_SCORES) && use_tri(desc) && desc->beta > 0 && desc->sim_threshold < 1.0f) c += 2;
     return c;

@@ -31,6 +31,8 @@ struct Params {
     int dtype;
     // hyper-parameters
     int pool_w, beta;
+    int head_mean;                  // Algorithm 1's aggregated selection: one kept set per sequence from the
+                                    // head-averaged Z (select_kernel then leaves Z in `imp` and a second kernel selects)
     int mean_then_pool;             // importance in Algorithm 1's order (mean over query rows, then pooling)
     float sim_threshold, eps, lambda;
     // workspace carve-up
@@ -39,7 +41,7 @@ struct Params {
     float *head_sum;     // [P][128]             sum over all candidate rows of r_i * k_i (the tile sums added up)
     float *logits;       // [P][alpha][cap_pad]  Eq. 2-3: group-max of scaled logits
     float *row_stat;     // [P][alpha][2]        Eq. 3 per row: max logit, 1 / sum of exp(logit - max)
-    float *imp;          // [P][cap_pad]         Eq. 4: importance I
+    float *imp;          // [P][cap_pad]         Eq. 4: importance I (head_mean: overwritten with Z by select_kernel)
     float *sbar;         // [P][cap_pad]         Eq. 6 column means after the retention rule.  With `tri` set the scoring
                          //                      kernels leave column SUMS minus the removed entries (the select stage
                          //                      divides by n)

@@ -130,6 +130,110 @@ __global__ void __launch_bounds__(kImpThreads) importance_kernel(Params p)
     }
 }
 
+// Exact top-k over n order-preserving keys in shared memory (written by the caller, one owner per slot; no barrier
+// needed before the call), later position first among equal keys.  Writes the k kept positions in ascending order and
+// then the alpha observation positions n .. n+alpha-1 into `copies` index lists of `budget` entries, `budget` apart.
+__device__ __forceinline__ void radix_select_emit(const uint32_t *keys, int n, int k, int alpha, int budget,
+                                                  int32_t *out, int copies)
+{
+    __shared__ uint32_t hist[256];
+    __shared__ uint32_t sel_prefix, sel_want;
+    __shared__ uint32_t warp_tot[kSelWarps];
+    const int tid = threadIdx.x;
+    if (tid == 0) {
+        sel_prefix = 0u;
+        sel_want = (uint32_t)k;
+    }
+
+    // ---- radix select: the k-th largest key, 8 bits at a time from the top
+    for (int shift = 24; shift >= 0; shift -= 8) {
+        if (tid < 256) hist[tid] = 0u;
+        __syncthreads();
+        const uint32_t prefix = sel_prefix;
+        const uint32_t high_mask = (shift == 24) ? 0u : (0xffffffffu << (shift + 8));
+        for (int i = tid; i < n; i += kSelThreads) {
+            const uint32_t key = keys[i];
+            if ((key & high_mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+        }
+        __syncthreads();
+        if (tid < 32) {
+            // lane l owns digits 255-8l .. 248-8l (descending); find the digit holding the want-th key
+            const uint32_t want = sel_want;        // read before any lane may overwrite it below
+            uint32_t local[8], sum = 0u;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                local[e] = hist[255 - (tid * 8 + e)];
+                sum += local[e];
+            }
+            uint32_t incl = sum;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const uint32_t o = __shfl_up_sync(0xffffffffu, incl, off);
+                if (tid >= off) incl += o;
+            }
+            uint32_t run = incl - sum;             // keys in larger digits, owned by earlier lanes
+            __syncwarp();
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {          // exactly one (lane, e) holds the want-th key
+                if (run < want && want <= run + local[e]) {
+                    sel_prefix = prefix | ((uint32_t)(255 - (tid * 8 + e)) << shift);
+                    sel_want = want - run;
+                }
+                run += local[e];
+            }
+        }
+        __syncthreads();
+    }
+    const uint32_t theta = sel_prefix;   // key of the k-th largest score
+    const uint32_t need_eq = sel_want;   // how many tokens equal to theta are kept (the latest ones)
+
+    // ---- emit the kept positions in ascending order
+    const int per = (n + kSelThreads - 1) / kSelThreads;      // contiguous tokens per thread
+    const int first = tid * per, last = min(first + per, n);
+    uint32_t gt = 0u, eq = 0u;
+    for (int i = first; i < last; ++i) {
+        const uint32_t key = keys[i];
+        gt += (key > theta);
+        eq += (key == theta);
+    }
+    uint32_t packed = (gt << 16) | eq;     // n <= 8192: both counts fit 16 bits, sums never carry across
+    uint32_t incl = packed;
+    const int lane = tid & 31, warp = tid >> 5;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const uint32_t o = __shfl_up_sync(0xffffffffu, incl, off);
+        if (lane >= off) incl += o;
+    }
+    if (lane == 31) warp_tot[warp] = incl;
+    __syncthreads();
+    uint32_t wsum = lane < kSelWarps ? warp_tot[lane] : 0u, wincl = wsum;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const uint32_t o = __shfl_up_sync(0xffffffffu, wincl, off);
+        if (lane >= off) wincl += o;
+    }
+    const uint32_t total = __shfl_sync(0xffffffffu, wincl, 31);
+    const uint32_t warp_excl = __shfl_sync(0xffffffffu, wincl - wsum, warp);
+    const uint32_t excl = warp_excl + incl - packed;
+    const uint32_t total_eq = total & 0xffffu;
+    const uint32_t skip_eq = total_eq - need_eq;    // the earliest ties are the ones dropped
+    uint32_t g = excl >> 16, q = excl & 0xffffu;
+    for (int i = first; i < last; ++i) {
+        const uint32_t key = keys[i];
+        const uint32_t kept_before = g + (q > skip_eq ? q - skip_eq : 0u);
+        if (key > theta) {
+            for (int c = 0; c < copies; ++c) out[(size_t)c * budget + kept_before] = i;
+            ++g;
+        } else if (key == theta) {
+            if (q >= skip_eq)
+                for (int c = 0; c < copies; ++c) out[(size_t)c * budget + kept_before] = i;
+            ++q;
+        }
+    }
+    for (int j = tid; j < alpha; j += kSelThreads)
+        for (int c = 0; c < copies; ++c) out[(size_t)c * budget + k + j] = n + j;   // observation tokens
+}
+
 // kFused: the block first does the work of row_stats_kernel and importance_kernel for its head, with the pooled
 // logits in shared memory (small caches only: one launch instead of three, all of them latency-bound there).
 template <bool kFused>
@@ -139,9 +243,6 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_kernel(Params p)
                                                    // kFused: then [cap_pad] importance and [alpha][cap_pad] logits
     __shared__ float stat_s[2 * RKV_MAX_GROUP_ROWS];
     __shared__ float scratch[kSelWarps];
-    __shared__ uint32_t hist[256];
-    __shared__ uint32_t sel_prefix, sel_want;
-    __shared__ uint32_t warp_tot[kSelWarps];
 
     const int head = blockIdx.x;
     const int b = head / p.hkv;
@@ -241,104 +342,46 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_kernel(Params p)
             if (p.dbg_Sbar) p.dbg_Sbar[dbg + i] = sb;
             if (p.dbg_R) p.dbg_R[dbg + i] = R;
             if (p.dbg_Z) p.dbg_Z[dbg + i] = Z;
+            if (p.head_mean) p.imp[(size_t)head * p.cap_pad + i] = Z;     // slot i is read (above) and written by this thread only
             keys[i] = order_key(Z);
         }
     }
-    if (tid == 0) {
-        sel_prefix = 0u;
-        sel_want = (uint32_t)k;
-    }
+    if (p.head_mean) return;      // Z of this head is in p.imp; select_mean_kernel picks the sequence's positions
+    radix_select_emit(keys, n, k, p.alpha, p.budget, out, 1);
+}
 
-    // ---- radix select: the k-th largest key, 8 bits at a time from the top
-    for (int shift = 24; shift >= 0; shift -= 8) {
-        if (tid < 256) hist[tid] = 0u;
-        __syncthreads();
-        const uint32_t prefix = sel_prefix;
-        const uint32_t high_mask = (shift == 24) ? 0u : (0xffffffffu << (shift + 8));
-        for (int i = tid; i < n; i += kSelThreads) {
-            const uint32_t key = keys[i];
-            if ((key & high_mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
-        }
-        __syncthreads();
-        if (tid < 32) {
-            // lane l owns digits 255-8l .. 248-8l (descending); find the digit holding the want-th key
-            const uint32_t want = sel_want;        // read before any lane may overwrite it below
-            uint32_t local[8], sum = 0u;
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                local[e] = hist[255 - (tid * 8 + e)];
-                sum += local[e];
-            }
-            uint32_t incl = sum;
-#pragma unroll
-            for (int off = 1; off < 32; off <<= 1) {
-                const uint32_t o = __shfl_up_sync(0xffffffffu, incl, off);
-                if (tid >= off) incl += o;
-            }
-            uint32_t run = incl - sum;             // keys in larger digits, owned by earlier lanes
-            __syncwarp();
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {          // exactly one (lane, e) holds the want-th key
-                if (run < want && want <= run + local[e]) {
-                    sel_prefix = prefix | ((uint32_t)(255 - (tid * 8 + e)) << shift);
-                    sel_want = want - run;
-                }
-                run += local[e];
-            }
-        }
-        __syncthreads();
+// Algorithm 1's aggregated selection, one block per sequence: AggScore_i = mean over the KV heads of Z_i^h (left in
+// p.imp by select_kernel), exact top-k on it, the same index list written for every head of the sequence.
+__global__ void __launch_bounds__(kSelThreads, 2) select_mean_kernel(Params p)
+{
+    extern __shared__ float row[];
+    const int b = blockIdx.x, tid = threadIdx.x;
+    const int L = p.meta[b];
+    if (L <= p.budget) return;      // select_kernel has written the identity lists
+    const int n = L - p.alpha;
+    uint32_t *keys = reinterpret_cast<uint32_t *>(row);
+    const float *z = p.imp + (size_t)b * p.hkv * p.cap_pad;
+    const float hkv = (float)p.hkv;
+    for (int i = tid; i < n; i += kSelThreads) {
+        float acc = 0.f;
+        for (int h = 0; h < p.hkv; ++h) acc += z[(size_t)h * p.cap_pad + i];      // fixed head order
+        keys[i] = order_key(acc / hkv);
     }
-    const uint32_t theta = sel_prefix;   // key of the k-th largest score
-    const uint32_t need_eq = sel_want;   // how many tokens equal to theta are kept (the latest ones)
-
-    // ---- emit the kept positions in ascending order
-    const int per = (n + kSelThreads - 1) / kSelThreads;      // contiguous tokens per thread
-    const int first = tid * per, last = min(first + per, n);
-    uint32_t gt = 0u, eq = 0u;
-    for (int i = first; i < last; ++i) {
-        const uint32_t key = keys[i];
-        gt += (key > theta);
-        eq += (key == theta);
-    }
-    uint32_t packed = (gt << 16) | eq;     // n <= 8192: both counts fit 16 bits, sums never carry across
-    uint32_t incl = packed;
-    const int lane = tid & 31, warp = tid >> 5;
-#pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-        const uint32_t o = __shfl_up_sync(0xffffffffu, incl, off);
-        if (lane >= off) incl += o;
-    }
-    if (lane == 31) warp_tot[warp] = incl;
-    __syncthreads();
-    uint32_t wsum = lane < kSelWarps ? warp_tot[lane] : 0u, wincl = wsum;
-#pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-        const uint32_t o = __shfl_up_sync(0xffffffffu, wincl, off);
-        if (lane >= off) wincl += o;
-    }
-    const uint32_t total = __shfl_sync(0xffffffffu, wincl, 31);
-    const uint32_t warp_excl = __shfl_sync(0xffffffffu, wincl - wsum, warp);
-    const uint32_t excl = warp_excl + incl - packed;
-    const uint32_t total_eq = total & 0xffffu;
-    const uint32_t skip_eq = total_eq - need_eq;    // the earliest ties are the ones dropped
-    uint32_t g = excl >> 16, q = excl & 0xffffu;
-    for (int i = first; i < last; ++i) {
-        const uint32_t key = keys[i];
-        const uint32_t kept_before = g + (q > skip_eq ? q - skip_eq : 0u);
-        if (key > theta) {
-            out[kept_before] = i;
-            ++g;
-        } else if (key == theta) {
-            if (q >= skip_eq) out[kept_before] = i;
-            ++q;
-        }
-    }
-    for (int j = tid; j < p.alpha; j += kSelThreads) out[k + j] = n + j;   // observation tokens
+    radix_select_emit(keys, n, p.budget - p.alpha, p.alpha, p.budget, p.out_idx + (size_t)b * p.hkv * p.budget, p.hkv);
 }
 
 }  // namespace
 
 bool select_is_fused(int cap_pad, int alpha) { return (size_t)(alpha + 2) * cap_pad * sizeof(float) <= kFusedSmemLimit; }
+
+static cudaError_t launch_select_mean(const Params &p, cudaStream_t s)
+{
+    const size_t smem = (size_t)p.cap_pad * sizeof(float);
+    cudaError_t e = cudaFuncSetAttribute(select_mean_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    select_mean_kernel<<<(unsigned)p.batch, kSelThreads, smem, s>>>(p);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_select(const Params &p, cudaStream_t s)
 {
@@ -352,7 +395,8 @@ cudaError_t launch_select(const Params &p, cudaStream_t s)
             cudaSuccess)
             return e;
         select_kernel<true><<<heads, kSelThreads, smem, s>>>(p);
-        return cudaGetLastError();
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        return p.head_mean ? launch_select_mean(p, s) : cudaSuccess;
     }
     row_stats_kernel<<<heads * (unsigned)p.alpha, kStatThreads, 0, s>>>(p);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
@@ -365,7 +409,8 @@ cudaError_t launch_select(const Params &p, cudaStream_t s)
         cudaSuccess)
         return e;
     select_kernel<false><<<heads, kSelThreads, smem, s>>>(p);
-    return cudaGetLastError();
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    return p.head_mean ? launch_select_mean(p, s) : cudaSuccess;
 }
 
 }  // namespace rkv

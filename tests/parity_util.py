@@ -10,6 +10,7 @@ k-th score) are written out here:
   kept   with z_k the oracle's k-th largest Z and tau = 1e-3 |z_k|: every candidate with Z_ref > z_k + tau is
          kept, every one with Z_ref < z_k - tau is evicted, exactly k are kept, ascending, then the alpha
          observation positions
+         (head_mean: the same rule on the head-averaged Z, and one list per sequence)
   K, V   rows [0, budget) bit-identical to the oracle's gather applied to the kept positions
 """
 from __future__ import annotations
@@ -69,7 +70,7 @@ def check_batch(k_in: torch.Tensor, v_in: torch.Tensor, q_in: torch.Tensor, seq_
                 budget: int, alpha: int, lam: float, W: int, beta: int, T: float, eps: float,
                 gpu_idx: torch.Tensor, gpu_k: Optional[torch.Tensor] = None, gpu_v: Optional[torch.Tensor] = None,
                 gpu_seq: Optional[torch.Tensor] = None, gpu_scores: Optional[torch.Tensor] = None,
-                max_errors: int = 10, mean_then_pool: bool = False) -> ParityReport:
+                max_errors: int = 10, mean_then_pool: bool = False, head_mean: bool = False) -> ParityReport:
     """All tensors are for the same (sub)batch: k_in/v_in [B,H,cap,d] and q_in [B,Hq,alpha,d] BEFORE the call,
     gpu_* AFTER it.  gpu_scores is [4,B,H,cap] (I, Sbar, R, Z) or None."""
     rep = ParityReport()
@@ -78,7 +79,7 @@ def check_batch(k_in: torch.Tensor, v_in: torch.Tensor, q_in: torch.Tensor, seq_
     seq = seq_in.detach().cpu().numpy().astype(np.int32)
     B, H, cap, d = K.shape
     res = oracle.oracle_batch(K, Q, seq, budget=budget, alpha=alpha, lam=lam, W=W, beta=beta, T=T, eps=eps,
-                              mean_then_pool=mean_then_pool)
+                              mean_then_pool=mean_then_pool, head_mean=head_mean)
     gidx = gpu_idx.detach().cpu().numpy()
     k_raw_in, v_raw_in = raw_rows(k_in), raw_rows(v_in)
     k_raw_out = raw_rows(gpu_k) if gpu_k is not None else None
@@ -152,6 +153,12 @@ def check_batch(k_in: torch.Tensor, v_in: torch.Tensor, q_in: torch.Tensor, seq_
                 err(f"{tag} index list not ascending / observation tail wrong: {gi[:4]}..{gi[-alpha - 1:]}")
                 continue
             ref_set = res.idx[b, h, :kk]
+            if head_mean:
+                # Algorithm 1's aggregated selection: the kept set is judged on the head-averaged score, and every
+                # head of the sequence carries the same list
+                Zr = res.Z[b, :, :n].mean(axis=0)
+                if not np.array_equal(gi, gidx[b, 0]):
+                    err(f"{tag} index list differs from head 0's although one set per sequence was asked for")
             z_k = Zr[ref_set].min()
             tau = 1e-3 * abs(z_k)
             must_keep = np.nonzero(Zr > z_k + tau)[0]

@@ -117,6 +117,7 @@ def test_rkv_compress_needs_a_current_descriptor(rkv):
     assert rkv.rkv_launch_count_for(_desc(rkv), 1024, 128, 8, rkv.RKV_STAGE_ALL) == 6
     assert rkv.rkv_launch_count_for(_desc(rkv), 64, 32, 8, rkv.RKV_STAGE_ALL) == 4          # one key tile: no second pass
     assert rkv.rkv_launch_count_for(_desc(rkv), 8, 128, 8, rkv.RKV_STAGE_ALL) == 0           # invalid sizes
+    assert rkv.rkv_launch_count_for(_desc(rkv, flags=rkv.RKV_FLAG_HEAD_MEAN), 1024, 128, 8, rkv.RKV_STAGE_ALL) == 7
 
 
 def test_product_package_does_not_touch_the_oracle():

@@ -41,7 +41,7 @@ def run_and_check(rkv, wl, *, flags=0, W=4, beta=1, T=0.5, eps=1e-8, lam=None, c
     rep = check_batch(k0[sel], v0[sel], q0[sel], s0[sel], budget=spec.budget, alpha=spec.alpha, lam=lam, W=W,
                       beta=beta, T=T, eps=eps, gpu_idx=idx[sel], gpu_k=wl.k_cache[sel], gpu_v=wl.v_cache[sel],
                       gpu_seq=wl.seq_lens[sel], gpu_scores=comp.scores[:, sel],
-                      mean_then_pool=bool(flags & 4))
+                      mean_then_pool=bool(flags & 4), head_mean=bool(flags & 8))
     return rep, comp
 
 
@@ -141,6 +141,22 @@ def test_mean_then_pool_variant(rkv, flags, W, budget, buffer):
     wl = ri.make_workload(small_spec("mtp", budget=budget, buffer=buffer), device="cuda", seed=151)
     rep, _ = run_and_check(rkv, wl, flags=flags, W=W)
     assert rep.ok(), rep.errors
+
+
+@pytest.mark.parametrize("flags", [pytest.param(8 | 1, id="simt"), pytest.param(8, id="tri"),
+                                   pytest.param(8 | 4, id="tri+mean_then_pool")])
+@pytest.mark.parametrize("hkv,hq,budget,buffer", [(2, 8, 256, 64), (4, 8, 300, 75), (3, 6, 1800, 128)])
+def test_head_mean_variant(rkv, flags, hkv, hq, budget, buffer):
+    """Algorithm 1's aggregated selection (flag RKV_FLAG_HEAD_MEAN): one kept set per sequence from the head-averaged
+    score, after both forms of the select stage; ragged lengths with one sequence left alone by the guard."""
+    spec = small_spec("hm", batch=3, hkv=hkv, hq=hq, budget=budget, buffer=buffer)
+    lens = torch.tensor([spec.cap, budget, budget + (buffer + 1) // 2])
+    wl = ri.make_workload(spec, device="cuda", seed=171, seq_lens=lens)
+    rep, comp = run_and_check(rkv, wl, flags=flags)
+    assert rep.ok(), rep.errors
+    assert rep.compressed_heads == 2 * hkv
+    assert rkv.rkv_launch_count_for(comp.desc, budget, buffer, spec.alpha, rkv.RKV_STAGE_SELECT) == \
+        (2 if budget < 1000 else 4)
 
 
 def test_fp32_small_shapes(rkv):
