@@ -32,8 +32,9 @@ UNIT = "tokens/s"
 # under profiles/: {workload: {kernel: bytes}}
 NCU_TRAFFIC = {
     # profiles/all_kernels_llama8b_b1.md (cold caches: the scoring passes read K from DRAM there)
-    "llama8b_b1": {"prep": 76.98e6, "scores_pass1": 85.13e6, "scores_list": 1.19e6, "scores_pass2": 72.39e6,
-                   "row_stats": 9.45e6, "importance": 9.46e6, "select": 2.39e6, "gather": 212.08e6},
+    # (the select stage is one kernel at this size: no row_stats / importance launches)
+    "llama8b_b1": {"prep": 76.72e6, "scores_pass1": 85.24e6, "scores_list": 1.19e6, "scores_pass2": 72.57e6,
+                   "select": 10.67e6, "gather": 212.71e6},
 }
 
 
