@@ -180,13 +180,13 @@ RKV_API int rkv_compress_host(const rkv_desc_t *desc, void *host_k_cache, void *
  * buffer fills -- an inference server whose memory pool already owns all of the GPU's memory and hands out
  * nothing beyond KV blocks, a plug-in running inside another framework's callback where allocation is
  * forbidden, a real-time loop that must not take the driver's allocation lock.  For them the scratch lives in
- * a fixed array inside the library's device image, RKV_STATIC_SCRATCH_BYTES (24 MiB) large.  Every GPU that
+ * a fixed array inside the library's device image, RKV_STATIC_SCRATCH_BYTES (32 MiB) large.  Every GPU that
  * loads the library carries that array until the process ends, used or not.
  *
  * Arguments, layouts, results and error codes are those of rkv_compress_ex; desc->workspace and
  * desc->workspace_bytes are ignored.  In addition:
  *   - a shape whose rkv_workspace_bytes() exceeds RKV_STATIC_SCRATCH_BYTES is refused with RKV_ERR_WORKSPACE
- *     before anything is launched (rkv_workspace_bytes() tells what a shape needs).  24 MiB covers, for example,
+ *     before anything is launched (rkv_workspace_bytes() tells what a shape needs).  32 MiB covers, for example,
  *     256 head-problems at budget 1024 + buffer 128 (all 32 layers of an 8-KV-head model, batch 1);
  *     larger batches are split into several calls over sub-ranges of the batch dimension, one after the other.
  *   - the call makes no cudaMalloc / cudaFree and calls no allocating library routine.
@@ -199,7 +199,7 @@ RKV_API int rkv_compress_host(const rkv_desc_t *desc, void *host_k_cache, void *
  *     it and corrupt each other's scores.  Serialise them, or give one of them a workspace of its own through
  *     rkv_compress_ex.
  */
-#define RKV_STATIC_SCRATCH_BYTES (24u << 20)
+#define RKV_STATIC_SCRATCH_BYTES (32u << 20)
 RKV_API int rkv_compress_static(const rkv_desc_t *desc, void *k_cache, void *v_cache, const void *q_window,
                         int32_t *seq_lens, int32_t budget, int32_t buffer, int32_t alpha, float lambda,
                         int32_t *out_idx, void *stream);

@@ -145,12 +145,12 @@ def rkv_compress_host(desc, host_k, host_v, host_q, host_seq_lens, budget, buffe
                                    _stream(stream))
 
 
-RKV_STATIC_SCRATCH_BYTES = 24 << 20
+RKV_STATIC_SCRATCH_BYTES = 32 << 20
 
 
 def rkv_compress_static(desc, k_cache, v_cache, q_window, seq_lens, budget, buffer, alpha, lam, out_idx,
                         stream=None) -> int:
-    """rkv_compress_ex with the scratch taken from the library's built-in 24 MiB device array, for callers that
+    """rkv_compress_ex with the scratch taken from the library's built-in 32 MiB device array, for callers that
     cannot allocate a workspace; desc.workspace is ignored.  Calls on one device share that array: do not let
     two of them overlap on the GPU."""
     return lib().rkv_compress_static(ctypes.byref(desc), _ptr(k_cache), _ptr(v_cache), _ptr(q_window),

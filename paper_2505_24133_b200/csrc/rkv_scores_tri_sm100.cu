@@ -68,10 +68,13 @@ enum {
     kBarREmpty = kBarRFull + 2,             // [2] ... and no longer read (8 epilogue warps)
     kNumBars = kBarREmpty + 2
 };
-// Pass 2 keeps one pair of resident tiles (its items are long) and uses the room of the second pair for the r_j of
-// the whole head, double-buffered across items, so its epilogue reads them in place.
-constexpr int kOffRHead = kOffA + 2 * kTileBytes;          // 2 x RKV_MAX_CAP floats
-static_assert(2 * RKV_MAX_CAP * 4 <= 2 * kTileBytes, "the head's r_j must fit the second resident pair");
+// Pass 2 keeps one pair of resident tiles (its items are long) and uses the room of the second pair for the extra
+// K = 16 slices of its operands: 128 rows x 32 bytes each (32-byte swizzle), one per resident tile and one per stage
+// of the ring.
+constexpr int kSliceBytes = kTile * 32;
+constexpr int kOffAugA = kOffA + 2 * kTileBytes;           // 2 slices, beside the resident tiles
+constexpr int kOffAugB = kOffAugA + 2 * kSliceBytes;       // kStagesB slices, beside the streamed tiles
+static_assert((2 + kStagesB) * kSliceBytes <= 2 * kTileBytes, "the slices must fit the second resident pair");
 constexpr int kOffItems = kOffBar + kNumBars * 8;          // kItemSlots x int4
 constexpr int kOffMisc = kOffItems + kItemSlots * 16;      // tmem base, abort flag, bail flag
 constexpr int kOffRj = kOffMisc + 16;                      // pass 1: [2 items][kPass1Depth * 128] r_j of the streamed tiles
@@ -128,7 +131,8 @@ struct Bars {
 template <bool kPass2>
 __global__ void __launch_bounds__(kThreads, 1)
 scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_q,
-                        const __grid_constant__ CUtensorMap map_hs, int items_per_head,
+                        const __grid_constant__ CUtensorMap map_hs, const __grid_constant__ CUtensorMap map_ns,
+                        int items_per_head,
                         unsigned long long total_items_host, int q_rows_pad)
 {
     extern __shared__ uint8_t smem_raw[];
@@ -225,17 +229,6 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
                 items[qs] = desc;
                 mbar_arrive(bar.at(kBarQFull + qs));
 
-                if (kPass2) {
-                    // r_j of the tiles this item streams (0 .. first_tile), straight into shared memory
-                    const uint32_t rb = k_item & 1;
-                    if (!mbar_wait(bar.at(kBarREmpty + rb), ((k_item >> 1) & 1) ^ 1, abort_flag, p.status)) break;
-                    const uint32_t bytes = (uint32_t)(first_tile + 1) * kTile * 4u;
-                    mbar_expect_tx(bar.at(kBarRFull + rb), bytes);
-                    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                                 ::"r"(sbase + kOffRHead + rb * RKV_MAX_CAP * 4), "l"(p.inv_norm + (size_t)head * p.cap_pad),
-                                   "r"(bytes), "r"(bar.at(kBarRFull + rb))
-                                 : "memory");
-                }
                 if (!kPass2 && rule_on) {
                     // r_j of the key tiles this item streams (first_tile down to first_tile + 2 - n_iter)
                     const uint32_t rb = k_item & 1;
@@ -281,9 +274,12 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
                     } else {
                         const int jt = first_tile - (kPass2 ? it : it - 1);
                         const int y = key_row_base + jt * kTile;
-                        mbar_expect_tx(bar.at(kBarBFull + s), kTileBytes);
+                        mbar_expect_tx(bar.at(kBarBFull + s), kTileBytes + (kPass2 ? kSliceBytes : 0));
                         tma_load_2d(dst, &map_k, 0, y, bar.at(kBarBFull + s));
                         tma_load_2d(dst + kHalfBytes, &map_k, 64, y, bar.at(kBarBFull + s));
+                        if (kPass2)     // the tile's extra slice: the norms of its keys in three bf16 parts
+                            tma_load_2d(sbase + kOffAugB + s * kSliceBytes, &map_ns, 0, head * p.cap_pad + jt * kTile,
+                                        bar.at(kBarBFull + s));
                     }
                     ++bcount;
                 }
@@ -346,6 +342,8 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
                         const uint32_t resident = sbase + kOffA + (ab * 2 + m) * kTileBytes;
                         const uint32_t d_tmem = tmem_base + a * 256 + m * 128;
                         umma_tile_k128(d_tmem, resident, stage, is_q ? idesc_q : idesc_k);
+                        if (kPass2)     // ... - (T / r_i) (||k_j|| + eps): the accumulator's sign is the threshold test
+                            umma_k16_sw32(d_tmem, sbase + kOffAugA + m * kSliceBytes, sbase + kOffAugB + s * kSliceBytes, idesc_k);
                         umma_commit(bar.at(kBarAccFull + a * 2 + m));
                         ++cnt[m];
                         if (!is_q) ++tiles_done;
@@ -432,6 +430,23 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
                             *reinterpret_cast<uint4 *>(tile + hb * kHalfBytes + lrow * 128 + ((c ^ (lrow & 7)) << 4)) = v;
                         }
                     }
+                    {
+                        // the row's extra slice: -T / r_i in three bf16 parts as (-t1, -t1, -t1, -t2, -t2, -t3, 0 ...),
+                        // which meets (n1, n2, n3, n1, n2, n1, 0 ...) of a key; 32-byte rows, 32-byte swizzle
+                        float rest = (row_ok && ri > 0.f) ? -__fdiv_rn(p.sim_threshold, ri) : 0.f;
+                        uint32_t part[3];
+#pragma unroll
+                        for (int c = 0; c < 3; ++c) {
+                            const __nv_bfloat16 h16 = __float2bfloat16_rn(rest);
+                            part[c] = (uint32_t)__bfloat16_as_ushort(h16);
+                            rest -= __bfloat162float(h16);
+                        }
+                        uint8_t *slice = smem + kOffAugA + m * kSliceBytes + lrow * 32;
+                        const int sw = (lrow >> 2) & 1;
+                        *reinterpret_cast<uint4 *>(slice + (sw << 4)) =
+                            make_uint4(part[0] | (part[0] << 16), part[0] | (part[1] << 16), part[1] | (part[2] << 16), 0u);
+                        *reinterpret_cast<uint4 *>(slice + ((sw ^ 1) << 4)) = make_uint4(0u, 0u, 0u, 0u);
+                    }
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> tensor-core reads
                 }
                 __syncwarp();
@@ -440,7 +455,7 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
 
             const bool scan = active && (kPass2 || rule_on);
             // r_j of the first key tile of the scan: loaded now, staged in shared memory when the tile is drained
-            const bool has_r = kPass2 || rule_on;
+            const bool has_r = !kPass2 && rule_on;
             if (has_r) {        // every warp waits for the item's r_j, and hands them back at the item's end
                 const bool r_ok = mbar_wait(bar.at(kBarRFull + (k_item & 1)), (k_item >> 1) & 1, abort_flag, p.status);
                 item_ok = item_ok && r_ok;
@@ -506,11 +521,16 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
             }
 
             float removed = 0.f;
+            // pass 2: how many partners were found; with beta = 1 the one partner's position and accumulator value
+            int nhit = 0, hit_j = -1;
+            float hit_h = 0.f;
             if (scan) {
                 // ---- key tiles, last to first; their r_j lie in shared memory
                 const float thr = (row_ok && ri > 0.f) ? __fdiv_rn(p.sim_threshold, ri) : kInf;   // g r_j vs T / r_i
                 // pass 2: the whole head from tile 0; pass 1: the item's tiles from its lowest one (that of row tile 0)
-                const float *r_base = kPass2 ? reinterpret_cast<const float *>(smem + kOffRHead) + (k_item & 1) * RKV_MAX_CAP
+                // pass 1: the r_j of the item's tiles in shared memory; pass 2: the head's, in global memory (read for
+                // the chunks with partners only)
+                const float *r_base = kPass2 ? inv_norm
                                              : reinterpret_cast<const float *>(smem + kOffRj) + (k_item & 1) * kPass1Depth * kTile -
                                                    (size_t)max(2 * d.y, first_tile + 1 - kPass1Depth) * kTile;
                 bool ok = item_ok;
@@ -532,11 +552,32 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
                         for (int ch = 3; ch >= 0; --ch) {
                             uint32_t g[32];
                             tmem_ld32(base + ch * 32, g);
+                            float v[32];
+                            uint32_t hits = 0u;
+                            if (kPass2) {
+                                // The accumulator holds h = k_i . k_j - (T / r_i) (||k_j|| + eps): S[j][i] > T exactly
+                                // when h > 0, so the screening is a maximum and a sign test, with nothing to load
+                                // per column (the loads of the r_j were what this epilogue's time went into: every
+                                // byte a thread receives, from TMEM or as a shared-memory broadcast, passes through
+                                // the same return path).  The listed tokens rarely have a partner in a given chunk.
+                                tmem_wait32(g);
+#pragma unroll
+                                for (int c = 0; c < 32; ++c) v[c] = __uint_as_float(g[c]);
+                                float m0 = 0.f, m1 = 0.f;
+#pragma unroll
+                                for (int c = 0; c < 32; c += 4) {
+                                    m0 = max3(m0, v[c], v[c + 1]);
+                                    m1 = max3(m1, v[c + 2], v[c + 3]);
+                                }
+                                const float cut = thr_row < kInf ? 0.f : kInf;
+                                if (!__any_sync(0xffffffffu, fmaxf(m0, m1) > cut)) continue;
+#pragma unroll
+                                for (int c = 0; c < 32; ++c) hits |= (v[c] > cut) ? (1u << c) : 0u;
+                            } else {
                             float4 R[8];
 #pragma unroll
                             for (int q = 0; q < 8; ++q) R[q] = rj4[ch * 8 + q];
                             tmem_wait32(g);
-                            float v[32];
 #pragma unroll
                             for (int q = 0; q < 8; ++q) {        // packed multiplies: two products per instruction
                                 const float2 p0 = __fmul2_rn(make_float2(__uint_as_float(g[4 * q]), __uint_as_float(g[4 * q + 1])),
@@ -548,22 +589,12 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
                                 v[4 * q + 2] = p1.x;
                                 v[4 * q + 3] = p1.y;
                             }
-                            if (kPass2) {
-                                // screening: the listed tokens rarely have a partner in a given chunk
-                                float m0 = 0.f, m1 = 0.f;
-#pragma unroll
-                                for (int c = 0; c < 32; c += 4) {
-                                    m0 = max3(m0, v[c], v[c + 1]);
-                                    m1 = max3(m1, v[c + 2], v[c + 3]);
-                                }
-                                if (!__any_sync(0xffffffffu, fmaxf(m0, m1) > thr_row)) continue;
-                            }   // (pass 1 meets every token's first partners here: it goes straight to the mask)
                             // some token of the warp has partners in this chunk: a bit mask of the entries above the
                             // threshold (no entry depends on another), cut down to the highest positions if they are
                             // more than the token still lacks, then their sum
-                            uint32_t hits = 0u;
 #pragma unroll
                             for (int c = 0; c < 32; ++c) hits |= (v[c] > thr_row) ? (1u << c) : 0u;
+                            }
                             const unsigned own = (unsigned)(i - (jbase + ch * 32));           // zero diagonal (Eq. 5)
                             if (own < 32u) hits &= ~(1u << own);
                             if (p.beta == 1) {
@@ -578,7 +609,12 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
 #pragma unroll
                                     for (int c = 0; c < 4; ++c) t4[c] = (top & 4) ? t8[4 + c] : t8[c];
                                     const float u0 = (top & 2) ? t4[2] : t4[0], u1 = (top & 2) ? t4[3] : t4[1];
-                                    removed += (top & 1) ? u1 : u0;
+                                    if (kPass2) {      // its r_j is fetched once, at the item's end
+                                        hit_h = (top & 1) ? u1 : u0;
+                                        hit_j = jbase + ch * 32 + top;
+                                    } else {
+                                        removed += (top & 1) ? u1 : u0;
+                                    }
                                     left = 0;
                                     thr_row = kInf;
                                 }
@@ -586,6 +622,18 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
                             }
                             int taken = __popc(hits);
                             for (; taken > left; --taken) hits &= hits - 1u;                   // drop the lowest positions
+                            if (kPass2) {
+                                // S = T + h r_i r_j per partner: the chunk's r_j, for once, from global memory
+                                nhit += taken;
+#pragma unroll
+                                for (int q = 0; q < 8; ++q) {
+                                    const float4 R = __ldg(rj4 + ch * 8 + q);
+                                    v[4 * q] *= R.x;
+                                    v[4 * q + 1] *= R.y;
+                                    v[4 * q + 2] *= R.z;
+                                    v[4 * q + 3] *= R.w;
+                                }
+                            }
                             float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll
                             for (int c = 0; c < 32; c += 4) {
@@ -620,7 +668,12 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
                     *out = total - removed * ri;
                     p.left[(size_t)head * p.cap_pad + i] = rule_on ? left : 0;
                 } else {
-                    *out -= removed * ri;
+                    // S = T + h r_i r_j for every partner found here
+                    if (p.beta == 1 && hit_j >= 0) {
+                        removed = hit_h * __ldg(inv_norm + hit_j);
+                        nhit = 1;
+                    }
+                    *out -= (float)nhit * p.sim_threshold + removed * ri;
                 }
             }
             ++k_item;
@@ -693,10 +746,11 @@ cudaError_t launch_scores_tri_sm100(const Params &p, cudaStream_t s)
 {
     const int q_rows = p.group * p.alpha;
     const int q_rows_pad = (q_rows + 15) / 16 * 16;
-    CUtensorMap map_k, map_q, map_hs;
+    CUtensorMap map_k, map_q, map_hs, map_ns;
     if (!make_map(&map_k, p.k_cache, (uint64_t)p.batch * p.hkv * p.cap, kTile) ||
         !make_map(&map_q, p.q_window, (uint64_t)p.batch * p.hq * p.alpha, (uint32_t)q_rows_pad) ||
-        !make_map(&map_hs, p.head_sum_bf16, (uint64_t)p.batch * p.hkv * 16, 16u))
+        !make_map(&map_hs, p.head_sum_bf16, (uint64_t)p.batch * p.hkv * 16, 16u) ||
+        !make_map_k16(&map_ns, p.norm_split, (uint64_t)p.batch * p.hkv * p.cap_pad))
         return cudaErrorInvalidValue;
     cudaError_t e;
     if ((e = cudaFuncSetAttribute(scores_tri_sm100_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -711,7 +765,7 @@ cudaError_t launch_scores_tri_sm100(const Params &p, cudaStream_t s)
     const int items_per_head = (p.tiles + 1) / 2;
     const unsigned long long total_items = (unsigned long long)items_per_head * (unsigned long long)heads;
     const unsigned grid1 = (unsigned)(total_items < (unsigned long long)sms ? total_items : (unsigned long long)sms);
-    scores_tri_sm100_kernel<false><<<grid1, kThreads, kSmemBytes, s>>>(p, map_k, map_q, map_hs, items_per_head,
+    scores_tri_sm100_kernel<false><<<grid1, kThreads, kSmemBytes, s>>>(p, map_k, map_q, map_hs, map_ns, items_per_head,
                                                                        total_items, q_rows_pad);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     if ((e = mark_kernel(p, 0, s)) != cudaSuccess) return e;
@@ -722,7 +776,7 @@ cudaError_t launch_scores_tri_sm100(const Params &p, cudaStream_t s)
     if ((e = mark_kernel(p, 1, s)) != cudaSuccess) return e;
     const unsigned long long max_items2 = (unsigned long long)heads * (unsigned long long)(p.cap_pad / kRowsPerItem + 1);
     const unsigned grid2 = (unsigned)(max_items2 < (unsigned long long)sms ? max_items2 : (unsigned long long)sms);
-    scores_tri_sm100_kernel<true><<<grid2, kThreads, kSmemBytes, s>>>(p, map_k, map_q, map_hs, 0, 0ull, q_rows_pad);
+    scores_tri_sm100_kernel<true><<<grid2, kThreads, kSmemBytes, s>>>(p, map_k, map_q, map_hs, map_ns, 0, 0ull, q_rows_pad);
     return cudaGetLastError();
 }
 

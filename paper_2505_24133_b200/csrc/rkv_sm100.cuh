@@ -123,6 +123,22 @@ __device__ __forceinline__ void umma_tile_k128(uint32_t d_tmem, uint32_t a_addr,
         ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc)
         : "memory");
 }
+// One more K = 16 step onto the accumulator at d_tmem: both operands are 128 rows x 16 bf16 (32-byte rows, 32-byte
+// swizzle, 8-row groups 256 bytes apart, 256-byte aligned).
+__device__ __forceinline__ void umma_k16_sw32(uint32_t d_tmem, uint32_t a_addr, uint32_t b_addr, uint32_t idesc)
+{
+    const uint32_t a_lo = ((a_addr & 0x3FFFFu) >> 4) | (1u << 16);
+    const uint32_t b_lo = ((b_addr & 0x3FFFFu) >> 4) | (1u << 16);
+    const uint32_t hi = (256u >> 4) | (1u << 14) | (6u << 29);       // stride 256 B, descriptor version, 32-byte swizzle
+    asm volatile(
+        "{\n\t.reg .pred p1;\n\t.reg .b64 da, db;\n\t"
+        "setp.eq.u32 p1, %3, %3;\n\t"
+        "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p1;\n\t"
+        "}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc)
+        : "memory");
+}
 __device__ __forceinline__ void umma_commit(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -186,6 +202,20 @@ inline bool make_map(CUtensorMap *map, const void *base, uint64_t rows, uint32_t
     const cuuint32_t estr[2] = {1u, 1u};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// 2-D bf16 view [rows][16] (32-byte rows), boxes of 128 rows, 32-byte swizzle: the extra K = 16 slices of key rows.
+inline bool make_map_k16(CUtensorMap *map, const void *base, uint64_t rows)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {16u, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {32u};
+    const cuuint32_t box[2] = {16u, (cuuint32_t)kTile};
+    const cuuint32_t estr[2] = {1u, 1u};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 

@@ -2,7 +2,7 @@
 
 Some users of this library are not allowed to call cudaMalloc when the decode buffer fills: a serving engine
 whose block pool already owns the whole GPU, code running inside another framework's callback, a latency-bound
-loop that must stay off the driver's allocation lock.  rkv_compress_static serves them from a 24 MiB scratch
+loop that must stay off the driver's allocation lock.  rkv_compress_static serves them from a 32 MiB scratch
 array that is part of the library itself.  This file checks, through the C ABI, that it gives exactly what
 rkv_compress_ex gives with a caller-allocated workspace -- on two calls in a row, because the array keeps the
 first call's contents and the second must not be disturbed by them.
