@@ -29,8 +29,8 @@
 //
 // Items are handed out by a global ticket counter, longest first within a head, so neighbouring blocks work on
 // the same head while its keys are in L2.
-// Warp roles (320 threads): warp 0 = ticket + TMA producer, warp 1 = MMA issuer and TMEM owner, warps 2..9 =
-// epilogue (warp w may touch TMEM lanes 32 (w % 4) .. +31; warps 2-5 serve row tile 0, warps 6-9 row tile 1).
+// Warp roles (352 threads): warp 0 = ticket + TMA producer, warp 1 = MMA issuer of row tile 0 and TMEM owner,
+// warp 10 = MMA issuer of row tile 1, warps 2..9 = epilogue (warp w may touch TMEM lanes 32 (w % 4) .. +31; warps 2-5 serve row tile 0, warps 6-9 row tile 1).
 // TMEM: four 128-column fp32 accumulators, two per row tile, so the tensor pipe fills one while the epilogue
 // drains the other.  Every wait on an mbarrier is bounded; on expiry the block records RKV_ERR_TIMEOUT, stops
 // issuing work and leaves through the common exit that frees TMEM.  No TMA multicast and no cluster launch.
@@ -42,7 +42,7 @@ namespace {
 
 using namespace sm100;
 
-constexpr int kThreads = 320;
+constexpr int kThreads = 352;                    // 11 warps: producer, 2 MMA issuers (warps 1 and 10), 8 epilogue
 constexpr int kStagesB = 3;                      // ring depth of streamed tiles
 constexpr int kItemSlots = 4;                    // ring depth of item descriptors
 constexpr int kHalfBytes = kTile * 64 * 2;       // one TMA box: 128 rows x 64 bf16 (128-byte swizzled rows)
@@ -57,7 +57,7 @@ constexpr int kOffB = kOffA + 2 * 2 * kTileBytes;          // kStagesB streamed 
 constexpr int kOffBar = kOffB + kStagesB * kTileBytes;     // mbarriers
 enum {
     kBarQFull = 0,                          // [kItemSlots] item descriptor written
-    kBarQEmpty = kBarQFull + kItemSlots,    // [kItemSlots] read by the MMA thread and the 8 epilogue warps
+    kBarQEmpty = kBarQFull + kItemSlots,    // [kItemSlots] read by the 2 MMA threads and the 8 epilogue warps
     kBarAFull = kBarQEmpty + kItemSlots,    // [2] resident tiles in place
     kBarAEmpty = kBarAFull + 2,             // [2] resident tiles no longer read
     kBarBFull = kBarAEmpty + 2,             // [kStagesB]
@@ -161,16 +161,16 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
     if (threadIdx.x == 0) {
         for (int s = 0; s < kItemSlots; ++s) {
             mbar_init(bar.at(kBarQFull + s), 1);
-            mbar_init(bar.at(kBarQEmpty + s), 9);
+            mbar_init(bar.at(kBarQEmpty + s), 10);
         }
         for (int s = 0; s < 2; ++s) {
             // pass 1: TMA fills the resident tiles; pass 2: the 8 epilogue warps do; the MMA thread reads them
             mbar_init(bar.at(kBarAFull + s), kPass2 ? 8 : 1);
-            mbar_init(bar.at(kBarAEmpty + s), 1);
+            mbar_init(bar.at(kBarAEmpty + s), 2);              // both MMA issuers
         }
         for (int s = 0; s < kStagesB; ++s) {
             mbar_init(bar.at(kBarBFull + s), 1);
-            mbar_init(bar.at(kBarBEmpty + s), 1);
+            mbar_init(bar.at(kBarBEmpty + s), 2);              // both MMA issuers
         }
         for (int s = 0; s < 4; ++s) {
             mbar_init(bar.at(kBarAccFull + s), 1);
@@ -295,11 +295,17 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
             }
         }
         __syncwarp();
-    } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
+    } else if (warp == 1 || warp == 10) {
+        // ------------------------------------------------------------------ MMA issuers
+        // One thread per row tile of the item (warp 1: row tile 0, warp 10: row tile 1).  With a single issuer the
+        // tensor pipe ran dry between tiles while the thread went through its barrier waits; two threads keep each
+        // other's products queued.  Both wait for every stage and every item (which keeps either from running a
+        // whole barrier phase ahead) and both release them: by a commit after products of their own, by a plain
+        // arrival otherwise.
         if (lane == 0) {
+            const int m = warp == 1 ? 0 : 1;
             const uint32_t idesc_k = instr_desc(kTile, kTile), idesc_q = instr_desc(kTile, q_rows_pad + 16);
-            uint32_t k_item = 0, bcount = 0, cnt[2] = {0u, 0u};
+            uint32_t k_item = 0, bcount = 0, cnt = 0;
             bool ok = true;
             while (ok) {
                 const uint32_t qs = k_item % kItemSlots;
@@ -319,10 +325,12 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
                     n_iter = d.w + 1;
                     skip_it = -1;
                 }
+                const bool mine = m < num_m;
                 const uint32_t ab = kPass2 ? 0u : (k_item & 1);                          // pass 2: one pair of tiles
                 const uint32_t a_par = kPass2 ? (k_item & 1) : ((k_item >> 1) & 1);
                 if (!mbar_wait(bar.at(kBarAFull + ab), a_par, abort_flag, p.status)) break;
                 if (kPass2) asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t resident = sbase + kOffA + (ab * 2 + m) * kTileBytes;
                 for (int it = 0; it < n_iter; ++it) {
                     const uint32_t s = bcount % kStagesB;
                     if (!mbar_wait(bar.at(kBarBFull + s), (bcount / kStagesB) & 1, abort_flag, p.status)) {
@@ -331,29 +339,29 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
                     }
                     const uint32_t stage = sbase + kOffB + s * kTileBytes;
                     const bool is_q = !kPass2 && it == 0;
-                    for (int m = 0; m < num_m; ++m) {
-                        if (m == 1 && it == skip_it && it > 0) continue;
-                        const uint32_t a = cnt[m] & 1;
-                        if (!mbar_wait(bar.at(kBarAccEmpty + a * 2 + m), ((cnt[m] >> 1) & 1) ^ 1, abort_flag, p.status)) {
+                    if (mine && !(m == 1 && it == skip_it && it > 0)) {
+                        const uint32_t a = cnt & 1;
+                        if (!mbar_wait(bar.at(kBarAccEmpty + a * 2 + m), ((cnt >> 1) & 1) ^ 1, abort_flag, p.status)) {
                             ok = false;
                             break;
                         }
                         tc_fence_after();
-                        const uint32_t resident = sbase + kOffA + (ab * 2 + m) * kTileBytes;
                         const uint32_t d_tmem = tmem_base + a * 256 + m * 128;
                         umma_tile_k128(d_tmem, resident, stage, is_q ? idesc_q : idesc_k);
                         if (kPass2)     // ... - (T / r_i) (||k_j|| + eps): the accumulator's sign is the threshold test
                             umma_k16_sw32(d_tmem, sbase + kOffAugA + m * kSliceBytes, sbase + kOffAugB + s * kSliceBytes, idesc_k);
                         umma_commit(bar.at(kBarAccFull + a * 2 + m));
-                        ++cnt[m];
+                        ++cnt;
                         if (!is_q) ++tiles_done;
+                        umma_commit(bar.at(kBarBEmpty + s));      // the stage may be refilled once these products have read it
+                    } else {
+                        mbar_arrive(bar.at(kBarBEmpty + s));
                     }
-                    if (!ok) break;
-                    umma_commit(bar.at(kBarBEmpty + s));          // the stage may be refilled once these MMAs have read it
                     ++bcount;
                 }
                 if (!ok) break;
-                umma_commit(bar.at(kBarAEmpty + ab));             // so may the resident tiles
+                if (mine) umma_commit(bar.at(kBarAEmpty + ab));   // so may the resident tiles
+                else mbar_arrive(bar.at(kBarAEmpty + ab));
                 ++k_item;
             }
         }
@@ -687,8 +695,8 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
         if (*abort_flag) __nanosleep(200000);      // error path only: let copies and MMAs in flight land
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
-        if (lane == 0 && !*abort_flag && tiles_done) atomicAdd(p.counters, tiles_done);
     }
+    if ((warp == 1 || warp == 10) && lane == 0 && !*abort_flag && tiles_done) atomicAdd(p.counters, tiles_done);
 }
 
 // ---- between the passes: list, per head, the tokens still short of partners with positions not yet looked at -----
