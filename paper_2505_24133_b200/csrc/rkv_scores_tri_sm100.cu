@@ -74,7 +74,10 @@ enum {
 constexpr int kSliceBytes = kTile * 32;
 constexpr int kOffAugA = kOffA + 2 * kTileBytes;           // 2 slices, beside the resident tiles
 constexpr int kOffAugB = kOffAugA + 2 * kSliceBytes;       // kStagesB slices, beside the streamed tiles
-static_assert((2 + kStagesB) * kSliceBytes <= 2 * kTileBytes, "the slices must fit the second resident pair");
+// ... and, when beta > 1 (several partners per token: their values need the r_j of whole chunks), for the r_j of
+// the head, one item at a time.
+constexpr int kOffRHead = kOffAugB + kStagesB * kSliceBytes;
+static_assert((2 + kStagesB) * kSliceBytes + RKV_MAX_CAP * 4 <= 2 * kTileBytes, "slices and r_j must fit the second resident pair");
 constexpr int kOffItems = kOffBar + kNumBars * 8;          // kItemSlots x int4
 constexpr int kOffMisc = kOffItems + kItemSlots * 16;      // tmem base, abort flag, bail flag
 constexpr int kOffRj = kOffMisc + 16;                      // pass 1: [2 items][kPass1Depth * 128] r_j of the streamed tiles
@@ -229,6 +232,16 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
                 items[qs] = desc;
                 mbar_arrive(bar.at(kBarQFull + qs));
 
+                if (kPass2 && p.beta > 1) {
+                    // r_j of the tiles this item streams (0 .. first_tile), straight into shared memory
+                    if (!mbar_wait(bar.at(kBarREmpty), (k_item & 1) ^ 1, abort_flag, p.status)) break;
+                    const uint32_t bytes = (uint32_t)(first_tile + 1) * kTile * 4u;
+                    mbar_expect_tx(bar.at(kBarRFull), bytes);
+                    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                                 ::"r"(sbase + kOffRHead), "l"(p.inv_norm + (size_t)head * p.cap_pad), "r"(bytes),
+                                   "r"(bar.at(kBarRFull))
+                                 : "memory");
+                }
                 if (!kPass2 && rule_on) {
                     // r_j of the key tiles this item streams (first_tile down to first_tile + 2 - n_iter)
                     const uint32_t rb = k_item & 1;
@@ -463,9 +476,10 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
 
             const bool scan = active && (kPass2 || rule_on);
             // r_j of the first key tile of the scan: loaded now, staged in shared memory when the tile is drained
-            const bool has_r = !kPass2 && rule_on;
+            const bool has_r = kPass2 ? p.beta > 1 : rule_on;
+            const uint32_t r_slot = kPass2 ? 0u : (k_item & 1), r_par = kPass2 ? (k_item & 1) : ((k_item >> 1) & 1);
             if (has_r) {        // every warp waits for the item's r_j, and hands them back at the item's end
-                const bool r_ok = mbar_wait(bar.at(kBarRFull + (k_item & 1)), (k_item >> 1) & 1, abort_flag, p.status);
+                const bool r_ok = mbar_wait(bar.at(kBarRFull + r_slot), r_par, abort_flag, p.status);
                 item_ok = item_ok && r_ok;
             }
 
@@ -536,9 +550,9 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
                 // ---- key tiles, last to first; their r_j lie in shared memory
                 const float thr = (row_ok && ri > 0.f) ? __fdiv_rn(p.sim_threshold, ri) : kInf;   // g r_j vs T / r_i
                 // pass 2: the whole head from tile 0; pass 1: the item's tiles from its lowest one (that of row tile 0)
-                // pass 1: the r_j of the item's tiles in shared memory; pass 2: the head's, in global memory (read for
-                // the chunks with partners only)
-                const float *r_base = kPass2 ? inv_norm
+                // pass 1: the r_j of the item's tiles in shared memory; pass 2: the head's (there only with beta > 1,
+                // and read for the chunks with partners only)
+                const float *r_base = kPass2 ? reinterpret_cast<const float *>(smem + kOffRHead)
                                              : reinterpret_cast<const float *>(smem + kOffRj) + (k_item & 1) * kPass1Depth * kTile -
                                                    (size_t)max(2 * d.y, first_tile + 1 - kPass1Depth) * kTile;
                 bool ok = item_ok;
@@ -631,11 +645,11 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
                             int taken = __popc(hits);
                             for (; taken > left; --taken) hits &= hits - 1u;                   // drop the lowest positions
                             if (kPass2) {
-                                // S = T + h r_i r_j per partner: the chunk's r_j, for once, from global memory
+                                // S = T + h r_i r_j per partner
                                 nhit += taken;
 #pragma unroll
                                 for (int q = 0; q < 8; ++q) {
-                                    const float4 R = __ldg(rj4 + ch * 8 + q);
+                                    const float4 R = rj4[ch * 8 + q];
                                     v[4 * q] *= R.x;
                                     v[4 * q + 1] *= R.y;
                                     v[4 * q + 2] *= R.z;
@@ -667,7 +681,7 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
             }
             if (has_r) {
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar.at(kBarREmpty + (k_item & 1)));
+                if (lane == 0) mbar_arrive(bar.at(kBarREmpty + r_slot));
             }
             if (!item_ok) break;              // (the epilogue warps meet at no barrier of their own: each may leave alone)
             if (row_ok) {
