@@ -111,21 +111,6 @@ __global__ void __launch_bounds__(kPrepThreads, 5) prep_kernel(Params p)
         const float r = (row < n) ? __fdividef(1.0f, nrm + p.eps) : 0.f;
         if (lane_in_row == 0) {
             inv_norm[row] = r;                       // row < cap_pad: the grid covers exactly cap_pad rows per head
-            {
-                // ||k|| + eps as three bf16 parts (their sum has fp32 accuracy), arranged so that the dot product
-                // with (-t1, -t1, -t1, -t2, -t2, -t3) is -t * (||k|| + eps) up to terms of relative size 2^-24
-                float rest = (row < n) ? nrm + p.eps : 0.f;
-                uint32_t part[3];
-#pragma unroll
-                for (int c = 0; c < 3; ++c) {
-                    const __nv_bfloat16 h16 = __float2bfloat16_rn(rest);
-                    part[c] = (uint32_t)__bfloat16_as_ushort(h16);
-                    rest -= __bfloat162float(h16);
-                }
-                uint4 *dst = reinterpret_cast<uint4 *>(p.norm_split + ((size_t)head * p.cap_pad + row) * 16);
-                dst[0] = make_uint4(part[0] | (part[1] << 16), part[2] | (part[0] << 16), part[1] | (part[0] << 16), 0u);
-                dst[1] = make_uint4(0u, 0u, 0u, 0u);
-            }
             p.self_dot[(size_t)head * p.cap_pad + row] = (r * r) * sq;     // Kbar_i . Kbar_i
         }
         const float2 r2 = make_float2(r, r);

@@ -689,6 +689,22 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
                 if (!kPass2) {
                     *out = total - removed * ri;
                     p.left[(size_t)head * p.cap_pad + i] = rule_on ? left : 0;
+                    if (rule_on) {
+                        // for pass 2: 1 / r_i = ||k_i|| + eps as three bf16 parts (their sum has fp32 accuracy), laid
+                        // out as the extra K = 16 slice of a key row, (n1, n2, n3, n1, n2, n1, 0 ...): its dot product
+                        // with a token's (-t1, -t1, -t1, -t2, -t2, -t3, 0 ...) is -t / r_i up to terms of size 2^-24
+                        float rest = ri > 0.f ? __fdiv_rn(1.0f, ri) : 0.f;
+                        uint32_t part[3];
+#pragma unroll
+                        for (int c = 0; c < 3; ++c) {
+                            const __nv_bfloat16 h16 = __float2bfloat16_rn(rest);
+                            part[c] = (uint32_t)__bfloat16_as_ushort(h16);
+                            rest -= __bfloat162float(h16);
+                        }
+                        uint4 *dst = reinterpret_cast<uint4 *>(p.norm_split + ((size_t)head * p.cap_pad + i) * 16);
+                        dst[0] = make_uint4(part[0] | (part[1] << 16), part[2] | (part[0] << 16), part[1] | (part[0] << 16), 0u);
+                        dst[1] = make_uint4(0u, 0u, 0u, 0u);
+                    }
                 } else {
                     // S = T + h r_i r_j for every partner found here
                     if (p.beta == 1 && hit_j >= 0) {
