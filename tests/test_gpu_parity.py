@@ -299,6 +299,48 @@ def test_thread_current_descriptor_entry_point(rkv):
     assert torch.equal(wl_a.k_cache.view(torch.int16), wl_b.k_cache.view(torch.int16))
 
 
+def test_call_is_capturable_in_a_cuda_graph_and_replays(rkv):
+    """The call only enqueues work on its stream (no synchronisation, no allocation), so a decode loop can capture
+    it in a CUDA graph: the replayed graph gives bit for bit what the eager call gives, also when replayed again on
+    restored inputs, and the result agrees with the oracle."""
+    spec = small_spec("graph", batch=2, budget=384, buffer=128)          # four key tiles: all eight kernels run
+    wl = ri.make_workload(spec, device="cuda", seed=181)
+    k0, v0, s0 = wl.k_cache.clone(), wl.v_cache.clone(), wl.seq_lens.clone()
+    comp = rkv.Compressor(spec.folded_batch, spec.n_kv_heads, spec.n_q_heads, spec.budget, spec.buffer, spec.alpha,
+                          spec.lam)
+    idx_eager = comp.compress(wl.k_cache, wl.v_cache, wl.q_window, wl.seq_lens).clone()
+    torch.cuda.synchronize()
+    comp.check_status()
+    k_eager, v_eager, s_eager = wl.k_cache.clone(), wl.v_cache.clone(), wl.seq_lens.clone()
+
+    def restore():
+        wl.k_cache.copy_(k0)
+        wl.v_cache.copy_(v0)
+        wl.seq_lens.copy_(s0)
+
+    restore()
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.graph(graph, stream=side):
+        comp.compress(wl.k_cache, wl.v_cache, wl.q_window, wl.seq_lens, stream=torch.cuda.current_stream())
+    torch.cuda.synchronize()
+    for _ in range(2):
+        restore()
+        comp.out_idx.fill_(-5)
+        graph.replay()
+        torch.cuda.synchronize()
+        comp.check_status()
+        assert torch.equal(comp.out_idx, idx_eager)
+        assert torch.equal(wl.seq_lens, s_eager)
+        nb = spec.budget
+        assert torch.equal(wl.k_cache[:, :, :nb].view(torch.int16), k_eager[:, :, :nb].view(torch.int16))
+        assert torch.equal(wl.v_cache[:, :, :nb].view(torch.int16), v_eager[:, :, :nb].view(torch.int16))
+    rep = check_batch(k0, v0, wl.q_window, s0, budget=spec.budget, alpha=spec.alpha, lam=spec.lam, W=4, beta=1, T=0.5,
+                      eps=1e-8, gpu_idx=comp.out_idx, gpu_k=wl.k_cache, gpu_v=wl.v_cache, gpu_seq=wl.seq_lens)
+    assert rep.ok(), rep.errors
+
+
 def test_kernel_events_and_executed_tile_counter(rkv):
     """The profiling hooks of the descriptor: nine event boundaries give eight non-negative kernel times, and the
     tensor-core kernels report how many 128 x 128 x 128 tile products they executed: at least one key tile per row
