@@ -234,6 +234,61 @@ __device__ __forceinline__ void radix_select_emit(const uint32_t *keys, int n, i
         for (int c = 0; c < copies; ++c) out[(size_t)c * budget + k + j] = n + j;   // observation tokens
 }
 
+// Eq. 4 with the default window W = 4 (positions i-4 .. i+3), eight consecutive tokens per thread: per query row
+// four 16-byte loads bring the 16 logits those windows cover, and the eight maxima come from a doubling scheme in
+// registers (the general kernel above reads each logit nine times).
+constexpr int kImp8Threads = 256;
+constexpr int kImp8Tokens = kImp8Threads * 8;
+
+__global__ void __launch_bounds__(kImp8Threads) importance_w4_kernel(Params p)
+{
+    const int chunks = (p.cap + kImp8Tokens - 1) / kImp8Tokens;
+    const int head = blockIdx.x / chunks;
+    const int i0 = (blockIdx.x % chunks) * kImp8Tokens + threadIdx.x * 8;     // first token of this thread
+    const int n = candidates_from_meta(p.meta[head / p.hkv], p.budget, p.alpha);
+    if (i0 >= n) return;
+    const float *logits = p.logits + (size_t)head * p.alpha * p.cap_pad;
+    const float *stat = p.row_stat + (size_t)head * p.alpha * 2;
+    const float kNegInf = -INFINITY;
+    const bool interior = i0 >= 4 && i0 + 11 < n;      // all 16 positions i0-4 .. i0+11 are candidates
+    float acc[8];
+#pragma unroll
+    for (int t = 0; t < 8; ++t) acc[t] = 0.f;
+    for (int j = 0; j < p.alpha; ++j) {
+        const float *row = logits + (size_t)j * p.cap_pad;
+        float x[16];                                    // x[u] = logit at position i0 - 4 + u
+        {
+            const float4 *r4 = reinterpret_cast<const float4 *>(row + i0);       // i0 is a multiple of 8
+            const float4 a = i0 >= 4 ? r4[-1] : make_float4(kNegInf, kNegInf, kNegInf, kNegInf);
+            const float4 b = r4[0], c = r4[1];          // i0 + 7 < cap_pad (a multiple of 128)
+            const float4 d = i0 + 8 < p.cap_pad ? r4[2] : make_float4(kNegInf, kNegInf, kNegInf, kNegInf);
+            x[0] = a.x, x[1] = a.y, x[2] = a.z, x[3] = a.w, x[4] = b.x, x[5] = b.y, x[6] = b.z, x[7] = b.w;
+            x[8] = c.x, x[9] = c.y, x[10] = c.z, x[11] = c.w, x[12] = d.x, x[13] = d.y, x[14] = d.z, x[15] = d.w;
+        }
+        if (!interior) {                                // the window is clipped to the candidates [0, n)
+#pragma unroll
+            for (int u = 0; u < 16; ++u) {
+                const int pos = i0 - 4 + u;
+                if (pos < 0 || pos >= n) x[u] = kNegInf;
+            }
+        }
+        float m2[15], m4[13];
+#pragma unroll
+        for (int u = 0; u < 15; ++u) m2[u] = fmaxf(x[u], x[u + 1]);
+#pragma unroll
+        for (int u = 0; u < 13; ++u) m4[u] = fmaxf(m2[u], m2[u + 2]);
+        const float mj = stat[2 * j], inv = stat[2 * j + 1];
+#pragma unroll
+        for (int t = 0; t < 8; ++t)                     // token i0 + t: positions i0 + t - 4 .. i0 + t + 3 = x[t .. t+7]
+            acc[t] += expf(fmaxf(m4[t], m4[t + 4]) - mj) * inv;
+    }
+    const float inv_alpha = 1.0f / (float)p.alpha;
+    float *out = p.imp + (size_t)head * p.cap_pad + i0;
+#pragma unroll
+    for (int t = 0; t < 8; ++t)
+        if (i0 + t < n) out[t] = acc[t] * inv_alpha;
+}
+
 // kFused: the block first does the work of row_stats_kernel and importance_kernel for its head, with the pooled
 // logits in shared memory (small caches only: one launch instead of three, all of them latency-bound there).
 template <bool kFused>
@@ -401,7 +456,10 @@ cudaError_t launch_select(const Params &p, cudaStream_t s)
     row_stats_kernel<<<heads * (unsigned)p.alpha, kStatThreads, 0, s>>>(p);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     if ((e = mark_kernel(p, 2, s)) != cudaSuccess) return e;
-    importance_kernel<<<heads * (unsigned)((p.cap + kImpTokens - 1) / kImpTokens), kImpThreads, 0, s>>>(p);
+    if (p.pool_w == 4 && !p.mean_then_pool)
+        importance_w4_kernel<<<heads * (unsigned)((p.cap + kImp8Tokens - 1) / kImp8Tokens), kImp8Threads, 0, s>>>(p);
+    else
+        importance_kernel<<<heads * (unsigned)((p.cap + kImpTokens - 1) / kImpTokens), kImpThreads, 0, s>>>(p);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     if ((e = mark_kernel(p, 3, s)) != cudaSuccess) return e;
     const size_t smem = (size_t)p.cap_pad * sizeof(float);
