@@ -19,8 +19,8 @@ namespace rkv {
 
 namespace {
 
-constexpr int kSelThreads = 512;
-constexpr int kSelWarps = kSelThreads / 32;
+constexpr int kSelThreadsFused = 512;     // single-kernel form (small caches, often few heads): more threads per head
+constexpr int kSelThreadsSplit = 256;     // three-kernel form: more blocks per SM hide the many block-wide barriers
 
 __device__ __forceinline__ uint32_t order_key(float z)
 {
@@ -29,6 +29,7 @@ __device__ __forceinline__ uint32_t order_key(float z)
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
+template <int kSelThreads>
 __device__ __forceinline__ float block_max(float v, float *scratch)
 {
 #pragma unroll
@@ -36,12 +37,14 @@ __device__ __forceinline__ float block_max(float v, float *scratch)
     __syncthreads();
     if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = v;
     __syncthreads();
+    constexpr int kSelWarps = kSelThreads / 32;
     float r = (threadIdx.x & 31) < kSelWarps ? scratch[threadIdx.x & 31] : -INFINITY;
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) r = fmaxf(r, __shfl_xor_sync(0xffffffffu, r, off));
     return r;
 }
 
+template <int kSelThreads>
 __device__ __forceinline__ float block_sum(float v, float *scratch)
 {
     // fixed reduction tree: the result does not depend on scheduling
@@ -50,6 +53,7 @@ __device__ __forceinline__ float block_sum(float v, float *scratch)
     __syncthreads();
     if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = v;
     __syncthreads();
+    constexpr int kSelWarps = kSelThreads / 32;
     float r = (threadIdx.x & 31) < kSelWarps ? scratch[threadIdx.x & 31] : 0.f;
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) r += __shfl_xor_sync(0xffffffffu, r, off);
@@ -133,9 +137,11 @@ __global__ void __launch_bounds__(kImpThreads) importance_kernel(Params p)
 // Exact top-k over n order-preserving keys in shared memory (written by the caller, one owner per slot; no barrier
 // needed before the call), later position first among equal keys.  Writes the k kept positions in ascending order and
 // then the alpha observation positions n .. n+alpha-1 into `copies` index lists of `budget` entries, `budget` apart.
+template <int kSelThreads>
 __device__ __forceinline__ void radix_select_emit(const uint32_t *keys, int n, int k, int alpha, int budget,
                                                   int32_t *out, int copies)
 {
+    constexpr int kSelWarps = kSelThreads / 32;
     __shared__ uint32_t hist[256];
     __shared__ uint32_t sel_prefix, sel_want;
     __shared__ uint32_t warp_tot[kSelWarps];
@@ -147,7 +153,7 @@ __device__ __forceinline__ void radix_select_emit(const uint32_t *keys, int n, i
 
     // ---- radix select: the k-th largest key, 8 bits at a time from the top
     for (int shift = 24; shift >= 0; shift -= 8) {
-        if (tid < 256) hist[tid] = 0u;
+        for (int t = tid; t < 256; t += kSelThreads) hist[t] = 0u;
         __syncthreads();
         const uint32_t prefix = sel_prefix;
         const uint32_t high_mask = (shift == 24) ? 0u : (0xffffffffu << (shift + 8));
@@ -292,8 +298,10 @@ __global__ void __launch_bounds__(kImp8Threads) importance_w4_kernel(Params p)
 // kFused: the block first does the work of row_stats_kernel and importance_kernel for its head, with the pooled
 // logits in shared memory (small caches only: one launch instead of three, all of them latency-bound there).
 template <bool kFused>
-__global__ void __launch_bounds__(kSelThreads, 2) select_kernel(Params p)
+__global__ void __launch_bounds__(kFused ? kSelThreadsFused : kSelThreadsSplit, kFused ? 2 : 4) select_kernel(Params p)
 {
+    constexpr int kSelThreads = kFused ? kSelThreadsFused : kSelThreadsSplit;
+    constexpr int kSelWarps = kSelThreads / 32;
     extern __shared__ float row[];                 // [cap_pad] one logits row / the Sbar row, then the keys;
                                                    // kFused: then [cap_pad] importance and [alpha][cap_pad] logits
     __shared__ float stat_s[2 * RKV_MAX_GROUP_ROWS];
@@ -378,10 +386,10 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_kernel(Params p)
         row[i] = v;
         m = fmaxf(m, v);
     }
-    m = block_max(m, scratch);
+    m = block_max<kSelThreads>(m, scratch);
     float s = 0.f;
     for (int i = tid; i < n; i += kSelThreads) s += expf(row[i] - m);
-    s = block_sum(s, scratch);
+    s = block_sum<kSelThreads>(s, scratch);
     const float inv = 1.0f / s;
 
     // ---- Eq. 7 and the integer keys (kept in the same shared row, one owner per slot)
@@ -402,13 +410,14 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_kernel(Params p)
         }
     }
     if (p.head_mean) return;      // Z of this head is in p.imp; select_mean_kernel picks the sequence's positions
-    radix_select_emit(keys, n, k, p.alpha, p.budget, out, 1);
+    radix_select_emit<kSelThreads>(keys, n, k, p.alpha, p.budget, out, 1);
 }
 
 // Algorithm 1's aggregated selection, one block per sequence: AggScore_i = mean over the KV heads of Z_i^h (left in
 // p.imp by select_kernel), exact top-k on it, the same index list written for every head of the sequence.
-__global__ void __launch_bounds__(kSelThreads, 2) select_mean_kernel(Params p)
+__global__ void __launch_bounds__(kSelThreadsSplit, 4) select_mean_kernel(Params p)
 {
+    constexpr int kSelThreads = kSelThreadsSplit;
     extern __shared__ float row[];
     const int b = blockIdx.x, tid = threadIdx.x;
     const int L = p.meta[b];
@@ -422,7 +431,7 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_mean_kernel(Params p)
         for (int h = 0; h < p.hkv; ++h) acc += z[(size_t)h * p.cap_pad + i];      // fixed head order
         keys[i] = order_key(acc / hkv);
     }
-    radix_select_emit(keys, n, p.budget - p.alpha, p.alpha, p.budget, p.out_idx + (size_t)b * p.hkv * p.budget, p.hkv);
+    radix_select_emit<kSelThreads>(keys, n, p.budget - p.alpha, p.alpha, p.budget, p.out_idx + (size_t)b * p.hkv * p.budget, p.hkv);
 }
 
 }  // namespace
@@ -434,7 +443,7 @@ static cudaError_t launch_select_mean(const Params &p, cudaStream_t s)
     const size_t smem = (size_t)p.cap_pad * sizeof(float);
     cudaError_t e = cudaFuncSetAttribute(select_mean_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    select_mean_kernel<<<(unsigned)p.batch, kSelThreads, smem, s>>>(p);
+    select_mean_kernel<<<(unsigned)p.batch, kSelThreadsSplit, smem, s>>>(p);
     return cudaGetLastError();
 }
 
@@ -449,7 +458,7 @@ cudaError_t launch_select(const Params &p, cudaStream_t s)
         if ((e = cudaFuncSetAttribute(select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) !=
             cudaSuccess)
             return e;
-        select_kernel<true><<<heads, kSelThreads, smem, s>>>(p);
+        select_kernel<true><<<heads, kSelThreadsFused, smem, s>>>(p);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
         return p.head_mean ? launch_select_mean(p, s) : cudaSuccess;
     }
@@ -466,7 +475,7 @@ cudaError_t launch_select(const Params &p, cudaStream_t s)
     if ((e = cudaFuncSetAttribute(select_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) !=
         cudaSuccess)
         return e;
-    select_kernel<false><<<heads, kSelThreads, smem, s>>>(p);
+    select_kernel<false><<<heads, kSelThreadsSplit, smem, s>>>(p);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     return p.head_mean ? launch_select_mean(p, s) : cudaSuccess;
 }
