@@ -45,13 +45,17 @@
 
 /* ---- Eq. 2-3 (Eq. 1 when G == 1): attention weights A[alpha][n] ---------- */
 static void attention_weights(const float *K, const float *Q, int n, int d,
-                              int G, int alpha, double *A)
+                              int G, int alpha, int mean_pool, double *A)
 {
     const double root_d = sqrt((double)d);
     for (int j = 0; j < alpha; ++j) {
-        /* Eq. 2: scaled logits of each query head g; Eq. 3: max over g */
+        /* Eq. 2: scaled logits of each query head g; Eq. 3: max over g.
+         * mean_pool (a variant, off by default): the mean over g instead, the
+         * pooling the paper's appendix ascribes to earlier work; read as Eq. 3
+         * with the max replaced, i.e. still on the logits and before the one
+         * softmax. */
         for (int i = 0; i < n; ++i) {
-            double pooled = -INFINITY;
+            double pooled = -INFINITY, total = 0.0;
             for (int g = 0; g < G; ++g) {
                 const float *q = Q + ((size_t)g * alpha + j) * d;
                 const float *k = K + (size_t)i * d;
@@ -61,8 +65,9 @@ static void attention_weights(const float *K, const float *Q, int n, int d,
                 double logit = dot / root_d;
                 if (logit > pooled)
                     pooled = logit;
+                total += logit;
             }
-            A[(size_t)j * n + i] = pooled;
+            A[(size_t)j * n + i] = mean_pool ? total / (double)G : pooled;
         }
         /* Eq. 3: softmax along the key dimension */
         double top = -INFINITY;
@@ -243,7 +248,9 @@ static int select_kept(const double *z, int n, int k, int alpha, int32_t *idx)
  *   S_raw, S_mod             optional [n][n] dumps of Eq. 5's matrix before and
  *                            after the retention rule; may be NULL
  *   variant                  0 = the method as the equations state it; bit 0 =
- *                            Algorithm 1's order for the importance (mean, then pool)
+ *                            Algorithm 1's order for the importance (mean, then pool);
+ *                            bit 2 = mean instead of max over the query heads of a
+ *                            group in Eq. 3
  * Returns 1 if the head was compressed, 0 if L <= budget (nothing to do:
  * idx = 0..L-1 then -1), -1 on bad arguments.
  */
@@ -275,7 +282,7 @@ int rkv_oracle_head(const float *K, const float *Q, int L, int d, int G,
         return -1;
     }
 
-    attention_weights(K, Q, n, d, G, alpha, A_);
+    attention_weights(K, Q, n, d, G, alpha, (variant & 4) != 0, A_);
     if (variant & 1) /* RKV_ORACLE_MEAN_THEN_POOL */
         importance_scores_mean_first(A_, n, alpha, W, I_);
     else
@@ -328,7 +335,7 @@ void rkv_oracle_gather(const uint8_t *in, const int32_t *idx, int count,
  *   belongs to KV head q / G), seq_lens [B], idx [B][Hkv][budget].
  *   scores: optional [4][B][Hkv][cap] doubles = I, Sbar, R, Z (first n used).
  *   compressed: optional [B] flags.
- *   variant: bit 0 as in rkv_oracle_head; bit 1 = one kept set per sequence
+ *   variant: bits 0 and 2 as in rkv_oracle_head; bit 1 = one kept set per sequence
  *   from the head-averaged score (Algorithm 1) instead of one per KV head.
  * Returns the number of OpenMP threads used, or -1 on bad arguments.
  */

@@ -71,7 +71,7 @@ class HeadResult:
 
 def oracle_head(K, Q, *, budget: int, alpha: int, lam: float, W: int, beta: int, T: float,
                 eps: float = 1e-8, L: Optional[int] = None, want_S: bool = False,
-                mean_then_pool: bool = False) -> HeadResult:
+                mean_then_pool: bool = False, gqa_mean_pool: bool = False) -> HeadResult:
     """One (sequence, KV head): K [>=L, d], Q [G, alpha, d]."""
     lib = _load()
     K = _f32(K)
@@ -92,7 +92,8 @@ def oracle_head(K, Q, *, budget: int, alpha: int, lam: float, W: int, beta: int,
                             _ptr(A, ctypes.c_double), _ptr(I, ctypes.c_double),
                             _ptr(Sbar, ctypes.c_double), _ptr(R, ctypes.c_double),
                             _ptr(Z, ctypes.c_double), _ptr(S_raw, ctypes.c_double),
-                            _ptr(S_mod, ctypes.c_double), 1 if mean_then_pool else 0)
+                            _ptr(S_mod, ctypes.c_double),
+                            (1 if mean_then_pool else 0) | (4 if gqa_mean_pool else 0))
     if r < 0:
         raise ValueError("rkv_oracle_head: bad arguments")
     return HeadResult(bool(r), idx, A, I, Sbar, R, Z, S_raw, S_mod)
@@ -111,7 +112,7 @@ class BatchResult:
 
 def oracle_batch(K, Q, seq_lens, *, budget: int, alpha: int, lam: float, W: int, beta: int,
                  T: float, eps: float = 1e-8, want_scores: bool = True,
-                 mean_then_pool: bool = False, head_mean: bool = False) -> BatchResult:
+                 mean_then_pool: bool = False, head_mean: bool = False, gqa_mean_pool: bool = False) -> BatchResult:
     """K [B, Hkv, cap, d], Q [B, Hq, alpha, d], seq_lens [B]."""
     lib = _load()
     K = _f32(K)
@@ -127,7 +128,7 @@ def oracle_batch(K, Q, seq_lens, *, budget: int, alpha: int, lam: float, W: int,
                              _ptr(seq, ctypes.c_int32), B, Hkv, Hq, cap, d, alpha, budget, W, beta,
                              float(T), float(eps), float(lam), _ptr(idx, ctypes.c_int32),
                              _ptr(scores, ctypes.c_double), _ptr(comp, ctypes.c_int32),
-                             (1 if mean_then_pool else 0) | (2 if head_mean else 0))
+                             (1 if mean_then_pool else 0) | (2 if head_mean else 0) | (4 if gqa_mean_pool else 0))
     if t < 0:
         raise ValueError("rkv_oracle_batch: bad arguments (seq_len > cap, or sizes)")
     if scores is None:

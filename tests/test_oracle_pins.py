@@ -502,3 +502,31 @@ def test_head_mean_aggregated_selection_variant():
     one = oracle.oracle_batch(K[:, :1], Q[:, :2], seq, head_mean=True, **kw)
     ref = oracle.oracle_batch(K[:, :1], Q[:, :2], seq, **kw)
     np.testing.assert_array_equal(one.idx, ref.idx)
+
+
+def test_gqa_mean_pool_variant():
+    """Mean instead of max over the query heads of a group (the pooling the paper's appendix ascribes to earlier work),
+    read as Eq. 3 with the max replaced: the attention weights are softmax(mean_g Q^g K^T / sqrt(d)), recomputed here
+    with numpy/scipy; G = 1 and a group of identical query heads give the max-pooled result; and on generic inputs
+    the two poolings differ (otherwise the pins above would not tell them apart)."""
+    from scipy.special import softmax
+    rng = np.random.default_rng(91)
+    L, alpha, G = 70, 8, 4
+    K, Q = _rand(rng, L, D), _rand(rng, G, alpha, D) * 2.0
+    n = L - alpha
+    mx = _run(K, Q, budget=40, alpha=alpha)
+    mp = _run(K, Q, budget=40, alpha=alpha, gqa_mean_pool=True)
+    logits = np.einsum("gjc,ic->gji", Q.astype(np.float64), K[:n].astype(np.float64)) / np.sqrt(D)
+    np.testing.assert_allclose(mp.A, softmax(logits.mean(axis=0), axis=1), rtol=1e-12, atol=1e-300)
+    np.testing.assert_allclose(mx.A, softmax(logits.max(axis=0), axis=1), rtol=1e-12, atol=1e-300)
+    np.testing.assert_allclose(mp.A.sum(axis=1), 1.0, rtol=1e-12)
+    assert np.abs(mp.A - mx.A).max() > 1e-3
+    np.testing.assert_array_equal(mp.S_raw, mx.S_raw)                        # the redundancy side does not change
+    one = _rand(rng, 1, alpha, D)
+    a = _run(K, one, budget=40, alpha=alpha)
+    b = _run(K, one, budget=40, alpha=alpha, gqa_mean_pool=True)
+    np.testing.assert_array_equal(a.idx, b.idx)
+    np.testing.assert_allclose(a.A, b.A, rtol=1e-15)
+    same = np.repeat(one, 3, axis=0)
+    c = _run(K, same, budget=40, alpha=alpha, gqa_mean_pool=True)
+    np.testing.assert_allclose(c.A, a.A, rtol=1e-12)
