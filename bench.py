@@ -49,6 +49,8 @@ def parse_args():
     ap.add_argument("--threshold", type=float, default=None)
     ap.add_argument("--pool-w", type=int, default=None)
     ap.add_argument("--mean-then-pool", action="store_true", help="importance in Algorithm 1's order (a variant)")
+    ap.add_argument("--gqa-mean-pool", action="store_true",
+                    help="mean instead of max over a group's query heads in Eq. 3 (a variant)")
     ap.add_argument("--head-mean", action="store_true",
                     help="Algorithm 1's aggregated selection: one kept set per sequence from the head-averaged score")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -155,7 +157,7 @@ def run_reference(args, rank: int):
     seq = wl.seq_lens.numpy()
     kw = dict(budget=spec.budget, alpha=spec.alpha, lam=spec.lam, W=4 if args.pool_w is None else args.pool_w,
               beta=1 if args.beta is None else args.beta, T=0.5 if args.threshold is None else args.threshold,
-              mean_then_pool=args.mean_then_pool, head_mean=args.head_mean)
+              mean_then_pool=args.mean_then_pool, head_mean=args.head_mean, gqa_mean_pool=args.gqa_mean_pool)
     oracle.build()
     steps, warm = max(1, min(args.steps, 5)), max(1, min(args.warmup, 1))
     for _ in range(warm):
@@ -276,9 +278,10 @@ def main():
         kw["sim_threshold"] = args.threshold
     if args.pool_w is not None:
         kw["pool_w"] = args.pool_w
-    if args.mean_then_pool or args.head_mean:
+    if args.mean_then_pool or args.head_mean or args.gqa_mean_pool:
         kw["flags"] = (rkv.RKV_FLAG_MEAN_THEN_POOL if args.mean_then_pool else 0) | \
-                      (rkv.RKV_FLAG_HEAD_MEAN if args.head_mean else 0)
+                      (rkv.RKV_FLAG_HEAD_MEAN if args.head_mean else 0) | \
+                      (rkv.RKV_FLAG_GQA_MEAN_POOL if args.gqa_mean_pool else 0)
     comp = rkv.Compressor(spec.folded_batch, spec.n_kv_heads, spec.n_q_heads, spec.budget, spec.buffer, spec.alpha,
                           spec.lam, dtype=spec.torch_dtype, device=dev, **kw)
     launches_per_step = rkv.rkv_launch_count_for(comp.desc, spec.budget, spec.buffer, spec.alpha, rkv.RKV_STAGE_ALL)
@@ -443,7 +446,7 @@ def main():
         while passes < 1 or (time.perf_counter() - t0 < 12.0 and passes < 200):      # about 12 s of CPU work
             res = oracle.oracle_batch(Kh, Qh, seq_h, budget=spec.budget, alpha=spec.alpha, lam=spec.lam, W=d.pool_w,
                                       beta=d.beta, T=d.sim_threshold, eps=d.eps, want_scores=False,
-                                      mean_then_pool=args.mean_then_pool, head_mean=args.head_mean)
+                                      mean_then_pool=args.mean_then_pool, head_mean=args.head_mean, gqa_mean_pool=args.gqa_mean_pool)
             passes += 1
         dt = time.perf_counter() - t0
         cpu = {"value": passes * seqs * spec.n_kv_heads * n / dt, "unit": UNIT, "cores": res.threads, "kind": "oracle",

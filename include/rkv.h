@@ -70,6 +70,10 @@ typedef enum { RKV_BF16 = 0, RKV_F32 = 1 } rkv_dtype_t;
                                    averaged and ONE set of positions is kept for all of them (every head's index
                                    list is the same); default is one set per KV head.  One more launch. */
 
+#define RKV_FLAG_GQA_MEAN_POOL 16u /* Eq. 3 with the mean instead of the max over the query heads of a group (the
+                                   pooling the paper's appendix ascribes to earlier work); still taken on the scaled
+                                   logits, before the one softmax.  Default is the max (Eq. 3). */
+
 /* stage bits for rkv_compress_stages */
 #define RKV_STAGE_PREP 1u    /* key inverse norms and per-tile sums of normalised keys */
 #define RKV_STAGE_SCORES 2u  /* Eq. 2-3 pooled logits; Eq. 5 matrix + retention rule + Eq. 6 column means */

@@ -117,6 +117,7 @@ int run(const rkv_desc_t *d, void *k_cache, void *v_cache, const void *q_window,
     p.beta = d->beta;
     p.mean_then_pool = (d->flags & RKV_FLAG_MEAN_THEN_POOL) ? 1 : 0;
     p.head_mean = (d->flags & RKV_FLAG_HEAD_MEAN) ? 1 : 0;
+    p.gqa_mean_pool = (d->flags & RKV_FLAG_GQA_MEAN_POOL) ? 1 : 0;
     p.sim_threshold = d->sim_threshold;
     p.eps = d->eps;
     p.lambda = lambda;

@@ -33,6 +33,7 @@ struct Params {
     int pool_w, beta;
     int head_mean;                  // Algorithm 1's aggregated selection: one kept set per sequence from the
                                     // head-averaged Z (select_kernel then leaves Z in `imp` and a second kernel selects)
+    int gqa_mean_pool;              // Eq. 3 with the mean over the group's query heads instead of the max
     int mean_then_pool;             // importance in Algorithm 1's order (mean over query rows, then pooling)
     float sim_threshold, eps, lambda;
     // workspace carve-up

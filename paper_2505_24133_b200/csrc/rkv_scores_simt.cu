@@ -102,15 +102,16 @@ __global__ void __launch_bounds__(kSimtThreads) scores_simt_kernel(Params p)
             const int i = jt * kTile + t;
             if (i < n) {
                 for (int j = 0; j < p.alpha; ++j) {
-                    float best = -INFINITY;
+                    float best = -INFINITY, total = 0.f;
                     for (int g = 0; g < p.group; ++g) {
                         const float *q = tileA + (g * p.alpha + j) * kPadRow;
                         float dot = 0.f;
 #pragma unroll 16
                         for (int c = 0; c < kHeadDim; ++c) dot = fmaf(q[c], tileB[t * kPadRow + c], dot);
                         best = fmaxf(best, dot * scale);
+                        total += dot * scale;
                     }
-                    logits[(size_t)j * p.cap_pad + i] = best;
+                    logits[(size_t)j * p.cap_pad + i] = p.gqa_mean_pool ? total / (float)p.group : best;
                 }
             }
         }

@@ -299,10 +299,13 @@ scores_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, const _
                     if (lane == 0) mbar_arrive(bar.acc_empty(a));
                     if (i < n) {
                         for (int j = 0; j < p.alpha; ++j) {
-                            float best = -INFINITY;
-                            for (int gq = 0; gq < p.group; ++gq)
-                                best = fmaxf(best, stage_f[(gq * p.alpha + j) * kTile + lrow] * scale);
-                            logits[(size_t)j * p.cap_pad + i] = best;
+                            float best = -INFINITY, total = 0.f;
+                            for (int gq = 0; gq < p.group; ++gq) {
+                                const float lg = stage_f[(gq * p.alpha + j) * kTile + lrow] * scale;
+                                best = fmaxf(best, lg);
+                                total += lg;
+                            }
+                            logits[(size_t)j * p.cap_pad + i] = p.gqa_mean_pool ? total / (float)p.group : best;
                         }
                     }
                 }

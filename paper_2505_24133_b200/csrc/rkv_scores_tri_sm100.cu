@@ -499,28 +499,36 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
                 if (p.alpha == 8) {
                     float best[8];
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) best[j] = -kInf;
+                    for (int j = 0; j < 8; ++j) best[j] = p.gqa_mean_pool ? 0.f : -kInf;
                     for (int g0 = 0; g0 < G; g0 += 2) {
                         uint32_t t0[8], t1[8];
                         tmem_ld8(qbase + g0 * 8, t0);
                         tmem_ld8(qbase + min(g0 + 1, G - 1) * 8, t1);     // an odd G reads its last head twice
                         tmem_wait8(t0);
                         tmem_wait8(t1);
+                        if (p.gqa_mean_pool) {        // the variant: sum over the group (scaled to the mean below)
+                            const bool both = g0 + 1 < G;
+#pragma unroll
+                            for (int j = 0; j < 8; ++j)
+                                best[j] += __uint_as_float(t0[j]) + (both ? __uint_as_float(t1[j]) : 0.f);
+                            continue;
+                        }
 #pragma unroll
                         for (int j = 0; j < 8; ++j)
                             best[j] = fmaxf(best[j], fmaxf(__uint_as_float(t0[j]), __uint_as_float(t1[j])));
                     }
+                    const float scale_q = p.gqa_mean_pool ? scale / (float)G : scale;
                     tmem_wait8(sp);
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar.at(kBarAccEmpty + a * 2 + m));
                     if (row_ok) {
 #pragma unroll
-                        for (int j = 0; j < 8; ++j) logits[(size_t)j * p.cap_pad + i] = best[j] * scale;
+                        for (int j = 0; j < 8; ++j) logits[(size_t)j * p.cap_pad + i] = best[j] * scale_q;
                     }
                 } else {
                     for (int j = 0; j < p.alpha; ++j) {
-                        float best = -kInf;
+                        float best = -kInf, sum = 0.f;
                         for (int g0 = 0; g0 < G; g0 += 4) {
                             uint32_t t[4];
 #pragma unroll
@@ -528,9 +536,13 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
                             asm volatile("tcgen05.wait::ld.sync.aligned;"
                                          : "+r"(t[0]), "+r"(t[1]), "+r"(t[2]), "+r"(t[3]) :: "memory");
 #pragma unroll
-                            for (int u = 0; u < 4; ++u) best = fmaxf(best, __uint_as_float(t[u]));
+                            for (int u = 0; u < 4; ++u) {
+                                best = fmaxf(best, __uint_as_float(t[u]));
+                                sum += (g0 + u < G) ? __uint_as_float(t[u]) : 0.f;
+                            }
                         }
-                        if (row_ok) logits[(size_t)j * p.cap_pad + i] = best * scale;
+                        if (row_ok)
+                            logits[(size_t)j * p.cap_pad + i] = p.gqa_mean_pool ? sum * scale / (float)G : best * scale;
                     }
                     tmem_wait8(sp);
                     tc_fence_before();

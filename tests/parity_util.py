@@ -70,7 +70,8 @@ def check_batch(k_in: torch.Tensor, v_in: torch.Tensor, q_in: torch.Tensor, seq_
                 budget: int, alpha: int, lam: float, W: int, beta: int, T: float, eps: float,
                 gpu_idx: torch.Tensor, gpu_k: Optional[torch.Tensor] = None, gpu_v: Optional[torch.Tensor] = None,
                 gpu_seq: Optional[torch.Tensor] = None, gpu_scores: Optional[torch.Tensor] = None,
-                max_errors: int = 10, mean_then_pool: bool = False, head_mean: bool = False) -> ParityReport:
+                max_errors: int = 10, mean_then_pool: bool = False, head_mean: bool = False,
+                gqa_mean_pool: bool = False) -> ParityReport:
     """All tensors are for the same (sub)batch: k_in/v_in [B,H,cap,d] and q_in [B,Hq,alpha,d] BEFORE the call,
     gpu_* AFTER it.  gpu_scores is [4,B,H,cap] (I, Sbar, R, Z) or None."""
     rep = ParityReport()
@@ -79,7 +80,7 @@ def check_batch(k_in: torch.Tensor, v_in: torch.Tensor, q_in: torch.Tensor, seq_
     seq = seq_in.detach().cpu().numpy().astype(np.int32)
     B, H, cap, d = K.shape
     res = oracle.oracle_batch(K, Q, seq, budget=budget, alpha=alpha, lam=lam, W=W, beta=beta, T=T, eps=eps,
-                              mean_then_pool=mean_then_pool, head_mean=head_mean)
+                              mean_then_pool=mean_then_pool, head_mean=head_mean, gqa_mean_pool=gqa_mean_pool)
     gidx = gpu_idx.detach().cpu().numpy()
     k_raw_in, v_raw_in = raw_rows(k_in), raw_rows(v_in)
     k_raw_out = raw_rows(gpu_k) if gpu_k is not None else None

@@ -41,7 +41,7 @@ def run_and_check(rkv, wl, *, flags=0, W=4, beta=1, T=0.5, eps=1e-8, lam=None, c
     rep = check_batch(k0[sel], v0[sel], q0[sel], s0[sel], budget=spec.budget, alpha=spec.alpha, lam=lam, W=W,
                       beta=beta, T=T, eps=eps, gpu_idx=idx[sel], gpu_k=wl.k_cache[sel], gpu_v=wl.v_cache[sel],
                       gpu_seq=wl.seq_lens[sel], gpu_scores=comp.scores[:, sel],
-                      mean_then_pool=bool(flags & 4), head_mean=bool(flags & 8))
+                      mean_then_pool=bool(flags & 4), head_mean=bool(flags & 8), gqa_mean_pool=bool(flags & 16))
     return rep, comp
 
 
@@ -157,6 +157,19 @@ def test_head_mean_variant(rkv, flags, hkv, hq, budget, buffer):
     assert rep.compressed_heads == 2 * hkv
     assert rkv.rkv_launch_count_for(comp.desc, budget, buffer, spec.alpha, rkv.RKV_STAGE_SELECT) == \
         (2 if budget < 1000 else 4)
+
+
+@pytest.mark.parametrize("flags", [pytest.param(16 | 1, id="simt"), pytest.param(16, id="tri"),
+                                   pytest.param(16 | 2, id="rowblock")])
+@pytest.mark.parametrize("hkv,hq,alpha", [(2, 8, 8), (1, 7, 8), (2, 6, 5), (2, 2, 8)])
+def test_gqa_mean_pool_variant(rkv, flags, hkv, hq, alpha):
+    """Mean instead of max over the query heads of a group in Eq. 3 (flag RKV_FLAG_GQA_MEAN_POOL), on all three
+    scoring routes: even and odd group sizes, the general query-window length, and G = 1."""
+    spec = small_spec("gmp", batch=2, hkv=hkv, hq=hq, budget=256, buffer=64, alpha=alpha)
+    wl = ri.make_workload(spec, device="cuda", seed=191)
+    rep, _ = run_and_check(rkv, wl, flags=flags)
+    assert rep.ok(), rep.errors
+    assert rep.compressed_heads == 2 * hkv
 
 
 def test_fp32_small_shapes(rkv):
