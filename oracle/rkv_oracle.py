@@ -147,3 +147,30 @@ def oracle_gather(rows: np.ndarray, idx: np.ndarray) -> np.ndarray:
     lib.rkv_oracle_gather(rows.ctypes.data, _ptr(idx, ctypes.c_int32), idx.shape[0], row_bytes,
                           out.ctypes.data)
     return out
+
+
+def oracle_append(k_cache: np.ndarray, v_cache: np.ndarray, k_new: np.ndarray, v_new: np.ndarray,
+                  seq_lens: np.ndarray):
+    """Section 3.1's decode step on the cache, written out: the new token of sequence b becomes row seq_lens[b] of
+    every KV head (k_cache, v_cache [B, H, cap, d] of any dtype; k_new, v_new [B, H, d]); seq_lens[b] grows by one.
+    A sequence whose cache is full stays as it is.  Returns new arrays (k, v, seq_lens)."""
+    k, v, s = k_cache.copy(), v_cache.copy(), np.array(seq_lens, dtype=np.int32, copy=True)
+    cap = k.shape[2]
+    for b in range(k.shape[0]):
+        L = int(s[b])
+        if 0 <= L < cap:
+            for h in range(k.shape[1]):
+                k[b, h, L] = k_new[b, h]
+                v[b, h, L] = v_new[b, h]
+            s[b] = L + 1
+    return k, v, s
+
+
+def oracle_push_query(q_window: np.ndarray, q_new: np.ndarray, slot: int) -> np.ndarray:
+    """Algorithm 1's observation buffer of the last alpha queries kept as a ring: q_new [B, Hq, d] replaces row `slot`
+    of every head's window in q_window [B, Hq, alpha, d].  Returns a new array."""
+    q = q_window.copy()
+    for b in range(q.shape[0]):
+        for h in range(q.shape[1]):
+            q[b, h, slot] = q_new[b, h]
+    return q

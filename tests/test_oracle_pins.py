@@ -530,3 +530,38 @@ def test_gqa_mean_pool_variant():
     same = np.repeat(one, 3, axis=0)
     c = _run(K, same, budget=40, alpha=alpha, gqa_mean_pool=True)
     np.testing.assert_allclose(c.A, a.A, rtol=1e-12)
+
+
+def test_append_and_query_ring_semantics():
+    """Section 3.1's decode step and Algorithm 1's observation buffer, pinned by what they must leave behind:
+    only row seq_lens[b] of each head changes and holds the new token, a full cache stays as it is, alpha pushes
+    with slots 0..alpha-1 rebuild the window from the pushed rows, and the scores do not depend on the slot order
+    (Eq. 4 averages over the window's rows)."""
+    rng = np.random.default_rng(101)
+    B, H, cap, alpha = 3, 2, 12, 4
+    K, V = _rand(rng, B, H, cap, D), _rand(rng, B, H, cap, D)
+    kn, vn = _rand(rng, B, H, D), _rand(rng, B, H, D)
+    seq = np.array([5, 12, 0], np.int32)
+    k2, v2, s2 = oracle.oracle_append(K, V, kn, vn, seq)
+    assert s2.tolist() == [6, 12, 1]
+    for b, L in enumerate(seq):
+        changed = np.any(k2[b] != K[b], axis=-1) | np.any(v2[b] != V[b], axis=-1)          # [H, cap]
+        if L < cap:
+            assert changed[:, L].all() and changed.sum() == H
+            np.testing.assert_array_equal(k2[b, :, L], kn[b])
+            np.testing.assert_array_equal(v2[b, :, L], vn[b])
+        else:
+            assert not changed.any()
+    Hq = 4
+    Qw = _rand(rng, B, Hq, alpha, D)
+    pushed = [_rand(rng, B, Hq, D) for _ in range(alpha)]
+    q = Qw
+    for step, row in enumerate(pushed):
+        q = oracle.oracle_push_query(q, row, step % alpha)
+    np.testing.assert_array_equal(q, np.stack(pushed, axis=2))
+    # a rotated window gives the same scores
+    Kh = _rand(rng, 40, D)
+    a = _run(Kh, q[0], budget=20, alpha=alpha)
+    b_ = _run(Kh, np.roll(q[0], 1, axis=1), budget=20, alpha=alpha)
+    np.testing.assert_allclose(a.I, b_.I, rtol=1e-12)
+    np.testing.assert_array_equal(a.idx, b_.idx)
