@@ -208,6 +208,26 @@ RKV_API int rkv_compress_static(const rkv_desc_t *desc, void *k_cache, void *v_c
                         int32_t *seq_lens, int32_t budget, int32_t buffer, int32_t alpha, float lambda,
                         int32_t *out_idx, void *stream);
 
+/* The two cache updates of a decode step that surround the compression, so that a whole decode segment (buffer
+ * appends, then rkv_compress when seq_lens reaches budget + buffer: Section 3.1) can be enqueued, or captured in a
+ * CUDA graph, through this library alone.  Both only enqueue work on `stream` (two launches / one launch) and use no
+ * workspace.
+ *
+ * rkv_append: the newly generated token of every sequence enters the buffer part of its cache.
+ *   k_new, v_new [batch, n_kv_heads, head_dim] (device, dtype of the cache, 16-byte aligned) are copied to row
+ *   seq_lens[b] of every KV head of sequence b in k_cache / v_cache [batch, n_kv_heads, budget + buffer, head_dim];
+ *   then seq_lens[b] += 1.  A sequence whose cache is full (seq_lens[b] == budget + buffer: the caller has to compress
+ *   first) or whose length is invalid is left unchanged and RKV_ERR_INVALID_ARG is written to desc->device_status.
+ * rkv_push_query: Algorithm 1's observation buffer M_alpha as a ring.
+ *   q_new [batch, n_q_heads, head_dim] becomes row `slot` (0 <= slot < alpha; the caller passes its step counter modulo
+ *   alpha) of every query head's window in q_window [batch, n_q_heads, alpha, head_dim].  The order of the alpha rows
+ *   plays no part in the scores (Eq. 4 averages over them), so no row is ever moved.
+ * Return codes as for rkv_compress_ex. */
+RKV_API int rkv_append(const rkv_desc_t *desc, void *k_cache, void *v_cache, const void *k_new, const void *v_new,
+                       int32_t *seq_lens, int32_t budget, int32_t buffer, void *stream);
+RKV_API int rkv_push_query(const rkv_desc_t *desc, void *q_window, const void *q_new, int32_t alpha, int32_t slot,
+                           void *stream);
+
 /* Number of kernels a call launches (for launch accounting; the memset that precedes the prep kernel is not
  * counted).  rkv_launch_count_for() is exact for the given sizes; rkv_launch_count(), which does not know them, gives
  * the count for large caches (small ones run the select stage as one kernel instead of three). */

@@ -68,6 +68,8 @@ def lib():
         L.rkv_compress_stages.restype, L.rkv_compress_stages.argtypes = ctypes.c_int, [P] + ten + [U32]
         L.rkv_compress_host.restype, L.rkv_compress_host.argtypes = ctypes.c_int, [P] + ten
         L.rkv_compress_static.restype, L.rkv_compress_static.argtypes = ctypes.c_int, [P] + ten
+        L.rkv_append.restype, L.rkv_append.argtypes = ctypes.c_int, [P, VP, VP, VP, VP, VP, I32, I32, VP]
+        L.rkv_push_query.restype, L.rkv_push_query.argtypes = ctypes.c_int, [P, VP, VP, I32, I32, VP]
         L.rkv_launch_count.restype, L.rkv_launch_count.argtypes = ctypes.c_int, [P, U32]
         L.rkv_launch_count_for.restype, L.rkv_launch_count_for.argtypes = ctypes.c_int, [P, I32, I32, I32, U32]
         L.rkv_status_string.restype, L.rkv_status_string.argtypes = ctypes.c_char_p, [ctypes.c_int]
@@ -157,6 +159,17 @@ def rkv_compress_static(desc, k_cache, v_cache, q_window, seq_lens, budget, buff
     return lib().rkv_compress_static(ctypes.byref(desc), _ptr(k_cache), _ptr(v_cache), _ptr(q_window),
                                      _ptr(seq_lens), budget, buffer, alpha, float(lam), _ptr(out_idx),
                                      _stream(stream))
+
+
+def rkv_append(desc, k_cache, v_cache, k_new, v_new, seq_lens, budget, buffer, stream=None) -> int:
+    """The new token of every sequence enters its cache at row seq_lens[b]; seq_lens[b] += 1 (Section 3.1)."""
+    return lib().rkv_append(ctypes.byref(desc), _ptr(k_cache), _ptr(v_cache), _ptr(k_new), _ptr(v_new), _ptr(seq_lens),
+                            budget, buffer, _stream(stream))
+
+
+def rkv_push_query(desc, q_window, q_new, alpha, slot, stream=None) -> int:
+    """q_new becomes row `slot` of every query head's observation window (Algorithm 1's M_alpha as a ring)."""
+    return lib().rkv_push_query(ctypes.byref(desc), _ptr(q_window), _ptr(q_new), alpha, slot, _stream(stream))
 
 
 class Compressor:

@@ -312,6 +312,33 @@ int rkv_compress_host(const rkv_desc_t *desc, void *host_k_cache, void *host_v_c
     return RKV_OK;
 }
 
+int rkv_append(const rkv_desc_t *d, void *k_cache, void *v_cache, const void *k_new, const void *v_new, int32_t *seq_lens,
+               int32_t budget, int32_t buffer, void *stream)
+{
+    // shape checks as for the compression (alpha plays no part here: any valid value)
+    int rc = check_shapes(d, budget, buffer, 1, nullptr);
+    if (rc != RKV_OK) return rc;
+    if (!k_cache || !v_cache || !k_new || !v_new || !seq_lens) return RKV_ERR_INVALID_ARG;
+    if (!aligned16(k_cache) || !aligned16(v_cache) || !aligned16(k_new) || !aligned16(v_new)) return RKV_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(seq_lens) & 3u) return RKV_ERR_INVALID_ARG;
+    const int row_bytes = kHeadDim * (d->dtype == RKV_BF16 ? 2 : 4);
+    const cudaError_t e = launch_append(k_cache, v_cache, k_new, v_new, seq_lens, d->batch, d->n_kv_heads, budget + buffer,
+                                        row_bytes, d->device_status, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? RKV_OK : cuda_fail(e, "append launch");
+}
+
+int rkv_push_query(const rkv_desc_t *d, void *q_window, const void *q_new, int32_t alpha, int32_t slot, void *stream)
+{
+    if (!d || alpha < 1 || slot < 0 || slot >= alpha) return RKV_ERR_INVALID_ARG;
+    int rc = check_shapes(d, alpha + 1, 1, alpha, nullptr);        // descriptor fields and alpha against the group limit
+    if (rc != RKV_OK) return rc;
+    if (!q_window || !q_new || !aligned16(q_window) || !aligned16(q_new)) return RKV_ERR_INVALID_ARG;
+    const int row_bytes = kHeadDim * (d->dtype == RKV_BF16 ? 2 : 4);
+    const cudaError_t e = launch_push_query(q_window, q_new, d->batch, d->n_q_heads, alpha, slot, row_bytes,
+                                            static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? RKV_OK : cuda_fail(e, "push_query launch");
+}
+
 int rkv_launch_count(const rkv_desc_t *desc, uint32_t stage_mask)
 {
     int c = 0;

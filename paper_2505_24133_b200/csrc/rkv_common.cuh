@@ -123,6 +123,10 @@ cudaError_t launch_scores_sm100(const Params &p, cudaStream_t s);
 cudaError_t launch_scores_tri_sm100(const Params &p, cudaStream_t s);
 cudaError_t launch_select(const Params &p, cudaStream_t s);
 cudaError_t launch_gather(const Params &p, cudaStream_t s);
+cudaError_t launch_append(void *k_cache, void *v_cache, const void *k_new, const void *v_new, int32_t *seq_lens, int batch,
+                          int hkv, int cap, int row_bytes, int32_t *status, cudaStream_t s);
+cudaError_t launch_push_query(void *q_window, const void *q_new, int batch, int hq, int alpha, int slot, int row_bytes,
+                              cudaStream_t s);
 bool scores_sm100_available();
 bool select_is_fused(int cap_pad, int alpha);   // the select stage is one kernel (small caches) instead of three
 

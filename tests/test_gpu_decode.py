@@ -1,0 +1,133 @@
+"""The decode-step updates around the compression (rkv_append, rkv_push_query) against the oracle, and one whole
+decode segment -- appends until the buffer is full, then the compression -- eagerly and as one CUDA graph."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import rkv_inputs as ri
+from parity_util import check_batch, raw_rows
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def rkv():
+    from paper_2505_24133_b200 import build as b
+    b.build()
+    import paper_2505_24133_b200 as r
+    assert r.lib() is not None
+    return r
+
+
+def _spec(dtype="bf16", batch=3, budget=256, buffer=64, alpha=8):
+    return ri.CacheSpec("decode", 1, batch, 2, 8, 128, budget, buffer, alpha, 0.1, dtype, 16, 0.3, 0.05, 4, 8.0)
+
+
+def _desc(rkv, spec, status):
+    d = rkv.rkv_desc_default()
+    d.batch, d.n_kv_heads, d.n_q_heads = spec.folded_batch, spec.n_kv_heads, spec.n_q_heads
+    d.dtype = rkv.RKV_BF16 if spec.dtype == "bf16" else rkv.RKV_F32
+    d.device_status = status.data_ptr()
+    return d
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_append_matches_oracle_bit_for_bit(rkv, dtype):
+    spec = _spec(dtype)
+    lens = torch.tensor([spec.budget, spec.cap, 17])                 # the second cache is full: refused, flagged
+    wl = ri.make_workload(spec, device="cuda", seed=211, seq_lens=lens)
+    gen = torch.Generator(device="cuda").manual_seed(5)
+    k_new = torch.randn(spec.folded_batch, spec.n_kv_heads, 128, device="cuda", generator=gen).to(wl.k_cache.dtype)
+    v_new = torch.randn(spec.folded_batch, spec.n_kv_heads, 128, device="cuda", generator=gen).to(wl.k_cache.dtype)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    want_k, want_v, want_s = oracle.oracle_append(raw_rows(wl.k_cache), raw_rows(wl.v_cache), raw_rows(k_new),
+                                                  raw_rows(v_new), wl.seq_lens.cpu().numpy())
+    rc = rkv.rkv_append(_desc(rkv, spec, status), wl.k_cache, wl.v_cache, k_new, v_new, wl.seq_lens, spec.budget,
+                        spec.buffer)
+    assert rc == rkv.RKV_OK, rkv.rkv_status_string(rc)
+    torch.cuda.synchronize()
+    assert np.array_equal(raw_rows(wl.k_cache), want_k) and np.array_equal(raw_rows(wl.v_cache), want_v)
+    assert wl.seq_lens.cpu().numpy().tolist() == want_s.tolist() == [spec.budget + 1, spec.cap, 18]
+    assert int(status.item()) == 1                                    # RKV_ERR_INVALID_ARG: a full cache was met
+
+
+def test_push_query_matches_oracle_and_rejects_bad_slots(rkv):
+    spec = _spec()
+    wl = ri.make_workload(spec, device="cuda", seed=212)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    d = _desc(rkv, spec, status)
+    gen = torch.Generator(device="cuda").manual_seed(6)
+    want = raw_rows(wl.q_window)
+    for step in range(spec.alpha + 3):
+        q_new = torch.randn(spec.folded_batch, spec.n_q_heads, 128, device="cuda", generator=gen).to(torch.bfloat16)
+        want = oracle.oracle_push_query(want, raw_rows(q_new), step % spec.alpha)
+        assert rkv.rkv_push_query(d, wl.q_window, q_new, spec.alpha, step % spec.alpha) == rkv.RKV_OK
+    torch.cuda.synchronize()
+    assert np.array_equal(raw_rows(wl.q_window), want)
+    assert rkv.rkv_push_query(d, wl.q_window, q_new, spec.alpha, spec.alpha) == 1       # slot out of range
+    assert rkv.rkv_push_query(d, wl.q_window, q_new, spec.alpha, -1) == 1
+
+
+def test_decode_segment_eager_and_as_one_cuda_graph(rkv):
+    """budget cached tokens, then `buffer` decode steps (append + query push), then the compression: the state after
+    the segment agrees with the oracle driven by the same inputs, and a CUDA graph of the whole segment replays to
+    the same bits."""
+    spec = _spec(batch=2, budget=256, buffer=32)
+    steps = spec.buffer
+    wl = ri.make_workload(spec, device="cuda", seed=213, seq_lens=torch.tensor([spec.budget, spec.budget]))
+    gen = torch.Generator(device="cuda").manual_seed(7)
+    B, H, Hq = spec.folded_batch, spec.n_kv_heads, spec.n_q_heads
+    # new tokens: every fourth repeats an earlier key with a little noise, so that the redundancy term has work to do
+    k_steps = torch.randn(steps, B, H, 128, device="cuda", generator=gen)
+    k_steps[3::4] = k_steps[0:steps:4][: k_steps[3::4].shape[0]] + 0.05 * torch.randn_like(k_steps[3::4])
+    k_steps = k_steps.to(torch.bfloat16)
+    v_steps = torch.randn(steps, B, H, 128, device="cuda", generator=gen).to(torch.bfloat16)
+    q_steps = (2.0 * torch.randn(steps, B, Hq, 128, device="cuda", generator=gen)).to(torch.bfloat16)
+    k0, v0, q0, s0 = wl.k_cache.clone(), wl.v_cache.clone(), wl.q_window.clone(), wl.seq_lens.clone()
+    comp = rkv.Compressor(B, H, Hq, spec.budget, spec.buffer, spec.alpha, spec.lam)
+
+    def segment():
+        for t in range(steps):
+            assert rkv.rkv_append(comp.desc, wl.k_cache, wl.v_cache, k_steps[t], v_steps[t], wl.seq_lens, spec.budget,
+                                  spec.buffer) == rkv.RKV_OK
+            assert rkv.rkv_push_query(comp.desc, wl.q_window, q_steps[t], spec.alpha, t % spec.alpha) == rkv.RKV_OK
+        comp.compress(wl.k_cache, wl.v_cache, wl.q_window, wl.seq_lens)
+
+    segment()
+    torch.cuda.synchronize()
+    comp.check_status()
+    # the oracle's view of the same segment, up to the compression's inputs
+    ok_, ov_, os_ = raw_rows(k0), raw_rows(v0), s0.cpu().numpy()
+    oq = raw_rows(q0)
+    for t in range(steps):
+        ok_, ov_, os_ = oracle.oracle_append(ok_, ov_, raw_rows(k_steps[t]), raw_rows(v_steps[t]), os_)
+        oq = oracle.oracle_push_query(oq, raw_rows(q_steps[t]), t % spec.alpha)
+    assert os_.tolist() == [spec.cap, spec.cap]
+    as_bf16 = lambda a: torch.from_numpy(a.view(np.int16).copy()).view(torch.bfloat16).cuda()
+    rep = check_batch(as_bf16(ok_), as_bf16(ov_), as_bf16(oq), torch.from_numpy(os_), budget=spec.budget,
+                      alpha=spec.alpha, lam=spec.lam, W=4, beta=1, T=0.5, eps=1e-8, gpu_idx=comp.out_idx,
+                      gpu_k=wl.k_cache, gpu_v=wl.v_cache, gpu_seq=wl.seq_lens)
+    assert rep.ok(), rep.errors
+    assert rep.compressed_heads == B * H and wl.seq_lens.tolist() == [spec.budget, spec.budget]
+    eager = (comp.out_idx.clone(), wl.k_cache.clone(), wl.v_cache.clone(), wl.q_window.clone())
+
+    # the same segment as one graph
+    def restore():
+        wl.k_cache.copy_(k0), wl.v_cache.copy_(v0), wl.q_window.copy_(q0), wl.seq_lens.copy_(s0)
+
+    restore()
+    graph, side = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.graph(graph, stream=side):
+        segment()
+    torch.cuda.synchronize()
+    restore()
+    graph.replay()
+    torch.cuda.synchronize()
+    comp.check_status()
+    nb = spec.budget
+    assert torch.equal(comp.out_idx, eager[0]) and wl.seq_lens.tolist() == [spec.budget, spec.budget]
+    assert torch.equal(wl.k_cache[:, :, :nb].view(torch.int16), eager[1][:, :, :nb].view(torch.int16))
+    assert torch.equal(wl.v_cache[:, :, :nb].view(torch.int16), eager[2][:, :, :nb].view(torch.int16))
+    assert torch.equal(wl.q_window.view(torch.int16), eager[3].view(torch.int16))
