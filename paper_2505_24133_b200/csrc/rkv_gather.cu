@@ -70,12 +70,17 @@ cudaError_t launch_gather(const Params &p, cudaStream_t s)
     cudaError_t e;
     if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
     if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
-    const bool small = streams < 8u * (unsigned)sms;        // fewer than 8 streams per SM: cut the rows in 4 slices
+    // Few streams: cut the rows into column slices, as many (4, 2) as still fit the SMs in one wave of resident blocks
+    // (8 per SM): a second, partly filled wave would leave SMs idle for much of the kernel.
+    const unsigned wave = 8u * (unsigned)sms;
+    const int split = streams * 4u <= wave ? 4 : (streams * 2u <= wave ? 2 : (streams < wave ? 4 : 1));
     if (p.dtype == RKV_BF16) {
-        if (small) gather_kernel<16, 4><<<streams * 4u, kGatherThreads, 0, s>>>(p);
+        if (split == 4) gather_kernel<16, 4><<<streams * 4u, kGatherThreads, 0, s>>>(p);
+        else if (split == 2) gather_kernel<16, 2><<<streams * 2u, kGatherThreads, 0, s>>>(p);
         else gather_kernel<16, 1><<<streams, kGatherThreads, 0, s>>>(p);
     } else {
-        if (small) gather_kernel<32, 4><<<streams * 4u, kGatherThreads, 0, s>>>(p);
+        if (split == 4) gather_kernel<32, 4><<<streams * 4u, kGatherThreads, 0, s>>>(p);
+        else if (split == 2) gather_kernel<32, 2><<<streams * 2u, kGatherThreads, 0, s>>>(p);
         else gather_kernel<32, 1><<<streams, kGatherThreads, 0, s>>>(p);
     }
     return cudaGetLastError();
