@@ -34,7 +34,7 @@ NCU_TRAFFIC = {
     # profiles/all_kernels_llama8b_b1.md (cold caches: the scoring passes read K from DRAM there)
     # (the select stage is one kernel at this size: no row_stats / importance launches)
     "llama8b_b1": {"prep": 76.80e6, "scores_pass1": 85.95e6, "scores_list": 1.19e6, "scores_pass2": 81.84e6,
-                   "select": 10.67e6, "gather": 212.43e6},
+                   "select": 10.67e6, "gather": 209.43e6},
 }
 
 
