@@ -3,9 +3,13 @@ select, gather) over one batch of synthetic caches.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
 
-Prints ONE JSON line (rank 0).  value = cached tokens scored per second over all ranks with the inputs already
-in HBM; e2e = the same through the host-buffer entry point with the copies inside the timed region; roofline =
-the dominant kernel against the measured peak; cpu_baseline = the CPU oracle timed on this machine's host cores.
+Prints ONE JSON line (rank 0).  The headline workload is the largest configuration (the Qwen-14B cache shape:
+12 288 head-problems of 4224 cached tokens, 26.6 GB of K+V; one compressing firing per step).  value = cached
+tokens scored per second over all ranks with the inputs already in HBM; e2e = the same through the host-buffer
+entry point with the copies inside the timed region; roofline = the slower of the two tensor-core scoring passes
+against the measured dense bf16 peak, roofline_hbm = the HBM-bound kernels against the measured copy bandwidth;
+cpu_baseline = the CPU oracle timed on this machine's host cores; configs = the other configurations (and the
+default one under settings that defeat the two-pass shortcut), each with its own per-kernel table.
 """
 from __future__ import annotations
 
@@ -28,22 +32,26 @@ import rkv_inputs as ri  # noqa: E402
 
 METRIC = "cached tokens scored/s (KV compressions/s alongside)"
 UNIT = "tokens/s"
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch, from the ncu captures summarised
-# under profiles/: {workload: {kernel: bytes}}
-NCU_TRAFFIC = {
-    # profiles/all_kernels_llama8b_b1.md (cold caches: the scoring passes read K from DRAM there)
-    # (the select stage is one kernel at this size: no row_stats / importance launches)
-    "llama8b_b1": {"prep": 76.80e6, "scores_pass1": 85.95e6, "scores_list": 1.19e6, "scores_pass2": 81.84e6,
-                   "select": 10.67e6, "gather": 209.43e6},
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per head-problem of one launch, from the ncu capture
+# of a 256-head-problem slice at n = 4216 summarised in profiles/all_kernels_llama8b_b16_batch1.md.  Every kernel
+# works head by head, so a full launch's traffic is this figure times the launch's head-problems (only taken for
+# workloads of that cache size).  None = the kernel has changed since the counters were taken.
+NCU_TRAFFIC_PER_HEAD_N4216 = {
+    "prep": (276.32e6 + 13.92e6) / 256, "scores_pass1": None, "scores_list": (4.33e6 + 0.0) / 256,
+    "scores_pass2": (323.53e6 + 6.96e6) / 256, "row_stats": 34.62e6 / 256, "importance": 34.63e6 / 256,
+    "select": 8.68e6 / 256, "gather": (531.44e6 + 472.86e6) / 256,
 }
+DEFAULT_WORKLOAD = "qwen14b_b32"
 
 
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=40)
+    ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="llama8b_b1", choices=[c for c in ri.CONFIG_ORDER if c != "tiny"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=[c for c in ri.CONFIG_ORDER if c != "tiny"])
+    ap.add_argument("--no-configs", action="store_true",
+                    help="only the named workload, without the other configurations under `configs`")
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--beta", type=int, default=None)
     ap.add_argument("--threshold", type=float, default=None)
@@ -132,11 +140,6 @@ def tokens_per_step(spec: ri.CacheSpec) -> int:
 def sim_flops_per_step(spec: ri.CacheSpec) -> float:
     n = spec.cap - spec.alpha
     return 2.0 * n * n * spec.head_dim * spec.head_problems    # Eq. 5: the full n x n x d product per head
-
-
-def local_spec(spec: ri.CacheSpec, rank: int, world: int) -> ri.CacheSpec:
-    """Weak scaling: every rank gets the whole workload's shape (its own sequences), seeded by rank."""
-    return spec
 
 
 # ------------------------------------------------------------------------------------------------- reference arm
@@ -234,6 +237,272 @@ def run_stream(args, rkv, rd, dev, rank, world, spec):
 
 
 # ------------------------------------------------------------------------------------------------- main arm
+def variant_kwargs(args, rkv):
+    kw = {}
+    if args.beta is not None:
+        kw["beta"] = args.beta
+    if args.threshold is not None:
+        kw["sim_threshold"] = args.threshold
+    if args.pool_w is not None:
+        kw["pool_w"] = args.pool_w
+    if args.mean_then_pool or args.head_mean or args.gqa_mean_pool:
+        kw["flags"] = (rkv.RKV_FLAG_MEAN_THEN_POOL if args.mean_then_pool else 0) | \
+                      (rkv.RKV_FLAG_HEAD_MEAN if args.head_mean else 0) | \
+                      (rkv.RKV_FLAG_GQA_MEAN_POOL if args.gqa_mean_pool else 0)
+    return kw
+
+
+class Timed:
+    """One workload resident in HBM with its pristine copy; steps restore the caches outside the timed events (or
+    cycle through replicas when they fit), so that every step compresses full caches that are not in L2."""
+
+    def __init__(self, rkv, rd, dev, wl, mem_gb, steps_needed):
+        self.rkv, self.rd, self.dev, self.wl, self.spec = rkv, rd, dev, wl, wl.spec
+        self.bytes_per_replica = 2 * wl.k_cache.numel() * wl.k_cache.element_size()
+        n_rep = max(1, min(steps_needed, int(mem_gb * 2 ** 30) // self.bytes_per_replica))
+        self.contiguous = n_rep >= steps_needed
+        self.reps = [(wl.k_cache.clone(), wl.v_cache.clone(), wl.seq_lens.clone()) for _ in range(n_rep)]
+        self.flush = torch.empty(256 * 2 ** 20, dtype=torch.uint8, device=dev)     # > L2 (126 MB)
+        self.stream = torch.cuda.current_stream()
+
+    def restore(self, i):
+        k, v, s = self.reps[i % len(self.reps)]
+        k.copy_(self.wl.k_cache)
+        v.copy_(self.wl.v_cache)
+        s.copy_(self.wl.seq_lens)
+
+    def step(self, comp, i):
+        k, v, s = self.reps[i % len(self.reps)]
+        comp.compress(k, v, self.wl.q_window, s, stream=self.stream)
+
+    def l2_note(self):
+        return (f"{len(self.reps)} input replicas of {self.bytes_per_replica / 2**20:.0f} MiB cycled, each used once"
+                if self.contiguous else "inputs restored and a 256 MiB buffer written between timed steps")
+
+    def run_timed(self, comp, K, W, sampler=None):
+        """W warm-up steps, then K steps timed with CUDA events on the launching stream; returns this rank's ms."""
+        rd = self.rd
+        for i in range(W):
+            if not self.contiguous:
+                self.restore(i)
+            self.step(comp, i)
+        torch.cuda.synchronize()
+        comp.check_status()
+        if sampler is not None:
+            sampler.start()
+            time.sleep(0.3)
+        rd.barrier()
+        torch.cuda.synchronize()
+        if self.contiguous:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(self.stream)
+            for i in range(K):
+                self.step(comp, W + i)
+            e1.record(self.stream)
+            torch.cuda.synchronize()
+            ms_total = e0.elapsed_time(e1)
+        else:
+            ms_total = 0.0
+            for i in range(K):
+                self.restore(i)
+                self.flush.fill_(i & 255)                   # evicts the restored caches from L2
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(self.stream)
+                self.step(comp, i)
+                e1.record(self.stream)
+                torch.cuda.synchronize()
+                ms_total += e0.elapsed_time(e1)
+        rd.barrier()
+        torch.cuda.synchronize()
+        comp.check_status()
+        return ms_total
+
+    def close(self):
+        self.reps = None
+        self.flush = None
+        torch.cuda.empty_cache()
+
+
+def kernel_table(rkv, timed: Timed, kw, KB, peaks):
+    """The same steps with an event after every kernel: per-kernel times, the work each launch had to do, and the
+    rate against the roofline that bounds it."""
+    spec, wl, dev = timed.spec, timed.wl, timed.dev
+    comp_ev = rkv.Compressor(spec.folded_batch, spec.n_kv_heads, spec.n_q_heads, spec.budget, spec.buffer, spec.alpha,
+                             spec.lam, dtype=spec.torch_dtype, device=dev, stage_events=True, **kw)
+    names = list(comp_ev.KERNEL_NAMES)
+    kernel_ms = [0.0] * len(names)
+    tiles_executed = pairs2 = moved_rows = 0
+    for i in range(KB):
+        timed.restore(i)
+        timed.flush.fill_(i & 255)
+        timed.step(comp_ev, i)
+        torch.cuda.synchronize()
+        for s_i, t in enumerate(comp_ev.kernel_ms()):
+            kernel_ms[s_i] += t / KB
+        if i == 0:
+            tiles_executed = int(comp_ev.counters[0].item())
+            pairs2 = int(comp_ev.counters[5].item())
+            idx = comp_ev.out_idx
+            moved_rows = int((idx != torch.arange(spec.budget, device=dev, dtype=idx.dtype)).sum().item())
+    comp_ev.check_status()
+    n = spec.cap - spec.alpha
+    esz = wl.k_cache.element_size()
+    row = spec.head_dim * esz
+    P = spec.head_problems
+    T = (n + 127) // 128
+    q_cols = -(-(spec.n_q_heads // spec.n_kv_heads) * spec.alpha // 16) * 16 + 16
+    tile_flops = 2.0 * 128 ** 3
+    rule_on = comp_ev.desc.beta > 0 and comp_ev.desc.sim_threshold < 1.0
+    pass1_tiles = P * T if rule_on else 0              # every row tile meets the last key tile once
+    pass1_flops = pass1_tiles * tile_flops + P * T * 2.0 * 128 * q_cols * 128
+    pass2_flops = max(tiles_executed - pass1_tiles, 0) * tile_flops
+    pass2_useful = pairs2 * 2.0 * 128 * 128            # listed tokens x keys of the streamed tiles x 2 d
+    # algorithmic work per launch: bytes a kernel has to move / flops it has to execute, nothing it merely could
+    work = {
+        "prep": ("hbm", P * (n * row + spec.cap * 8)),                          # K once; r_i and Kbar_i.Kbar_i out
+        "scores_pass1": ("tensor", pass1_flops),
+        "scores_list": ("hbm", P * n * 8),
+        "scores_pass2": ("tensor", pass2_flops),
+        "row_stats": ("hbm", P * spec.alpha * n * 4),
+        "importance": ("hbm", P * (spec.alpha + 1) * n * 4),
+        "select": ("hbm", P * (2 * n * 4 + spec.budget * 4)),
+        "gather": ("hbm", moved_rows * row * 2 * 2 + P * spec.budget * 4),      # K and V rows that move: read + write
+    }
+    kernels = {}
+    for nm, ms in zip(names, kernel_ms):
+        bound, amount = work[nm]
+        rate = amount / (ms * 1e-3) if ms > 0 else 0.0
+        if bound == "tensor":
+            kernels[nm] = {"ms": ms, "tflops": rate / 1e12, "frac_of_bf16_peak": rate / 1e12 / peaks["bf16_tflops"],
+                           "flops_per_launch": amount}
+        else:
+            kernels[nm] = {"ms": ms, "gbs": rate / 1e9, "frac_of_hbm_peak": rate / 1e9 / peaks["hbm_gbs"],
+                           "bytes_per_launch": amount}
+    if kernel_ms[3] > 0:
+        kernels["scores_pass2"]["useful_tflops"] = pass2_useful / (kernel_ms[3] * 1e-3) / 1e12
+    scoring_ms = kernel_ms[1] + kernel_ms[2] + kernel_ms[3]
+    scoring = {"tiles_executed": tiles_executed, "tiles_full_matrix": P * T * T,
+               "pass2_token_tile_pairs": pairs2,
+               "executed_tflops": (pass1_flops + pass2_flops) / (scoring_ms * 1e-3) / 1e12,
+               "full_matrix_equivalent_tflops": sim_flops_per_step(spec) / (scoring_ms * 1e-3) / 1e12}
+    del comp_ev
+    return kernels, scoring
+
+
+def rooflines(spec, kernels, scoring, peaks):
+    """roofline: the slower (lower fraction of its peak) of the two tcgen05 scoring passes on the tile products it
+    executed.  roofline_hbm: the HBM-bound kernels that move the bulk of the bytes."""
+    cands = [nm for nm in ("scores_pass1", "scores_pass2") if kernels[nm]["ms"] > 0 and kernels[nm]["flops_per_launch"] > 0]
+    n = spec.cap - spec.alpha
+    per_head = NCU_TRAFFIC_PER_HEAD_N4216 if n == 4216 else {}
+
+    def traffic(nm):
+        t = per_head.get(nm)
+        return None if t is None else t * spec.head_problems
+
+    roofline = None
+    if cands:
+        nm = min(cands, key=lambda c: kernels[c]["frac_of_bf16_peak"])
+        k = kernels[nm]
+        roofline = {"kernel": nm, "bound": "tensor", "achieved": k["tflops"], "peak": peaks["bf16_tflops"],
+                    "unit": "TFLOP/s", "frac": k["frac_of_bf16_peak"],
+                    "peak_source": f"{peaks['source']} burst cuBLAS bf16",
+                    "traffic": traffic(nm), "flops_per_launch": k["flops_per_launch"],
+                    "counts": "128x128x128 tile products the kernel executed (counted by the kernel)",
+                    "full_matrix_equivalent_tflops": scoring["full_matrix_equivalent_tflops"],
+                    "other_pass": {c: kernels[c]["frac_of_bf16_peak"] for c in cands if c != nm}}
+    hbm = {}
+    for nm in ("gather", "prep"):
+        k = kernels[nm]
+        hbm[nm] = {"bound": "hbm", "achieved": k["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                   "frac": k["frac_of_hbm_peak"], "peak_source": f"{peaks['source']} copy",
+                   "traffic": traffic(nm), "bytes_per_launch": k["bytes_per_launch"]}
+    return roofline, hbm
+
+
+def measure_e2e(rkv, rd, dev, wl, kw, KE, toks):
+    """The host-buffer entry point, copies inside the timed region (wall clock around call + synchronise)."""
+    spec = wl.spec
+    esz = wl.k_cache.element_size()
+    row = spec.head_dim * esz
+    ch = rkv.Compressor(spec.folded_batch, spec.n_kv_heads, spec.n_q_heads, spec.budget, spec.buffer, spec.alpha,
+                        spec.lam, dtype=spec.torch_dtype, device=dev, host_staging=True, **kw)
+    hk = torch.empty(wl.k_cache.shape, dtype=wl.k_cache.dtype, pin_memory=True)
+    hv = torch.empty(wl.v_cache.shape, dtype=wl.v_cache.dtype, pin_memory=True)
+    hq = wl.q_window.cpu().pin_memory()
+    hs = wl.seq_lens.cpu().pin_memory()
+    hi = torch.empty(spec.folded_batch, spec.n_kv_heads, spec.budget, dtype=torch.int32).pin_memory()
+    stream = torch.cuda.current_stream()
+    ms_e2e = 0.0
+    for i in range(KE + 1):                       # the first step warms up
+        hk.copy_(wl.k_cache)
+        hv.copy_(wl.v_cache)
+        hs.copy_(wl.seq_lens)
+        rd.barrier()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        ch.compress_host(hk, hv, hq, hs, hi, stream=stream)
+        torch.cuda.synchronize()                  # the step's results are on the host from here
+        if i > 0:
+            ms_e2e += (time.perf_counter() - t0) * 1e3
+    ch.check_status()
+    e2e_value, _ = rd.whole_job_rate(toks * KE, ms_e2e, dev)
+    h2d = 2 * wl.k_cache.numel() * esz + wl.q_window.numel() * esz + wl.seq_lens.numel() * 4
+    d2h = 2 * spec.head_problems * spec.budget * row + spec.head_problems * spec.budget * 4 + wl.seq_lens.numel() * 4
+    del ch, hk, hv
+    torch.cuda.empty_cache()
+    return {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+            "steps": KE, "ms_per_step": ms_e2e / KE,
+            "how": "rkv_compress_host from pinned host buffers; wall clock around the call and a synchronise"}
+
+
+def measure_cpu(wl, desc, args):
+    """The oracle as it stands on this machine's cores: a bounded sample (about 12 s) of the same workload."""
+    import oracle
+    spec = wl.spec
+    n = spec.cap - spec.alpha
+    cores = os.cpu_count() or 1
+    heads = max(spec.n_kv_heads, min(spec.head_problems, int(cores * 2.5e9 / (n * n * spec.head_dim))))
+    seqs = max(1, heads // spec.n_kv_heads)
+    Kh = wl.k_cache[:seqs].float().cpu().numpy()
+    Qh = wl.q_window[:seqs].float().cpu().numpy()
+    oracle.build()
+    seq_h = wl.seq_lens[:seqs].cpu().numpy()
+    passes, t0 = 0, time.perf_counter()
+    while passes < 1 or (time.perf_counter() - t0 < 12.0 and passes < 200):
+        res = oracle.oracle_batch(Kh, Qh, seq_h, budget=spec.budget, alpha=spec.alpha, lam=spec.lam, W=desc.pool_w,
+                                  beta=desc.beta, T=desc.sim_threshold, eps=desc.eps, want_scores=False,
+                                  mean_then_pool=args.mean_then_pool, head_mean=args.head_mean,
+                                  gqa_mean_pool=args.gqa_mean_pool)
+        passes += 1
+    dt = time.perf_counter() - t0
+    return {"value": passes * seqs * spec.n_kv_heads * n / dt, "unit": UNIT, "cores": res.threads, "kind": "oracle",
+            "sample": f"first {seqs * spec.n_kv_heads} of {spec.head_problems} head-problems, {passes} passes, {dt:.1f} s"}
+
+
+def side_config(rkv, rd, dev, wl, kw, K, W, mem_gb, peaks):
+    """A configuration other than the headline one: ms per step, rates and the per-kernel table."""
+    spec = wl.spec
+    timed = Timed(rkv, rd, dev, wl, mem_gb, K + W)
+    comp = rkv.Compressor(spec.folded_batch, spec.n_kv_heads, spec.n_q_heads, spec.budget, spec.buffer, spec.alpha,
+                          spec.lam, dtype=spec.torch_dtype, device=dev, **kw)
+    ms_total = timed.run_timed(comp, K, W)
+    toks = tokens_per_step(spec)
+    value, ms_slowest = rd.whole_job_rate(toks * K, ms_total, dev)
+    kernels, scoring = kernel_table(rkv, timed, kw, min(K, 5), peaks)
+    roofline, hbm = rooflines(spec, kernels, scoring, peaks)
+    out = {"head_problems": spec.head_problems, "n": spec.cap - spec.alpha, "steps": K,
+           "ms_per_step": ms_slowest / K, "tokens_per_s": value,
+           "compressions_per_s": value / toks * spec.folded_batch,
+           "beta": comp.desc.beta, "sim_threshold": comp.desc.sim_threshold, "l2": timed.l2_note(),
+           "kernels": {nm: {k2: v2 for k2, v2 in kv.items() if not k2.endswith("_per_launch")} for nm, kv in kernels.items()},
+           "scoring": scoring, "roofline": roofline and {k2: roofline[k2] for k2 in ("kernel", "achieved", "frac")},
+           "roofline_hbm": {nm: {"achieved": h["achieved"], "frac": h["frac"]} for nm, h in hbm.items()}}
+    del comp
+    timed.close()
+    return out
+
+
 def main():
     args = parse_args()
     from paper_2505_24133_b200 import dist as rd
@@ -256,201 +525,49 @@ def main():
         return
     K, W = args.steps, max(args.warmup, 3)
     peaks = measured_peaks()
+    kw = variant_kwargs(args, rkv)
 
-    # ---- inputs: one pristine workload per rank, replicated so that every step compresses fresh caches
+    # ---- the headline workload: one pristine copy per rank, restored (or replicated) so that every step compresses
+    # full caches
     wl = ri.make_workload(spec, device=dev, seed=ri.BASE_SEED + 1000 * rank + ri.CONFIG_ORDER.index(args.workload))
-    bytes_per_replica = 2 * wl.k_cache.numel() * wl.k_cache.element_size()
-    budget_bytes = int(args.mem_gb * 2 ** 30)
-    n_rep = max(1, min(K + W, budget_bytes // bytes_per_replica))
-    contiguous = n_rep >= K + W                     # else: restore between steps, outside the timed events
-    reps = [(wl.k_cache.clone(), wl.v_cache.clone(), wl.seq_lens.clone()) for _ in range(n_rep)]
-    flush = torch.empty(256 * 2 ** 20, dtype=torch.uint8, device=dev)     # > L2 (126 MB)
-
-    def restore(i):
-        reps[i][0].copy_(wl.k_cache)
-        reps[i][1].copy_(wl.v_cache)
-        reps[i][2].copy_(wl.seq_lens)
-
-    kw = {}
-    if args.beta is not None:
-        kw["beta"] = args.beta
-    if args.threshold is not None:
-        kw["sim_threshold"] = args.threshold
-    if args.pool_w is not None:
-        kw["pool_w"] = args.pool_w
-    if args.mean_then_pool or args.head_mean or args.gqa_mean_pool:
-        kw["flags"] = (rkv.RKV_FLAG_MEAN_THEN_POOL if args.mean_then_pool else 0) | \
-                      (rkv.RKV_FLAG_HEAD_MEAN if args.head_mean else 0) | \
-                      (rkv.RKV_FLAG_GQA_MEAN_POOL if args.gqa_mean_pool else 0)
+    timed = Timed(rkv, rd, dev, wl, args.mem_gb, K + W)
     comp = rkv.Compressor(spec.folded_batch, spec.n_kv_heads, spec.n_q_heads, spec.budget, spec.buffer, spec.alpha,
                           spec.lam, dtype=spec.torch_dtype, device=dev, **kw)
     launches_per_step = rkv.rkv_launch_count_for(comp.desc, spec.budget, spec.buffer, spec.alpha, rkv.RKV_STAGE_ALL)
-    stream = torch.cuda.current_stream()
-
-    def step(i, c=comp):
-        k, v, s = reps[i % n_rep]
-        c.compress(k, v, wl.q_window, s, stream=stream)
-
-    # ---- pass A: the headline number
-    for i in range(W):
-        step(i)
-    torch.cuda.synchronize()
-    comp.check_status()
     sampler = ClockSampler(local_rank)
-    sampler.start()
-    time.sleep(0.3)
-    rd.barrier()
-    torch.cuda.synchronize()
-    if contiguous:
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        for i in range(K):
-            step(W + i)
-        e1.record(stream)
-        torch.cuda.synchronize()
-        ms_total = e0.elapsed_time(e1)
-    else:
-        ms_total = 0.0
-        for i in range(K):
-            restore(i % n_rep)
-            flush.fill_(i & 255)                   # evicts the restored caches from L2
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record(stream)
-            step(i)
-            e1.record(stream)
-            torch.cuda.synchronize()
-            ms_total += e0.elapsed_time(e1)
-    rd.barrier()
-    torch.cuda.synchronize()
+    ms_total = timed.run_timed(comp, K, W, sampler)
     clocks = sampler.stop()
-    comp.check_status()
     toks = tokens_per_step(spec)
     value, ms_slowest = rd.whole_job_rate(toks * K, ms_total, dev)
     ms_per_step = ms_slowest / K
-
-    # ---- pass B: the same steps with per-kernel events, for the roofline of the dominant kernel
-    comp_ev = rkv.Compressor(spec.folded_batch, spec.n_kv_heads, spec.n_q_heads, spec.budget, spec.buffer, spec.alpha,
-                             spec.lam, dtype=spec.torch_dtype, device=dev, stage_events=True, **kw)
-    names = list(comp_ev.KERNEL_NAMES)
-    kernel_ms = [0.0] * len(names)
-    KB = min(K, 20)
-    tiles_executed = moved_rows = 0
-    for i in range(KB):
-        restore(i % n_rep)
-        flush.fill_(i & 255)
-        step(i, comp_ev)
-        torch.cuda.synchronize()
-        for s_i, t in enumerate(comp_ev.kernel_ms()):
-            kernel_ms[s_i] += t / KB
-        if i == 0:
-            tiles_executed = int(comp_ev.counters[0].item())
-            idx = comp_ev.out_idx
-            moved_rows = int((idx != torch.arange(spec.budget, device=dev, dtype=idx.dtype)).sum().item())
     n = spec.cap - spec.alpha
-    esz = wl.k_cache.element_size()
-    row = spec.head_dim * esz
-    P = spec.head_problems
-    T = (n + 127) // 128
-    depth = 1                                          # key tiles every token meets in the first scoring pass
-    q_cols = -(-(spec.n_q_heads // spec.n_kv_heads) * spec.alpha // 16) * 16 + 16
-    tile_flops = 2.0 * 128 ** 3
-    pass1_tiles = P * sum(min(T - I, depth) for I in range(T))
-    pass1_flops = pass1_tiles * tile_flops + P * T * 2.0 * 128 * q_cols * 128
-    pass2_flops = max(tiles_executed - pass1_tiles, 0) * tile_flops
-    # algorithmic work per launch: bytes a kernel has to move / flops it has to execute, nothing it merely could
-    work = {
-        "prep": ("hbm", P * (n * row + spec.cap * 8)),                          # K once; r_i and Kbar_i.Kbar_i out
-        "scores_pass1": ("tensor", pass1_flops),
-        "scores_list": ("hbm", P * n * 8),
-        "scores_pass2": ("tensor", pass2_flops),
-        "row_stats": ("hbm", P * spec.alpha * n * 4),
-        "importance": ("hbm", P * (spec.alpha + 1) * n * 4),
-        "select": ("hbm", P * (2 * n * 4 + spec.budget * 4)),
-        "gather": ("hbm", moved_rows * row * 2 * 2 + P * spec.budget * 4),      # K and V rows that move: read + write
-    }
-    kernels = {}
-    for nm, ms in zip(names, kernel_ms):
-        bound, amount = work[nm]
-        rate = amount / (ms * 1e-3) if ms > 0 else 0.0
-        kernels[nm] = {"ms": ms, ("tflops" if bound == "tensor" else "gbs"): rate / (1e12 if bound == "tensor" else 1e9)}
-    dom = max(range(len(names)), key=lambda s_i: kernel_ms[s_i])
-    dom_name = names[dom]
-    bound, amount = work[dom_name]
-    full_matrix_tflops = sim_flops_per_step(spec) / ((kernel_ms[1] + kernel_ms[2] + kernel_ms[3]) * 1e-3) / 1e12
-    if bound == "tensor":
-        ach = kernels[dom_name]["tflops"]
-        roofline = {"kernel": dom_name, "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"],
-                    "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops"],
-                    "peak_source": f"{peaks['source']} burst cuBLAS bf16",
-                    "traffic": NCU_TRAFFIC.get(spec.name, {}).get(dom_name),
-                    "flops_per_launch": amount}
-    else:
-        ach = kernels[dom_name]["gbs"]
-        roofline = {"kernel": dom_name, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                    "frac": ach / peaks["hbm_gbs"], "peak_source": f"{peaks['source']} copy",
-                    "traffic": NCU_TRAFFIC.get(spec.name, {}).get(dom_name), "bytes_per_launch": amount}
-    scoring = {"tiles_executed": tiles_executed, "tiles_full_matrix": P * T * T,
-               "executed_tflops": (pass1_flops + pass2_flops) / ((kernel_ms[1] + kernel_ms[2] + kernel_ms[3]) * 1e-3) / 1e12,
-               "full_matrix_equivalent_tflops": full_matrix_tflops}
 
-    # ---- e2e: the host-buffer entry point, copies inside the timed region
+    kernels, scoring = kernel_table(rkv, timed, kw, min(K, 10), peaks)
+    roofline, roofline_hbm = rooflines(spec, kernels, scoring, peaks)
+    desc_view = {"pool_w": comp.desc.pool_w, "beta": comp.desc.beta, "sim_threshold": comp.desc.sim_threshold}
+    l2_note = timed.l2_note()
+    timed.close()
+
     e2e = None
     if not args.no_e2e:
-        KE = min(K, 8)
-        ch = rkv.Compressor(spec.folded_batch, spec.n_kv_heads, spec.n_q_heads, spec.budget, spec.buffer, spec.alpha,
-                            spec.lam, dtype=spec.torch_dtype, device=dev, host_staging=True, **kw)
-        hk0, hv0 = wl.k_cache.cpu(), wl.v_cache.cpu()
-        hq = wl.q_window.cpu().pin_memory()
-        hosts = [(hk0.clone().pin_memory(), hv0.clone().pin_memory(), wl.seq_lens.cpu().pin_memory(),
-                  torch.empty(spec.folded_batch, spec.n_kv_heads, spec.budget, dtype=torch.int32).pin_memory())
-                 for _ in range(min(KE + 1, 3))]
-
-        def host_step(i):
-            hk, hv, hs, hi = hosts[i % len(hosts)]
-            ch.compress_host(hk, hv, hq, hs, hi, stream=stream)
-
-        host_step(0)
-        torch.cuda.synchronize()
-        ms_e2e = 0.0
-        for i in range(KE):
-            hk, hv, hs, hi = hosts[i % len(hosts)]
-            hk.copy_(hk0)
-            hv.copy_(hv0)
-            hs.copy_(wl.seq_lens.cpu())
-            rd.barrier()
-            torch.cuda.synchronize()
-            t0 = time.perf_counter()
-            host_step(i)
-            torch.cuda.synchronize()              # the step's results are on the host from here
-            ms_e2e += (time.perf_counter() - t0) * 1e3
-        ch.check_status()
-        e2e_value, _ = rd.whole_job_rate(toks * KE, ms_e2e, dev)
-        h2d = 2 * wl.k_cache.numel() * esz + wl.q_window.numel() * esz + wl.seq_lens.numel() * 4
-        d2h = 2 * spec.head_problems * spec.budget * row + spec.head_problems * spec.budget * 4 + wl.seq_lens.numel() * 4
-        e2e = {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-               "steps": KE, "ms_per_step": ms_e2e / KE}
-
-    # ---- cpu baseline: the oracle on this machine's cores, a bounded sample of the same workload (rank 0, N = 1)
+        e2e = measure_e2e(rkv, rd, dev, wl, kw, min(K, 2 if spec.head_problems > 4096 else 8), toks)
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        import oracle
-        cores = os.cpu_count() or 1
-        heads = max(spec.n_kv_heads, min(spec.head_problems, int(cores * 2.5e9 / (n * n * spec.head_dim))))
-        seqs = max(1, heads // spec.n_kv_heads)
-        d = comp.desc
-        Kh = wl.k_cache[:seqs].float().cpu().numpy()
-        Qh = wl.q_window[:seqs].float().cpu().numpy()
-        oracle.build()
-        seq_h = wl.seq_lens[:seqs].cpu().numpy()
-        passes, t0 = 0, time.perf_counter()
-        while passes < 1 or (time.perf_counter() - t0 < 12.0 and passes < 200):      # about 12 s of CPU work
-            res = oracle.oracle_batch(Kh, Qh, seq_h, budget=spec.budget, alpha=spec.alpha, lam=spec.lam, W=d.pool_w,
-                                      beta=d.beta, T=d.sim_threshold, eps=d.eps, want_scores=False,
-                                      mean_then_pool=args.mean_then_pool, head_mean=args.head_mean, gqa_mean_pool=args.gqa_mean_pool)
-            passes += 1
-        dt = time.perf_counter() - t0
-        cpu = {"value": passes * seqs * spec.n_kv_heads * n / dt, "unit": UNIT, "cores": res.threads, "kind": "oracle",
-               "sample": f"first {seqs * spec.n_kv_heads} of {spec.head_problems} head-problems, {passes} passes, {dt:.1f} s"}
+        cpu = measure_cpu(wl, comp.desc, args)
+    del comp, wl
+    torch.cuda.empty_cache()
+
+    # ---- the other configurations, and the settings that defeat the two-pass shortcut, in the same run
+    configs = {}
+    if not args.no_configs and args.workload == DEFAULT_WORKLOAD and args.batch is None and args.layers is None and not kw:
+        for name, k_side in (("llama8b_b1", 20), ("llama8b_b16", 5), ("qwen7b_b64", 5)):
+            swl = ri.make_workload(ri.SPECS[name], device=dev, seed=ri.BASE_SEED + 1000 * rank + ri.CONFIG_ORDER.index(name))
+            configs[name] = side_config(rkv, rd, dev, swl, {}, k_side, 3, args.mem_gb, peaks)
+            if name == "llama8b_b16":
+                configs[name + " threshold=0.9"] = side_config(rkv, rd, dev, swl, {"sim_threshold": 0.9}, 3, 3, args.mem_gb, peaks)
+                configs[name + " beta=8"] = side_config(rkv, rd, dev, swl, {"beta": 8}, 3, 3, args.mem_gb, peaks)
+            del swl
+            torch.cuda.empty_cache()
 
     if rank == 0:
         line = {
@@ -460,13 +577,12 @@ def main():
             "config": {"workload": spec.name, "head_problems_per_gpu": spec.head_problems,
                        "layers": spec.layers, "batch": spec.batch, "n_kv_heads": spec.n_kv_heads,
                        "n_q_heads": spec.n_q_heads, "budget": spec.budget, "buffer": spec.buffer, "alpha": spec.alpha,
-                       "lambda": spec.lam, "pool_w": comp.desc.pool_w, "beta": comp.desc.beta,
-                       "sim_threshold": comp.desc.sim_threshold, "importance_order": "mean, then pool (Algorithm 1)"
+                       "lambda": spec.lam, **desc_view, "importance_order": "mean, then pool (Algorithm 1)"
                        if args.mean_then_pool else "pool, then mean (Eq. 4)",
                        "selection": "one set per sequence, head-averaged score (Algorithm 1)" if args.head_mean
                        else "one set per KV head",
-                       "l2": (f"{n_rep} input replicas of {bytes_per_replica / 2**20:.0f} MiB cycled, each used once"
-                              if contiguous else "inputs restored and a 256 MiB buffer written between timed steps"),
+                       "step": "one compressing firing: every cache full (budget + buffer tokens)",
+                       "l2": l2_note,
                        "parallelism": f"{world} independent replicas, no collective"},
             "compressions_per_s": value / toks * spec.folded_batch,
             "head_problems_per_s": value / n,
@@ -474,12 +590,16 @@ def main():
             "kernels": kernels,
             "scoring": scoring,
             "roofline": roofline,
+            "roofline_hbm": roofline_hbm,
             "clocks": clocks,
+            "peaks": {"hbm_gbs": peaks["hbm_gbs"], "bf16_tflops": peaks["bf16_tflops"], "source": peaks["source"]},
         }
         if e2e is not None:
             line["e2e"] = e2e
         if cpu is not None:
             line["cpu_baseline"] = cpu
+        if configs:
+            line["configs"] = configs
         print(json.dumps(line))
     if torch.distributed.is_initialized():
         torch.distributed.destroy_process_group()

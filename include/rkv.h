@@ -59,9 +59,9 @@ typedef enum { RKV_BF16 = 0, RKV_F32 = 1 } rkv_dtype_t;
 #define RKV_FLAG_SIMT_SCORES 1u /* score with the plain fp32 CUDA-core kernel instead of the tcgen05
                                    kernels (always used for RKV_F32; a debugging aid for RKV_BF16) */
 #define RKV_FLAG_ROWBLOCK_SCORES 2u /* bf16: score with the row-block tcgen05 kernel (forms the full similarity
-                                   matrix) instead of the default triangle kernels (upper-triangular tiles, then
-                                   only the tokens still short of partners against the tiles to their left);
-                                   a cross-check */
+                                   matrix) instead of the default two-pass kernels (every token against the last
+                                   key tile first, then only the tokens still short of partners against the
+                                   earlier tiles, last to first); a cross-check */
 
 #define RKV_FLAG_MEAN_THEN_POOL 4u /* importance in Algorithm 1's order: mean over the alpha query rows first, then the
                                    pooling (read as Eq. 4's max over the same window); default is Eq. 4's order */
@@ -102,10 +102,11 @@ typedef struct rkv_desc {
     void *workspace;     /* device scratch, 256-byte aligned, >= rkv_workspace_bytes(); contents are
                             undefined between calls; two calls that overlap on the GPU need two workspaces */
     size_t workspace_bytes;
-    int32_t *device_status; /* optional device int32; kernels store the first error they meet
+    int32_t *device_status; /* optional device int32; kernels store the first error they meet into it if it holds 0
                                (RKV_ERR_INVALID_ARG for seq_lens[b] > cap or < 0, RKV_ERR_TIMEOUT).  The caller
-                               zeroes it and reads it after synchronising the stream; while it is non-zero the
-                               scoring stage does no work (after an error the results are invalid anyway) */
+                               zeroes it and reads it after synchronising the stream.  The library only ever
+                               writes it: a value left over from an earlier call changes nothing in a later one.
+                               What a call does after an error is stated with rkv_compress below. */
     /* optional device dumps of the scores, each [batch][n_kv_heads][cap] float, first n entries written */
     float *dbg_I, *dbg_Sbar, *dbg_R, *dbg_Z;
     /* optional: 5 cudaEvent_t handles; event s is recorded before stage s (prep, scores, select, gather)
@@ -115,9 +116,15 @@ typedef struct rkv_desc {
        pass, after the listing kernel between the passes, after the row statistics and after the importance
        kernel (with a scoring kernel that is a single launch the first two coincide with the stage's start) */
     void *const *kernel_events;
-    /* optional device uint64[4], written at the end of the scoring stage: [0] = 128 x 128 x 128 tile products the
-       tensor-core kernels executed in this call, [2] = work items of the second scoring pass */
+    /* optional device uint64[8], written at the end of the scoring stage: [0] = 128 x 128 x 128 tile products the
+       tensor-core kernels executed in this call, [2] = work items of the second scoring pass, [5] = (listed token,
+       key tile) pairs the second pass had to form (its useful work: items pad the tokens to whole 128-row tiles);
+       the other words are internal */
     unsigned long long *dbg_counters;
+    /* limit of every bounded wait inside the kernels, in GPU clock ticks; 0 = the default (about two seconds).
+       A wait that runs out is an error (RKV_ERR_TIMEOUT), never a hang.  Values below about a million ticks can
+       expire during ordinary memory latency: leave it at 0 outside of tests. */
+    int64_t wait_limit_cycles;
 } rkv_desc_t;
 
 /* Fill *desc with the defaults above (pool_w 4, beta 1, T 0.5, eps 1e-8, head_dim 128, bf16), zero elsewhere. */
@@ -144,8 +151,13 @@ RKV_API int rkv_set_desc(const rkv_desc_t *desc);
  * original position, rows [budget, cap) are unspecified, out_idx[b][h] lists the kept original positions
  * (ascending; the last alpha are L-alpha .. L-1) and seq_lens[b] becomes budget.
  * For seq_lens[b] <= budget (Algorithm 1's guard) nothing changes; out_idx[b][h][j] = j for j < L, -1 after.
- * seq_lens[b] > cap or < 0 cannot be seen without a sync: that sequence is skipped, out_idx[b] = -1 and
- * RKV_ERR_INVALID_ARG is stored to device_status.
+ * seq_lens[b] > cap or < 0 cannot be seen without a sync: that sequence alone is skipped (its caches and length
+ * stay as they are, out_idx[b] = -1), RKV_ERR_INVALID_ARG is stored to device_status, and every other sequence
+ * of the batch is compressed as usual.
+ * If a bounded wait inside a kernel runs out (RKV_ERR_TIMEOUT in device_status), the scores of the call are
+ * incomplete: the remaining kernels then leave ALL caches and lengths of the batch unmodified and set every
+ * entry of out_idx to -1.  The state that carries this between the kernels lives in the workspace and is reset by
+ * each call, so nothing has to be cleared before the next one.
  * Requires 1 <= alpha < budget, buffer >= 1, cap <= RKV_MAX_CAP, G * alpha <= RKV_MAX_GROUP_ROWS,
  * lambda in [0, 1].  Host-detectable errors return before anything is launched.
  * Uses the thread's current descriptor (rkv_set_desc).
@@ -195,7 +207,8 @@ RKV_API int rkv_compress_host(const rkv_desc_t *desc, void *host_k_cache, void *
  *     larger batches are split into several calls over sub-ranges of the batch dimension, one after the other.
  *   - the call makes no cudaMalloc / cudaFree and calls no allocating library routine.
  *   - the FIRST call on each device looks up the array's device address (with that device current) and caches
- *     it; make that first call outside any stream capture.
+ *     it; make that first call outside any stream capture (a first call that arrives while `stream` is being
+ *     captured is refused with RKV_ERR_INVALID_ARG before the lookup).
  *   - all calls on a device share the one array, which still holds the previous call's contents.  The few
  *     words that have to start at zero (work counters, per-head tickets) are cleared by the call itself, on the
  *     stream, before its first kernel; everything else is written by one stage before the next reads it.  But
@@ -227,6 +240,22 @@ RKV_API int rkv_append(const rkv_desc_t *desc, void *k_cache, void *v_cache, con
                        int32_t *seq_lens, int32_t budget, int32_t buffer, void *stream);
 RKV_API int rkv_push_query(const rkv_desc_t *desc, void *q_window, const void *q_new, int32_t alpha, int32_t slot,
                            void *stream);
+
+/*
+ * Self-test of the kernels' failure detection (no counterpart in the paper).  Every wait inside the tensor-core
+ * kernels is bounded; this call makes such a wait run out on purpose, in a tiny kernel of its own (one block that
+ * allocates tensor memory, waits with the given limit on a barrier nothing arrives at, calls off a second waiting
+ * thread through the block's abort flag and leaves through the scoring kernels' kind of exit).  Nothing hangs,
+ * faults or traps; the context stays usable and later calls on the stream run normally.
+ *   device_status  device int32, must hold 0: receives RKV_ERR_TIMEOUT
+ *   report_words   device uint64[8], 8-byte aligned, zeroed by the call: [0] != 0: abort recorded, [1] ticks the
+ *                  first wait lasted, [2] = 0: it returned "failed", [3] ticks the second wait lasted, [4] = 1: the
+ *                  second wait was called off before its own limit, [5] = 1: the block reached its end
+ *   limit_cycles   limit of the first wait in GPU clock ticks, 1000 .. the default limit (about two seconds)
+ * Enqueues one memset and one launch on `stream`; returns RKV_ERR_INVALID_ARG for bad arguments.
+ */
+RKV_API int rkv_selftest_wait_expiry(int32_t *device_status, unsigned long long *report_words, int64_t limit_cycles,
+                                     void *stream);
 
 /* Number of kernels a call launches (for launch accounting; the memset that precedes the prep kernel is not
  * counted).  rkv_launch_count_for() is exact for the given sizes; rkv_launch_count(), which does not know them, gives

@@ -41,6 +41,7 @@ class RkvDesc(ctypes.Structure):
         ("device_status", ctypes.c_void_p), ("dbg_I", ctypes.c_void_p), ("dbg_Sbar", ctypes.c_void_p),
         ("dbg_R", ctypes.c_void_p), ("dbg_Z", ctypes.c_void_p), ("stage_events", ctypes.c_void_p),
         ("kernel_events", ctypes.c_void_p), ("dbg_counters", ctypes.c_void_p),
+        ("wait_limit_cycles", ctypes.c_int64),
     ]
 
 
@@ -70,6 +71,7 @@ def lib():
         L.rkv_compress_static.restype, L.rkv_compress_static.argtypes = ctypes.c_int, [P] + ten
         L.rkv_append.restype, L.rkv_append.argtypes = ctypes.c_int, [P, VP, VP, VP, VP, VP, I32, I32, VP]
         L.rkv_push_query.restype, L.rkv_push_query.argtypes = ctypes.c_int, [P, VP, VP, I32, I32, VP]
+        L.rkv_selftest_wait_expiry.restype, L.rkv_selftest_wait_expiry.argtypes = ctypes.c_int, [VP, VP, ctypes.c_int64, VP]
         L.rkv_launch_count.restype, L.rkv_launch_count.argtypes = ctypes.c_int, [P, U32]
         L.rkv_launch_count_for.restype, L.rkv_launch_count_for.argtypes = ctypes.c_int, [P, I32, I32, I32, U32]
         L.rkv_status_string.restype, L.rkv_status_string.argtypes = ctypes.c_char_p, [ctypes.c_int]
@@ -172,6 +174,11 @@ def rkv_push_query(desc, q_window, q_new, alpha, slot, stream=None) -> int:
     return lib().rkv_push_query(ctypes.byref(desc), _ptr(q_window), _ptr(q_new), alpha, slot, _stream(stream))
 
 
+def rkv_selftest_wait_expiry(device_status, report_words, limit_cycles: int, stream=None) -> int:
+    """Make a bounded device-side wait run out on purpose in a tiny kernel of its own (failure-detection self-test)."""
+    return lib().rkv_selftest_wait_expiry(_ptr(device_status), _ptr(report_words), int(limit_cycles), _stream(stream))
+
+
 class Compressor:
     """Convenience holder of a descriptor, its workspace and optional score dumps for one cache shape.
 
@@ -222,7 +229,7 @@ class Compressor:
             self._kevent_array = (ctypes.c_void_p * 4)(*[ev.cuda_event for ev in self.kevents])
             d.stage_events = ctypes.cast(self._event_array, ctypes.c_void_p)
             d.kernel_events = ctypes.cast(self._kevent_array, ctypes.c_void_p)
-            self.counters = torch.zeros(4, dtype=torch.int64, device=self.device)
+            self.counters = torch.zeros(8, dtype=torch.int64, device=self.device)
             d.dbg_counters = self.counters.data_ptr()
         self.desc = d
         self.out_idx = torch.empty(batch, n_kv_heads, budget, dtype=torch.int32, device=self.device)

@@ -69,7 +69,7 @@ int check_shapes(const rkv_desc_t *d, int budget, int buffer, int alpha, Layout 
         lay->head_sum_bf16 = off; off = align_up(off + P * 16 * kHeadDim * sizeof(__nv_bfloat16), 256);
         lay->meta = off;        off = align_up(off + (size_t)d->batch * sizeof(int32_t), 256);
         // the region the prep stage zeroes: counters and per-head tile tickets
-        lay->counters = off;    off = align_up(off + 4 * sizeof(unsigned long long), 256);
+        lay->counters = off;    off = align_up(off + 8 * sizeof(unsigned long long), 256);
         lay->tile_done = off;   off = align_up(off + P * sizeof(uint32_t), 256);
         lay->zero_bytes = off - lay->counters;
         lay->total = off;
@@ -142,6 +142,7 @@ int run(const rkv_desc_t *d, void *k_cache, void *v_cache, const void *q_window,
     p.zero_bytes = lay.zero_bytes;
     p.tri = lay.tri;
     p.status = d->device_status;
+    p.wait_cycles = d->wait_limit_cycles > 0 ? (long long)d->wait_limit_cycles : sm100_default_wait_cycles();
     p.kernel_events = d->kernel_events;
     p.dbg_counters = d->dbg_counters;
     p.dbg_I = d->dbg_I;
@@ -168,7 +169,7 @@ int run(const rkv_desc_t *d, void *k_cache, void *v_cache, const void *q_window,
         if (!p.tri && ((e = mark_kernel(p, 0, s)) != cudaSuccess || (e = mark_kernel(p, 1, s)) != cudaSuccess))
             return cuda_fail(e, "cudaEventRecord");
         if (p.dbg_counters &&
-            (e = cudaMemcpyAsync(p.dbg_counters, p.counters, 4 * sizeof(unsigned long long), cudaMemcpyDeviceToDevice, s)) !=
+            (e = cudaMemcpyAsync(p.dbg_counters, p.counters, 8 * sizeof(unsigned long long), cudaMemcpyDeviceToDevice, s)) !=
                 cudaSuccess)
             return cuda_fail(e, "cudaMemcpyAsync");
     }

@@ -58,9 +58,12 @@ struct Params {
     __nv_bfloat16 *head_sum_bf16;   // [P][16][128] head_sum split into three bf16 rows (hi, mid, lo), 13 zero rows
     int32_t *meta;       // [batch]              snapshot of seq_lens (kMetaInvalid if out of range)
     // zeroed by the prep stage's memset, in this order, contiguous:
-    unsigned long long *counters;   // [4]       [0] = similarity tiles computed by the tcgen05 kernels, [1] = item
+    unsigned long long *counters;   // [8]       [0] = similarity tiles computed by the tcgen05 kernels, [1] = item
                                     //           ticket of the first scoring pass, [2] = entries in strag_items,
-                                    //           [3] = item ticket of the second pass
+                                    //           [3] = item ticket of the second pass, [4] = the call's abort word
+                                    //           (non-zero once a bounded wait ran out: later kernels of the call
+                                    //           then leave the caches, lengths and index lists alone),
+                                    //           [5] = listed-token x key-tile pairs the second pass has to form
     uint32_t *tile_done;            // [P]       tiles of the head finished by the prep stage
     size_t zero_bytes;              // bytes from `counters` to the end of `tile_done`
     int tri;                        // 1: the triangle kernels score (bf16 default); 0: another kernel does
@@ -68,6 +71,7 @@ struct Params {
     void *const *kernel_events;     // see rkv_desc_t
     unsigned long long *dbg_counters;
     int32_t *status;
+    long long wait_cycles;          // limit of every bounded wait, in clock64() ticks
     float *dbg_I, *dbg_Sbar, *dbg_R, *dbg_Z;
 };
 
@@ -83,6 +87,31 @@ inline cudaError_t mark_kernel(const Params &p, int i, cudaStream_t s)
 __device__ __forceinline__ void report(int32_t *status, int code)
 {
     if (status) atomicCAS(status, 0, code);
+}
+
+constexpr int kAbortWord = 4;       // index of the call's abort word in Params::counters
+constexpr int kPairsWord = 5;       // index of the second pass's useful-work count
+
+// Where a bounded wait records that it ran out: the caller's optional status word, and the call's own abort word
+// in the workspace, which the later kernels of the same call read.
+struct ErrSink {
+    int32_t *status;
+    unsigned long long *abort_word;
+    long long wait_cycles;
+};
+__device__ __forceinline__ ErrSink make_sink(const Params &p)
+{
+    return ErrSink{p.status, p.counters + kAbortWord, p.wait_cycles};
+}
+__device__ __forceinline__ void report_timeout(const ErrSink &sink)
+{
+    report(sink.status, RKV_ERR_TIMEOUT);
+    atomicExch(sink.abort_word, 1ull);
+}
+// True once some kernel of this call has given up on a wait.
+__device__ __forceinline__ bool call_aborted(const Params &p)
+{
+    return *reinterpret_cast<volatile unsigned long long *>(p.counters + kAbortWord) != 0ull;
 }
 
 // Number of candidates of sequence b as every stage after prep sees it: 0 = nothing to compress.
@@ -128,6 +157,7 @@ cudaError_t launch_append(void *k_cache, void *v_cache, const void *k_new, const
 cudaError_t launch_push_query(void *q_window, const void *q_new, int batch, int hq, int alpha, int slot, int row_bytes,
                               cudaStream_t s);
 bool scores_sm100_available();
+long long sm100_default_wait_cycles();          // default limit of the kernels' bounded waits (about two seconds)
 bool select_is_fused(int cap_pad, int alpha);   // the select stage is one kernel (small caches) instead of three
 
 }  // namespace rkv

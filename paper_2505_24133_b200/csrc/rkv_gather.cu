@@ -33,6 +33,7 @@ __global__ void __launch_bounds__(kGatherThreads) gather_kernel(Params p)
     const int b = head / p.hkv;
     const int L = p.meta[b];
     if (L <= p.budget) return;                      // nothing was selected for this sequence
+    if (call_aborted(p)) return;                    // a bounded wait ran out earlier in this call: caches and lengths stay as they are
     if (which == 0 && slice == 0 && head % p.hkv == 0 && threadIdx.x == 0) p.seq_lens[b] = p.budget;
 
     uint4 *base = reinterpret_cast<uint4 *>(which ? p.v_cache : p.k_cache) + (size_t)head * p.cap * kVecPerRow +

@@ -27,6 +27,7 @@ __global__ void __launch_bounds__(kPrepThreads, 5) prep_kernel(Params p)
     extern __shared__ __align__(128) uint8_t prep_smem[];       // the tile's candidate rows, then one mbarrier
     constexpr int kTileBytesT = kTile * kHeadDim * (int)sizeof(T);
     __shared__ int abort_flag;
+    const ErrSink sink = make_sink(p);
     constexpr int kPerVec = Elem<T>::kPerVec;            // elements per 16-byte vector
     constexpr int kVecPerLane = 2;                       // 16-byte vectors of a row held by one lane
     constexpr int kLanesPerRow = kHeadDim / (kPerVec * kVecPerLane);     // 8 (bf16) or 16 (fp32)
@@ -72,7 +73,7 @@ __global__ void __launch_bounds__(kPrepThreads, 5) prep_kernel(Params p)
         }
     }
     __syncthreads();
-    const bool landed = rows_here == 0 || mbar_wait(bar, 0, &abort_flag, p.status);
+    const bool landed = rows_here == 0 || mbar_wait(bar, 0, &abort_flag, sink);
     if (!__syncthreads_and(landed)) {      // the block leaves as a whole, or not at all
         __nanosleep(200000);               // error path only: let the copy land before the block's memory is reused
         return;

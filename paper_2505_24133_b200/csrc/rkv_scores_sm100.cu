@@ -82,7 +82,8 @@ scores_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, const _
     // Once any block has recorded an error (a wait that ran out), the blocks still to run return at once
     // instead of each waiting out its own limit.
     __shared__ int bail;
-    if (threadIdx.x == 0) bail = (p.status != nullptr && *reinterpret_cast<volatile int32_t *>(p.status) != 0);
+    const ErrSink sink = make_sink(p);
+    if (threadIdx.x == 0) bail = call_aborted(p) ? 1 : 0;      // a wait of this call has run out: nothing more is started
     __syncthreads();
     if (bail) return;
 
@@ -144,7 +145,7 @@ scores_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, const _
             for (int t = 0; t < n_iter; ++t) {
                 const int s = t % kStages;
                 const int jt = n_tiles - 1 - t;                       // last tile first
-                if (!mbar_wait(bar.empty(s), ((t / kStages) & 1) ^ 1, abort_flag, p.status)) break;
+                if (!mbar_wait(bar.empty(s), ((t / kStages) & 1) ^ 1, abort_flag, sink)) break;
                 mbar_expect_tx(bar.full(s), kTileBytes);
                 const uint32_t dst = sbase + kOffB + s * kTileBytes;
                 const int y = key_row_base + jt * kTile;
@@ -156,11 +157,11 @@ scores_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, const _
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             const uint32_t idesc = is_q ? instr_desc(kTile, q_rows_pad) : instr_desc(kTile, kTile);
-            bool ok = mbar_wait(bar.resident(), 0, abort_flag, p.status);
+            bool ok = mbar_wait(bar.resident(), 0, abort_flag, sink);
             for (int t = 0; ok && t < n_iter; ++t) {
                 const int s = t % kStages, a = t & 1;
-                if (!mbar_wait(bar.full(s), (t / kStages) & 1, abort_flag, p.status)) break;
-                if (!mbar_wait(bar.acc_empty(a), ((t >> 1) & 1) ^ 1, abort_flag, p.status)) break;
+                if (!mbar_wait(bar.full(s), (t / kStages) & 1, abort_flag, sink)) break;
+                if (!mbar_wait(bar.acc_empty(a), ((t >> 1) & 1) ^ 1, abort_flag, sink)) break;
                 tc_fence_after();
                 const uint32_t stage = sbase + kOffB + s * kTileBytes;
                 for (int m = 0; m < num_m; ++m) {
@@ -202,7 +203,7 @@ scores_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, const _
             const bool row_ok = warp_active && i < n;
             const float ri = row_ok ? r_s[i] : 0.f;
             float total = 0.f;
-            bool ok = mbar_wait(bar.resident(), 0, abort_flag, p.status);
+            bool ok = mbar_wait(bar.resident(), 0, abort_flag, sink);
             if (ok && warp_active) {
                 // Kbar_i . s - Kbar_i . Kbar_i from the resident (swizzled) tile: 16-byte chunk c of row r sits at
                 // chunk position c ^ (r & 7) of the row's 128 bytes
@@ -234,7 +235,7 @@ scores_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, const _
             for (int t = 0; ok && t < n_iter; ++t) {
                 const int a = t & 1;
                 const int jt = n_tiles - 1 - t;
-                if (!mbar_wait(bar.acc_full(a), (t >> 1) & 1, abort_flag, p.status)) break;
+                if (!mbar_wait(bar.acc_full(a), (t >> 1) & 1, abort_flag, sink)) break;
                 if (warp_active) {
                     tc_fence_after();
                     const bool any_live = __any_sync(0xffffffffu, thr < kInf);
@@ -283,7 +284,7 @@ scores_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, const _
             for (int t = 0; t < n_iter; ++t) {
                 const int a = t & 1;
                 const int jt = n_tiles - 1 - t;
-                if (!mbar_wait(bar.acc_full(a), (t >> 1) & 1, abort_flag, p.status)) break;
+                if (!mbar_wait(bar.acc_full(a), (t >> 1) & 1, abort_flag, sink)) break;
                 if (warp_active) {
                     tc_fence_after();
                     const int i = jt * kTile + lrow;
@@ -328,6 +329,7 @@ scores_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, const _
 }  // namespace
 
 bool scores_sm100_available() { return true; }
+long long sm100_default_wait_cycles() { return sm100::kWaitCycles; }
 
 cudaError_t launch_scores_sm100(const Params &p, cudaStream_t s)
 {

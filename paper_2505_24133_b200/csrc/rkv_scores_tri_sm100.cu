@@ -147,10 +147,12 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
     volatile int *bail = reinterpret_cast<volatile int *>(smem + kOffMisc + 8);
     const Bars bar{sbase + kOffBar};
 
-    // Once any block has recorded an error, the blocks still to start return at once.  Pass 2 has nothing to do
-    // when the list is empty.
+    // Once a bounded wait of this call has run out, the blocks still to start return at once (a sequence with an
+    // invalid length does not stop the others: it just has no candidates).  Pass 2 has nothing to do when the list
+    // is empty.
+    const ErrSink sink = make_sink(p);
     if (threadIdx.x == 0) {
-        int b = (p.status != nullptr && *reinterpret_cast<volatile int32_t *>(p.status) != 0);
+        int b = call_aborted(p) ? 1 : 0;
         if (kPass2 && p.counters[2] == 0ull) b = 1;
         *bail = b;
     }
@@ -228,13 +230,13 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
                 const int key_row_base = head * p.cap;                         // first row of the head in the 2-D key view
 
                 const uint32_t qs = k_item % kItemSlots;
-                if (!mbar_wait(bar.at(kBarQEmpty + qs), ((k_item / kItemSlots) & 1) ^ 1, abort_flag, p.status)) break;
+                if (!mbar_wait(bar.at(kBarQEmpty + qs), ((k_item / kItemSlots) & 1) ^ 1, abort_flag, sink)) break;
                 items[qs] = desc;
                 mbar_arrive(bar.at(kBarQFull + qs));
 
                 if (kPass2 && p.beta > 1) {
                     // r_j of the tiles this item streams (0 .. first_tile), straight into shared memory
-                    if (!mbar_wait(bar.at(kBarREmpty), (k_item & 1) ^ 1, abort_flag, p.status)) break;
+                    if (!mbar_wait(bar.at(kBarREmpty), (k_item & 1) ^ 1, abort_flag, sink)) break;
                     const uint32_t bytes = (uint32_t)(first_tile + 1) * kTile * 4u;
                     mbar_expect_tx(bar.at(kBarRFull), bytes);
                     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
@@ -245,7 +247,7 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
                 if (!kPass2 && rule_on) {
                     // r_j of the key tiles this item streams (first_tile down to first_tile + 2 - n_iter)
                     const uint32_t rb = k_item & 1;
-                    if (!mbar_wait(bar.at(kBarREmpty + rb), ((k_item >> 1) & 1) ^ 1, abort_flag, p.status)) break;
+                    if (!mbar_wait(bar.at(kBarREmpty + rb), ((k_item >> 1) & 1) ^ 1, abort_flag, sink)) break;
                     const int low_tile = first_tile + 2 - n_iter;
                     const uint32_t bytes = (uint32_t)(n_iter - 1) * kTile * 4u;
                     mbar_expect_tx(bar.at(kBarRFull + rb), bytes);
@@ -259,7 +261,7 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
                     const int row0 = desc.y * kRowsPerItem;
                     const int num_m = (desc.z - row0 > kTile) ? 2 : 1;
                     const uint32_t ab = k_item & 1;
-                    if (!mbar_wait(bar.at(kBarAEmpty + ab), ((k_item >> 1) & 1) ^ 1, abort_flag, p.status)) break;
+                    if (!mbar_wait(bar.at(kBarAEmpty + ab), ((k_item >> 1) & 1) ^ 1, abort_flag, sink)) break;
                     mbar_expect_tx(bar.at(kBarAFull + ab), (uint32_t)(num_m * kTileBytes));
                     for (int m = 0; m < num_m; ++m) {
                         const uint32_t dst = sbase + kOffA + (ab * 2 + m) * kTileBytes;
@@ -270,7 +272,7 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
                 }
                 for (int it = 0; it < n_iter; ++it) {
                     const uint32_t s = bcount % kStagesB;
-                    if (!mbar_wait(bar.at(kBarBEmpty + s), ((bcount / kStagesB) & 1) ^ 1, abort_flag, p.status)) {
+                    if (!mbar_wait(bar.at(kBarBEmpty + s), ((bcount / kStagesB) & 1) ^ 1, abort_flag, sink)) {
                         ok = false;
                         break;
                     }
@@ -301,7 +303,7 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
             // terminator: tells the other roles that no item follows (skipped when the block is aborting)
             if (!*abort_flag) {
                 const uint32_t qs = k_item % kItemSlots;
-                if (mbar_wait(bar.at(kBarQEmpty + qs), ((k_item / kItemSlots) & 1) ^ 1, abort_flag, p.status)) {
+                if (mbar_wait(bar.at(kBarQEmpty + qs), ((k_item / kItemSlots) & 1) ^ 1, abort_flag, sink)) {
                     items[qs] = make_int4(-1, 0, 0, 0);
                     mbar_arrive(bar.at(kBarQFull + qs));
                 }
@@ -322,7 +324,7 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
             bool ok = true;
             while (ok) {
                 const uint32_t qs = k_item % kItemSlots;
-                if (!mbar_wait(bar.at(kBarQFull + qs), (k_item / kItemSlots) & 1, abort_flag, p.status)) break;
+                if (!mbar_wait(bar.at(kBarQFull + qs), (k_item / kItemSlots) & 1, abort_flag, sink)) break;
                 const int4 d = items[qs];
                 mbar_arrive(bar.at(kBarQEmpty + qs));
                 if (d.x < 0) break;
@@ -341,12 +343,12 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
                 const bool mine = m < num_m;
                 const uint32_t ab = kPass2 ? 0u : (k_item & 1);                          // pass 2: one pair of tiles
                 const uint32_t a_par = kPass2 ? (k_item & 1) : ((k_item >> 1) & 1);
-                if (!mbar_wait(bar.at(kBarAFull + ab), a_par, abort_flag, p.status)) break;
+                if (!mbar_wait(bar.at(kBarAFull + ab), a_par, abort_flag, sink)) break;
                 if (kPass2) asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t resident = sbase + kOffA + (ab * 2 + m) * kTileBytes;
                 for (int it = 0; it < n_iter; ++it) {
                     const uint32_t s = bcount % kStagesB;
-                    if (!mbar_wait(bar.at(kBarBFull + s), (bcount / kStagesB) & 1, abort_flag, p.status)) {
+                    if (!mbar_wait(bar.at(kBarBFull + s), (bcount / kStagesB) & 1, abort_flag, sink)) {
                         ok = false;
                         break;
                     }
@@ -354,7 +356,7 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
                     const bool is_q = !kPass2 && it == 0;
                     if (mine && !(m == 1 && it == skip_it && it > 0)) {
                         const uint32_t a = cnt & 1;
-                        if (!mbar_wait(bar.at(kBarAccEmpty + a * 2 + m), ((cnt >> 1) & 1) ^ 1, abort_flag, p.status)) {
+                        if (!mbar_wait(bar.at(kBarAccEmpty + a * 2 + m), ((cnt >> 1) & 1) ^ 1, abort_flag, sink)) {
                             ok = false;
                             break;
                         }
@@ -393,7 +395,7 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
 
         while (true) {
             const uint32_t qs = k_item % kItemSlots;
-            if (!mbar_wait(bar.at(kBarQFull + qs), (k_item / kItemSlots) & 1, abort_flag, p.status)) break;
+            if (!mbar_wait(bar.at(kBarQFull + qs), (k_item / kItemSlots) & 1, abort_flag, sink)) break;
             const int4 d = items[qs];
             __syncwarp();
             if (lane == 0) mbar_arrive(bar.at(kBarQEmpty + qs));
@@ -438,7 +440,7 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
 
                 // gather this thread's key row into the resident tile (same swizzled layout as a TMA load); every
                 // warp waits and arrives, also one without rows of its own, so that no arrival runs ahead
-                item_ok = mbar_wait(bar.at(kBarAEmpty + ab), a_par ^ 1, abort_flag, p.status);
+                item_ok = mbar_wait(bar.at(kBarAEmpty + ab), a_par ^ 1, abort_flag, sink);
                 if (active && item_ok) {
                     uint8_t *tile = smem + kOffA + (ab * 2 + m) * kTileBytes;
                     const uint4 *src = reinterpret_cast<const uint4 *>(
@@ -479,13 +481,13 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
             const bool has_r = kPass2 ? p.beta > 1 : rule_on;
             const uint32_t r_slot = kPass2 ? 0u : (k_item & 1), r_par = kPass2 ? (k_item & 1) : ((k_item >> 1) & 1);
             if (has_r) {        // every warp waits for the item's r_j, and hands them back at the item's end
-                const bool r_ok = mbar_wait(bar.at(kBarRFull + r_slot), r_par, abort_flag, p.status);
+                const bool r_ok = mbar_wait(bar.at(kBarRFull + r_slot), r_par, abort_flag, sink);
                 item_ok = item_ok && r_ok;
             }
 
             if (!kPass2 && active) {
                 const uint32_t a = cnt & 1;
-                item_ok = mbar_wait(bar.at(kBarAccFull + a * 2 + m), (cnt >> 1) & 1, abort_flag, p.status);
+                item_ok = mbar_wait(bar.at(kBarAccFull + a * 2 + m), (cnt >> 1) & 1, abort_flag, sink);
             }
             if (!kPass2 && active && item_ok) {
                 // ---- iteration 0, Eq. 2-3: thread = key, all G * alpha logits of that key in its accumulator row,
@@ -572,7 +574,7 @@ scores_tri_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, con
                     const int jbase = jt * kTile;
                     const float4 *rj4 = reinterpret_cast<const float4 *>(r_base + jbase);
                     const uint32_t a = cnt & 1;
-                    if (ok) ok = mbar_wait(bar.at(kBarAccFull + a * 2 + m), (cnt >> 1) & 1, abort_flag, p.status);
+                    if (ok) ok = mbar_wait(bar.at(kBarAccFull + a * 2 + m), (cnt >> 1) & 1, abort_flag, sink);
                     ++cnt;
                     if (!ok) continue;
                     tc_fence_after();
@@ -781,11 +783,14 @@ __global__ void __launch_bounds__(kCompactThreads) strag_compact_kernel(Params p
             const unsigned long long at = atomicAdd(&p.counters[2], (unsigned long long)chunks);
             // complete item descriptors, longest scans (largest positions) first: pass 1 took the chunk's last token
             // down to tile max(its own, n_tiles - depth), so the chunk's scan starts one tile below that
+            unsigned long long pairs = 0ull;
             for (int q = 0; q < chunks; ++q) {
                 const int c = chunks - 1 - q, k0 = c * kRowsPerItem, rows = min(count - k0, kRowsPerItem);
                 const int first_tile = max(list[k0 + rows - 1] / kTile, low) - 1;     // >= 0 for every listed token
                 p.strag_items[at + q] = make_int4(head, k0, rows, first_tile);
+                pairs += (unsigned long long)rows * (unsigned long long)(first_tile + 1);
             }
+            atomicAdd(&p.counters[kPairsWord], pairs);      // listed tokens x key tiles: the work pass 2 cannot avoid
         }
     }
 }

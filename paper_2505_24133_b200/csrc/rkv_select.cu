@@ -313,6 +313,10 @@ __global__ void __launch_bounds__(kFused ? kSelThreadsFused : kSelThreadsSplit, 
     const int L = p.meta[b];
     int32_t *out = p.out_idx + (size_t)head * p.budget;
 
+    if (call_aborted(p)) {    // a bounded wait of an earlier stage ran out: the scores are incomplete, nothing is selected
+        for (int j = tid; j < p.budget; j += kSelThreads) out[j] = -1;
+        return;
+    }
     if (L <= p.budget) {      // Algorithm 1's guard (or an invalid length): nothing is compressed
         for (int j = tid; j < p.budget; j += kSelThreads) out[j] = (j < L) ? j : -1;
         return;
@@ -421,6 +425,7 @@ __global__ void __launch_bounds__(kSelThreadsSplit, 4) select_mean_kernel(Params
     extern __shared__ float row[];
     const int b = blockIdx.x, tid = threadIdx.x;
     const int L = p.meta[b];
+    if (call_aborted(p)) return;    // select_kernel has written -1 everywhere
     if (L <= p.budget) return;      // select_kernel has written the identity lists
     const int n = L - p.alpha;
     uint32_t *keys = reinterpret_cast<uint32_t *>(row);

@@ -9,7 +9,7 @@
 namespace rkv {
 namespace sm100 {
 
-constexpr long long kWaitCycles = 4000000000ll;   // about two seconds: far beyond any legitimate wait
+constexpr long long kWaitCycles = 4000000000ll;   // default limit of a wait, about two seconds: far beyond any legitimate wait
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -39,7 +39,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 }
 
 // Bounded wait.  Returns false if the block is aborting (this wait ran out of time, or another one did).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int32_t *status)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, const ErrSink &sink)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const long long start = clock64();
@@ -47,11 +47,11 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 63u) == 0u) {
             if (*abort_flag) return false;
-            if (clock64() - start > kWaitCycles) break;
+            if (clock64() - start > sink.wait_cycles) break;
         }
     }
     *abort_flag = 1;
-    report(status, RKV_ERR_TIMEOUT);
+    report_timeout(sink);
     return false;
 }
 

@@ -22,13 +22,18 @@ bool g_scratch_ready[kMaxDevices];
 
 // Device address of the scratch array on the current device.  The first call on a device asks the runtime
 // for it (which also makes the runtime load this library's device image there); later calls read the cache.
-int scratch_address(void **out)
+int scratch_address(void **out, cudaStream_t stream)
 {
     int dev = -1;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess || dev < 0 || dev >= kMaxDevices) return RKV_ERR_CUDA;
     std::lock_guard<std::mutex> guard(g_lock);
     if (!g_scratch_ready[dev]) {
+        // the lookup may load the device image: not something to do in the middle of a stream capture
+        cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+        e = cudaStreamIsCapturing(stream, &capturing);
+        if (e != cudaSuccess) return RKV_ERR_CUDA;
+        if (capturing != cudaStreamCaptureStatusNone) return RKV_ERR_INVALID_ARG;
         void *ptr = nullptr;
         e = cudaGetSymbolAddress(&ptr, g_static_scratch);
         if (e != cudaSuccess || ptr == nullptr) return RKV_ERR_CUDA;
@@ -63,7 +68,7 @@ int rkv_compress_static(const rkv_desc_t *desc, void *k_cache, void *v_cache, co
     }
     if (need > (size_t)RKV_STATIC_SCRATCH_BYTES) return RKV_ERR_WORKSPACE;
     void *scratch = nullptr;
-    const int rc = scratch_address(&scratch);
+    const int rc = scratch_address(&scratch, static_cast<cudaStream_t>(stream));
     if (rc != RKV_OK) return rc;
     rkv_desc_t inner = *desc;       // the caller's workspace fields, if any, are ignored
     inner.workspace = scratch;

@@ -43,11 +43,13 @@ def test_config2_simt_and_tcgen05_agree(rkv):
     assert same > 0.5
 
 
-@pytest.mark.parametrize("name,rows", [("llama8b_b16", [0, 311]), ("qwen7b_b64", [0, 7, 1000, 1791]),
-                                       ("qwen14b_b32", [5, 1535])])
+@pytest.mark.parametrize("name,rows", [("llama8b_b16", [0, 63, 130, 205, 311, 402, 450, 511]),
+                                       ("qwen7b_b64", [0, 7, 100, 333, 512, 640, 700, 815, 999, 1000, 1111, 1290, 1400,
+                                                       1555, 1700, 1791]),
+                                       ("qwen14b_b32", [5, 200, 410, 777, 901, 1203, 1400, 1535])])
 def test_full_size_configs_sampled(rkv, name, rows):
-    """Configs 3, 4 and (one firing of) 5 at full size (about 9, 8 and 27 GB of K+V), oracle on sampled sequences
-    (all KV heads)."""
+    """Configs 3, 4 and (one firing of) 5 at full size (about 9, 8 and 27 GB of K+V), oracle on 64 sampled
+    head-problems each (sampled sequences, all their KV heads)."""
     wl = ri.make_workload(ri.SPECS[name], device="cuda")
     rep, comp = run_and_check(rkv, wl, check_rows=rows)
     print(rep.summary())
@@ -63,6 +65,20 @@ def test_full_size_configs_sampled(rkv, name, rows):
     assert bool((wl.seq_lens == spec.budget).all())
     del wl, comp
     torch.cuda.empty_cache()
+
+
+@pytest.mark.slow
+def test_full_coverage_at_the_largest_cache_size(rkv):
+    """Every head-problem of a batch through the oracle at the largest cache size of the configurations
+    (budget 4096 + buffer 128, n = 4216, 33 key tiles): the Llama-8B shape with one sequence per layer, 256
+    head-problems.  About a minute of oracle time on 16 host threads."""
+    spec = ri.scaled(ri.SPECS["llama8b_b16"], batch=1)
+    wl = ri.make_workload(spec, device="cuda", seed=ri.BASE_SEED + 303)
+    rep, comp = run_and_check(rkv, wl)
+    print(rep.summary())
+    assert rep.ok(), rep.errors
+    assert rep.compressed_heads == 256
+    comp.check_status()
 
 
 def test_config5_stream_stepwise(rkv):

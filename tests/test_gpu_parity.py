@@ -75,8 +75,8 @@ def test_tiny_shape_other_seeds_and_margin(rkv, seed):
 
 
 # ----------------------------------------------------------------------------- small shapes, both score kernels
-# the three scoring kernels: fp32 CUDA cores; symmetric tcgen05 (default; beta > 4 falls back to the row-block
-# kernel by itself); row-block tcgen05 forced
+# the three scoring routes: fp32 CUDA cores; the two-pass tcgen05 kernels (default for bf16, whatever beta and T);
+# the row-block tcgen05 kernel that forms the full matrix
 SCORE_FLAGS = [pytest.param(1, id="simt"), pytest.param(0, id="sym"), pytest.param(2, id="rowblock")]
 
 
@@ -262,20 +262,90 @@ def test_second_call_is_a_no_op(rkv):
     comp.check_status()
 
 
-def test_length_beyond_capacity_is_reported_not_clamped(rkv):
+@pytest.mark.parametrize("flags", SCORE_FLAGS)
+def test_length_beyond_capacity_is_reported_not_clamped(rkv, flags):
+    """One sequence with an impossible length: it alone is skipped and reported; the other sequences of the batch are
+    compressed exactly as if it were not there (full parity on them), on every scoring route."""
     spec = small_spec("bad", batch=3)
     wl = ri.make_workload(spec, device="cuda", seed=111, seq_lens=torch.tensor([spec.cap, spec.cap, spec.cap]))
     wl.seq_lens[1] = spec.cap + 1
-    k0 = wl.k_cache.clone()
-    comp = rkv.Compressor(3, 2, 8, spec.budget, spec.buffer, spec.alpha, 0.1, flags=1)
+    k0, v0, q0, s0 = wl.k_cache.clone(), wl.v_cache.clone(), wl.q_window.clone(), wl.seq_lens.clone()
+    comp = rkv.Compressor(3, 2, 8, spec.budget, spec.buffer, spec.alpha, 0.1, flags=flags, dump_scores=True)
     idx = comp.compress(wl.k_cache, wl.v_cache, wl.q_window, wl.seq_lens)
     torch.cuda.synchronize()
     assert int(comp.status.item()) == 1                      # RKV_ERR_INVALID_ARG
     assert bool((idx[1] == -1).all())
     assert torch.equal(k0[1].view(torch.int16), wl.k_cache[1].view(torch.int16))
+    assert torch.equal(v0[1].view(torch.int16), wl.v_cache[1].view(torch.int16))
     assert wl.seq_lens.tolist() == [spec.budget, spec.cap + 1, spec.budget]
+    sel = torch.tensor([0, 2], device="cuda")
+    d = comp.desc
+    rep = check_batch(k0[sel], v0[sel], q0[sel], s0[sel], budget=spec.budget, alpha=spec.alpha, lam=0.1, W=d.pool_w,
+                      beta=d.beta, T=d.sim_threshold, eps=d.eps, gpu_idx=idx[sel], gpu_k=wl.k_cache[sel],
+                      gpu_v=wl.v_cache[sel], gpu_seq=wl.seq_lens[sel], gpu_scores=comp.scores[:, sel])
+    assert rep.ok(), rep.errors
+    assert rep.compressed_heads == 4
     with pytest.raises(rkv.RkvError):
         comp.check_status()
+
+
+@pytest.mark.parametrize("flags", SCORE_FLAGS)
+def test_stale_status_word_does_not_disturb_a_call(rkv, flags):
+    """The status word is write-only for the library: a value left over from an earlier call (here planted by hand)
+    changes nothing in the next call, and stays as it is."""
+    spec = small_spec("stale", batch=2, budget=384, buffer=128)
+    wl = ri.make_workload(spec, device="cuda", seed=113)
+    k0, v0, q0, s0 = wl.k_cache.clone(), wl.v_cache.clone(), wl.q_window.clone(), wl.seq_lens.clone()
+    comp = rkv.Compressor(spec.folded_batch, 2, 8, spec.budget, spec.buffer, spec.alpha, 0.1, flags=flags)
+    comp.status.fill_(5)
+    idx = comp.compress(wl.k_cache, wl.v_cache, wl.q_window, wl.seq_lens)
+    torch.cuda.synchronize()
+    assert int(comp.status.item()) == 5
+    rep = check_batch(k0, v0, q0, s0, budget=spec.budget, alpha=spec.alpha, lam=0.1, gpu_idx=idx, gpu_k=wl.k_cache,
+                      gpu_v=wl.v_cache, gpu_seq=wl.seq_lens, **DEFAULTS)
+    assert rep.ok(), rep.errors
+    assert rep.compressed_heads == 4
+
+
+def test_bounded_wait_runs_out_and_the_context_stays_usable(rkv):
+    """Failure detection without a fault: a device-side wait on a barrier that nothing arrives at gives up after its
+    limit (about a millisecond here), records RKV_ERR_TIMEOUT, calls off the other waiting thread of the block, and
+    the kernel ends normally with its tensor memory freed.  A compression enqueued right behind it on the same stream
+    is unaffected."""
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    words = torch.full((8,), 77, dtype=torch.int64, device="cuda")
+    limit = 2_000_000                                       # about 1 ms at 1.9 GHz
+    assert rkv.rkv_selftest_wait_expiry(status, words, 10, None) == 1       # limit out of range: refused
+    assert rkv.rkv_selftest_wait_expiry(status, words, limit) == rkv.RKV_OK
+    spec = small_spec("after_timeout", batch=2, budget=384, buffer=128)
+    wl = ri.make_workload(spec, device="cuda", seed=115)
+    rep, comp = run_and_check(rkv, wl)                      # same (current) stream, straight behind the self-test
+    w = words.tolist()
+    assert int(status.item()) == 5                          # RKV_ERR_TIMEOUT
+    assert w[0] != 0                                        # abort recorded
+    assert w[2] == 0 and limit < w[1] < 50 * limit          # the first wait failed, after its limit and not much later
+    assert w[4] == 1 and w[3] < 100 * limit                 # the second was called off long before two seconds
+    assert w[5] == 1                                        # the block reached its end
+    assert rep.ok(), rep.errors
+    comp.check_status()
+
+
+# ----------------------------------------------------------------------------- hard inputs at benchmark sizes
+@pytest.mark.parametrize("flags", [pytest.param(0, id="sym"), pytest.param(2, id="rowblock")])
+@pytest.mark.parametrize("T,beta,budget", [(0.9, 1, 2048), (0.5, 8, 2048), (1.0, 1, 2048), (0.5, 400, 2048),
+                                           (0.9, 1, 4096), (0.5, 8, 4096)])
+def test_hard_retention_settings_at_benchmark_sizes(rkv, flags, T, beta, budget):
+    """The settings that defeat the two-pass shortcut -- a high threshold (few partners: nearly every token is listed
+    for the second pass), several partners per token (their r_j staged per head in shared memory), the rule switched
+    off by T = 1 -- at the cache sizes of the benchmark configurations (17 and 33 key tiles), not only on small
+    shapes."""
+    spec = small_spec("hard", batch=1, hkv=2, hq=8, budget=budget, buffer=128, span=32)
+    wl = ri.make_workload(spec, device="cuda", seed=211 + budget)
+    rep, comp = run_and_check(rkv, wl, flags=flags, T=T, beta=beta)
+    print(rep.summary())
+    assert rep.ok(), rep.errors
+    assert rep.compressed_heads == 2
+    comp.check_status()
 
 
 def test_host_buffer_entry_point_matches_device_entry_point(rkv):

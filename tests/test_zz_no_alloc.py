@@ -31,7 +31,7 @@ def _spec(name, batch, budget, buffer):
     return ri.CacheSpec(name, 1, batch, 2, 8, 128, budget, buffer, 8, 0.1, "bf16", 16, 0.3, 0.05, 4, 8.0)
 
 
-def _run_both(rkv, spec, seed, seq_lens):
+def _run_both(rkv, spec, seed, seq_lens, check_memory=False):
     """One compression of the same seeded caches through rkv_compress_ex (torch-allocated workspace) and through
     rkv_compress_static (no workspace); returns both results."""
     a = ri.make_workload(spec, device="cuda", seed=seed, seq_lens=seq_lens)
@@ -48,10 +48,20 @@ def _run_both(rkv, spec, seed, seq_lens):
     d.device_status = status.data_ptr()
     assert d.workspace is None and d.workspace_bytes == 0          # nothing allocated for scratch
     idx = torch.full((spec.folded_batch, spec.n_kv_heads, spec.budget), -7, dtype=torch.int32, device="cuda")
+    if check_memory:
+        # the descriptor's workspace fields are ignored: a bogus, far too small one must make no difference, and
+        # the pointer is never dereferenced
+        d.workspace, d.workspace_bytes = 0x1000, 16
+        torch.cuda.synchronize()
+        free_before, _ = torch.cuda.mem_get_info()
     rc = rkv.rkv_compress_static(d, b.k_cache, b.v_cache, b.q_window, b.seq_lens, spec.budget, spec.buffer,
                                  spec.alpha, spec.lam, idx)
     assert rc == rkv.RKV_OK, rkv.rkv_status_string(rc)
     torch.cuda.synchronize()
+    if check_memory:
+        # a warm call (the device image is loaded, the array's address cached) takes no device memory at all
+        free_after, _ = torch.cuda.mem_get_info()
+        assert free_after == free_before
     assert int(status.item()) == 0
     return (ref_idx, a), (idx, b)
 
@@ -77,7 +87,7 @@ def test_static_scratch_matches_workspace_entry_point_twice_in_a_row(rkv):
     # budget, so Algorithm 1's guard leaves it alone), so that stale scores of the first call sit right
     # behind the rows this one uses
     small = _spec("static_b", batch=4, budget=200, buffer=60)
-    ref, got = _run_both(rkv, small, seed=202, seq_lens=torch.tensor([260, 201, 150, 233]))
+    ref, got = _run_both(rkv, small, seed=202, seq_lens=torch.tensor([260, 201, 150, 233]), check_memory=True)
     _assert_same(small, ref, got)
     assert got[1].seq_lens.tolist() == [200, 200, 150, 200]
 
