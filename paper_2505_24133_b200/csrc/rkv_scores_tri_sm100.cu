@@ -85,43 +85,6 @@ constexpr int kSmemBytes = kOffRj + 2 * kPass1Depth * kTile * 4 + 1024;  // + sl
 static_assert(kOffItems % 16 == 0 && kOffRj % 16 == 0, "item descriptors are read as int4, r_j as float4");
 static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
 
-__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&r)[8])
-{
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
-                 : "r"(taddr)
-                 : "memory");
-}
-__device__ __forceinline__ void tmem_ld1(uint32_t taddr, uint32_t &r)
-{
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(r) : "r"(taddr) : "memory");
-}
-// Wait for the thread's TMEM loads; the loaded registers pass through the statement so that nothing that uses
-// them can be scheduled ahead of it.
-__device__ __forceinline__ void tmem_wait8(uint32_t (&r)[8])
-{
-    asm volatile("tcgen05.wait::ld.sync.aligned;"
-                 : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7])
-                 :: "memory");
-}
-__device__ __forceinline__ void tmem_wait32(uint32_t (&r)[32])
-{
-    asm volatile("tcgen05.wait::ld.sync.aligned;"
-                 : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
-                   "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
-                   "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
-                   "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
-                 :: "memory");
-}
-
-// max(a, b, c), NaN operands ignored
-__device__ __forceinline__ float max3(float a, float b, float c)
-{
-    float d;
-    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
-    return d;
-}
-
 struct Bars {
     uint32_t bar0;
     __device__ __forceinline__ uint32_t at(int idx) const { return bar0 + 8 * idx; }
@@ -820,9 +783,8 @@ cudaError_t launch_scores_tri_sm100(const Params &p, cudaStream_t s)
     const int items_per_head = (p.tiles + 1) / 2;
     const unsigned long long total_items = (unsigned long long)items_per_head * (unsigned long long)heads;
     const unsigned grid1 = (unsigned)(total_items < (unsigned long long)sms ? total_items : (unsigned long long)sms);
-    scores_tri_sm100_kernel<false><<<grid1, kThreads, kSmemBytes, s>>>(p, map_k, map_q, map_hs, map_ns, items_per_head,
-                                                                       total_items, q_rows_pad);
-    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    (void)grid1;
+    if ((e = launch_scores_pass1_sm100(p, s, map_k, map_q, map_hs, q_rows_pad, sms)) != cudaSuccess) return e;
     if ((e = mark_kernel(p, 0, s)) != cudaSuccess) return e;
     const bool rule_on = p.beta > 0 && p.sim_threshold < 1.0f;
     if (!rule_on || p.tiles < 2) return mark_kernel(p, 1, s);       // nobody can lack partners / pass 1 has seen everything

@@ -123,6 +123,39 @@ __device__ __forceinline__ void umma_tile_k128(uint32_t d_tmem, uint32_t a_addr,
         ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc)
         : "memory");
 }
+// The same product with the second 64-column half of each operand at its own distance from the first (a_half,
+// b_half bytes; multiples of 1024): for operand blocks with fewer than 128 rows packed back to back.
+__device__ __forceinline__ void umma_tile_k128_halves(uint32_t d_tmem, uint32_t a_addr, uint32_t a_half, uint32_t b_addr,
+                                                      uint32_t b_half, uint32_t idesc)
+{
+    const uint32_t a0 = ((a_addr & 0x3FFFFu) >> 4) | (1u << 16);
+    const uint32_t b0 = ((b_addr & 0x3FFFFu) >> 4) | (1u << 16);
+    const uint32_t a1 = (((a_addr + a_half) & 0x3FFFFu) >> 4) | (1u << 16);
+    const uint32_t b1 = (((b_addr + b_half) & 0x3FFFFu) >> 4) | (1u << 16);
+    const uint32_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);      // stride 1024 B, descriptor version, 128-byte swizzle
+    asm volatile(
+        "{\n\t.reg .pred p0, p1;\n\t.reg .b64 da, db;\n\t.reg .b32 ta, tb;\n\t"
+        "setp.ne.u32 p0, %3, %3;\n\tsetp.eq.u32 p1, %3, %3;\n\t"
+        "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p0;\n\t"
+        "add.u32 ta, %1, 2;\n\tadd.u32 tb, %2, 2;\n\tmov.b64 da, {ta, %3};\n\tmov.b64 db, {tb, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p1;\n\t"
+        "add.u32 ta, %1, 4;\n\tadd.u32 tb, %2, 4;\n\tmov.b64 da, {ta, %3};\n\tmov.b64 db, {tb, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p1;\n\t"
+        "add.u32 ta, %1, 6;\n\tadd.u32 tb, %2, 6;\n\tmov.b64 da, {ta, %3};\n\tmov.b64 db, {tb, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p1;\n\t"
+        "mov.b64 da, {%5, %3};\n\tmov.b64 db, {%6, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p1;\n\t"
+        "add.u32 ta, %5, 2;\n\tadd.u32 tb, %6, 2;\n\tmov.b64 da, {ta, %3};\n\tmov.b64 db, {tb, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p1;\n\t"
+        "add.u32 ta, %5, 4;\n\tadd.u32 tb, %6, 4;\n\tmov.b64 da, {ta, %3};\n\tmov.b64 db, {tb, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p1;\n\t"
+        "add.u32 ta, %5, 6;\n\tadd.u32 tb, %6, 6;\n\tmov.b64 da, {ta, %3};\n\tmov.b64 db, {tb, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p1;\n\t"
+        "}"
+        ::"r"(d_tmem), "r"(a0), "r"(b0), "r"(hi), "r"(idesc), "r"(a1), "r"(b1)
+        : "memory");
+}
 // One more K = 16 step onto the accumulator at d_tmem: both operands are 128 rows x 16 bf16 (32-byte rows, 32-byte
 // swizzle, 8-row groups 256 bytes apart, 256-byte aligned).
 __device__ __forceinline__ void umma_k16_sw32(uint32_t d_tmem, uint32_t a_addr, uint32_t b_addr, uint32_t idesc)
@@ -170,6 +203,43 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16])
         : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&r)[8])
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_ld1(uint32_t taddr, uint32_t &r)
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(r) : "r"(taddr) : "memory");
+}
+// Wait for the thread's TMEM loads; the loaded registers pass through the statement so that nothing that uses
+// them can be scheduled ahead of it.
+__device__ __forceinline__ void tmem_wait8(uint32_t (&r)[8])
+{
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7])
+                 :: "memory");
+}
+__device__ __forceinline__ void tmem_wait32(uint32_t (&r)[32])
+{
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                   "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+                   "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
+                   "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+                 :: "memory");
+}
+
+// max(a, b, c), NaN operands ignored
+__device__ __forceinline__ float max3(float a, float b, float c)
+{
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
 
 
 // ---- host side: tensor maps -------------------------------------------------------------------------------
@@ -220,4 +290,9 @@ inline bool make_map_k16(CUtensorMap *map, const void *base, uint64_t rows)
 }
 
 }  // namespace sm100
+
+// first scoring pass of the two-pass tensor-core route (its own file); the maps are built by the caller
+cudaError_t launch_scores_pass1_sm100(const Params &p, cudaStream_t s, const CUtensorMap &map_k, const CUtensorMap &map_q,
+                                      const CUtensorMap &map_hs, int q_rows_pad, int sms);
+
 }  // namespace rkv
