@@ -69,7 +69,7 @@ int check_shapes(const rkv_desc_t *d, int budget, int buffer, int alpha, Layout 
         lay->head_sum_bf16 = off; off = align_up(off + P * 16 * kHeadDim * sizeof(__nv_bfloat16), 256);
         lay->meta = off;        off = align_up(off + (size_t)d->batch * sizeof(int32_t), 256);
         // the region the prep stage zeroes: counters and per-head tile tickets
-        lay->counters = off;    off = align_up(off + 8 * sizeof(unsigned long long), 256);
+        lay->counters = off;    off = align_up(off + 32 * sizeof(unsigned long long), 256);
         lay->tile_done = off;   off = align_up(off + P * sizeof(uint32_t), 256);
         lay->zero_bytes = off - lay->counters;
         lay->total = off;
@@ -346,8 +346,9 @@ int rkv_launch_count(const rkv_desc_t *desc, uint32_t stage_mask)
     for (uint32_t bit = 1; bit <= RKV_STAGE_GATHER; bit <<= 1) c += (stage_mask & bit) ? 1 : 0;
     if (stage_mask & RKV_STAGE_SELECT) c += 2;      // row statistics and importance run ahead of the selection kernel
     if (desc && (stage_mask & RKV_STAGE_SELECT) && (desc->flags & RKV_FLAG_HEAD_MEAN)) c += 1;   // per-sequence selection
-    // the triangle scoring path is three kernels (pass 1, listing, pass 2) while the retention rule is on
-    if (desc && (stage_mask & RKV_STAGE_SCORES) && use_tri(desc) && desc->beta > 0 && desc->sim_threshold < 1.0f) c += 2;
+    // the two-pass scoring path is the first pass plus up to three rounds of (listing, second pass) while the
+    // retention rule is on
+    if (desc && (stage_mask & RKV_STAGE_SCORES) && use_tri(desc) && desc->beta > 0 && desc->sim_threshold < 1.0f) c += 6;
     return c;
 }
 
@@ -357,8 +358,9 @@ int rkv_launch_count_for(const rkv_desc_t *desc, int32_t budget, int32_t buffer,
     if (check_shapes(desc, budget, buffer, alpha, &lay) != RKV_OK) return 0;
     int c = rkv_launch_count(desc, stage_mask);
     if ((stage_mask & RKV_STAGE_SELECT) && select_is_fused(lay.cap_pad, alpha)) c -= 2;
-    if ((stage_mask & RKV_STAGE_SCORES) && use_tri(desc) && desc->beta > 0 && desc->sim_threshold < 1.0f && lay.tiles < 2)
-        c -= 2;                                     // one key tile: the first scoring pass has seen everything
+    if ((stage_mask & RKV_STAGE_SCORES) && use_tri(desc) && desc->beta > 0 && desc->sim_threshold < 1.0f)
+        c -= lay.tiles < 2 ? 6                                      // one key tile: the first scoring pass has seen everything
+                           : 2 * (3 - scores_pass2_rounds(lay.tiles));   // small caches take fewer rounds
     return c;
 }
 

@@ -63,7 +63,8 @@ struct Params {
                                     //           [3] = item ticket of the second pass, [4] = the call's abort word
                                     //           (non-zero once a bounded wait ran out: later kernels of the call
                                     //           then leave the caches, lengths and index lists alone),
-                                    //           [5] = listed-token x key-tile pairs the second pass has to form
+                                    //           [5] = listed-token x key-tile pairs the second pass has to form,
+                                    //           [8 + 2 r], [9 + 2 r] = work items and item ticket of its round r
     uint32_t *tile_done;            // [P]       tiles of the head finished by the prep stage
     size_t zero_bytes;              // bytes from `counters` to the end of `tile_done`
     int tri;                        // 1: the triangle kernels score (bf16 default); 0: another kernel does
@@ -158,6 +159,7 @@ cudaError_t launch_push_query(void *q_window, const void *q_new, int batch, int 
                               cudaStream_t s);
 bool scores_sm100_available();
 long long sm100_default_wait_cycles();          // default limit of the kernels' bounded waits (about two seconds)
+int scores_pass2_rounds(int tiles);            // list + scan rounds of the second scoring pass for caches of `tiles` key tiles
 bool select_is_fused(int cap_pad, int alpha);   // the select stage is one kernel (small caches) instead of three
 
 }  // namespace rkv
