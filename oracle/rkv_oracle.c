@@ -418,3 +418,67 @@ int rkv_oracle_batch(const float *K, const float *Q, const int32_t *seq_lens,
     free(zown);
     return bad ? -1 : threads;
 }
+
+/*
+ * Section 3.1's decode step on the cache as it stands (retained tokens plus the
+ * buffer): the new token's query of every query head attends over the cached
+ * keys of its KV head, Eq. 1 with a single query row,
+ *   out[b][q] = sum_j softmax_j( q . K[b][q / G][j] / sqrt(d) ) V[b][q / G][j],
+ *   j < seq_lens[b].
+ * K, V [B][Hkv][cap][d] float, Qn [B][Hq][d] float, out [B][Hq][d] double.
+ * A sequence with no cached token gives a zero row.  Returns 0, or -1 on bad
+ * arguments.
+ */
+int rkv_oracle_decode_attention(const float *K, const float *V, const float *Qn,
+                                const int32_t *seq_lens, int B, int Hkv, int Hq,
+                                int cap, int d, double *out)
+{
+    if (B < 1 || Hkv < 1 || Hq % Hkv != 0 || d < 1 || cap < 1)
+        return -1;
+    const int G = Hq / Hkv;
+    int bad = 0;
+#ifdef _OPENMP
+#pragma omp parallel for schedule(dynamic, 1)
+#endif
+    for (int bq = 0; bq < B * Hq; ++bq) {
+        const int b = bq / Hq, q = bq % Hq, h = q / G;
+        const int L = seq_lens[b];
+        double *o = out + (size_t)bq * d;
+        for (int c = 0; c < d; ++c)
+            o[c] = 0.0;
+        if (L < 0 || L > cap) {
+#ifdef _OPENMP
+#pragma omp atomic write
+#endif
+            bad = 1;
+            continue;
+        }
+        if (L == 0)
+            continue;
+        const float *Kh = K + ((size_t)b * Hkv + h) * cap * d;
+        const float *Vh = V + ((size_t)b * Hkv + h) * cap * d;
+        const float *qv = Qn + (size_t)bq * d;
+        double *w = (double *)malloc((size_t)L * sizeof(double));
+        double mx = -INFINITY;
+        for (int j = 0; j < L; ++j) {
+            double dot = 0.0;
+            for (int c = 0; c < d; ++c)
+                dot += (double)qv[c] * (double)Kh[(size_t)j * d + c];
+            w[j] = dot / sqrt((double)d);
+            if (w[j] > mx)
+                mx = w[j];
+        }
+        double sum = 0.0;
+        for (int j = 0; j < L; ++j) {
+            w[j] = exp(w[j] - mx);
+            sum += w[j];
+        }
+        for (int j = 0; j < L; ++j) {
+            const double a = w[j] / sum;
+            for (int c = 0; c < d; ++c)
+                o[c] += a * (double)Vh[(size_t)j * d + c];
+        }
+        free(w);
+    }
+    return bad ? -1 : 0;
+}

@@ -44,6 +44,8 @@ def _load():
         lib.rkv_oracle_gather.restype = None
         lib.rkv_oracle_gather.argtypes = [ctypes.c_void_p, ip, ctypes.c_int, ctypes.c_size_t,
                                           ctypes.c_void_p]
+        lib.rkv_oracle_decode_attention.restype = ctypes.c_int
+        lib.rkv_oracle_decode_attention.argtypes = [fp, fp, fp, ip] + [ctypes.c_int] * 5 + [dp]
         _lib = lib
     return _lib
 
@@ -112,8 +114,15 @@ class BatchResult:
 
 def oracle_batch(K, Q, seq_lens, *, budget: int, alpha: int, lam: float, W: int, beta: int,
                  T: float, eps: float = 1e-8, want_scores: bool = True,
-                 mean_then_pool: bool = False, head_mean: bool = False, gqa_mean_pool: bool = False) -> BatchResult:
-    """K [B, Hkv, cap, d], Q [B, Hq, alpha, d], seq_lens [B]."""
+                 mean_then_pool: bool = False, head_mean: bool = False, gqa_mean_pool: bool = False,
+                 budgets=None) -> BatchResult:
+    """K [B, Hkv, cap, d], Q [B, Hq, alpha, d], seq_lens [B].
+    budgets: optional [B], a budget of its own per sequence (Section 4.2's budget ratios); `budget` is then only
+    the row length of idx (entries beyond a sequence's own budget are -1)."""
+    if budgets is not None:
+        return _oracle_batch_per_sequence(K, Q, seq_lens, budgets, budget=budget, alpha=alpha, lam=lam, W=W, beta=beta,
+                                          T=T, eps=eps, want_scores=want_scores, mean_then_pool=mean_then_pool,
+                                          head_mean=head_mean, gqa_mean_pool=gqa_mean_pool)
     lib = _load()
     K = _f32(K)
     Q = _f32(Q)
@@ -134,6 +143,46 @@ def oracle_batch(K, Q, seq_lens, *, budget: int, alpha: int, lam: float, W: int,
     if scores is None:
         return BatchResult(idx, comp.astype(bool), None, None, None, None, t)
     return BatchResult(idx, comp.astype(bool), scores[0], scores[1], scores[2], scores[3], t)
+
+
+def _oracle_batch_per_sequence(K, Q, seq_lens, budgets, *, budget, want_scores, **kw) -> BatchResult:
+    """Every sequence with its own budget: the sequences are independent, so each goes through the C oracle alone
+    with its budget, and the results are put side by side (marshalling only)."""
+    K = _f32(K)
+    Q = _f32(Q)
+    B, Hkv, cap, _ = K.shape
+    idx = np.full((B, Hkv, budget), -1, dtype=np.int32)
+    comp = np.zeros(B, dtype=bool)
+    scores = [np.zeros((B, Hkv, cap)) for _ in range(4)] if want_scores else [None] * 4
+    threads = 1
+    for b in range(B):
+        nb = int(budgets[b])
+        assert kw["alpha"] < nb <= budget
+        r = oracle_batch(K[b:b + 1], Q[b:b + 1], np.asarray(seq_lens)[b:b + 1], budget=nb, want_scores=want_scores, **kw)
+        idx[b, :, :nb] = r.idx[0]
+        comp[b] = r.compressed[0]
+        threads = max(threads, r.threads)
+        if want_scores:
+            for t, part in enumerate((r.I, r.Sbar, r.R, r.Z)):
+                scores[t][b] = part[0]
+    return BatchResult(idx, comp, scores[0], scores[1], scores[2], scores[3], threads)
+
+
+def oracle_decode_attention(K, V, q_new, seq_lens) -> np.ndarray:
+    """Section 3.1's decode step: the new query of every query head over the cached keys and values of its KV head
+    (Eq. 1 with one query row).  K, V [B, Hkv, cap, d], q_new [B, Hq, d], seq_lens [B] -> [B, Hq, d] float64."""
+    lib = _load()
+    K, V, q_new = _f32(K), _f32(V), _f32(q_new)
+    seq = np.ascontiguousarray(np.asarray(seq_lens, dtype=np.int32))
+    B, Hkv, cap, d = K.shape
+    Hq = q_new.shape[1]
+    assert V.shape == K.shape and q_new.shape == (B, Hq, d) and seq.shape == (B,)
+    out = np.zeros((B, Hq, d))
+    rc = lib.rkv_oracle_decode_attention(_ptr(K, ctypes.c_float), _ptr(V, ctypes.c_float), _ptr(q_new, ctypes.c_float),
+                                         _ptr(seq, ctypes.c_int32), B, Hkv, Hq, cap, d, _ptr(out, ctypes.c_double))
+    if rc != 0:
+        raise ValueError("rkv_oracle_decode_attention: bad arguments")
+    return out
 
 
 def oracle_gather(rows: np.ndarray, idx: np.ndarray) -> np.ndarray:

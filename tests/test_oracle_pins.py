@@ -565,3 +565,68 @@ def test_append_and_query_ring_semantics():
     b_ = _run(Kh, np.roll(q[0], 1, axis=1), budget=20, alpha=alpha)
     np.testing.assert_allclose(a.I, b_.I, rtol=1e-12)
     np.testing.assert_array_equal(a.idx, b_.idx)
+
+
+def test_decode_attention_against_library_softmax_and_closed_forms():
+    """Section 3.1's decode step (Eq. 1 with one query row) pinned to what fixes it from outside: scipy's softmax and
+    numpy's matrix product per query head with the GQA head mapping written out; one cached token returns its value
+    row; identical keys give the mean of the values; adding a constant vector's worth of logit to every key changes
+    nothing; tokens at and beyond the cached length are never read (NaN there)."""
+    from scipy.special import softmax
+    import oracle
+    rng = np.random.default_rng(17)
+    B, Hkv, Hq, cap, d = 3, 2, 6, 37, 16
+    G = Hq // Hkv
+    K = rng.standard_normal((B, Hkv, cap, d)).astype(np.float32)
+    V = rng.standard_normal((B, Hkv, cap, d)).astype(np.float32)
+    q = rng.standard_normal((B, Hq, d)).astype(np.float32)
+    seq = np.array([37, 1, 20], dtype=np.int32)
+    K[2, :, 20:] = np.nan
+    V[2, :, 20:] = np.nan
+    out = oracle.oracle_decode_attention(K, V, q, seq)
+    for b in range(B):
+        L = int(seq[b])
+        for h in range(Hq):
+            kv = h // G
+            w = softmax(q[b, h].astype(np.float64) @ K[b, kv, :L].astype(np.float64).T / np.sqrt(d))
+            want = w @ V[b, kv, :L].astype(np.float64)
+            assert np.allclose(out[b, h], want, rtol=1e-12, atol=1e-14)
+    assert np.allclose(out[1], np.repeat(V[1, :, 0].astype(np.float64), G, axis=0))          # one token: its value row
+    Ks = K.copy()
+    Ks[0] = Ks[0, :, :1]                                                                     # identical keys
+    same = oracle.oracle_decode_attention(Ks, V, q, seq)
+    assert np.allclose(same[0], np.repeat(V[0].astype(np.float64).mean(axis=1), G, axis=0))
+    # softmax is shift-invariant: a key component that is the same for every token moves every logit alike
+    Kc, qc = np.concatenate([K, np.full((B, Hkv, cap, 1), 3.0, np.float32)], -1), \
+        np.concatenate([q * np.sqrt((d + 1) / d), np.full((B, Hq, 1), 0.7, np.float32)], -1).astype(np.float32)
+    Vc = np.concatenate([V, np.zeros((B, Hkv, cap, 1), np.float32)], -1)
+    Kc[2, :, 20:] = np.nan
+    shifted = oracle.oracle_decode_attention(Kc, Vc, qc, seq)
+    assert np.allclose(shifted[..., :d], out, rtol=1e-5, atol=1e-6)
+    empty = oracle.oracle_decode_attention(K, V, q, np.array([0, 0, 0], dtype=np.int32))
+    assert not empty.any()
+
+
+def test_per_sequence_budgets_equal_independent_calls():
+    """Budgets of their own per sequence (Section 4.2's budget ratios): every sequence's result is the one a call with
+    that budget alone gives, index rows are padded with -1 beyond the sequence's budget, and a sequence at or below its
+    budget is left alone."""
+    import oracle
+    rng = np.random.default_rng(23)
+    B, Hkv, Hq, cap, d, alpha = 3, 2, 4, 60, 16, 4
+    K = rng.standard_normal((B, Hkv, cap, d)).astype(np.float32)
+    Q = rng.standard_normal((B, Hq, alpha, d)).astype(np.float32)
+    seq = np.array([60, 50, 33], dtype=np.int32)
+    budgets = np.array([40, 24, 33], dtype=np.int32)
+    kw = dict(alpha=alpha, lam=0.1, W=2, beta=1, T=0.3)
+    res = oracle.oracle_batch(K, Q, seq, budget=40, budgets=budgets, **kw)
+    assert res.compressed.tolist() == [True, True, False]
+    for b in range(B):
+        one = oracle.oracle_batch(K[b:b + 1], Q[b:b + 1], seq[b:b + 1], budget=int(budgets[b]), **kw)
+        nb = int(budgets[b])
+        assert np.array_equal(res.idx[b, :, :nb], one.idx[0])
+        assert (res.idx[b, :, nb:] == -1).all()
+        assert np.array_equal(res.Z[b], one.Z[0])
+    kept = res.idx[1, 0, :24]
+    assert np.all(np.diff(kept) > 0) and np.array_equal(kept[-alpha:], np.arange(46, 50))    # 24 kept, observation tail
+    assert np.array_equal(res.idx[2, 0, :33], np.arange(33))                                 # L = budget: the guard
