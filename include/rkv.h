@@ -125,6 +125,13 @@ typedef struct rkv_desc {
        A wait that runs out is an error (RKV_ERR_TIMEOUT), never a hang.  Values below about a million ticks can
        expire during ordinary memory latency: leave it at 0 outside of tests. */
     int64_t wait_limit_cycles;
+    /* optional device int32[batch]: a budget of its own for every sequence (the budget-ratio experiments of Section
+       4.2: the budget as a share of each sequence's length), alpha < budgets[b] <= budget.  NULL: every sequence
+       uses the call's `budget`.  The call's `budget` stays the maximum: it fixes the cache capacity (budget +
+       buffer) and the row length of out_idx.  Sequence b is compressed when seq_lens[b] > budgets[b]; it keeps
+       budgets[b] tokens, out_idx[b][h][budgets[b] ..] = -1, and seq_lens[b] becomes budgets[b].  A value out of
+       range is treated like an invalid length: the sequence is skipped and RKV_ERR_INVALID_ARG recorded. */
+    const int32_t *budgets;
 } rkv_desc_t;
 
 /* Fill *desc with the defaults above (pool_w 4, beta 1, T 0.5, eps 1e-8, head_dim 128, bf16), zero elsewhere. */
@@ -240,6 +247,27 @@ RKV_API int rkv_append(const rkv_desc_t *desc, void *k_cache, void *v_cache, con
                        int32_t *seq_lens, int32_t budget, int32_t buffer, void *stream);
 RKV_API int rkv_push_query(const rkv_desc_t *desc, void *q_window, const void *q_new, int32_t alpha, int32_t slot,
                            void *stream);
+
+/*
+ * The attention of a decode step over the cache as it stands (Section 3.1: between two firings the model decodes
+ * against the retained tokens plus the buffer; Eq. 1 with one query row per head), so that a whole decode segment --
+ * rkv_push_query, rkv_decode_attention, rkv_append, and rkv_compress when the buffer is full -- runs through this
+ * library:
+ *   out[b][q] = sum_j softmax_j( q_new[b][q] . K[b][q / G][j] / sqrt(head_dim) ) V[b][q / G][j],  j < seq_lens[b]
+ *   k_cache, v_cache  [batch][n_kv_heads][budget + buffer][head_dim] (device, desc->dtype), read only
+ *   q_new             [batch][n_q_heads][head_dim] (device, desc->dtype, 16-byte aligned)
+ *   seq_lens          [batch] int32 (device), read only; 0 gives a zero output row; a value outside
+ *                     [0, budget + buffer] gives a zero row and RKV_ERR_INVALID_ARG in desc->device_status
+ *   out               [batch][n_q_heads][head_dim] float32 (device, 16-byte aligned)
+ * fp32 arithmetic throughout.  G = n_q_heads / n_kv_heads up to 8 (RKV_ERR_UNSUPPORTED beyond).  With few
+ * head-problems the rows of a head are cut into splits whose partial results go through desc->workspace:
+ * rkv_decode_workspace_bytes() says how much that needs (0 for large batches; never more than a compression of the
+ * same shape needs, so one workspace serves both).  Enqueues one or two kernels on `stream`; return codes as for
+ * rkv_compress_ex.
+ */
+RKV_API size_t rkv_decode_workspace_bytes(const rkv_desc_t *desc, int32_t budget, int32_t buffer);
+RKV_API int rkv_decode_attention(const rkv_desc_t *desc, const void *k_cache, const void *v_cache, const void *q_new,
+                                 const int32_t *seq_lens, float *out, int32_t budget, int32_t buffer, void *stream);
 
 /*
  * Self-test of the kernels' failure detection (no counterpart in the paper).  Every wait inside the tensor-core

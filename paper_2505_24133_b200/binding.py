@@ -41,7 +41,7 @@ class RkvDesc(ctypes.Structure):
         ("device_status", ctypes.c_void_p), ("dbg_I", ctypes.c_void_p), ("dbg_Sbar", ctypes.c_void_p),
         ("dbg_R", ctypes.c_void_p), ("dbg_Z", ctypes.c_void_p), ("stage_events", ctypes.c_void_p),
         ("kernel_events", ctypes.c_void_p), ("dbg_counters", ctypes.c_void_p),
-        ("wait_limit_cycles", ctypes.c_int64),
+        ("wait_limit_cycles", ctypes.c_int64), ("budgets", ctypes.c_void_p),
     ]
 
 
@@ -71,6 +71,8 @@ def lib():
         L.rkv_compress_static.restype, L.rkv_compress_static.argtypes = ctypes.c_int, [P] + ten
         L.rkv_append.restype, L.rkv_append.argtypes = ctypes.c_int, [P, VP, VP, VP, VP, VP, I32, I32, VP]
         L.rkv_push_query.restype, L.rkv_push_query.argtypes = ctypes.c_int, [P, VP, VP, I32, I32, VP]
+        L.rkv_decode_workspace_bytes.restype, L.rkv_decode_workspace_bytes.argtypes = SZ, [P, I32, I32]
+        L.rkv_decode_attention.restype, L.rkv_decode_attention.argtypes = ctypes.c_int, [P, VP, VP, VP, VP, VP, I32, I32, VP]
         L.rkv_selftest_wait_expiry.restype, L.rkv_selftest_wait_expiry.argtypes = ctypes.c_int, [VP, VP, ctypes.c_int64, VP]
         L.rkv_launch_count.restype, L.rkv_launch_count.argtypes = ctypes.c_int, [P, U32]
         L.rkv_launch_count_for.restype, L.rkv_launch_count_for.argtypes = ctypes.c_int, [P, I32, I32, I32, U32]
@@ -174,6 +176,17 @@ def rkv_push_query(desc, q_window, q_new, alpha, slot, stream=None) -> int:
     return lib().rkv_push_query(ctypes.byref(desc), _ptr(q_window), _ptr(q_new), alpha, slot, _stream(stream))
 
 
+def rkv_decode_workspace_bytes(desc, budget: int, buffer: int) -> int:
+    return int(lib().rkv_decode_workspace_bytes(ctypes.byref(desc), budget, buffer))
+
+
+def rkv_decode_attention(desc, k_cache, v_cache, q_new, seq_lens, out, budget, buffer, stream=None) -> int:
+    """The new token's queries attend over the cached keys and values of their KV heads (Section 3.1, Eq. 1);
+    out [batch, n_q_heads, head_dim] float32."""
+    return lib().rkv_decode_attention(ctypes.byref(desc), _ptr(k_cache), _ptr(v_cache), _ptr(q_new), _ptr(seq_lens),
+                                      _ptr(out), budget, buffer, _stream(stream))
+
+
 def rkv_selftest_wait_expiry(device_status, report_words, limit_cycles: int, stream=None) -> int:
     """Make a bounded device-side wait run out on purpose in a tiny kernel of its own (failure-detection self-test)."""
     return lib().rkv_selftest_wait_expiry(_ptr(device_status), _ptr(report_words), int(limit_cycles), _stream(stream))
@@ -189,7 +202,7 @@ class Compressor:
                  lam: float = 0.1, dtype: torch.dtype = torch.bfloat16, pool_w: Optional[int] = None,
                  beta: Optional[int] = None, sim_threshold: Optional[float] = None, eps: Optional[float] = None,
                  flags: int = 0, device="cuda", dump_scores: bool = False, host_staging: bool = False,
-                 stage_events: bool = False):
+                 stage_events: bool = False, budgets: Optional[torch.Tensor] = None):
         self.budget, self.buffer, self.alpha, self.lam = budget, buffer, alpha, lam
         self.cap = budget + buffer
         self.device = torch.device(device)
@@ -231,6 +244,11 @@ class Compressor:
             d.kernel_events = ctypes.cast(self._kevent_array, ctypes.c_void_p)
             self.counters = torch.zeros(8, dtype=torch.int64, device=self.device)
             d.dbg_counters = self.counters.data_ptr()
+        self.budgets = None
+        if budgets is not None:          # per-sequence budgets (device int32 [batch]); `budget` stays the maximum
+            self.budgets = budgets.to(device=self.device, dtype=torch.int32).contiguous()
+            assert self.budgets.shape == (batch,)
+            d.budgets = self.budgets.data_ptr()
         self.desc = d
         self.out_idx = torch.empty(batch, n_kv_heads, budget, dtype=torch.int32, device=self.device)
 

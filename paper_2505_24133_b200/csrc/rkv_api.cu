@@ -67,7 +67,7 @@ int check_shapes(const rkv_desc_t *d, int budget, int buffer, int alpha, Layout 
         lay->strag_items = off; off = align_up(off + tri * P * (lay->cap_pad / 256 + 1) * sizeof(int4), 256);
         lay->self_dot = off;    off = align_up(off + P * lay->cap_pad * sizeof(float), 256);
         lay->head_sum_bf16 = off; off = align_up(off + P * 16 * kHeadDim * sizeof(__nv_bfloat16), 256);
-        lay->meta = off;        off = align_up(off + (size_t)d->batch * sizeof(int32_t), 256);
+        lay->meta = off;        off = align_up(off + 2 * (size_t)d->batch * sizeof(int32_t), 256);
         // the region the prep stage zeroes: counters and per-head tile tickets
         lay->counters = off;    off = align_up(off + 32 * sizeof(unsigned long long), 256);
         lay->tile_done = off;   off = align_up(off + P * sizeof(uint32_t), 256);
@@ -87,7 +87,8 @@ int run(const rkv_desc_t *d, void *k_cache, void *v_cache, const void *q_window,
     if (rc != RKV_OK) return rc;
     if (!k_cache || !v_cache || !q_window || !seq_lens || !out_idx) return RKV_ERR_INVALID_ARG;
     if (!aligned16(k_cache) || !aligned16(v_cache) || !aligned16(q_window)) return RKV_ERR_INVALID_ARG;
-    if ((reinterpret_cast<uintptr_t>(seq_lens) & 3u) || (reinterpret_cast<uintptr_t>(out_idx) & 3u))
+    if ((reinterpret_cast<uintptr_t>(seq_lens) & 3u) || (reinterpret_cast<uintptr_t>(out_idx) & 3u) ||
+        (reinterpret_cast<uintptr_t>(d->budgets) & 3u))
         return RKV_ERR_INVALID_ARG;
     if (!(lambda >= 0.f && lambda <= 1.f)) return RKV_ERR_INVALID_ARG;
     if ((stages & ~RKV_STAGE_ALL) != 0u || stages == 0u) return RKV_ERR_INVALID_ARG;
@@ -142,6 +143,7 @@ int run(const rkv_desc_t *d, void *k_cache, void *v_cache, const void *q_window,
     p.zero_bytes = lay.zero_bytes;
     p.tri = lay.tri;
     p.status = d->device_status;
+    p.budgets = d->budgets;
     p.wait_cycles = d->wait_limit_cycles > 0 ? (long long)d->wait_limit_cycles : sm100_default_wait_cycles();
     p.kernel_events = d->kernel_events;
     p.dbg_counters = d->dbg_counters;
@@ -338,6 +340,48 @@ int rkv_push_query(const rkv_desc_t *d, void *q_window, const void *q_new, int32
     const cudaError_t e = launch_push_query(q_window, q_new, d->batch, d->n_q_heads, alpha, slot, row_bytes,
                                             static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? RKV_OK : cuda_fail(e, "push_query launch");
+}
+
+static int attend_plan(const rkv_desc_t *d, int32_t budget, int32_t buffer, int *splits, size_t *bytes)
+{
+    int rc = check_shapes(d, budget, buffer, 1, nullptr);
+    if (rc != RKV_OK) return rc;
+    const int G = d->n_q_heads / d->n_kv_heads;
+    if (G > attend_max_group()) return RKV_ERR_UNSUPPORTED;
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+        sms = 148;       // sizing only (no device here): the B200's count
+    *splits = attend_splits(d->batch * d->n_kv_heads, budget + buffer, sms);
+    *bytes = attend_partial_bytes(d->batch * d->n_kv_heads, *splits, G);
+    return RKV_OK;
+}
+
+size_t rkv_decode_workspace_bytes(const rkv_desc_t *desc, int32_t budget, int32_t buffer)
+{
+    int splits = 1;
+    size_t bytes = 0;
+    return attend_plan(desc, budget, buffer, &splits, &bytes) == RKV_OK ? bytes : 0;
+}
+
+int rkv_decode_attention(const rkv_desc_t *d, const void *k_cache, const void *v_cache, const void *q_new,
+                         const int32_t *seq_lens, float *out, int32_t budget, int32_t buffer, void *stream)
+{
+    int splits = 1;
+    size_t bytes = 0;
+    int rc = attend_plan(d, budget, buffer, &splits, &bytes);
+    if (rc != RKV_OK) return rc;
+    if (!k_cache || !v_cache || !q_new || !seq_lens || !out) return RKV_ERR_INVALID_ARG;
+    if (!aligned16(k_cache) || !aligned16(v_cache) || !aligned16(q_new) || !aligned16(out)) return RKV_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(seq_lens) & 3u) return RKV_ERR_INVALID_ARG;
+    if (bytes > 0) {
+        if (!d->workspace || d->workspace_bytes < bytes) return RKV_ERR_WORKSPACE;
+        if (reinterpret_cast<uintptr_t>(d->workspace) & 255u) return RKV_ERR_WORKSPACE;
+    }
+    const long long wait = d->wait_limit_cycles > 0 ? (long long)d->wait_limit_cycles : sm100_default_wait_cycles();
+    const cudaError_t e = launch_attend(k_cache, v_cache, q_new, seq_lens, out, static_cast<float *>(d->workspace), d->batch,
+                                        d->n_kv_heads, d->n_q_heads, budget + buffer, splits, d->dtype, d->device_status,
+                                        wait, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? RKV_OK : cuda_fail(e, "decode attention launch");
 }
 
 int rkv_launch_count(const rkv_desc_t *desc, uint32_t stage_mask)

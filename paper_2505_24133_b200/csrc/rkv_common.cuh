@@ -56,7 +56,9 @@ struct Params {
                          //                      token, tokens (1..256), first streamed tile}
     float *self_dot;     // [P][cap_pad]         Kbar_i . Kbar_i (1 up to rounding and eps; 0 for a zero key)
     __nv_bfloat16 *head_sum_bf16;   // [P][16][128] head_sum split into three bf16 rows (hi, mid, lo), 13 zero rows
-    int32_t *meta;       // [batch]              snapshot of seq_lens (kMetaInvalid if out of range)
+    int32_t *meta;       // [2][batch]           snapshot of seq_lens (kMetaInvalid if out of range), then each
+                         //                      sequence's budget (p.budget unless the caller gave per-sequence ones)
+    const int32_t *budgets;   // optional [batch]: per-sequence budgets (alpha < budgets[b] <= budget), else null
     // zeroed by the prep stage's memset, in this order, contiguous:
     unsigned long long *counters;   // [8]       [0] = similarity tiles computed by the tcgen05 kernels, [1] = item
                                     //           ticket of the first scoring pass, [2] = entries in strag_items,
@@ -107,7 +109,7 @@ __device__ __forceinline__ ErrSink make_sink(const Params &p)
 __device__ __forceinline__ void report_timeout(const ErrSink &sink)
 {
     report(sink.status, RKV_ERR_TIMEOUT);
-    atomicExch(sink.abort_word, 1ull);
+    if (sink.abort_word) atomicExch(sink.abort_word, 1ull);
 }
 // True once some kernel of this call has given up on a wait.
 __device__ __forceinline__ bool call_aborted(const Params &p)
@@ -115,10 +117,16 @@ __device__ __forceinline__ bool call_aborted(const Params &p)
     return *reinterpret_cast<volatile unsigned long long *>(p.counters + kAbortWord) != 0ull;
 }
 
-// Number of candidates of sequence b as every stage after prep sees it: 0 = nothing to compress.
+// Number of candidates of a sequence of length L with the given budget: 0 = nothing to compress.
 __device__ __forceinline__ int candidates_from_meta(int L, int budget, int alpha)
 {
     return (L > budget) ? (L - alpha) : 0;
+}
+// The same for sequence b as every stage after prep sees it (length and budget snapshots left by the prep stage).
+__device__ __forceinline__ int seq_budget(const Params &p, int b) { return p.meta[p.batch + b]; }
+__device__ __forceinline__ int seq_candidates(const Params &p, int b)
+{
+    return candidates_from_meta(p.meta[b], p.meta[p.batch + b], p.alpha);
 }
 
 template <typename T> struct Elem;
@@ -157,6 +165,12 @@ cudaError_t launch_append(void *k_cache, void *v_cache, const void *k_new, const
                           int hkv, int cap, int row_bytes, int32_t *status, cudaStream_t s);
 cudaError_t launch_push_query(void *q_window, const void *q_new, int batch, int hq, int alpha, int slot, int row_bytes,
                               cudaStream_t s);
+cudaError_t launch_attend(const void *k_cache, const void *v_cache, const void *q_new, const int32_t *seq_lens, float *out,
+                          float *partial, int batch, int hkv, int hq, int cap, int splits, int dtype, int32_t *status,
+                          long long wait_cycles, cudaStream_t s);
+int attend_max_group();
+int attend_splits(int heads, int cap, int sms);
+size_t attend_partial_bytes(int heads, int splits, int G);
 bool scores_sm100_available();
 long long sm100_default_wait_cycles();          // default limit of the kernels' bounded waits (about two seconds)
 int scores_pass2_rounds(int tiles);            // list + scan rounds of the second scoring pass for caches of `tiles` key tiles

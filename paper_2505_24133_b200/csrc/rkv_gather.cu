@@ -32,9 +32,10 @@ __global__ void __launch_bounds__(kGatherThreads) gather_kernel(Params p)
     const int which = stream & 1;
     const int b = head / p.hkv;
     const int L = p.meta[b];
-    if (L <= p.budget) return;                      // nothing was selected for this sequence
+    const int budget_b = seq_budget(p, b);
+    if (L <= budget_b) return;                      // nothing was selected for this sequence
     if (call_aborted(p)) return;                    // a bounded wait ran out earlier in this call: caches and lengths stay as they are
-    if (which == 0 && slice == 0 && head % p.hkv == 0 && threadIdx.x == 0) p.seq_lens[b] = p.budget;
+    if (which == 0 && slice == 0 && head % p.hkv == 0 && threadIdx.x == 0) p.seq_lens[b] = budget_b;
 
     uint4 *base = reinterpret_cast<uint4 *>(which ? p.v_cache : p.k_cache) + (size_t)head * p.cap * kVecPerRow +
                   slice * kVecPerSlice;
@@ -42,8 +43,8 @@ __global__ void __launch_bounds__(kGatherThreads) gather_kernel(Params p)
     const int lane_vec = threadIdx.x % kVecPerSlice;
     const int lane_row = threadIdx.x / kVecPerSlice;
 
-    for (int j0 = 0; j0 < p.budget; j0 += kRows) {
-        const int j_end = min(j0 + kRows, p.budget);
+    for (int j0 = 0; j0 < budget_b; j0 += kRows) {
+        const int j_end = min(j0 + kRows, budget_b);
         if (idx[j_end - 1] == j_end - 1) continue;   // ascending and idx[j] >= j: the whole chunk is in place
         uint4 held[kVecPerThread];
         int src[kVecPerThread];

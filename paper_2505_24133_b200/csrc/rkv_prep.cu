@@ -42,12 +42,17 @@ __global__ void __launch_bounds__(kPrepThreads, 5) prep_kernel(Params p)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     int L = p.seq_lens[b];
-    if (L < 0 || L > p.cap) {
+    int budget_b = p.budgets ? p.budgets[b] : p.budget;             // Section 4.2's per-sequence (ratio) budgets
+    if (L < 0 || L > p.cap || budget_b <= p.alpha || budget_b > p.budget) {
         report(p.status, RKV_ERR_INVALID_ARG);
         L = kMetaInvalid;
+        budget_b = p.budget;
     }
-    if (tile == 0 && head % p.hkv == 0 && threadIdx.x == 0) p.meta[b] = L;
-    const int n = candidates_from_meta(L, p.budget, p.alpha);
+    if (tile == 0 && head % p.hkv == 0 && threadIdx.x == 0) {
+        p.meta[b] = L;
+        p.meta[p.batch + b] = budget_b;
+    }
+    const int n = candidates_from_meta(L, budget_b, p.alpha);
 
     const T *K = static_cast<const T *>(p.k_cache) + (size_t)head * p.cap * kHeadDim;
     float *inv_norm = p.inv_norm + (size_t)head * p.cap_pad;

@@ -141,7 +141,7 @@ scores_stream_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, 
                 next_ticket = atomicAdd(&p.counters[1], 1ull);
                 const int head = (int)(ticket / (unsigned)splits);
                 const int part = (int)(ticket % (unsigned)splits);
-                const int n = candidates_from_meta(p.meta[head / p.hkv], p.budget, p.alpha);
+                const int n = seq_candidates(p, head / p.hkv);
                 if (n == 0) continue;
                 const int n_tiles = (n + kTile - 1) / kTile;
                 const int t0 = (int)((long long)part * n_tiles / splits), t1 = (int)((long long)(part + 1) * n_tiles / splits);

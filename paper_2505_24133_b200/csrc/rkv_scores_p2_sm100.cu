@@ -517,7 +517,7 @@ __global__ void __launch_bounds__(kCompactThreads) strag_compact_kernel(Params p
     __shared__ int warp_tot[kCompactThreads / 32];
     __shared__ int running;
     const int head = blockIdx.x;
-    const int n = candidates_from_meta(p.meta[head / p.hkv], p.budget, p.alpha);
+    const int n = seq_candidates(p, head / p.hkv);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int32_t *left = p.left + (size_t)head * p.cap_pad;
     int32_t *list = p.strag + (size_t)head * p.cap_pad;

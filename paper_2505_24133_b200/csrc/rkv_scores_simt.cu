@@ -51,7 +51,7 @@ __global__ void __launch_bounds__(kSimtThreads) scores_simt_kernel(Params p)
     const int head = blockIdx.x / blocks_per_head;
     const int x = blockIdx.x % blocks_per_head;
     const int b = head / p.hkv, h = head % p.hkv;
-    const int n = candidates_from_meta(p.meta[b], p.budget, p.alpha);
+    const int n = seq_candidates(p, b);
     if (n == 0) return;
     const int n_tiles = (n + kTile - 1) / kTile;
     const T *K = static_cast<const T *>(p.k_cache) + (size_t)head * p.cap * kHeadDim;

@@ -92,7 +92,7 @@ scores_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, const _
     const int head = blockIdx.x / items;
     const int x = blockIdx.x % items;
     const int b = head / p.hkv, h = head % p.hkv;
-    const int n = candidates_from_meta(p.meta[b], p.budget, p.alpha);
+    const int n = seq_candidates(p, b);
     const bool is_q = (x == row_blocks);
     const int row0 = x * kRowsPerBlock;
     if (n == 0 || (!is_q && row0 >= n)) return;            // uniform for the block; nothing allocated yet

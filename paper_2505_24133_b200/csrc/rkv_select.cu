@@ -70,7 +70,7 @@ __global__ void __launch_bounds__(kStatThreads) row_stats_kernel(Params p)
 {
     __shared__ float scratch[kStatThreads / 32];
     const int head = blockIdx.x / p.alpha, j = blockIdx.x % p.alpha;
-    const int n = candidates_from_meta(p.meta[head / p.hkv], p.budget, p.alpha);
+    const int n = seq_candidates(p, head / p.hkv);
     if (n == 0) return;
     const float *row = p.logits + ((size_t)head * p.alpha + j) * p.cap_pad;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -103,7 +103,7 @@ __global__ void __launch_bounds__(kImpThreads) importance_kernel(Params p)
 {
     const int chunks = (p.cap + kImpTokens - 1) / kImpTokens;
     const int head = blockIdx.x / chunks, i0 = (blockIdx.x % chunks) * kImpTokens;
-    const int n = candidates_from_meta(p.meta[head / p.hkv], p.budget, p.alpha);
+    const int n = seq_candidates(p, head / p.hkv);
     if (i0 >= n) return;
     const int W = p.pool_w;
     const float *logits = p.logits + (size_t)head * p.alpha * p.cap_pad;
@@ -238,6 +238,8 @@ __device__ __forceinline__ void radix_select_emit(const uint32_t *keys, int n, i
     }
     for (int j = tid; j < alpha; j += kSelThreads)
         for (int c = 0; c < copies; ++c) out[(size_t)c * budget + k + j] = n + j;   // observation tokens
+    for (int j = k + alpha + tid; j < budget; j += kSelThreads)                     // a sequence with a smaller budget of its own
+        for (int c = 0; c < copies; ++c) out[(size_t)c * budget + j] = -1;
 }
 
 // Eq. 4 with the default window W = 4 (positions i-4 .. i+3), eight consecutive tokens per thread: per query row
@@ -251,7 +253,7 @@ __global__ void __launch_bounds__(kImp8Threads) importance_w4_kernel(Params p)
     const int chunks = (p.cap + kImp8Tokens - 1) / kImp8Tokens;
     const int head = blockIdx.x / chunks;
     const int i0 = (blockIdx.x % chunks) * kImp8Tokens + threadIdx.x * 8;     // first token of this thread
-    const int n = candidates_from_meta(p.meta[head / p.hkv], p.budget, p.alpha);
+    const int n = seq_candidates(p, head / p.hkv);
     if (i0 >= n) return;
     const float *logits = p.logits + (size_t)head * p.alpha * p.cap_pad;
     const float *stat = p.row_stat + (size_t)head * p.alpha * 2;
@@ -317,12 +319,13 @@ __global__ void __launch_bounds__(kFused ? kSelThreadsFused : kSelThreadsSplit, 
         for (int j = tid; j < p.budget; j += kSelThreads) out[j] = -1;
         return;
     }
-    if (L <= p.budget) {      // Algorithm 1's guard (or an invalid length): nothing is compressed
+    const int budget_b = seq_budget(p, b);
+    if (L <= budget_b) {      // Algorithm 1's guard (or an invalid length): nothing is compressed
         for (int j = tid; j < p.budget; j += kSelThreads) out[j] = (j < L) ? j : -1;
         return;
     }
     const int n = L - p.alpha;
-    const int k = p.budget - p.alpha;
+    const int k = budget_b - p.alpha;
 
     const float *imp = p.imp + (size_t)head * p.cap_pad;
     if (kFused) {
@@ -426,7 +429,7 @@ __global__ void __launch_bounds__(kSelThreadsSplit, 4) select_mean_kernel(Params
     const int b = blockIdx.x, tid = threadIdx.x;
     const int L = p.meta[b];
     if (call_aborted(p)) return;    // select_kernel has written -1 everywhere
-    if (L <= p.budget) return;      // select_kernel has written the identity lists
+    if (L <= seq_budget(p, b)) return;      // select_kernel has written the identity lists
     const int n = L - p.alpha;
     uint32_t *keys = reinterpret_cast<uint32_t *>(row);
     const float *z = p.imp + (size_t)b * p.hkv * p.cap_pad;
@@ -436,7 +439,7 @@ __global__ void __launch_bounds__(kSelThreadsSplit, 4) select_mean_kernel(Params
         for (int h = 0; h < p.hkv; ++h) acc += z[(size_t)h * p.cap_pad + i];      // fixed head order
         keys[i] = order_key(acc / hkv);
     }
-    radix_select_emit<kSelThreads>(keys, n, p.budget - p.alpha, p.alpha, p.budget, p.out_idx + (size_t)b * p.hkv * p.budget, p.hkv);
+    radix_select_emit<kSelThreads>(keys, n, seq_budget(p, b) - p.alpha, p.alpha, p.budget, p.out_idx + (size_t)b * p.hkv * p.budget, p.hkv);
 }
 
 }  // namespace

@@ -71,7 +71,7 @@ def check_batch(k_in: torch.Tensor, v_in: torch.Tensor, q_in: torch.Tensor, seq_
                 gpu_idx: torch.Tensor, gpu_k: Optional[torch.Tensor] = None, gpu_v: Optional[torch.Tensor] = None,
                 gpu_seq: Optional[torch.Tensor] = None, gpu_scores: Optional[torch.Tensor] = None,
                 max_errors: int = 10, mean_then_pool: bool = False, head_mean: bool = False,
-                gqa_mean_pool: bool = False) -> ParityReport:
+                gqa_mean_pool: bool = False, budgets=None) -> ParityReport:
     """All tensors are for the same (sub)batch: k_in/v_in [B,H,cap,d] and q_in [B,Hq,alpha,d] BEFORE the call,
     gpu_* AFTER it.  gpu_scores is [4,B,H,cap] (I, Sbar, R, Z) or None."""
     rep = ParityReport()
@@ -79,32 +79,39 @@ def check_batch(k_in: torch.Tensor, v_in: torch.Tensor, q_in: torch.Tensor, seq_
     Q = to_numpy_f32(q_in)
     seq = seq_in.detach().cpu().numpy().astype(np.int32)
     B, H, cap, d = K.shape
+    nb_all = np.full(B, budget, np.int32) if budgets is None else np.asarray(budgets, dtype=np.int32)
     res = oracle.oracle_batch(K, Q, seq, budget=budget, alpha=alpha, lam=lam, W=W, beta=beta, T=T, eps=eps,
-                              mean_then_pool=mean_then_pool, head_mean=head_mean, gqa_mean_pool=gqa_mean_pool)
+                              mean_then_pool=mean_then_pool, head_mean=head_mean, gqa_mean_pool=gqa_mean_pool,
+                              budgets=None if budgets is None else nb_all)
     gidx = gpu_idx.detach().cpu().numpy()
     k_raw_in, v_raw_in = raw_rows(k_in), raw_rows(v_in)
     k_raw_out = raw_rows(gpu_k) if gpu_k is not None else None
     v_raw_out = raw_rows(gpu_v) if gpu_v is not None else None
     sc = gpu_scores.detach().cpu().numpy().astype(np.float64) if gpu_scores is not None else None
-    kk = budget - alpha
 
     def err(msg):
         if len(rep.errors) < max_errors:
             rep.errors.append(msg)
 
     if gpu_seq is not None:
-        want = np.where(seq > budget, budget, seq)
+        want = np.where(seq > nb_all, nb_all, seq)
         got = gpu_seq.detach().cpu().numpy()
         if not np.array_equal(got, want):
             err(f"seq_lens after the call: got {got[:8]}, want {want[:8]}")
 
     for b in range(B):
         L = int(seq[b])
+        nb = int(nb_all[b])            # this sequence's budget (Section 4.2's per-sequence budgets; else the call's)
+        kk = nb - alpha
         for h in range(H):
             rep.heads += 1
             tag = f"[b={b},h={h},L={L}]"
             gi = gidx[b, h]
-            if L <= budget:
+            if L > nb and not np.all(gi[nb:] == -1):
+                err(f"{tag} index entries beyond the sequence's budget {nb} are not -1")
+            if L > nb:
+                gi = gi[:nb]
+            if L <= nb:
                 if not np.array_equal(gi, res.idx[b, h]):
                     err(f"{tag} no-op index list differs")
                 if k_raw_out is not None and not (np.array_equal(k_raw_out[b, h], k_raw_in[b, h]) and
@@ -158,7 +165,7 @@ def check_batch(k_in: torch.Tensor, v_in: torch.Tensor, q_in: torch.Tensor, seq_
                 # Algorithm 1's aggregated selection: the kept set is judged on the head-averaged score, and every
                 # head of the sequence carries the same list
                 Zr = res.Z[b, :, :n].mean(axis=0)
-                if not np.array_equal(gi, gidx[b, 0]):
+                if not np.array_equal(gi, gidx[b, 0][:nb]):
                     err(f"{tag} index list differs from head 0's although one set per sequence was asked for")
             z_k = Zr[ref_set].min()
             tau = 1e-3 * abs(z_k)
@@ -179,8 +186,8 @@ def check_batch(k_in: torch.Tensor, v_in: torch.Tensor, q_in: torch.Tensor, seq_
                 rep.sets_identical += 1
             # ---- compacted rows: the oracle's gather on the positions the GPU kept
             if k_raw_out is not None:
-                if not np.array_equal(k_raw_out[b, h, :budget], oracle.oracle_gather(k_raw_in[b, h], gi)):
+                if not np.array_equal(k_raw_out[b, h, :nb], oracle.oracle_gather(k_raw_in[b, h], gi)):
                     err(f"{tag} compacted K rows differ from the gather of the kept positions")
-                if not np.array_equal(v_raw_out[b, h, :budget], oracle.oracle_gather(v_raw_in[b, h], gi)):
+                if not np.array_equal(v_raw_out[b, h, :nb], oracle.oracle_gather(v_raw_in[b, h], gi)):
                     err(f"{tag} compacted V rows differ from the gather of the kept positions")
     return rep

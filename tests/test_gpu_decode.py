@@ -131,3 +131,67 @@ def test_decode_segment_eager_and_as_one_cuda_graph(rkv):
     assert torch.equal(wl.k_cache[:, :, :nb].view(torch.int16), eager[1][:, :, :nb].view(torch.int16))
     assert torch.equal(wl.v_cache[:, :, :nb].view(torch.int16), eager[2][:, :, :nb].view(torch.int16))
     assert torch.equal(wl.q_window.view(torch.int16), eager[3].view(torch.int16))
+
+
+# ----------------------------------------------------------------------------- decode-step attention over the cache
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("hkv,hq", [(2, 2), (2, 8), (2, 10), (1, 7), (1, 8), (3, 9)])
+def test_decode_attention_matches_the_oracle(rkv, dtype, hkv, hq):
+    """Section 3.1's decode step, Eq. 1 with one query row: all group sizes the kernel serves, ragged lengths (a full
+    cache, a single token, an empty cache, a length that ends inside a tile), rows beyond the length filled with NaN
+    to prove they are never read.  Few head-problems: the rows of a head are cut into splits and merged."""
+    spec = ri.CacheSpec("att", 1, 5, hkv, hq, 128, 300, 84, 8, 0.1, dtype, 16, 0.3, 0.05, 4, 8.0)
+    lens = [spec.cap, 1, 0, 200, 129]
+    wl = ri.make_workload(spec, device="cuda", seed=301 + hq, seq_lens=torch.tensor(lens))
+    for b, L in enumerate(lens):
+        wl.k_cache[b, :, L:] = float("nan")
+        wl.v_cache[b, :, L:] = float("nan")
+    g = torch.Generator(device="cuda").manual_seed(5)
+    q_new = torch.randn(5, hq, 128, generator=g, device="cuda").to(spec.torch_dtype)
+    comp = rkv.Compressor(5, hkv, hq, spec.budget, spec.buffer, spec.alpha, 0.1, dtype=spec.torch_dtype)
+    assert rkv.rkv_decode_workspace_bytes(comp.desc, spec.budget, spec.buffer) <= comp.workspace.numel()
+    out = torch.full((5, hq, 128), 7.0, dtype=torch.float32, device="cuda")
+    rc = rkv.rkv_decode_attention(comp.desc, wl.k_cache, wl.v_cache, q_new, wl.seq_lens, out, spec.budget, spec.buffer)
+    assert rc == rkv.RKV_OK, rkv.rkv_status_string(rc)
+    torch.cuda.synchronize()
+    comp.check_status()
+    K, V = (torch.nan_to_num(t.float(), nan=0.0).cpu().numpy() for t in (wl.k_cache, wl.v_cache))
+    ref = oracle.oracle_decode_attention(K, V, q_new.float().cpu().numpy(), np.array(lens, dtype=np.int32))
+    got = out.cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all()
+    scale = np.maximum(np.abs(ref).max(axis=-1, keepdims=True), 1e-30)
+    assert (np.abs(got - ref) <= 1e-3 * scale + 1e-7).all(), float((np.abs(got - ref) / scale).max())
+    assert not got[2].any()                                   # empty cache: zero rows
+
+
+def test_decode_attention_large_batch_single_split(rkv):
+    """Enough head-problems for one block per head (no splits, no workspace): the Llama-8B group size at the cache
+    size of the first benchmark configuration, checked on sampled sequences."""
+    spec = ri.scaled(ri.SPECS["llama8b_b1"], layers=1, batch=80)
+    lens = torch.randint(1, spec.cap + 1, (80,), generator=torch.Generator().manual_seed(9))
+    lens[0], lens[1] = spec.cap, 1
+    wl = ri.make_workload(spec, device="cuda", seed=311, seq_lens=lens)
+    g = torch.Generator(device="cuda").manual_seed(6)
+    q_new = torch.randn(80, spec.n_q_heads, 128, generator=g, device="cuda").to(torch.bfloat16)
+    d = rkv.rkv_desc_default()
+    d.batch, d.n_kv_heads, d.n_q_heads = 80, spec.n_kv_heads, spec.n_q_heads
+    assert rkv.rkv_decode_workspace_bytes(d, spec.budget, spec.buffer) == 0
+    out = torch.empty(80, spec.n_q_heads, 128, dtype=torch.float32, device="cuda")
+    rc = rkv.rkv_decode_attention(d, wl.k_cache, wl.v_cache, q_new, wl.seq_lens, out, spec.budget, spec.buffer)
+    assert rc == rkv.RKV_OK, rkv.rkv_status_string(rc)
+    torch.cuda.synchronize()
+    rows = [0, 1, 17, 42, 79]
+    ref = oracle.oracle_decode_attention(wl.k_cache[rows].float().cpu().numpy(), wl.v_cache[rows].float().cpu().numpy(),
+                                         q_new[rows].float().cpu().numpy(), lens[rows].numpy().astype(np.int32))
+    got = out[rows].cpu().numpy().astype(np.float64)
+    scale = np.maximum(np.abs(ref).max(axis=-1, keepdims=True), 1e-30)
+    assert (np.abs(got - ref) <= 1e-3 * scale + 1e-7).all()
+
+
+def test_decode_attention_argument_checks(rkv):
+    d = rkv.rkv_desc_default()
+    d.batch, d.n_kv_heads, d.n_q_heads = 2, 1, 9           # G = 9: beyond what one block serves
+    assert rkv.rkv_decode_attention(d, 0x20000, 0x20000, 0x20000, 0x30000, 0x40000, 256, 64, 0) == 2
+    d.n_q_heads = 4
+    assert rkv.rkv_decode_attention(d, 0x20000, 0x20000, 0x20000, 0x30000, 0, 256, 64, 0) == 1       # null output
+    assert rkv.rkv_decode_attention(d, 0x20000, 0x20000, 0x20000, 0x30000, 0x40000, 256, 64, 0) == 3  # splits need a workspace

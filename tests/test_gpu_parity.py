@@ -21,7 +21,8 @@ def rkv():
     return r
 
 
-def run_and_check(rkv, wl, *, flags=0, W=4, beta=1, T=0.5, eps=1e-8, lam=None, check_rows=None, stages=None):
+def run_and_check(rkv, wl, *, flags=0, W=4, beta=1, T=0.5, eps=1e-8, lam=None, check_rows=None, stages=None,
+                  budgets=None):
     """Compress wl on the GPU through the C ABI and compare with the oracle.  check_rows: indices of the
     leading (folded batch) dimension to verify (default: all)."""
     spec = wl.spec
@@ -29,7 +30,7 @@ def run_and_check(rkv, wl, *, flags=0, W=4, beta=1, T=0.5, eps=1e-8, lam=None, c
     k0, v0, q0, s0 = wl.k_cache.clone(), wl.v_cache.clone(), wl.q_window.clone(), wl.seq_lens.clone()
     comp = rkv.Compressor(spec.folded_batch, spec.n_kv_heads, spec.n_q_heads, spec.budget, spec.buffer, spec.alpha,
                           lam, dtype=spec.torch_dtype, pool_w=W, beta=beta, sim_threshold=T, eps=eps, flags=flags,
-                          dump_scores=True)
+                          dump_scores=True, budgets=None if budgets is None else torch.tensor(budgets))
     if stages is None:
         idx = comp.compress(wl.k_cache, wl.v_cache, wl.q_window, wl.seq_lens)
     else:
@@ -41,7 +42,8 @@ def run_and_check(rkv, wl, *, flags=0, W=4, beta=1, T=0.5, eps=1e-8, lam=None, c
     rep = check_batch(k0[sel], v0[sel], q0[sel], s0[sel], budget=spec.budget, alpha=spec.alpha, lam=lam, W=W,
                       beta=beta, T=T, eps=eps, gpu_idx=idx[sel], gpu_k=wl.k_cache[sel], gpu_v=wl.v_cache[sel],
                       gpu_seq=wl.seq_lens[sel], gpu_scores=comp.scores[:, sel],
-                      mean_then_pool=bool(flags & 4), head_mean=bool(flags & 8), gqa_mean_pool=bool(flags & 16))
+                      mean_then_pool=bool(flags & 4), head_mean=bool(flags & 8), gqa_mean_pool=bool(flags & 16),
+                      budgets=None if budgets is None else [budgets[r] for r in rows])
     return rep, comp
 
 
@@ -328,6 +330,40 @@ def test_bounded_wait_runs_out_and_the_context_stays_usable(rkv):
     assert w[5] == 1                                        # the block reached its end
     assert rep.ok(), rep.errors
     comp.check_status()
+
+
+# ----------------------------------------------------------------------------- per-sequence budgets
+@pytest.mark.parametrize("flags", [pytest.param(1, id="simt"), pytest.param(0, id="sym"), pytest.param(2, id="rowblock"),
+                                   pytest.param(8, id="sym+head_mean")])
+@pytest.mark.parametrize("budget,buffer", [(256, 64), (1800, 128)])
+def test_per_sequence_budgets(rkv, flags, budget, buffer):
+    """A budget of its own for every sequence (Section 4.2's budget ratios): each sequence keeps exactly its own
+    budget, the rest of its index rows is -1, its new length is its budget; a sequence at or below its budget is left
+    alone; both forms of the select stage."""
+    spec = small_spec("pseq", batch=4, hkv=2, hq=8, budget=budget, buffer=buffer)
+    lens = [spec.cap, spec.cap - 7, budget // 2 + 40, budget // 2]
+    budgets = [budget, budget - 55, budget // 2, budget // 2 + 10]
+    wl = ri.make_workload(spec, device="cuda", seed=231, seq_lens=torch.tensor(lens))
+    rep, comp = run_and_check(rkv, wl, flags=flags, budgets=budgets)
+    print(rep.summary())
+    assert rep.ok(), rep.errors
+    assert rep.compressed_heads == 6
+    assert wl.seq_lens.tolist() == [budget, budget - 55, budget // 2, budget // 2]
+    comp.check_status()
+
+
+def test_per_sequence_budget_out_of_range_is_reported(rkv):
+    spec = small_spec("pseq_bad", batch=3)
+    wl = ri.make_workload(spec, device="cuda", seed=233)
+    k0 = wl.k_cache.clone()
+    comp = rkv.Compressor(3, 2, 8, spec.budget, spec.buffer, spec.alpha, 0.1,
+                          budgets=torch.tensor([spec.budget, spec.budget + 1, spec.alpha]))
+    idx = comp.compress(wl.k_cache, wl.v_cache, wl.q_window, wl.seq_lens)
+    torch.cuda.synchronize()
+    assert int(comp.status.item()) == 1
+    assert bool((idx[1:] == -1).all()) and bool((idx[0] >= 0).all())
+    assert torch.equal(k0[1:].view(torch.int16), wl.k_cache[1:].view(torch.int16))
+    assert wl.seq_lens.tolist() == [spec.budget, spec.cap, spec.cap]
 
 
 # ----------------------------------------------------------------------------- hard inputs at benchmark sizes
