@@ -480,6 +480,37 @@ def measure_cpu(wl, desc, args):
             "sample": f"first {seqs * spec.n_kv_heads} of {spec.head_problems} head-problems, {passes} passes, {dt:.1f} s"}
 
 
+def measure_attention(rkv, dev, wl, peaks, reps=5):
+    """rkv_decode_attention over the workload's full caches (every K and V row read once): ms and GB/s."""
+    spec = wl.spec
+    d = rkv.rkv_desc_default()
+    d.batch, d.n_kv_heads, d.n_q_heads = spec.folded_batch, spec.n_kv_heads, spec.n_q_heads
+    need = rkv.rkv_decode_workspace_bytes(d, spec.budget, spec.buffer)
+    ws = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
+    d.workspace, d.workspace_bytes = ws.data_ptr(), ws.numel()
+    gen = torch.Generator(device=dev).manual_seed(ri.BASE_SEED + 99)
+    q_new = torch.randn(spec.folded_batch, spec.n_q_heads, spec.head_dim, generator=gen, device=dev).to(spec.torch_dtype)
+    out = torch.empty(spec.folded_batch, spec.n_q_heads, spec.head_dim, dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream()
+    flush = torch.empty(256 * 2 ** 20, dtype=torch.uint8, device=dev)
+    ms = 0.0
+    for i in range(reps + 1):
+        flush.fill_(i & 255)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        rc = rkv.rkv_decode_attention(d, wl.k_cache, wl.v_cache, q_new, wl.seq_lens, out, spec.budget, spec.buffer, stream)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        if rc != rkv.RKV_OK:
+            return {"error": rkv.rkv_status_string(rc)}
+        if i > 0:
+            ms += e0.elapsed_time(e1) / reps
+    nbytes = 2 * wl.k_cache.numel() * wl.k_cache.element_size() + q_new.numel() * q_new.element_size() + out.numel() * 4
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    return {"ms": ms, "gbs": gbs, "frac_of_hbm_peak": gbs / peaks["hbm_gbs"], "bytes_per_launch": nbytes,
+            "what": "one decode step's attention of every sequence over its full cache (K and V read once)"}
+
+
 def side_config(rkv, rd, dev, wl, kw, K, W, mem_gb, peaks):
     """A configuration other than the headline one: ms per step, rates and the per-kernel table."""
     spec = wl.spec
@@ -548,6 +579,7 @@ def main():
     l2_note = timed.l2_note()
     timed.close()
 
+    attention = measure_attention(rkv, dev, wl, peaks)
     e2e = None
     if not args.no_e2e:
         e2e = measure_e2e(rkv, rd, dev, wl, kw, min(K, 2 if spec.head_problems > 4096 else 8), toks)
@@ -594,6 +626,7 @@ def main():
             "clocks": clocks,
             "peaks": {"hbm_gbs": peaks["hbm_gbs"], "bf16_tflops": peaks["bf16_tflops"], "source": peaks["source"]},
         }
+        line["decode_attention"] = attention
         if e2e is not None:
             line["e2e"] = e2e
         if cpu is not None:

@@ -9,8 +9,11 @@
 // (cp.async.bulk, three stages in flight, bounded waits), all G query heads of the group served from the same tile.
 //   scores   8 lanes per row, 16 dims each (two or four 16-byte shared-memory loads), the G partial dot products of a
 //            row folded over the 8 lanes by 3 shuffle steps; four rows per warp instruction
-//   softmax  online, per tile: block-wide tile maximum per query head, running maximum and sum, base-2 exponentials
+//   softmax  online and per WARP: each of the 8 compute warps keeps its own running maximum and sum over its 8 rows
+//            of every tile (base-2 exponentials), so the tile loop has no block-wide barrier; the warps' results are
+//            merged once, at the end
 //   values   lanes over d: a lane owns 4 dims of the output of every query head, a warp walks its 8 rows of the tile
+// A ninth warp is the producer of the bulk copies; stages are handed back through mbarriers.
 // With few head-problems the rows of a head are cut into splits (more blocks than SMs); a second small kernel merges
 // the splits' partial results.
 #include "rkv_sm100.cuh"
@@ -21,9 +24,9 @@ namespace {
 
 using namespace sm100;
 
-constexpr int kAttThreads = 256;
-constexpr int kAttWarps = kAttThreads / 32;
-constexpr int kAttRows = 64;            // rows per tile
+constexpr int kAttWarps = 7;             // compute warps
+constexpr int kAttThreads = (kAttWarps + 1) * 32;     // + the producer warp
+constexpr int kAttRows = 56;            // rows per tile: 8 per compute warp
 constexpr int kAttStages = 3;
 constexpr int kAttMaxG = 8;             // query heads per KV head served by one block
 
@@ -45,11 +48,13 @@ __global__ void __launch_bounds__(kAttThreads, (G <= 4 && sizeof(T) == 2) ? 2 : 
     constexpr int kPerVec = Elem<T>::kPerVec;               // elements per 16-byte vector
     constexpr int kVecPerRow = kHeadDim / kPerVec;          // 16 (bf16) or 32 (fp32)
     constexpr int kVecPerLane = kVecPerRow / 8;             // vectors of a row held by one of its 8 lanes
+    constexpr int GP = (G + 3) / 4 * 4;                     // query heads padded to whole float4s
+    constexpr int kRowsPerWarp = kAttRows / kAttWarps;      // 8
+    static_assert(kRowsPerWarp == 8, "a warp takes its rows four at a time, twice");
     extern __shared__ __align__(128) uint8_t att_smem[];    // kAttStages x (K tile, V tile), then the small arrays
-    float *sc = reinterpret_cast<float *>(att_smem + kAttStages * 2 * kTileBytesT);      // [G][kAttRows] scores, then weights
-    float *red = sc + G * kAttRows;                          // [kAttWarps][G] per-warp maxima / sums
-    float *stat = red + kAttWarps * G;                       // [G][3]: running maximum, running sum, rescale factor
-    unsigned long long *bars = reinterpret_cast<unsigned long long *>(stat + 3 * G + ((3 * G) & 1));
+    float *wts = reinterpret_cast<float *>(att_smem + kAttStages * 2 * kTileBytesT);     // [kAttWarps][kRowsPerWarp][GP] weights
+    float *wstat = wts + kAttWarps * kRowsPerWarp * GP;     // [kAttWarps][G][2] per-warp running maximum and sum
+    unsigned long long *bars = reinterpret_cast<unsigned long long *>(wstat + kAttWarps * G * 2);   // full[stages], empty[stages]
     __shared__ int abort_flag;
 
     const int head = blockIdx.x / p.splits, split = blockIdx.x % p.splits;
@@ -70,179 +75,203 @@ __global__ void __launch_bounds__(kAttThreads, (G <= 4 && sizeof(T) == 2) ? 2 : 
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
-        for (int s = 0; s < kAttStages; ++s) mbar_init(smem_u32(bars + s), 1);
+        for (int s = 0; s < kAttStages; ++s) {
+            mbar_init(smem_u32(bars + s), 1);                          // full: the producer's arrival + the copies' bytes
+            mbar_init(smem_u32(bars + kAttStages + s), kAttWarps);     // empty: every compute warp is done with the stage
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (threadIdx.x < G) {
-        stat[threadIdx.x * 3] = -INFINITY;
-        stat[threadIdx.x * 3 + 1] = 0.f;
-    }
     __syncthreads();
 
-    auto issue = [&](int t) {           // tile t of this block into stage t % kAttStages (one thread)
-        const int s = t % kAttStages;
-        const int row0 = (t_begin + t) * kAttRows;
-        const uint32_t bytes = (uint32_t)min(kAttRows, Lc - row0) * kRowBytes;
-        const uint32_t bar = smem_u32(bars + s);
-        mbar_expect_tx(bar, 2 * bytes);
-        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                     ::"r"(smem_u32(att_smem + (size_t)s * 2 * kTileBytesT)), "l"(K + (size_t)row0 * kHeadDim), "r"(bytes), "r"(bar)
-                     : "memory");
-        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                     ::"r"(smem_u32(att_smem + (size_t)s * 2 * kTileBytesT + kTileBytesT)), "l"(V + (size_t)row0 * kHeadDim), "r"(bytes),
-                       "r"(bar)
-                     : "memory");
-    };
-    if (threadIdx.x == 0)
-        for (int t = 0; t < min(n_tiles, kAttStages); ++t) issue(t);
+    float2 acc[G][2];                    // compute warps: lane owns dims 4 lane .. 4 lane + 3 of every head's output
+#pragma unroll
+    for (int g = 0; g < G; ++g) acc[g][0] = acc[g][1] = make_float2(0.f, 0.f);
 
-    // the group's queries, scaled by log2(e) / sqrt(d): lane j of a row's 8 lanes holds vectors j, j + 8, ...
-    const int sub = lane >> 3, j8 = lane & 7;
-    float qreg[G][kVecPerLane * kPerVec];
-    {
-        const float qscale = 1.4426950408889634f * rsqrtf((float)kHeadDim);
-        const T *Q = static_cast<const T *>(p.q_new) + ((size_t)b * p.hq + (size_t)h * G) * kHeadDim;
-#pragma unroll
-        for (int g = 0; g < G; ++g)
-#pragma unroll
-            for (int u = 0; u < kVecPerLane; ++u) {
-                const uint4 vec = *reinterpret_cast<const uint4 *>(Q + (size_t)g * kHeadDim + (j8 + 8 * u) * kPerVec);
-                Elem<T>::unpack(vec, &qreg[g][u * kPerVec]);
-#pragma unroll
-                for (int e = 0; e < kPerVec; ++e) qreg[g][u * kPerVec + e] *= qscale;
+    if (warp == kAttWarps) {
+        // ------------------------------------------------------------------ producer warp: the tiles of K and V
+        if (lane == 0) {
+            for (int t = 0; t < n_tiles; ++t) {
+                const int s = t % kAttStages;
+                if (!mbar_wait(smem_u32(bars + kAttStages + s), ((t / kAttStages) & 1) ^ 1, &abort_flag, sink)) break;
+                const int row0 = (t_begin + t) * kAttRows;
+                const uint32_t bytes = (uint32_t)min(kAttRows, Lc - row0) * kRowBytes;
+                const uint32_t bar = smem_u32(bars + s);
+                mbar_expect_tx(bar, 2 * bytes);
+                asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                             ::"r"(smem_u32(att_smem + (size_t)s * 2 * kTileBytesT)), "l"(K + (size_t)row0 * kHeadDim), "r"(bytes),
+                               "r"(bar)
+                             : "memory");
+                asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                             ::"r"(smem_u32(att_smem + (size_t)s * 2 * kTileBytesT + kTileBytesT)), "l"(V + (size_t)row0 * kHeadDim),
+                               "r"(bytes), "r"(bar)
+                             : "memory");
             }
-    }
-    float acc[G][4];                     // lane owns dims 4 lane .. 4 lane + 3 of every head's output (this warp's rows)
-#pragma unroll
-    for (int g = 0; g < G; ++g)
-#pragma unroll
-        for (int e = 0; e < 4; ++e) acc[g][e] = 0.f;
-
-    for (int t = 0; t < n_tiles; ++t) {
-        const int s = t % kAttStages;
-        const int row0 = (t_begin + t) * kAttRows;
-        const int rows_here = min(kAttRows, Lc - row0);
-        const bool landed = mbar_wait(smem_u32(bars + s), (t / kAttStages) & 1, &abort_flag, sink);
-        if (!__syncthreads_and(landed)) {            // the block leaves as a whole, or not at all
-            __nanosleep(200000);                     // error path only: let copies in flight land
-            return;
         }
-        const uint8_t *kt = att_smem + (size_t)s * 2 * kTileBytesT, *vt = kt + kTileBytesT;
-
-        // ---- scores of the tile: warp w takes rows 8 w .. 8 w + 7, four at a time
-        float wmax[G];
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------------ compute warps
+        // Every warp runs its own online softmax over its 8 rows of each tile (no block-wide barrier in the loop); the
+        // warps' results are merged once, at the end.
+        // The group's queries, scaled by log2(e) / sqrt(d): lane j of a row's 8 lanes holds vectors j, j + 8, ...
+        const int sub = lane >> 3, j8 = lane & 7;
+        float qreg[G][kVecPerLane * kPerVec];     // (used in pairs: packed fp32 multiply-adds, two per instruction)
+        {
+            const float qscale = 1.4426950408889634f * rsqrtf((float)kHeadDim);
+            const T *Q = static_cast<const T *>(p.q_new) + ((size_t)b * p.hq + (size_t)h * G) * kHeadDim;
 #pragma unroll
-        for (int g = 0; g < G; ++g) wmax[g] = -INFINITY;
-#pragma unroll
-        for (int it = 0; it < 2; ++it) {
-            const int r = warp * 8 + it * 4 + sub;
-            float dot[G];
-#pragma unroll
-            for (int g = 0; g < G; ++g) dot[g] = 0.f;
-            if (r < rows_here) {
+            for (int g = 0; g < G; ++g)
 #pragma unroll
                 for (int u = 0; u < kVecPerLane; ++u) {
-                    float kf[kPerVec];
-                    Elem<T>::unpack(*reinterpret_cast<const uint4 *>(kt + (size_t)r * kRowBytes + (j8 + 8 * u) * 16), kf);
+                    const uint4 vec = *reinterpret_cast<const uint4 *>(Q + (size_t)g * kHeadDim + (j8 + 8 * u) * kPerVec);
+                    Elem<T>::unpack(vec, &qreg[g][u * kPerVec]);
 #pragma unroll
-                    for (int g = 0; g < G; ++g)
+                    for (int e = 0; e < kPerVec; ++e) qreg[g][u * kPerVec + e] *= qscale;
+                }
+        }
+        float m_run[G], l_run[G];            // running maximum (base-2 domain) and sum of this warp, the same in every lane
 #pragma unroll
-                        for (int e = 0; e < kPerVec; ++e) dot[g] = fmaf(qreg[g][u * kPerVec + e], kf[e], dot[g]);
+        for (int g = 0; g < G; ++g) {
+            m_run[g] = -INFINITY;
+            l_run[g] = 0.f;
+        }
+        float *my_w = wts + warp * kRowsPerWarp * GP;
+        bool ok = true;
+
+        for (int t = 0; t < n_tiles && ok; ++t) {
+            const int s = t % kAttStages;
+            const int row0 = (t_begin + t) * kAttRows;
+            const int rows_here = min(kAttRows, Lc - row0);
+            ok = mbar_wait(smem_u32(bars + s), (t / kAttStages) & 1, &abort_flag, sink);
+            if (!ok) break;
+            const uint8_t *kt = att_smem + (size_t)s * 2 * kTileBytesT, *vt = kt + kTileBytesT;
+
+            // ---- scores of this warp's rows 8 w .. 8 w + 7, four at a time; every lane of a row's 8 ends up with them
+            float sv[2][G];
+#pragma unroll
+            for (int it = 0; it < 2; ++it) {
+                const int r = warp * kRowsPerWarp + it * 4 + sub;
+                float2 dot2[G];
+#pragma unroll
+                for (int g = 0; g < G; ++g) dot2[g] = make_float2(0.f, 0.f);
+                if (r < rows_here) {
+#pragma unroll
+                    for (int u = 0; u < kVecPerLane; ++u) {
+                        float kf[kPerVec];
+                        Elem<T>::unpack(*reinterpret_cast<const uint4 *>(kt + (size_t)r * kRowBytes + (j8 + 8 * u) * 16), kf);
+#pragma unroll
+                        for (int g = 0; g < G; ++g)
+#pragma unroll
+                            for (int e = 0; e < kPerVec; e += 2)
+                                dot2[g] = __ffma2_rn(make_float2(qreg[g][u * kPerVec + e], qreg[g][u * kPerVec + e + 1]),
+                                                     make_float2(kf[e], kf[e + 1]), dot2[g]);
+                    }
+                }
+#pragma unroll
+                for (int g = 0; g < G; ++g) {
+                    float dot = dot2[g].x + dot2[g].y;
+#pragma unroll
+                    for (int off = 4; off > 0; off >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, off);
+                    sv[it][g] = r < rows_here ? dot : -INFINITY;          // rows beyond the cached length take no part
                 }
             }
+            // ---- online softmax of the warp: new maximum over its 8 rows, rescale, the rows' weights
+            __syncwarp();                       // the previous tile's weights are no longer read
 #pragma unroll
             for (int g = 0; g < G; ++g) {
-#pragma unroll
-                for (int off = 4; off > 0; off >>= 1) dot[g] += __shfl_xor_sync(0xffffffffu, dot[g], off);
-                const float sv = r < rows_here ? dot[g] : -INFINITY;      // rows beyond the cached length take no part
-                if (j8 == 0) sc[g * kAttRows + r] = sv;
-                wmax[g] = fmaxf(wmax[g], sv);
+                float m = fmaxf(sv[0][g], sv[1][g]);
+                m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 8));
+                m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 16));
+                const float m_new = fmaxf(m_run[g], m);
+                // (a warp whose rows all lie beyond the length keeps m = -inf: nothing to rescale, weights 0)
+                const float a = m_new == -INFINITY ? 1.f : exp2f(m_run[g] - m_new);
+                const float w0 = m_new == -INFINITY ? 0.f : exp2f(sv[0][g] - m_new);
+                const float w1 = m_new == -INFINITY ? 0.f : exp2f(sv[1][g] - m_new);
+                float wsum = j8 == 0 ? w0 + w1 : 0.f;                    // one lane per row counts
+                wsum += __shfl_xor_sync(0xffffffffu, wsum, 8);
+                wsum += __shfl_xor_sync(0xffffffffu, wsum, 16);
+                l_run[g] = l_run[g] * a + wsum;
+                m_run[g] = m_new;
+                const float2 a2 = make_float2(a, a);
+                acc[g][0] = __fmul2_rn(acc[g][0], a2);
+                acc[g][1] = __fmul2_rn(acc[g][1], a2);
+                if (j8 == 0) {
+                    my_w[sub * GP + g] = w0;
+                    my_w[(4 + sub) * GP + g] = w1;
+                }
             }
-        }
+            __syncwarp();
+            // ---- values: this warp's rows, lanes over d
+            const int r_lo = warp * kRowsPerWarp, r_hi = min(r_lo + kRowsPerWarp, rows_here);
+            for (int r = r_lo; r < r_hi; ++r) {
+                float2 v01, v23;
+                if (sizeof(T) == 2) {
+                    const uint2 raw = *reinterpret_cast<const uint2 *>(vt + (size_t)r * kRowBytes + lane * 8);
+                    const __nv_bfloat162 *h2 = reinterpret_cast<const __nv_bfloat162 *>(&raw);
+                    v01 = __bfloat1622float2(h2[0]);
+                    v23 = __bfloat1622float2(h2[1]);
+                } else {
+                    const float4 raw = *reinterpret_cast<const float4 *>(vt + (size_t)r * kRowBytes + lane * 16);
+                    v01 = make_float2(raw.x, raw.y);
+                    v23 = make_float2(raw.z, raw.w);
+                }
+                float w[GP];                 // the row's weights of all query heads: one or two 16-byte broadcasts
 #pragma unroll
-        for (int g = 0; g < G; ++g) {
-            float m = wmax[g];
+                for (int g4 = 0; g4 < GP; g4 += 4) {
+                    const float4 w4 = *reinterpret_cast<const float4 *>(my_w + (r - r_lo) * GP + g4);
+                    w[g4] = w4.x, w[g4 + 1] = w4.y, w[g4 + 2] = w4.z, w[g4 + 3] = w4.w;
+                }
 #pragma unroll
-            for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
-            if (lane == 0) red[warp * G + g] = m;
-        }
-        __syncthreads();
-        // ---- online softmax: new running maximum, rescale factor, the tile's weights and their sum
-        if (threadIdx.x < G) {
-            const int g = threadIdx.x;
-            float m = stat[g * 3];
-#pragma unroll
-            for (int w = 0; w < kAttWarps; ++w) m = fmaxf(m, red[w * G + g]);
-            stat[g * 3 + 2] = exp2f(stat[g * 3] - m);          // 0 on the first tile (old maximum -inf)
-            stat[g * 3] = m;
-        }
-        __syncthreads();
-        for (int x = threadIdx.x; x < G * kAttRows; x += kAttThreads) {
-            const int g = x / kAttRows;
-            sc[x] = exp2f(sc[x] - stat[g * 3]);                 // -inf rows give 0
-        }
-        __syncthreads();
-        if (warp < G) {          // one warp per query head adds up the tile's weights, in a fixed order
-            const int g = warp;
-            float sum = sc[g * kAttRows + lane] + sc[g * kAttRows + 32 + lane];
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
-            if (lane == 0) stat[g * 3 + 1] = stat[g * 3 + 1] * stat[g * 3 + 2] + sum;
-        }
-        static_assert(G <= kAttWarps, "every query head of the group needs a warp of its own for the sum");
-
-        // ---- values: this warp's 8 rows, lanes over d
-#pragma unroll
-        for (int g = 0; g < G; ++g) {
-            const float a = stat[g * 3 + 2];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) acc[g][e] *= a;
-        }
-        const int r_lo = warp * 8, r_hi = min(r_lo + 8, rows_here);
-        for (int r = r_lo; r < r_hi; ++r) {
-            float vf[4];
-            if (sizeof(T) == 2) {
-                const uint2 raw = *reinterpret_cast<const uint2 *>(vt + (size_t)r * kRowBytes + lane * 8);
-                const __nv_bfloat162 *h2 = reinterpret_cast<const __nv_bfloat162 *>(&raw);
-                const float2 x0 = __bfloat1622float2(h2[0]), x1 = __bfloat1622float2(h2[1]);
-                vf[0] = x0.x, vf[1] = x0.y, vf[2] = x1.x, vf[3] = x1.y;
-            } else {
-                const float4 raw = *reinterpret_cast<const float4 *>(vt + (size_t)r * kRowBytes + lane * 16);
-                vf[0] = raw.x, vf[1] = raw.y, vf[2] = raw.z, vf[3] = raw.w;
+                for (int g = 0; g < G; ++g) {
+                    const float2 w2 = make_float2(w[g], w[g]);
+                    acc[g][0] = __ffma2_rn(w2, v01, acc[g][0]);
+                    acc[g][1] = __ffma2_rn(w2, v23, acc[g][1]);
+                }
             }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(bars + kAttStages + s));       // this warp is done with the stage
+        }
+        if (lane == 0) {
 #pragma unroll
             for (int g = 0; g < G; ++g) {
-                const float w = sc[g * kAttRows + r];
-#pragma unroll
-                for (int e = 0; e < 4; ++e) acc[g][e] = fmaf(w, vf[e], acc[g][e]);
+                wstat[(warp * G + g) * 2] = m_run[g];
+                wstat[(warp * G + g) * 2 + 1] = ok ? l_run[g] : 0.f;      // error path: zeros (the status word says why)
             }
         }
-        __syncthreads();                 // the stage and the score array are free again
-        if (threadIdx.x == 0 && t + kAttStages < n_tiles) issue(t + kAttStages);
     }
+    if (*reinterpret_cast<volatile int *>(&abort_flag)) __nanosleep(200000);   // error path only: let copies in flight land
+    __syncthreads();                     // every warp is through with the tile stages
+    if (warp < kAttWarps) {
+        float *fold_w = reinterpret_cast<float *>(att_smem);      // [kAttWarps][G][128], in the room of the stages
+#pragma unroll
+        for (int g = 0; g < G; ++g)
+            *reinterpret_cast<float4 *>(fold_w + ((size_t)warp * G + g) * kHeadDim + lane * 4) =
+                make_float4(acc[g][0].x, acc[g][0].y, acc[g][1].x, acc[g][1].y);
+    }
+    __syncthreads();
 
-    // ---- fold the warps' partial outputs (fixed order), then write the result of this block
-    float *fold = reinterpret_cast<float *>(att_smem);        // [kAttWarps][G][128], the tile stages are free now
-    __syncthreads();
-#pragma unroll
-    for (int g = 0; g < G; ++g)
-        *reinterpret_cast<float4 *>(fold + ((size_t)warp * G + g) * kHeadDim + lane * 4) =
-            make_float4(acc[g][0], acc[g][1], acc[g][2], acc[g][3]);
-    __syncthreads();
-    for (int x = threadIdx.x; x < G * kHeadDim; x += kAttThreads) {
+    // ---- merge the warps' results (fixed order): out = sum_w 2^(m_w - m) acc_w / sum_w 2^(m_w - m) l_w
+    const float *fold = reinterpret_cast<const float *>(att_smem);
+    for (int x = threadIdx.x; x < G * kHeadDim; x += blockDim.x) {
         const int g = x / kHeadDim, c = x % kHeadDim;
-        float sum = 0.f;
+        float m = -INFINITY;
 #pragma unroll
-        for (int w = 0; w < kAttWarps; ++w) sum += fold[((size_t)w * G + g) * kHeadDim + c];
+        for (int w = 0; w < kAttWarps; ++w) m = fmaxf(m, wstat[(w * G + g) * 2]);
+        float num = 0.f, den = 0.f;
+#pragma unroll
+        for (int w = 0; w < kAttWarps; ++w) {
+            const float mw = wstat[(w * G + g) * 2];
+            const float f = mw == -INFINITY ? 0.f : exp2f(mw - m);
+            num = fmaf(f, fold[((size_t)w * G + g) * kHeadDim + c], num);
+            den = fmaf(f, wstat[(w * G + g) * 2 + 1], den);
+        }
         if (p.splits == 1) {
-            const float l = stat[g * 3 + 1];
-            p.out[((size_t)b * p.hq + (size_t)h * G + g) * kHeadDim + c] = l > 0.f ? sum / l : 0.f;
+            p.out[((size_t)b * p.hq + (size_t)h * G + g) * kHeadDim + c] = den > 0.f ? num / den : 0.f;
         } else {
             float *part = p.partial + (((size_t)head * p.splits + split) * G + g) * (kHeadDim + 2);
-            part[c] = sum;
+            part[c] = num;
             if (c == 0) {
-                part[kHeadDim] = stat[g * 3];
-                part[kHeadDim + 1] = stat[g * 3 + 1];
+                part[kHeadDim] = m;
+                part[kHeadDim + 1] = den;
             }
         }
     }
@@ -272,7 +301,8 @@ template <typename T, int G>
 cudaError_t launch_one(const AttendParams &p, cudaStream_t s)
 {
     const int tile_bytes = kAttRows * kHeadDim * (int)sizeof(T);
-    const int smem = kAttStages * 2 * tile_bytes + (G * kAttRows + kAttWarps * G + 3 * G + 1) * 4 + kAttStages * 8 + 16;
+    const int smem = kAttStages * 2 * tile_bytes + (kAttWarps * (kAttRows / kAttWarps) * ((G + 3) / 4 * 4) + kAttWarps * G * 2) * 4 +
+                     2 * kAttStages * 8 + 16;
     cudaError_t e = cudaFuncSetAttribute(attend_kernel<T, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     attend_kernel<T, G><<<(unsigned)(p.batch * p.hkv * p.splits), kAttThreads, smem, s>>>(p);
