@@ -49,7 +49,7 @@ def parse_args():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=[c for c in ri.CONFIG_ORDER if c != "tiny"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=[c for c in ri.SPECS if c != "tiny"])
     ap.add_argument("--no-configs", action="store_true",
                     help="only the named workload, without the other configurations under `configs`")
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
@@ -560,7 +560,7 @@ def main():
 
     # ---- the headline workload: one pristine copy per rank, restored (or replicated) so that every step compresses
     # full caches
-    wl = ri.make_workload(spec, device=dev, seed=ri.BASE_SEED + 1000 * rank + ri.CONFIG_ORDER.index(args.workload))
+    wl = ri.make_workload(spec, device=dev, seed=ri.BASE_SEED + 1000 * rank + list(ri.SPECS).index(args.workload))
     timed = Timed(rkv, rd, dev, wl, args.mem_gb, K + W)
     comp = rkv.Compressor(spec.folded_batch, spec.n_kv_heads, spec.n_q_heads, spec.budget, spec.buffer, spec.alpha,
                           spec.lam, dtype=spec.torch_dtype, device=dev, **kw)
@@ -592,8 +592,8 @@ def main():
     # ---- the other configurations, and the settings that defeat the two-pass shortcut, in the same run
     configs = {}
     if not args.no_configs and args.workload == DEFAULT_WORKLOAD and args.batch is None and args.layers is None and not kw:
-        for name, k_side in (("llama8b_b1", 20), ("llama8b_b16", 5), ("qwen7b_b64", 5)):
-            swl = ri.make_workload(ri.SPECS[name], device=dev, seed=ri.BASE_SEED + 1000 * rank + ri.CONFIG_ORDER.index(name))
+        for name, k_side in (("llama8b_b1", 20), ("llama8b_b16", 5), ("qwen7b_b64", 5), ("mha7b_b8", 5)):
+            swl = ri.make_workload(ri.SPECS[name], device=dev, seed=ri.BASE_SEED + 1000 * rank + list(ri.SPECS).index(name))
             configs[name] = side_config(rkv, rd, dev, swl, {}, k_side, 3, args.mem_gb, peaks)
             if name == "llama8b_b16":
                 configs[name + " threshold=0.9"] = side_config(rkv, rd, dev, swl, {"sim_threshold": 0.9}, 3, 3, args.mem_gb, peaks)

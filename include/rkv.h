@@ -47,7 +47,7 @@ extern "C" {
 typedef enum {
     RKV_OK = 0,
     RKV_ERR_INVALID_ARG = 1, /* null / misaligned pointer, size out of range */
-    RKV_ERR_UNSUPPORTED = 2, /* head_dim != 128, unknown dtype, cap too large, device is not sm_100 */
+    RKV_ERR_UNSUPPORTED = 2, /* head_dim not 64 / 128 / 256, unknown dtype, cap or query group too large */
     RKV_ERR_WORKSPACE = 3,   /* workspace missing or too small */
     RKV_ERR_CUDA = 4,        /* a CUDA runtime / driver call failed */
     RKV_ERR_TIMEOUT = 5      /* device status only: a bounded wait inside a kernel ran out */
@@ -92,7 +92,8 @@ typedef struct rkv_desc {
     int32_t batch;       /* sequences; layers that fire together are folded into this dimension */
     int32_t n_kv_heads;  /* KV heads per sequence */
     int32_t n_q_heads;   /* query heads; G = n_q_heads / n_kv_heads must be integral (G = 1: Eq. 1) */
-    int32_t head_dim;    /* d; only 128 */
+    int32_t head_dim;    /* d: 64, 128 or 256.  The tensor-core scoring kernels serve bf16 caches with d = 128; other
+                            head dimensions are scored by the CUDA-core kernel (correct, but far slower) */
     int32_t dtype;       /* rkv_dtype_t of k_cache, v_cache and q_window */
     int32_t pool_w;      /* W of Eq. 4; 0 = no pooling.  Range [0, 64].  Default 4 (the paper prints no value) */
     int32_t beta;        /* beta of Section 3.3; 0 = rule off.  Default 1 (the paper prints no value) */
@@ -259,7 +260,7 @@ RKV_API int rkv_push_query(const rkv_desc_t *desc, void *q_window, const void *q
  *   seq_lens          [batch] int32 (device), read only; 0 gives a zero output row; a value outside
  *                     [0, budget + buffer] gives a zero row and RKV_ERR_INVALID_ARG in desc->device_status
  *   out               [batch][n_q_heads][head_dim] float32 (device, 16-byte aligned)
- * fp32 arithmetic throughout.  G = n_q_heads / n_kv_heads up to 8 (RKV_ERR_UNSUPPORTED beyond).  With few
+ * fp32 arithmetic throughout.  head_dim 128 and G = n_q_heads / n_kv_heads up to 8 (RKV_ERR_UNSUPPORTED otherwise).  With few
  * head-problems the rows of a head are cut into splits whose partial results go through desc->workspace:
  * rkv_decode_workspace_bytes() says how much that needs (0 for large batches; never more than a compression of the
  * same shape needs, so one workspace serves both).  Enqueues one or two kernels on `stream`; return codes as for

@@ -202,12 +202,13 @@ class Compressor:
                  lam: float = 0.1, dtype: torch.dtype = torch.bfloat16, pool_w: Optional[int] = None,
                  beta: Optional[int] = None, sim_threshold: Optional[float] = None, eps: Optional[float] = None,
                  flags: int = 0, device="cuda", dump_scores: bool = False, host_staging: bool = False,
-                 stage_events: bool = False, budgets: Optional[torch.Tensor] = None):
+                 stage_events: bool = False, budgets: Optional[torch.Tensor] = None, head_dim: int = 128):
         self.budget, self.buffer, self.alpha, self.lam = budget, buffer, alpha, lam
         self.cap = budget + buffer
         self.device = torch.device(device)
         d = rkv_desc_default()
         d.batch, d.n_kv_heads, d.n_q_heads = batch, n_kv_heads, n_q_heads
+        d.head_dim = head_dim
         d.dtype = RKV_BF16 if dtype == torch.bfloat16 else RKV_F32
         if dtype not in (torch.bfloat16, torch.float32):
             raise ValueError("dtype must be bfloat16 or float32")

@@ -25,7 +25,12 @@ struct Layout {
     int cap, cap_pad, tiles, tri;
 };
 
-bool use_simt(const rkv_desc_t *d) { return d->dtype == RKV_F32 || (d->flags & RKV_FLAG_SIMT_SCORES); }
+// The tensor-core scoring kernels serve bf16 caches with head dimension 128; everything else (fp32 caches, head
+// dimensions 64 and 256, or on request) is scored by the CUDA-core kernel.
+bool use_simt(const rkv_desc_t *d)
+{
+    return d->dtype == RKV_F32 || d->head_dim != kHeadDim || (d->flags & RKV_FLAG_SIMT_SCORES);
+}
 
 // 1 when the triangle tensor-core kernels score (bf16 caches, unless a cross-check kernel is asked for).
 int use_tri(const rkv_desc_t *d) { return !(use_simt(d) || (d->flags & RKV_FLAG_ROWBLOCK_SCORES)); }
@@ -39,7 +44,7 @@ int check_shapes(const rkv_desc_t *d, int budget, int buffer, int alpha, Layout 
     if (alpha < 1 || budget <= alpha || buffer < 1) return RKV_ERR_INVALID_ARG;
     if (d->pool_w < 0 || d->pool_w > 64 || d->beta < 0) return RKV_ERR_INVALID_ARG;
     if (!(d->sim_threshold >= 0.f && d->sim_threshold <= 1.f) || !(d->eps >= 0.f)) return RKV_ERR_INVALID_ARG;
-    if (d->head_dim != kHeadDim) return RKV_ERR_UNSUPPORTED;
+    if (d->head_dim != 64 && d->head_dim != 128 && d->head_dim != 256) return RKV_ERR_UNSUPPORTED;
     if (d->dtype != RKV_BF16 && d->dtype != RKV_F32) return RKV_ERR_UNSUPPORTED;
     const long long cap = (long long)budget + buffer;
     if (cap > RKV_MAX_CAP) return RKV_ERR_UNSUPPORTED;
@@ -53,8 +58,9 @@ int check_shapes(const rkv_desc_t *d, int budget, int buffer, int alpha, Layout 
         size_t off = 0;
         lay->inv_norm = off;  off = align_up(off + P * lay->cap_pad * sizeof(float), 256);
         lay->norm_split = off;  off = align_up(off + P * lay->cap_pad * 16 * sizeof(__nv_bfloat16), 256);
-        lay->tile_sum = off;  off = align_up(off + P * lay->tiles * kHeadDim * sizeof(float), 256);
-        lay->head_sum = off;  off = align_up(off + P * kHeadDim * sizeof(float), 256);
+        const size_t hd = (size_t)d->head_dim;
+        lay->tile_sum = off;  off = align_up(off + P * lay->tiles * hd * sizeof(float), 256);
+        lay->head_sum = off;  off = align_up(off + P * hd * sizeof(float), 256);
         lay->logits = off;    off = align_up(off + P * alpha * lay->cap_pad * sizeof(float), 256);
         lay->row_stat = off;  off = align_up(off + P * alpha * 2 * sizeof(float), 256);
         lay->imp = off;       off = align_up(off + P * lay->cap_pad * sizeof(float), 256);
@@ -66,7 +72,7 @@ int check_shapes(const rkv_desc_t *d, int budget, int buffer, int alpha, Layout 
         lay->strag_count = off; off = align_up(off + tri * P * sizeof(int32_t), 256);
         lay->strag_items = off; off = align_up(off + tri * P * (lay->cap_pad / 256 + 1) * sizeof(int4), 256);
         lay->self_dot = off;    off = align_up(off + P * lay->cap_pad * sizeof(float), 256);
-        lay->head_sum_bf16 = off; off = align_up(off + P * 16 * kHeadDim * sizeof(__nv_bfloat16), 256);
+        lay->head_sum_bf16 = off; off = align_up(off + P * 16 * hd * sizeof(__nv_bfloat16), 256);
         lay->meta = off;        off = align_up(off + 2 * (size_t)d->batch * sizeof(int32_t), 256);
         // the region the prep stage zeroes: counters and per-head tile tickets
         lay->counters = off;    off = align_up(off + 32 * sizeof(unsigned long long), 256);
@@ -107,6 +113,7 @@ int run(const rkv_desc_t *d, void *k_cache, void *v_cache, const void *q_window,
     p.hkv = d->n_kv_heads;
     p.hq = d->n_q_heads;
     p.group = d->n_q_heads / d->n_kv_heads;
+    p.d = d->head_dim;
     p.cap = lay.cap;
     p.cap_pad = lay.cap_pad;
     p.tiles = lay.tiles;
@@ -197,7 +204,7 @@ int host_layout(const rkv_desc_t *d, int budget, int buffer, int alpha, HostLayo
     if (rc != RKV_OK) return rc;
     const size_t esz = d->dtype == RKV_BF16 ? 2 : 4;
     const size_t P = (size_t)d->batch * d->n_kv_heads;
-    h->row_bytes = kHeadDim * esz;
+    h->row_bytes = (size_t)d->head_dim * esz;
     h->kv_bytes = P * lay.cap * h->row_bytes;
     h->q_bytes = (size_t)d->batch * d->n_q_heads * alpha * h->row_bytes;
     h->seq_bytes = (size_t)d->batch * sizeof(int32_t);
@@ -324,7 +331,7 @@ int rkv_append(const rkv_desc_t *d, void *k_cache, void *v_cache, const void *k_
     if (!k_cache || !v_cache || !k_new || !v_new || !seq_lens) return RKV_ERR_INVALID_ARG;
     if (!aligned16(k_cache) || !aligned16(v_cache) || !aligned16(k_new) || !aligned16(v_new)) return RKV_ERR_INVALID_ARG;
     if (reinterpret_cast<uintptr_t>(seq_lens) & 3u) return RKV_ERR_INVALID_ARG;
-    const int row_bytes = kHeadDim * (d->dtype == RKV_BF16 ? 2 : 4);
+    const int row_bytes = d->head_dim * (d->dtype == RKV_BF16 ? 2 : 4);
     const cudaError_t e = launch_append(k_cache, v_cache, k_new, v_new, seq_lens, d->batch, d->n_kv_heads, budget + buffer,
                                         row_bytes, d->device_status, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? RKV_OK : cuda_fail(e, "append launch");
@@ -336,7 +343,7 @@ int rkv_push_query(const rkv_desc_t *d, void *q_window, const void *q_new, int32
     int rc = check_shapes(d, alpha + 1, 1, alpha, nullptr);        // descriptor fields and alpha against the group limit
     if (rc != RKV_OK) return rc;
     if (!q_window || !q_new || !aligned16(q_window) || !aligned16(q_new)) return RKV_ERR_INVALID_ARG;
-    const int row_bytes = kHeadDim * (d->dtype == RKV_BF16 ? 2 : 4);
+    const int row_bytes = d->head_dim * (d->dtype == RKV_BF16 ? 2 : 4);
     const cudaError_t e = launch_push_query(q_window, q_new, d->batch, d->n_q_heads, alpha, slot, row_bytes,
                                             static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? RKV_OK : cuda_fail(e, "push_query launch");
@@ -347,7 +354,7 @@ static int attend_plan(const rkv_desc_t *d, int32_t budget, int32_t buffer, int 
     int rc = check_shapes(d, budget, buffer, 1, nullptr);
     if (rc != RKV_OK) return rc;
     const int G = d->n_q_heads / d->n_kv_heads;
-    if (G > attend_max_group()) return RKV_ERR_UNSUPPORTED;
+    if (G > attend_max_group() || d->head_dim != kHeadDim) return RKV_ERR_UNSUPPORTED;
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
         sms = 148;       // sizing only (no device here): the B200's count

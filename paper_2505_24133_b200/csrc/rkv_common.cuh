@@ -10,7 +10,7 @@
 
 namespace rkv {
 
-constexpr int kHeadDim = 128;   // d
+constexpr int kHeadDim = 128;   // d of the tensor-core kernels (other head dimensions go through the CUDA-core kernels)
 constexpr int kTile = 128;      // keys per tile (rows of one tensor-core operand tile)
 
 // meta[b] values
@@ -26,6 +26,7 @@ struct Params {
     int32_t *out_idx;
     // shapes
     int batch, hkv, hq, group;      // group = G
+    int d;                          // head dimension: 64, 128 or 256
     int cap, cap_pad, tiles;        // cap_pad = tiles * kTile
     int budget, buffer, alpha;
     int dtype;

@@ -76,15 +76,21 @@ cudaError_t launch_gather(const Params &p, cudaStream_t s)
     // (8 per SM): a second, partly filled wave would leave SMs idle for much of the kernel.
     const unsigned wave = 8u * (unsigned)sms;
     const int split = streams * 4u <= wave ? 4 : (streams * 2u <= wave ? 2 : (streams < wave ? 4 : 1));
-    if (p.dtype == RKV_BF16) {
-        if (split == 4) gather_kernel<16, 4><<<streams * 4u, kGatherThreads, 0, s>>>(p);
-        else if (split == 2) gather_kernel<16, 2><<<streams * 2u, kGatherThreads, 0, s>>>(p);
-        else gather_kernel<16, 1><<<streams, kGatherThreads, 0, s>>>(p);
-    } else {
-        if (split == 4) gather_kernel<32, 4><<<streams * 4u, kGatherThreads, 0, s>>>(p);
-        else if (split == 2) gather_kernel<32, 2><<<streams * 2u, kGatherThreads, 0, s>>>(p);
-        else gather_kernel<32, 1><<<streams, kGatherThreads, 0, s>>>(p);
+    const int vec_per_row = p.d * (p.dtype == RKV_BF16 ? 2 : 4) / 16;      // 16-byte vectors per row: 8 .. 64
+#define RKV_GATHER_CASE(V)                                                                      \
+    case V:                                                                                     \
+        if (split == 4) gather_kernel<V, 4><<<streams * 4u, kGatherThreads, 0, s>>>(p);         \
+        else if (split == 2) gather_kernel<V, 2><<<streams * 2u, kGatherThreads, 0, s>>>(p);    \
+        else gather_kernel<V, 1><<<streams, kGatherThreads, 0, s>>>(p);                         \
+        break;
+    switch (vec_per_row) {
+        RKV_GATHER_CASE(8)
+        RKV_GATHER_CASE(16)
+        RKV_GATHER_CASE(32)
+        RKV_GATHER_CASE(64)
+        default: return cudaErrorInvalidValue;
     }
+#undef RKV_GATHER_CASE
     return cudaGetLastError();
 }
 

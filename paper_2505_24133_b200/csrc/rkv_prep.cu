@@ -20,18 +20,18 @@ namespace {
 constexpr int kPrepThreads = 256;
 constexpr int kPrepWarps = kPrepThreads / 32;
 
-template <typename T>
-__global__ void __launch_bounds__(kPrepThreads, 5) prep_kernel(Params p)
+template <typename T, int D>
+__global__ void __launch_bounds__(kPrepThreads, D <= 128 ? 5 : 2) prep_kernel(Params p)
 {
     using namespace sm100;
     extern __shared__ __align__(128) uint8_t prep_smem[];       // the tile's candidate rows, then one mbarrier
-    constexpr int kTileBytesT = kTile * kHeadDim * (int)sizeof(T);
+    constexpr int kTileBytesT = kTile * D * (int)sizeof(T);
     __shared__ int abort_flag;
     const ErrSink sink = make_sink(p);
     constexpr int kPerVec = Elem<T>::kPerVec;            // elements per 16-byte vector
     constexpr int kVecPerLane = 2;                       // 16-byte vectors of a row held by one lane
-    constexpr int kLanesPerRow = kHeadDim / (kPerVec * kVecPerLane);     // 8 (bf16) or 16 (fp32)
-    constexpr int kVecPerRow = kHeadDim / kPerVec;
+    constexpr int kLanesPerRow = D / (kPerVec * kVecPerLane);     // 8 (bf16) or 16 (fp32)
+    constexpr int kVecPerRow = D / kPerVec;
     constexpr int kRowsPerPass = 32 / kLanesPerRow;      // rows a warp covers with one load
     constexpr int kRowsPerWarp = kTile / kPrepWarps;     // 16
     constexpr int kPasses = kRowsPerWarp / kRowsPerPass;
@@ -54,7 +54,7 @@ __global__ void __launch_bounds__(kPrepThreads, 5) prep_kernel(Params p)
     }
     const int n = candidates_from_meta(L, budget_b, p.alpha);
 
-    const T *K = static_cast<const T *>(p.k_cache) + (size_t)head * p.cap * kHeadDim;
+    const T *K = static_cast<const T *>(p.k_cache) + (size_t)head * p.cap * D;
     float *inv_norm = p.inv_norm + (size_t)head * p.cap_pad;
 
     const int sub = lane / kLanesPerRow;                 // which of the rows of this pass
@@ -70,10 +70,10 @@ __global__ void __launch_bounds__(kPrepThreads, 5) prep_kernel(Params p)
         mbar_init(bar, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         if (rows_here > 0) {
-            const uint32_t bytes = (uint32_t)rows_here * kHeadDim * (uint32_t)sizeof(T);
+            const uint32_t bytes = (uint32_t)rows_here * D * (uint32_t)sizeof(T);
             mbar_expect_tx(bar, bytes);
             asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                         ::"r"(smem_u32(prep_smem)), "l"(K + (size_t)tile * kTile * kHeadDim), "r"(bytes), "r"(bar)
+                         ::"r"(smem_u32(prep_smem)), "l"(K + (size_t)tile * kTile * D), "r"(bytes), "r"(bar)
                          : "memory");
         }
     }
@@ -133,7 +133,7 @@ __global__ void __launch_bounds__(kPrepThreads, 5) prep_kernel(Params p)
             acc2[e].y += __shfl_xor_sync(0xffffffffu, acc2[e].y, off);
         }
     }
-    __shared__ float part[kPrepWarps][kHeadDim];
+    __shared__ float part[kPrepWarps][D];
     if (sub == 0) {
 #pragma unroll
         for (int u = 0; u < kVecPerLane; ++u) {
@@ -146,11 +146,11 @@ __global__ void __launch_bounds__(kPrepThreads, 5) prep_kernel(Params p)
         }
     }
     __syncthreads();
-    if (threadIdx.x < kHeadDim) {
+    if (threadIdx.x < D) {
         float s = 0.f;
 #pragma unroll
         for (int w = 0; w < kPrepWarps; ++w) s += part[w][threadIdx.x];
-        p.tile_sum[((size_t)head * p.tiles + tile) * kHeadDim + threadIdx.x] = s;
+        p.tile_sum[((size_t)head * p.tiles + tile) * D + threadIdx.x] = s;
     }
 
     // The block that finishes a head's last tile adds the tile sums up, always in tile order, so the result does
@@ -162,45 +162,48 @@ __global__ void __launch_bounds__(kPrepThreads, 5) prep_kernel(Params p)
         last_block = (atomicAdd(&p.tile_done[head], 1u) == (unsigned)p.tiles - 1u);
     }
     __syncthreads();
-    if (last_block && threadIdx.x < kHeadDim) {
+    if (last_block && threadIdx.x < D) {
         __threadfence();
-        const float *ts = p.tile_sum + (size_t)head * p.tiles * kHeadDim + threadIdx.x;
+        const float *ts = p.tile_sum + (size_t)head * p.tiles * D + threadIdx.x;
         float s = 0.f;
-        for (int t = 0; t < p.tiles; ++t) s += __ldcg(ts + (size_t)t * kHeadDim);
-        p.head_sum[(size_t)head * kHeadDim + threadIdx.x] = s;
+        for (int t = 0; t < p.tiles; ++t) s += __ldcg(ts + (size_t)t * D);
+        p.head_sum[(size_t)head * D + threadIdx.x] = s;
         // the same vector as three bf16 rows whose sum is s to fp32 accuracy (rows 3..15 of the 16-row block are
         // zero): appended to the query rows, it lets the tensor cores form Kbar_i . s along with the logits
-        __nv_bfloat16 *hs = p.head_sum_bf16 + (size_t)head * 16 * kHeadDim + threadIdx.x;
+        __nv_bfloat16 *hs = p.head_sum_bf16 + (size_t)head * 16 * D + threadIdx.x;
         float rest = s;
 #pragma unroll
         for (int part_i = 0; part_i < 3; ++part_i) {
             const __nv_bfloat16 h16 = __float2bfloat16_rn(rest);
-            hs[part_i * kHeadDim] = h16;
+            hs[part_i * D] = h16;
             rest -= __bfloat162float(h16);
         }
-        for (int z = 3; z < 16; ++z) hs[z * kHeadDim] = __float2bfloat16_rn(0.f);
+        for (int z = 3; z < 16; ++z) hs[z * D] = __float2bfloat16_rn(0.f);
     }
 }
 
 }  // namespace
 
-cudaError_t launch_prep(const Params &p, cudaStream_t s)
+template <typename T, int D>
+static cudaError_t launch_prep_for(const Params &p, cudaStream_t s)
 {
     const unsigned grid = (unsigned)p.tiles * (unsigned)(p.batch * p.hkv);
-    cudaError_t e;
-    if (p.dtype == RKV_BF16) {
-        const int smem = kTile * kHeadDim * 2 + 16;
-        if ((e = cudaFuncSetAttribute(prep_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)) !=
-            cudaSuccess)
-            return e;
-        prep_kernel<__nv_bfloat16><<<grid, kPrepThreads, smem, s>>>(p);
-    } else {
-        const int smem = kTile * kHeadDim * 4 + 16;
-        if ((e = cudaFuncSetAttribute(prep_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)) != cudaSuccess)
-            return e;
-        prep_kernel<float><<<grid, kPrepThreads, smem, s>>>(p);
-    }
+    const int smem = kTile * D * (int)sizeof(T) + 16;
+    cudaError_t e = cudaFuncSetAttribute(prep_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    prep_kernel<T, D><<<grid, kPrepThreads, smem, s>>>(p);
     return cudaGetLastError();
+}
+
+cudaError_t launch_prep(const Params &p, cudaStream_t s)
+{
+    const bool bf16 = p.dtype == RKV_BF16;
+    switch (p.d) {
+        case 64: return bf16 ? launch_prep_for<__nv_bfloat16, 64>(p, s) : launch_prep_for<float, 64>(p, s);
+        case 128: return bf16 ? launch_prep_for<__nv_bfloat16, 128>(p, s) : launch_prep_for<float, 128>(p, s);
+        case 256: return bf16 ? launch_prep_for<__nv_bfloat16, 256>(p, s) : launch_prep_for<float, 256>(p, s);
+        default: return cudaErrorInvalidValue;
+    }
 }
 
 }  // namespace rkv

@@ -16,15 +16,17 @@ namespace rkv {
 namespace {
 
 constexpr int kSimtThreads = 128;
-constexpr int kPadRow = kHeadDim + 1;   // padded smem row: thread-per-row reads hit distinct banks
 
-template <typename T>
-__device__ void load_tile_rows(const T *src, int first_row, int valid_rows, float *dst /*[128][kPadRow]*/)
+// kRows rows of D elements into shared memory as fp32, rows padded to D + 1 floats (thread-per-row reads then hit
+// distinct banks); rows >= valid_rows are zero-filled.
+template <typename T, int D, int kRows>
+__device__ void load_tile_rows(const T *src, int first_row, int valid_rows, float *dst /*[kRows][D + 1]*/)
 {
-    // rows >= valid_rows are zero-filled
+    constexpr int kPadRow = D + 1;
+    constexpr int kHeadDim = D;
     constexpr int kPerVec = Elem<T>::kPerVec;
     constexpr int kVecPerRow = kHeadDim / kPerVec;
-    for (int v = threadIdx.x; v < kTile * kVecPerRow; v += kSimtThreads) {
+    for (int v = threadIdx.x; v < kRows * kVecPerRow; v += kSimtThreads) {
         const int r = v / kVecPerRow, c = (v % kVecPerRow) * kPerVec;
         float f[kPerVec];
         if (first_row + r < valid_rows) {
@@ -39,12 +41,17 @@ __device__ void load_tile_rows(const T *src, int first_row, int valid_rows, floa
     }
 }
 
-template <typename T>
+// D: head dimension (64, 128, 256).  The streamed keys come in sub-tiles of kRowsB rows (64 at D = 256, where two
+// whole tiles would not fit shared memory).
+template <typename T, int D>
 __global__ void __launch_bounds__(kSimtThreads) scores_simt_kernel(Params p)
 {
+    constexpr int kHeadDim = D;
+    constexpr int kPadRow = D + 1;
+    constexpr int kRowsB = D <= 128 ? kTile : kTile / 2;
     extern __shared__ float smem[];
     float *tileA = smem;                       // [128][kPadRow]
-    float *tileB = smem + kTile * kPadRow;     // [128][kPadRow]
+    float *tileB = smem + kTile * kPadRow;     // [kRowsB][kPadRow]
     __shared__ float rB[kTile];
 
     const int blocks_per_head = p.tiles + 1;
@@ -62,18 +69,18 @@ __global__ void __launch_bounds__(kSimtThreads) scores_simt_kernel(Params p)
         // ---------------- Eq. 5-6 + retention rule for rows [128 x, 128 x + 128)
         if (x >= n_tiles) return;
         const int i = x * kTile + t;
-        load_tile_rows<T>(K, x * kTile, n, tileA);
+        load_tile_rows<T, D, kTile>(K, x * kTile, n, tileA);
         const float ri = (i < n) ? inv_norm[i] : 0.f;
         float total = 0.f, removed = 0.f;
         int left = p.beta;
-        for (int jt = n_tiles - 1; jt >= 0; --jt) {          // descending j: "largest positions first"
+        for (int jt = (n_tiles * kTile) / kRowsB - 1; jt >= 0; --jt) {          // descending j: "largest positions first"
             __syncthreads();
-            load_tile_rows<T>(K, jt * kTile, n, tileB);
-            rB[t] = (jt * kTile + t < n) ? inv_norm[jt * kTile + t] : 0.f;
+            load_tile_rows<T, D, kRowsB>(K, jt * kRowsB, n, tileB);
+            if (t < kRowsB) rB[t] = (jt * kRowsB + t < n) ? inv_norm[jt * kRowsB + t] : 0.f;
             __syncthreads();
             if (i < n) {
-                for (int jj = kTile - 1; jj >= 0; --jj) {
-                    const int j = jt * kTile + jj;
+                for (int jj = kRowsB - 1; jj >= 0; --jj) {
+                    const int j = jt * kRowsB + jj;
                     if (j >= n || j == i) continue;           // zero diagonal (Eq. 5)
                     float dot = 0.f;
 #pragma unroll 16
@@ -92,15 +99,15 @@ __global__ void __launch_bounds__(kSimtThreads) scores_simt_kernel(Params p)
         // ---------------- Eq. 2-3: max over the group of scaled logits, per (query row, key)
         const int rows = p.group * p.alpha;
         const T *Q = static_cast<const T *>(p.q_window) + ((size_t)b * p.hq + (size_t)h * p.group) * p.alpha * kHeadDim;
-        load_tile_rows<T>(Q, 0, rows, tileA);                 // query rows g * alpha + j
+        load_tile_rows<T, D, kTile>(Q, 0, rows, tileA);       // query rows g * alpha + j
         const float scale = rsqrtf((float)kHeadDim);
         float *logits = p.logits + (size_t)head * p.alpha * p.cap_pad;
-        for (int jt = 0; jt < n_tiles; ++jt) {
+        for (int jt = 0; jt < (n_tiles * kTile) / kRowsB; ++jt) {
             __syncthreads();
-            load_tile_rows<T>(K, jt * kTile, n, tileB);
+            load_tile_rows<T, D, kRowsB>(K, jt * kRowsB, n, tileB);
             __syncthreads();
-            const int i = jt * kTile + t;
-            if (i < n) {
+            const int i = jt * kRowsB + t;
+            if (t < kRowsB && i < n) {
                 for (int j = 0; j < p.alpha; ++j) {
                     float best = -INFINITY, total = 0.f;
                     for (int g = 0; g < p.group; ++g) {
@@ -118,26 +125,28 @@ __global__ void __launch_bounds__(kSimtThreads) scores_simt_kernel(Params p)
     }
 }
 
-constexpr size_t kSimtSmem = 2ull * kTile * kPadRow * sizeof(float);
+template <typename T, int D>
+cudaError_t launch_simt_for(const Params &p, cudaStream_t s)
+{
+    const unsigned grid = (unsigned)(p.tiles + 1) * (unsigned)(p.batch * p.hkv);
+    const size_t smem = (size_t)(kTile + (D <= 128 ? kTile : kTile / 2)) * (D + 1) * sizeof(float);
+    cudaError_t e = cudaFuncSetAttribute(scores_simt_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    scores_simt_kernel<T, D><<<grid, kSimtThreads, smem, s>>>(p);
+    return cudaGetLastError();
+}
 
 }  // namespace
 
 cudaError_t launch_scores_simt(const Params &p, cudaStream_t s)
 {
-    const unsigned grid = (unsigned)(p.tiles + 1) * (unsigned)(p.batch * p.hkv);
-    cudaError_t e;
-    if (p.dtype == RKV_BF16) {
-        e = cudaFuncSetAttribute(scores_simt_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)kSimtSmem);
-        if (e != cudaSuccess) return e;
-        scores_simt_kernel<__nv_bfloat16><<<grid, kSimtThreads, kSimtSmem, s>>>(p);
-    } else {
-        e = cudaFuncSetAttribute(scores_simt_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)kSimtSmem);
-        if (e != cudaSuccess) return e;
-        scores_simt_kernel<float><<<grid, kSimtThreads, kSimtSmem, s>>>(p);
+    const bool bf16 = p.dtype == RKV_BF16;
+    switch (p.d) {
+        case 64: return bf16 ? launch_simt_for<__nv_bfloat16, 64>(p, s) : launch_simt_for<float, 64>(p, s);
+        case 128: return bf16 ? launch_simt_for<__nv_bfloat16, 128>(p, s) : launch_simt_for<float, 128>(p, s);
+        case 256: return bf16 ? launch_simt_for<__nv_bfloat16, 256>(p, s) : launch_simt_for<float, 256>(p, s);
+        default: return cudaErrorInvalidValue;
     }
-    return cudaGetLastError();
 }
 
 }  // namespace rkv

@@ -70,6 +70,9 @@ SPECS: Dict[str, CacheSpec] = {
     "qwen14b_b32": CacheSpec("qwen14b_b32", 48, 32, 8, 40, 128, 4096, 128, 8, 0.1, "bf16", 32, 0.30, 0.05, 4, 8.0),
 }
 CONFIG_ORDER = ["tiny", "llama8b_b1", "llama8b_b16", "qwen7b_b64", "qwen14b_b32"]
+# a multi-head-attention cache (G = 1, Eq. 1: every query head has its own KV head), shaped like a 7B model with 32
+# layers x 32 heads, batch 8, budget 2048: beside the five configurations above, which are all grouped-query
+SPECS["mha7b_b8"] = CacheSpec("mha7b_b8", 32, 8, 32, 32, 128, 2048, 128, 8, 0.1, "bf16", 32, 0.30, 0.05, 4, 8.0)
 
 
 def scaled(spec: CacheSpec, *, layers: Optional[int] = None, batch: Optional[int] = None,

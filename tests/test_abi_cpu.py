@@ -50,7 +50,9 @@ def test_workspace_size_rules(rkv):
     assert rkv.rkv_host_workspace_bytes(d, 1024, 128, 8) > a + 2 * 2 * 8 * 1152 * 256
     # invalid shapes give 0
     assert rkv.rkv_workspace_bytes(_desc(rkv, n_q_heads=30), 1024, 128, 8) == 0      # G not integral
-    assert rkv.rkv_workspace_bytes(_desc(rkv, head_dim=64), 1024, 128, 8) == 0
+    assert rkv.rkv_workspace_bytes(_desc(rkv, head_dim=96), 1024, 128, 8) == 0
+    assert 0 < rkv.rkv_workspace_bytes(_desc(rkv, head_dim=64), 1024, 128, 8) < \
+        rkv.rkv_workspace_bytes(_desc(rkv, head_dim=256), 1024, 128, 8)
     assert rkv.rkv_workspace_bytes(d, 8, 128, 8) == 0                                # budget <= alpha
     assert rkv.rkv_workspace_bytes(d, 8192, 128, 8) == 0                             # cap > RKV_MAX_CAP
     assert rkv.rkv_workspace_bytes(_desc(rkv, n_q_heads=8 * 17), 1024, 128, 8) == 0  # G * alpha = 136 > 112
@@ -86,7 +88,7 @@ def test_host_detectable_errors_return_before_any_launch(rkv, case, want):
     elif case == "group":
         d.n_q_heads = 30
     elif case == "head_dim":
-        d.head_dim = 256
+        d.head_dim = 96
     elif case == "dtype":
         d.dtype = 7
     elif case == "no_workspace":

@@ -30,7 +30,8 @@ def run_and_check(rkv, wl, *, flags=0, W=4, beta=1, T=0.5, eps=1e-8, lam=None, c
     k0, v0, q0, s0 = wl.k_cache.clone(), wl.v_cache.clone(), wl.q_window.clone(), wl.seq_lens.clone()
     comp = rkv.Compressor(spec.folded_batch, spec.n_kv_heads, spec.n_q_heads, spec.budget, spec.buffer, spec.alpha,
                           lam, dtype=spec.torch_dtype, pool_w=W, beta=beta, sim_threshold=T, eps=eps, flags=flags,
-                          dump_scores=True, budgets=None if budgets is None else torch.tensor(budgets))
+                          dump_scores=True, budgets=None if budgets is None else torch.tensor(budgets),
+                          head_dim=spec.head_dim)
     if stages is None:
         idx = comp.compress(wl.k_cache, wl.v_cache, wl.q_window, wl.seq_lens)
     else:
@@ -48,8 +49,8 @@ def run_and_check(rkv, wl, *, flags=0, W=4, beta=1, T=0.5, eps=1e-8, lam=None, c
 
 
 def small_spec(name, *, layers=1, batch=2, hkv=2, hq=8, budget=256, buffer=64, alpha=8, dtype="bf16", span=16,
-               copy_frac=0.3, sigma=0.05, lam=0.1):
-    return ri.CacheSpec(name, layers, batch, hkv, hq, 128, budget, buffer, alpha, lam, dtype, span, copy_frac, sigma,
+               copy_frac=0.3, sigma=0.05, lam=0.1, head_dim=128):
+    return ri.CacheSpec(name, layers, batch, hkv, hq, head_dim, budget, buffer, alpha, lam, dtype, span, copy_frac, sigma,
                         4, 8.0)
 
 
@@ -329,6 +330,26 @@ def test_bounded_wait_runs_out_and_the_context_stays_usable(rkv):
     assert w[4] == 1 and w[3] < 100 * limit                 # the second was called off long before two seconds
     assert w[5] == 1                                        # the block reached its end
     assert rep.ok(), rep.errors
+    comp.check_status()
+
+
+# ----------------------------------------------------------------------------- other head dimensions
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("head_dim", [64, 256])
+@pytest.mark.parametrize("hkv,hq,budget,buffer,lens", [(2, 8, 256, 64, [320, 300, 256]), (2, 2, 120, 17, [137, 129, 121]),
+                                                       (1, 5, 1800, 128, [1928, 1900, 1801])])
+def test_head_dimensions_64_and_256(rkv, dtype, head_dim, hkv, hq, budget, buffer, lens):
+    """Head dimensions other than 128 (every stage: prep, CUDA-core scoring, both forms of the select stage, in-place
+    compaction with 128- to 1024-byte rows), grouped and multi-head (G = 1, Eq. 1) queries, ragged lengths."""
+    spec = small_spec("hd", batch=3, hkv=hkv, hq=hq, budget=budget, buffer=buffer, dtype=dtype, head_dim=head_dim)
+    wl = ri.make_workload(spec, device="cuda", seed=241 + head_dim, seq_lens=torch.tensor(lens))
+    for b, L in enumerate(lens):
+        wl.k_cache[b, :, L:] = float("nan")
+        wl.v_cache[b, :, L:] = float("nan")
+    rep, comp = run_and_check(rkv, wl)
+    print(rep.summary())
+    assert rep.ok(), rep.errors
+    assert rep.compressed_heads == hkv * sum(L > budget for L in lens)
     comp.check_status()
 
 
