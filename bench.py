@@ -351,15 +351,17 @@ def kernel_table(rkv, timed: Timed, kw, KB, peaks):
     P = spec.head_problems
     T = (n + 127) // 128
     q_cols = -(-(spec.n_q_heads // spec.n_kv_heads) * spec.alpha // 16) * 16 + 16
-    tile_flops = 2.0 * 128 ** 3
+    # one tile product = 128 x 128 outputs over K = 128 + 16: the head dimension plus the one extra K = 16 step that
+    # folds the threshold test into the accumulator (both scoring passes issue it for every key tile)
+    tile_flops = 2.0 * 128 * 128 * (128 + 16)
     rule_on = comp_ev.desc.beta > 0 and comp_ev.desc.sim_threshold < 1.0
     pass1_tiles = P * T if rule_on else 0              # every row tile meets the last key tile once
     pass1_flops = pass1_tiles * tile_flops + P * T * 2.0 * 128 * q_cols * 128
     pass2_flops = max(tiles_executed - pass1_tiles, 0) * tile_flops
-    pass2_useful = pairs2 * 2.0 * 128 * 128            # listed tokens x keys of the streamed tiles x 2 d
+    pass2_useful = pairs2 * 2.0 * 128 * (128 + 16)     # listed tokens x keys of the streamed tiles x 2 (d + 16)
     # algorithmic work per launch: bytes a kernel has to move / flops it has to execute, nothing it merely could
     work = {
-        "prep": ("hbm", P * (n * row + spec.cap * 8)),                          # K once; r_i and Kbar_i.Kbar_i out
+        "prep": ("hbm", P * (n * row + spec.cap * (8 + 32))),                   # K once; r_i, Kbar_i.Kbar_i and the 32-byte slice out
         "scores_pass1": ("tensor", pass1_flops),
         "scores_list": ("hbm", P * n * 8),
         "scores_pass2": ("tensor", pass2_flops),
@@ -408,7 +410,7 @@ def rooflines(spec, kernels, scoring, peaks):
                     "unit": "TFLOP/s", "frac": k["frac_of_bf16_peak"],
                     "peak_source": f"{peaks['source']} burst cuBLAS bf16",
                     "traffic": traffic(nm), "flops_per_launch": k["flops_per_launch"],
-                    "counts": "128x128x128 tile products the kernel executed (counted by the kernel)",
+                    "counts": "128x128x(128+16) tile products the kernel executed (counted by the kernel) + its query products",
                     "full_matrix_equivalent_tflops": scoring["full_matrix_equivalent_tflops"],
                     "other_pass": {c: kernels[c]["frac_of_bf16_peak"] for c in cands if c != nm}}
     hbm = {}

@@ -20,7 +20,7 @@ int cuda_fail(cudaError_t e, const char *where)
 }
 
 struct Layout {
-    size_t inv_norm, norm_split, tile_sum, head_sum, logits, row_stat, imp, sbar, left, strag, strag_count, strag_items, self_dot, head_sum_bf16, meta, counters,
+    size_t inv_norm, norm_split, thr_split, tile_sum, head_sum, logits, row_stat, imp, sbar, left, strag, strag_count, strag_items, self_dot, head_sum_bf16, meta, counters,
         tile_done, zero_bytes, total;
     int cap, cap_pad, tiles, tri;
 };
@@ -58,6 +58,7 @@ int check_shapes(const rkv_desc_t *d, int budget, int buffer, int alpha, Layout 
         size_t off = 0;
         lay->inv_norm = off;  off = align_up(off + P * lay->cap_pad * sizeof(float), 256);
         lay->norm_split = off;  off = align_up(off + P * lay->cap_pad * 16 * sizeof(__nv_bfloat16), 256);
+        lay->thr_split = off;   off = align_up(off + P * kTile * 16 * sizeof(__nv_bfloat16), 256);
         const size_t hd = (size_t)d->head_dim;
         lay->tile_sum = off;  off = align_up(off + P * lay->tiles * hd * sizeof(float), 256);
         lay->head_sum = off;  off = align_up(off + P * hd * sizeof(float), 256);
@@ -132,6 +133,7 @@ int run(const rkv_desc_t *d, void *k_cache, void *v_cache, const void *q_window,
     char *ws = static_cast<char *>(d->workspace);
     p.inv_norm = reinterpret_cast<float *>(ws + lay.inv_norm);
     p.norm_split = reinterpret_cast<__nv_bfloat16 *>(ws + lay.norm_split);
+    p.thr_split = reinterpret_cast<__nv_bfloat16 *>(ws + lay.thr_split);
     p.tile_sum = reinterpret_cast<float *>(ws + lay.tile_sum);
     p.head_sum = reinterpret_cast<float *>(ws + lay.head_sum);
     p.logits = reinterpret_cast<float *>(ws + lay.logits);

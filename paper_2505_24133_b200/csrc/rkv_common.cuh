@@ -40,8 +40,11 @@ struct Params {
     // workspace carve-up
     float *inv_norm;     // [P][cap_pad]         r_i = 1 / (||k_i|| + eps); 0 for i >= n
     __nv_bfloat16 *norm_split;    // [P][cap_pad][16]  (n1, n2, n3, n1, n2, n1, 0 ...): 1 / r_i as three bf16 parts, laid
-                                  // out as the extra K = 16 slice the second scoring pass appends to a key row
-                                  // (written by the first pass for the candidates, i < n)
+                                  // out as the extra K = 16 slice the scoring passes append to a key row
+    __nv_bfloat16 *thr_split;     // [P][128][16]      (-t1, -t1, -t1, -t2, -t2, -t3, 0 ...): -T / r_j of the keys of the
+                                  // head's LAST key tile as three bf16 parts, the slice the first scoring pass appends
+                                  // to that tile's rows; the dot product of the two kinds of slice is -T / (r_i r_j)
+                                  // to fp32 accuracy.  Both are written by the prep stage (two-pass route only).
     float *tile_sum;     // [P][tiles][128]      sum over the tile's candidate rows of r_i * k_i
     float *head_sum;     // [P][128]             sum over all candidate rows of r_i * k_i (the tile sums added up)
     float *logits;       // [P][alpha][cap_pad]  Eq. 2-3: group-max of scaled logits

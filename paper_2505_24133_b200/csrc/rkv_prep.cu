@@ -91,7 +91,8 @@ __global__ void __launch_bounds__(kPrepThreads, D <= 128 ? 5 : 2) prep_kernel(Pa
 #pragma unroll
     for (int e = 0; e < kHeld / 2; ++e) acc2[e] = make_float2(0.f, 0.f);
 
-#pragma unroll 2
+    float r_keep[kPasses];               // r of this lane's row in every pass (for the slices written after the loop)
+#pragma unroll
     for (int q = 0; q < kPasses; ++q) {
         const int lr = warp * kRowsPerWarp + q * kRowsPerPass + sub;       // row within the tile
         const int row = tile * kTile + lr;
@@ -119,9 +120,50 @@ __global__ void __launch_bounds__(kPrepThreads, D <= 128 ? 5 : 2) prep_kernel(Pa
             inv_norm[row] = r;                       // row < cap_pad: the grid covers exactly cap_pad rows per head
             p.self_dot[(size_t)head * p.cap_pad + row] = (r * r) * sq;     // Kbar_i . Kbar_i
         }
+        r_keep[q] = r;
         const float2 r2 = make_float2(r, r);
 #pragma unroll
         for (int e = 0; e < kHeld / 2; ++e) acc2[e] = __ffma2_rn(r2, make_float2(f[2 * e], f[2 * e + 1]), acc2[e]);
+    }
+
+    if (p.tri) {
+        // The threshold test of Section 3.3, S[j][i] > T, as the sign of k_i . k_j - T / (r_i r_j): the tensor-core kernels
+        // append one K = 16 step to a tile product whose operands are these slices.  1 / r = ||k|| + eps in three bf16
+        // parts (their sum has fp32 accuracy) as (n1, n2, n3, n1, n2, n1, 0 ...) for a key row; its dot product with a
+        // row's (-t1, -t1, -t1, -t2, -t2, -t3, 0 ...), the parts of T / r, is -T / (r_i r_j) up to terms of size 2^-24.
+        // One lane per row of the warp's 16 rows: lane l takes row l, whose r sits with the first lane of its group.
+        float r_mine = 0.f;
+#pragma unroll
+        for (int q = 0; q < kPasses; ++q) {
+            const float v = __shfl_sync(0xffffffffu, r_keep[q], (lane % kRowsPerPass) * kLanesPerRow);
+            if (lane / kRowsPerPass == q) r_mine = v;
+        }
+        if (lane < kRowsPerWarp) {
+            const int lr = warp * kRowsPerWarp + lane, row = tile * kTile + lr;
+            float rest = r_mine > 0.f ? __fdiv_rn(1.0f, r_mine) : 0.f;
+            uint32_t part[3];
+#pragma unroll
+            for (int c = 0; c < 3; ++c) {
+                const __nv_bfloat16 h16 = __float2bfloat16_rn(rest);
+                part[c] = (uint32_t)__bfloat16_as_ushort(h16);
+                rest -= __bfloat162float(h16);
+            }
+            uint4 *dst = reinterpret_cast<uint4 *>(p.norm_split + ((size_t)head * p.cap_pad + row) * 16);
+            dst[0] = make_uint4(part[0] | (part[1] << 16), part[2] | (part[0] << 16), part[1] | (part[0] << 16), 0u);
+            dst[1] = make_uint4(0u, 0u, 0u, 0u);
+            if (tile == (n + kTile - 1) / kTile - 1) {       // the head's last key tile: the first pass's resident operand
+                rest = r_mine > 0.f ? -__fdiv_rn(p.sim_threshold, r_mine) : 0.f;
+#pragma unroll
+                for (int c = 0; c < 3; ++c) {
+                    const __nv_bfloat16 h16 = __float2bfloat16_rn(rest);
+                    part[c] = (uint32_t)__bfloat16_as_ushort(h16);
+                    rest -= __bfloat162float(h16);
+                }
+                uint4 *thr = reinterpret_cast<uint4 *>(p.thr_split + ((size_t)head * kTile + lr) * 16);
+                thr[0] = make_uint4(part[0] | (part[0] << 16), part[0] | (part[1] << 16), part[1] | (part[2] << 16), 0u);
+                thr[1] = make_uint4(0u, 0u, 0u, 0u);
+            }
+        }
     }
 
     // fold the row groups of a warp, then the warps, in a fixed order (deterministic sums)

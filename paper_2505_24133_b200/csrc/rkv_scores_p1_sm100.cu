@@ -35,6 +35,7 @@ using namespace sm100;
 constexpr int kThreadsP1 = 320;
 constexpr int kHalfBytes = kTile * 64 * 2;       // one TMA box: 128 rows x 64 bf16 (128-byte swizzled rows)
 constexpr int kTileBytes = 2 * kHalfBytes;       // 32 KB: a 128 x 128 bf16 operand tile
+constexpr int kSliceBytes = kTile * 32;          // the extra K = 16 slice of an operand: 128 rows x 32 bytes (32-byte swizzle)
 constexpr int kMaxStagesA = 6;
 constexpr uint32_t kTmemColsP1 = 512;            // 2 buffers x (128 key columns + up to 128 query columns)
 constexpr int kSmemLimit = 227 * 1024;
@@ -53,8 +54,11 @@ enum {
 struct SmemPlan {
     int stages;          // ring depth
     int q_bytes;         // bytes of the query block: (q_rows_pad + 16) rows x 256 B
-    int off_slot;        // 2 x B block: rows [0, 128) the last key tile, then the query block; as two 64-column halves
+    int off_aug;         // stages x slice of a streamed tile
+    int off_slot;        // 2 x [B block: rows [0, 128) the last key tile, then the query block; as two 64-column halves |
+                         //      slice of the last key tile]
     int slot_bytes;      // (128 + q_rows_pad + 16) rows x 256 B; a half is slot_bytes / 2
+    int slot_stride;     // slot_bytes + kSliceBytes
     int off_rj;          // 2 x 128 floats: r_j of the last key tile
     int off_bar, off_items, off_misc, total;
 };
@@ -64,11 +68,13 @@ __host__ __device__ inline SmemPlan make_plan(int q_rows_pad)
     SmemPlan pl;
     pl.q_bytes = (q_rows_pad + 16) * 256;
     pl.slot_bytes = kTileBytes + pl.q_bytes;
-    const int fixed = 2 * pl.slot_bytes + 2 * kTile * 4 + kNumBarsP1 * 8 + 2 * 16 + 16 + 1024;   // + alignment slack
-    int stages = (kSmemLimit - fixed) / kTileBytes;
+    pl.slot_stride = pl.slot_bytes + kSliceBytes;
+    const int fixed = 2 * pl.slot_stride + 2 * kTile * 4 + kNumBarsP1 * 8 + 2 * 16 + 16 + 1024;   // + alignment slack
+    int stages = (kSmemLimit - fixed) / (kTileBytes + kSliceBytes);
     pl.stages = stages > kMaxStagesA ? kMaxStagesA : stages;
-    pl.off_slot = pl.stages * kTileBytes;
-    pl.off_rj = pl.off_slot + 2 * pl.slot_bytes;
+    pl.off_aug = pl.stages * kTileBytes;
+    pl.off_slot = pl.off_aug + pl.stages * kSliceBytes;
+    pl.off_rj = pl.off_slot + 2 * pl.slot_stride;
     pl.off_bar = pl.off_rj + 2 * kTile * 4;
     pl.off_items = pl.off_bar + kNumBarsP1 * 8;
     pl.off_misc = pl.off_items + 2 * 16;
@@ -79,7 +85,8 @@ __host__ __device__ inline SmemPlan make_plan(int q_rows_pad)
 // Item descriptor (int4): {head, first row tile, one past the last row tile, n}.  x < 0: no more items.
 __global__ void __launch_bounds__(kThreadsP1, 1)
 scores_stream_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_q,
-                           const __grid_constant__ CUtensorMap map_hs, int splits, unsigned long long total_items,
+                           const __grid_constant__ CUtensorMap map_hs, const __grid_constant__ CUtensorMap map_ns,
+                           const __grid_constant__ CUtensorMap map_ts, int splits, unsigned long long total_items,
                            int q_rows_pad)
 {
     extern __shared__ uint8_t smem_raw[];
@@ -151,10 +158,10 @@ scores_stream_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, 
                 const uint32_t slot = k_item & 1;
                 if (!mbar_wait(bar(kBarSlotEmpty + slot), ((k_item >> 1) & 1) ^ 1, abort_flag, sink)) break;
                 items[slot] = make_int4(head, t0, t1, n);
-                const uint32_t slot_addr = sbase + pl.off_slot + slot * pl.slot_bytes;
+                const uint32_t slot_addr = sbase + pl.off_slot + slot * pl.slot_stride;
                 const uint32_t full = bar(kBarSlotFull + slot);
                 // the descriptor is published by this arrival; the barrier completes when the operands have landed too
-                mbar_expect_tx(full, (uint32_t)pl.q_bytes + (rule_on ? (uint32_t)(kTileBytes + kTile * 4) : 0u));
+                mbar_expect_tx(full, (uint32_t)pl.q_bytes + (rule_on ? (uint32_t)(kTileBytes + kSliceBytes + kTile * 4) : 0u));
                 {
                     const int b = head / p.hkv, h = head % p.hkv;
                     const int q_row = (b * p.hq + h * p.group) * p.alpha;
@@ -170,6 +177,8 @@ scores_stream_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, 
                     const int y = key_row_base + (n_tiles - 1) * kTile;
                     tma_load_2d(slot_addr, &map_k, 0, y, full);
                     tma_load_2d(slot_addr + (uint32_t)pl.slot_bytes / 2, &map_k, 64, y, full);
+                    // the tile's extra slice: -T / r_j of its keys in three bf16 parts
+                    tma_load_2d(slot_addr + (uint32_t)pl.slot_bytes, &map_ts, 0, head * kTile, full);
                     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                                  ::"r"(sbase + pl.off_rj + slot * kTile * 4),
                                    "l"(p.inv_norm + (size_t)head * p.cap_pad + (size_t)(n_tiles - 1) * kTile),
@@ -184,9 +193,12 @@ scores_stream_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, 
                     }
                     const uint32_t dst = sbase + s * kTileBytes;
                     const int y = key_row_base + t * kTile;
-                    mbar_expect_tx(bar(kBarAFull + s), kTileBytes);
+                    mbar_expect_tx(bar(kBarAFull + s), kTileBytes + (rule_on ? kSliceBytes : 0));
                     tma_load_2d(dst, &map_k, 0, y, bar(kBarAFull + s));
                     tma_load_2d(dst + kHalfBytes, &map_k, 64, y, bar(kBarAFull + s));
+                    if (rule_on)    // the tile's extra slice: 1 / r_i of its keys in three bf16 parts
+                        tma_load_2d(sbase + pl.off_aug + s * kSliceBytes, &map_ns, 0, head * p.cap_pad + t * kTile,
+                                    bar(kBarAFull + s));
                     ++acount;
                 }
                 ++k_item;
@@ -207,6 +219,7 @@ scores_stream_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, 
             // one product per streamed tile: N = the 128 keys of the last tile + the query block (the query block alone
             // while the retention rule is off)
             const uint32_t idesc_kq = instr_desc(kTile, kTile + q_rows_pad + 16), idesc_q = instr_desc(kTile, q_rows_pad + 16);
+            const uint32_t idesc_k = instr_desc(kTile, kTile);
             uint32_t k_item = 0, acount = 0;
             bool ok = true;
             while (ok) {
@@ -214,7 +227,7 @@ scores_stream_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, 
                 if (!mbar_wait(bar(kBarSlotFull + slot), (k_item >> 1) & 1, abort_flag, sink)) break;
                 const int4 d = items[slot];
                 if (d.x < 0) break;
-                const uint32_t b_block = sbase + pl.off_slot + slot * pl.slot_bytes, b_half = (uint32_t)pl.slot_bytes / 2;
+                const uint32_t b_block = sbase + pl.off_slot + slot * pl.slot_stride, b_half = (uint32_t)pl.slot_bytes / 2;
                 for (int t = d.y; t < d.z; ++t) {
                     const uint32_t s = acount % (uint32_t)stages;
                     if (!mbar_wait(bar(kBarAFull + s), (acount / (uint32_t)stages) & 1, abort_flag, sink)) {
@@ -231,6 +244,8 @@ scores_stream_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, 
                     const uint32_t d_tmem = tmem_base + a * 256;
                     if (rule_on) {
                         umma_tile_k128_halves(d_tmem, tile, kHalfBytes, b_block, b_half, idesc_kq);
+                        // ... - T / (r_i r_j) onto the key columns: the accumulator's sign is the threshold test
+                        umma_k16_sw32(d_tmem, sbase + pl.off_aug + s * kSliceBytes, b_block + (uint32_t)pl.slot_bytes, idesc_k);
                         ++tiles_done;
                     } else {
                         umma_tile_k128_halves(d_tmem + 128, tile, kHalfBytes, b_block + kTile * 128, b_half, idesc_q);
@@ -354,73 +369,101 @@ scores_stream_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, 
                 // sum_j S[j][i] before the retention rule: Kbar_i . s - Kbar_i . Kbar_i
                 const float total = ri * ((__uint_as_float(sp[0]) + __uint_as_float(sp[1])) + __uint_as_float(sp[2])) - self;
 
-                // ---- the last key tile, last position first; its r_j lie in shared memory
-                float removed = 0.f;
+                // ---- the last key tile, last position first.  The accumulator holds h = k_i . k_j - T / (r_i r_j):
+                // S[j][i] > T exactly when h > 0, so the screening is a sign test with nothing to load per column; a
+                // partner's value is S = T + h r_i r_j, with the r_j of the tile in shared memory.
+                float removed = 0.f;             // sum of h r_j over the partners found
+                int nhit = 0;
                 int left = row_ok ? p.beta : 0;
                 if (rule_on) {
-                    const float thr = (row_ok && ri > 0.f) ? __fdiv_rn(p.sim_threshold, ri) : kInf;   // g r_j vs T / r_i
-                    float thr_row = left > 0 ? thr : kInf;
-                    if (__any_sync(0xffffffffu, thr_row < kInf)) {
-                        // 32-column chunks, last first; kept rolled: the roles share the instruction cache
-#pragma unroll 1
-                        for (int ch = 3; ch >= 0; --ch) {
-                            if (ch < 3 && !__any_sync(0xffffffffu, thr_row < kInf)) break;   // every token of the warp is served
-                            uint32_t g[32];
-                            tmem_ld32(lane_base + ch * 32, g);
-                            float v[32];
-                            uint32_t hits = 0u;
-                            float4 R[8];
+                    bool want = left > 0;
+                    const int valid = n - jbase;                  // columns [0, valid) of the tile are candidates
+                    const float *rj = reinterpret_cast<const float *>(rj4);
+                    // 32-column chunks, last first.  The TMEM load of the next chunk is issued before the current one is
+                    // looked at, so its latency passes under the work (two register sets, used alternately).
+                    auto chunk = [&](const uint32_t (&g)[32], int ch) {
+                        const int nv = valid - ch * 32;
+                        uint32_t colmask = nv >= 32 ? 0xffffffffu : (nv <= 0 ? 0u : ((1u << nv) - 1u));
+                        const unsigned own = (unsigned)(i - (jbase + ch * 32));           // zero diagonal (Eq. 5)
+                        if (own < 32u) colmask &= ~(1u << own);
+                        // bit c of `neg` = sign bit of entry c: one funnel shift per entry, four independent chains
+                        uint32_t n0 = 0u, n1 = 0u, n2 = 0u, n3 = 0u;
 #pragma unroll
-                            for (int q = 0; q < 8; ++q) R[q] = rj4[ch * 8 + q];
-                            tmem_wait32(g);
+                        for (int c = 7; c >= 0; --c) {
+                            n0 = __funnelshift_l(g[c], n0, 1);
+                            n1 = __funnelshift_l(g[8 + c], n1, 1);
+                            n2 = __funnelshift_l(g[16 + c], n2, 1);
+                            n3 = __funnelshift_l(g[24 + c], n3, 1);
+                        }
+                        const uint32_t neg = (n0 | (n1 << 8)) | ((n2 << 16) | (n3 << 24));
+                        // entries with a clear sign bit (h > 0, but also +0 and some NaN patterns of rows that are not
+                        // candidates: confirmed one by one below)
+                        uint32_t pos = want ? (~neg & colmask) : 0u;
+                        if (p.beta == 1) {
+                            // one partner at most: the candidate at the highest set bit, its value picked by a select
+                            // tree (nearly always a single turn)
+                            while (pos != 0u) {
+                                const int top = 31 - __clz(pos);
+                                uint32_t t16[16], t8[8], t4[4];
 #pragma unroll
-                            for (int q = 0; q < 8; ++q) {        // packed multiplies: two products per instruction
-                                const float2 p0 = __fmul2_rn(make_float2(__uint_as_float(g[4 * q]), __uint_as_float(g[4 * q + 1])),
-                                                             make_float2(R[q].x, R[q].y));
-                                const float2 p1 = __fmul2_rn(make_float2(__uint_as_float(g[4 * q + 2]), __uint_as_float(g[4 * q + 3])),
-                                                             make_float2(R[q].z, R[q].w));
-                                v[4 * q] = p0.x;
-                                v[4 * q + 1] = p0.y;
-                                v[4 * q + 2] = p1.x;
-                                v[4 * q + 3] = p1.y;
-                            }
-                            // a bit mask of the entries above the threshold (no entry depends on another), cut down to
-                            // the highest positions if they are more than the token still lacks, then their sum
+                                for (int c = 0; c < 16; ++c) t16[c] = (top & 16) ? g[16 + c] : g[c];
 #pragma unroll
-                            for (int c = 0; c < 32; ++c) hits |= (v[c] > thr_row) ? (1u << c) : 0u;
-                            const unsigned own = (unsigned)(i - (jbase + ch * 32));           // zero diagonal (Eq. 5)
-                            if (own < 32u) hits &= ~(1u << own);
-                            if (p.beta == 1) {
-                                // one partner at most: the entry at the highest set bit, picked by a select tree
-                                if (left > 0 && hits != 0u) {
-                                    const int top = 31 - __clz(hits);
-                                    float t16[16], t8[8], t4[4];
+                                for (int c = 0; c < 8; ++c) t8[c] = (top & 8) ? t16[8 + c] : t16[c];
 #pragma unroll
-                                    for (int c = 0; c < 16; ++c) t16[c] = (top & 16) ? v[16 + c] : v[c];
-#pragma unroll
-                                    for (int c = 0; c < 8; ++c) t8[c] = (top & 8) ? t16[8 + c] : t16[c];
-#pragma unroll
-                                    for (int c = 0; c < 4; ++c) t4[c] = (top & 4) ? t8[4 + c] : t8[c];
-                                    const float u0 = (top & 2) ? t4[2] : t4[0], u1 = (top & 2) ? t4[3] : t4[1];
-                                    removed += (top & 1) ? u1 : u0;
+                                for (int c = 0; c < 4; ++c) t4[c] = (top & 4) ? t8[4 + c] : t8[c];
+                                const uint32_t u0 = (top & 2) ? t4[2] : t4[0], u1 = (top & 2) ? t4[3] : t4[1];
+                                const float hv = __uint_as_float((top & 1) ? u1 : u0);
+                                if (hv > 0.f) {
+                                    removed = hv * rj[ch * 32 + top];
+                                    nhit = 1;
                                     left = 0;
-                                    thr_row = kInf;
+                                    want = false;
+                                    break;
                                 }
-                                continue;
+                                pos &= ~(1u << top);
                             }
-                            int taken = __popc(hits);
-                            for (; taken > left; --taken) hits &= hits - 1u;                   // drop the lowest positions
-                            float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+                            return;
+                        }
+                        // several partners per token: the exact mask, cut down to the highest positions if they are more
+                        // than the token still lacks, then the sum of their h r_j
+                        if (!__any_sync(0xffffffffu, pos != 0u)) return;
+                        uint32_t hits = 0u;
 #pragma unroll
-                            for (int c = 0; c < 32; c += 4) {
-                                s0 += (hits >> c & 1u) ? v[c] : 0.f;
-                                s1 += (hits >> (c + 1) & 1u) ? v[c + 1] : 0.f;
-                                s2 += (hits >> (c + 2) & 1u) ? v[c + 2] : 0.f;
-                                s3 += (hits >> (c + 3) & 1u) ? v[c + 3] : 0.f;
+                        for (int c = 0; c < 32; ++c) hits |= (__uint_as_float(g[c]) > 0.f) ? (1u << c) : 0u;
+                        hits &= pos;
+                        int taken = __popc(hits);
+                        for (; taken > left; --taken) hits &= hits - 1u;                   // drop the lowest positions
+                        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) {
+                            const float4 R = rj4[ch * 8 + q];
+                            s0 += (hits >> (4 * q) & 1u) ? __uint_as_float(g[4 * q]) * R.x : 0.f;
+                            s1 += (hits >> (4 * q + 1) & 1u) ? __uint_as_float(g[4 * q + 1]) * R.y : 0.f;
+                            s2 += (hits >> (4 * q + 2) & 1u) ? __uint_as_float(g[4 * q + 2]) * R.z : 0.f;
+                            s3 += (hits >> (4 * q + 3) & 1u) ? __uint_as_float(g[4 * q + 3]) * R.w : 0.f;
+                        }
+                        removed += (s0 + s1) + (s2 + s3);
+                        nhit += taken;
+                        left -= taken;
+                        if (left == 0) want = false;
+                    };
+                    if (__any_sync(0xffffffffu, want)) {
+                        uint32_t ga[32], gb[32];
+                        tmem_ld32(lane_base + 3 * 32, ga);
+                        tmem_wait32(ga);
+                        tmem_ld32(lane_base + 2 * 32, gb);
+                        chunk(ga, 3);
+                        tmem_wait32(gb);
+                        if (__any_sync(0xffffffffu, want)) {                              // else every token of the warp is served
+                            tmem_ld32(lane_base + 1 * 32, ga);
+                            chunk(gb, 2);
+                            tmem_wait32(ga);
+                            if (__any_sync(0xffffffffu, want)) {
+                                tmem_ld32(lane_base, gb);
+                                chunk(ga, 1);
+                                tmem_wait32(gb);
+                                if (__any_sync(0xffffffffu, want)) chunk(gb, 0);
                             }
-                            removed += (s0 + s1) + (s2 + s3);
-                            left -= taken;
-                            if (left == 0) thr_row = kInf;
                         }
                     }
                 }
@@ -434,24 +477,8 @@ scores_stream_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, 
 #pragma unroll
                         for (int j = 0; j < 8; ++j) logits[(size_t)j * p.cap_pad + i] = pooled[j];
                     }
-                    p.sbar[(size_t)head * p.cap_pad + i] = total - removed * ri;
+                    p.sbar[(size_t)head * p.cap_pad + i] = total - ((float)nhit * p.sim_threshold + removed * ri);
                     p.left[(size_t)head * p.cap_pad + i] = rule_on ? left : 0;
-                    if (rule_on) {
-                        // for pass 2: 1 / r_i = ||k_i|| + eps as three bf16 parts (their sum has fp32 accuracy), laid
-                        // out as the extra K = 16 slice of a key row, (n1, n2, n3, n1, n2, n1, 0 ...): its dot product
-                        // with a token's (-t1, -t1, -t1, -t2, -t2, -t3, 0 ...) is -t / r_i up to terms of size 2^-24
-                        float rest = ri > 0.f ? __fdiv_rn(1.0f, ri) : 0.f;
-                        uint32_t part[3];
-#pragma unroll
-                        for (int c = 0; c < 3; ++c) {
-                            const __nv_bfloat16 h16 = __float2bfloat16_rn(rest);
-                            part[c] = (uint32_t)__bfloat16_as_ushort(h16);
-                            rest -= __bfloat162float(h16);
-                        }
-                        uint4 *dst = reinterpret_cast<uint4 *>(p.norm_split + ((size_t)head * p.cap_pad + i) * 16);
-                        dst[0] = make_uint4(part[0] | (part[1] << 16), part[2] | (part[0] << 16), part[1] | (part[0] << 16), 0u);
-                        dst[1] = make_uint4(0u, 0u, 0u, 0u);
-                    }
                 }
             }
             if (!ok) break;
@@ -476,7 +503,8 @@ scores_stream_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, 
 }  // namespace
 
 cudaError_t launch_scores_pass1_sm100(const Params &p, cudaStream_t s, const CUtensorMap &map_k, const CUtensorMap &map_q,
-                                      const CUtensorMap &map_hs, int q_rows_pad, int sms)
+                                      const CUtensorMap &map_hs, const CUtensorMap &map_ns, const CUtensorMap &map_ts,
+                                      int q_rows_pad, int sms)
 {
     const SmemPlan pl = make_plan(q_rows_pad);
     if (pl.stages < 2) return cudaErrorInvalidConfiguration;
@@ -490,7 +518,8 @@ cudaError_t launch_scores_pass1_sm100(const Params &p, cudaStream_t s, const CUt
     splits = splits < 1 ? 1 : (splits > p.tiles ? p.tiles : splits);
     const unsigned long long total_items = (unsigned long long)splits * (unsigned long long)heads;
     const unsigned grid = (unsigned)(total_items < (unsigned long long)sms ? total_items : (unsigned long long)sms);
-    scores_stream_sm100_kernel<<<grid, kThreadsP1, pl.total, s>>>(p, map_k, map_q, map_hs, splits, total_items, q_rows_pad);
+    scores_stream_sm100_kernel<<<grid, kThreadsP1, pl.total, s>>>(p, map_k, map_q, map_hs, map_ns, map_ts, splits, total_items,
+                                                                  q_rows_pad);
     return cudaGetLastError();
 }
 

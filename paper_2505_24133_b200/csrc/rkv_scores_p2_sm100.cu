@@ -577,11 +577,12 @@ cudaError_t launch_scores_tri_sm100(const Params &p, cudaStream_t s)
 {
     const int q_rows = p.group * p.alpha;
     const int q_rows_pad = (q_rows + 15) / 16 * 16;
-    CUtensorMap map_k, map_q, map_hs, map_ns;
+    CUtensorMap map_k, map_q, map_hs, map_ns, map_ts;
     if (!make_map(&map_k, p.k_cache, (uint64_t)p.batch * p.hkv * p.cap, kTile) ||
         !make_map(&map_q, p.q_window, (uint64_t)p.batch * p.hq * p.alpha, (uint32_t)q_rows_pad) ||
         !make_map(&map_hs, p.head_sum_bf16, (uint64_t)p.batch * p.hkv * 16, 16u) ||
-        !make_map_k16(&map_ns, p.norm_split, (uint64_t)p.batch * p.hkv * p.cap_pad))
+        !make_map_k16(&map_ns, p.norm_split, (uint64_t)p.batch * p.hkv * p.cap_pad) ||
+        !make_map_k16(&map_ts, p.thr_split, (uint64_t)p.batch * p.hkv * kTile))
         return cudaErrorInvalidValue;
     cudaError_t e;
     if ((e = cudaFuncSetAttribute(scores_pass2_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)) !=
@@ -591,7 +592,7 @@ cudaError_t launch_scores_tri_sm100(const Params &p, cudaStream_t s)
     if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
     if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
     const int heads = p.batch * p.hkv;
-    if ((e = launch_scores_pass1_sm100(p, s, map_k, map_q, map_hs, q_rows_pad, sms)) != cudaSuccess) return e;
+    if ((e = launch_scores_pass1_sm100(p, s, map_k, map_q, map_hs, map_ns, map_ts, q_rows_pad, sms)) != cudaSuccess) return e;
     if ((e = mark_kernel(p, 0, s)) != cudaSuccess) return e;
     const bool rule_on = p.beta > 0 && p.sim_threshold < 1.0f;
     if (!rule_on || p.tiles < 2) return mark_kernel(p, 1, s);       // nobody can lack partners / the first pass has seen everything

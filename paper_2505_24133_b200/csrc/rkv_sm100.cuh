@@ -293,6 +293,7 @@ inline bool make_map_k16(CUtensorMap *map, const void *base, uint64_t rows)
 
 // first scoring pass of the two-pass tensor-core route (its own file); the maps are built by the caller
 cudaError_t launch_scores_pass1_sm100(const Params &p, cudaStream_t s, const CUtensorMap &map_k, const CUtensorMap &map_q,
-                                      const CUtensorMap &map_hs, int q_rows_pad, int sms);
+                                      const CUtensorMap &map_hs, const CUtensorMap &map_ns, const CUtensorMap &map_ts,
+                                      int q_rows_pad, int sms);
 
 }  // namespace rkv
