@@ -35,11 +35,12 @@ UNIT = "tokens/s"
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per head-problem of one launch, from the ncu capture
 # of a 256-head-problem slice at n = 4216 summarised in profiles/all_kernels_llama8b_b16_batch1.md.  Every kernel
 # works head by head, so a full launch's traffic is this figure times the launch's head-problems (only taken for
-# workloads of that cache size).  None = the kernel has changed since the counters were taken.
+# workloads of that cache size; the capture has G = 4, other group sizes differ only in the few KB of queries per head).
+# None = the kernel has changed since the counters were taken.
 NCU_TRAFFIC_PER_HEAD_N4216 = {
-    "prep": (276.32e6 + 13.92e6) / 256, "scores_pass1": None, "scores_list": (4.33e6 + 0.0) / 256,
-    "scores_pass2": (323.53e6 + 6.96e6) / 256, "row_stats": 34.62e6 / 256, "importance": 34.63e6 / 256,
-    "select": 8.68e6 / 256, "gather": (531.44e6 + 472.86e6) / 256,
+    "prep": 315.80e6 / 256, "scores_pass1": 359.09e6 / 256, "scores_list": 4.33e6 / 256,
+    "scores_pass2": 402.12e6 / 256,          # three scans and the two later listings, as bench.py's interval has them
+    "row_stats": 34.61e6 / 256, "importance": 34.63e6 / 256, "select": 8.69e6 / 256, "gather": 1003.60e6 / 256,
 }
 DEFAULT_WORKLOAD = "qwen14b_b32"
 
