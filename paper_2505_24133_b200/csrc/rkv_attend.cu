@@ -5,15 +5,15 @@
 //
 // HBM-bound: every cached K and V row is read once, 2 * 2 * G * d flop per 2 * d * sizeof(T) bytes (5 flop per byte
 // for G = 5 at bf16), so the arithmetic stays on the CUDA cores in fp32 and the work goes into the data path: one
-// block per (KV head, split of the rows), 64-row tiles of K and of V brought into shared memory by bulk copies
+// block per (KV head, split of the rows), 56-row tiles of K and of V brought into shared memory by bulk copies
 // (cp.async.bulk, three stages in flight, bounded waits), all G query heads of the group served from the same tile.
 //   scores   8 lanes per row, 16 dims each (two or four 16-byte shared-memory loads), the G partial dot products of a
 //            row folded over the 8 lanes by 3 shuffle steps; four rows per warp instruction
-//   softmax  online and per WARP: each of the 8 compute warps keeps its own running maximum and sum over its 8 rows
+//   softmax  online and per WARP: each of the 7 compute warps keeps its own running maximum and sum over its 8 rows
 //            of every tile (base-2 exponentials), so the tile loop has no block-wide barrier; the warps' results are
 //            merged once, at the end
 //   values   lanes over d: a lane owns 4 dims of the output of every query head, a warp walks its 8 rows of the tile
-// A ninth warp is the producer of the bulk copies; stages are handed back through mbarriers.
+// An eighth warp is the producer of the bulk copies; stages are handed back through mbarriers.
 // With few head-problems the rows of a head are cut into splits (more blocks than SMs); a second small kernel merges
 // the splits' partial results.
 #include "rkv_sm100.cuh"

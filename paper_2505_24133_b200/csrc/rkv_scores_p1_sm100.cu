@@ -3,22 +3,24 @@
 // downwards).  tcgen05.mma with TMEM accumulators, fed by TMA, one persistent block per SM.
 //
 // The pass is a single sweep over the keys, so it is organised as a stream: the 128-row key tiles of a head flow
-// through a ring of shared-memory stages as the A operand (one token per TMEM lane), while the two B operands of the
-// head stay put: its G * alpha query rows followed by 16 rows that hold sum_j Kbar_j split into bf16 parts, and its
-// last key tile.  Per streamed tile the tensor cores form two products into one accumulator buffer:
+// through a ring of shared-memory stages as the A operand (one token per TMEM lane), while ONE B operand block of the
+// head stays put: the rows of its last key tile, then its G * alpha query rows, then 16 rows that hold sum_j Kbar_j
+// split into bf16 parts.  Per streamed tile the tensor cores form one product of N = 128 + query rows + 16 (a product
+// with few columns costs nearly as much as one with 128), plus one K = 16 step on the key columns that folds the
+// threshold test into the accumulator (slices of both operands written by the prep stage):
 //
-//   columns [0, 128)         k_i . k_j for the 128 keys j of the last tile: the thread that owns token i scans them
-//                            from the last position downwards, "the first beta hits" are Section 3.3's partners
+//   columns [0, 128)         h = k_i . k_j - T / (r_i r_j) for the 128 keys j of the last tile: S[j][i] > T exactly
+//                            when h > 0.  The thread that owns token i scans them from the last position downwards,
+//                            "the first beta hits" are Section 3.3's partners; a partner's value is T + h r_i r_j
 //   columns [128, 128 + q)   k_i . q for every query row (a thread ends up with all logits of its key and takes the max,
 //                            or the mean, over the group: Eq. 3), then k_i . s in three parts, which gives
 //                            sum_j S[j][i] = Kbar_i . (sum_j Kbar_j) - Kbar_i . Kbar_i without forming the matrix
 //
-// Out, per token: the pooled logits, the column sum minus the removed entries (sbar), the partners still lacking
-// (left), and 1 / r_i in three bf16 parts (norm_split), the extra K = 16 slice the second pass appends to a key row.
+// Out, per token: the pooled logits, the column sum minus the removed entries (sbar), the partners still lacking (left).
 //
 // Work item = (head, range of row tiles); items are handed out by a global ticket counter, head-major.  The operands
 // that stay put are double-buffered across items, so the next item's arrive while the current one is streamed, and
-// the ring never drains at an item boundary: the kernel is bound by the one read of K from HBM.
+// the ring never drains at an item boundary.
 // Warp roles (320 threads): warp 0 = tickets + TMA producer, warp 1 = MMA issuer and TMEM owner, warps 2..9 = epilogue
 // in two groups of four (warp w may touch TMEM lanes 32 (w % 4) .. +31); group g drains accumulator buffer g, i.e.
 // every second tile of the stream.  Every wait on an mbarrier is bounded; on expiry the block records
