@@ -133,6 +133,17 @@ typedef struct rkv_desc {
        budgets[b] tokens, out_idx[b][h][budgets[b] ..] = -1, and seq_lens[b] becomes budgets[b].  A value out of
        range is treated like an invalid length: the sequence is skipped and RKV_ERR_INVALID_ARG recorded. */
     const int32_t *budgets;
+    /* optional: PAGED caches (the paper's last section names the reallocation cost of paged serving frameworks as the
+       method's limitation; here the compaction stays in place, page by page).  block_table is a device int32
+       [batch][n_kv_heads][(budget + buffer) / 128]: the page that holds rows [128 t, 128 t + 128) of head (b, h).
+       k_cache and v_cache are then page POOLS [pool_pages][128][head_dim] (same dtype, 16-byte aligned), a page
+       holding 128 consecutive rows of one (sequence, KV head); budget + buffer must be a multiple of 128; the pages of
+       one call must be distinct.  Every entry point that takes k_cache / v_cache follows the table (rkv_compress*,
+       rkv_append, rkv_decode_attention; not rkv_compress_host).  The compaction moves rows between a head's own pages
+       only and never changes the table: after a compression the head's first budget rows, in table order, are the kept
+       ones.  NULL: contiguous caches as described with rkv_compress. */
+    const int32_t *block_table;
+    int64_t pool_pages;
 } rkv_desc_t;
 
 /* Fill *desc with the defaults above (pool_w 4, beta 1, T 0.5, eps 1e-8, head_dim 128, bf16), zero elsewhere. */

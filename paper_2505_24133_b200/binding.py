@@ -41,7 +41,8 @@ class RkvDesc(ctypes.Structure):
         ("device_status", ctypes.c_void_p), ("dbg_I", ctypes.c_void_p), ("dbg_Sbar", ctypes.c_void_p),
         ("dbg_R", ctypes.c_void_p), ("dbg_Z", ctypes.c_void_p), ("stage_events", ctypes.c_void_p),
         ("kernel_events", ctypes.c_void_p), ("dbg_counters", ctypes.c_void_p),
-        ("wait_limit_cycles", ctypes.c_int64), ("budgets", ctypes.c_void_p),
+        ("wait_limit_cycles", ctypes.c_int64), ("budgets", ctypes.c_void_p), ("block_table", ctypes.c_void_p),
+        ("pool_pages", ctypes.c_int64),
     ]
 
 
@@ -202,7 +203,8 @@ class Compressor:
                  lam: float = 0.1, dtype: torch.dtype = torch.bfloat16, pool_w: Optional[int] = None,
                  beta: Optional[int] = None, sim_threshold: Optional[float] = None, eps: Optional[float] = None,
                  flags: int = 0, device="cuda", dump_scores: bool = False, host_staging: bool = False,
-                 stage_events: bool = False, budgets: Optional[torch.Tensor] = None, head_dim: int = 128):
+                 stage_events: bool = False, budgets: Optional[torch.Tensor] = None, head_dim: int = 128,
+                 block_table: Optional[torch.Tensor] = None, pool_pages: int = 0):
         self.budget, self.buffer, self.alpha, self.lam = budget, buffer, alpha, lam
         self.cap = budget + buffer
         self.device = torch.device(device)
@@ -250,6 +252,11 @@ class Compressor:
             self.budgets = budgets.to(device=self.device, dtype=torch.int32).contiguous()
             assert self.budgets.shape == (batch,)
             d.budgets = self.budgets.data_ptr()
+        self.block_table = None
+        if block_table is not None:      # paged caches: [batch, n_kv_heads, cap / 128] page ids into pools of pool_pages pages
+            self.block_table = block_table.to(device=self.device, dtype=torch.int32).contiguous()
+            assert self.block_table.shape == (batch, n_kv_heads, self.cap // 128)
+            d.block_table, d.pool_pages = self.block_table.data_ptr(), pool_pages
         self.desc = d
         self.out_idx = torch.empty(batch, n_kv_heads, budget, dtype=torch.int32, device=self.device)
 

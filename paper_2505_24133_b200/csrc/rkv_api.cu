@@ -50,6 +50,10 @@ int check_shapes(const rkv_desc_t *d, int budget, int buffer, int alpha, Layout 
     if (cap > RKV_MAX_CAP) return RKV_ERR_UNSUPPORTED;
     if ((long long)(d->n_q_heads / d->n_kv_heads) * alpha > RKV_MAX_GROUP_ROWS) return RKV_ERR_UNSUPPORTED;
     if ((long long)d->batch * d->n_kv_heads > (1ll << 24)) return RKV_ERR_UNSUPPORTED;
+    if (d->block_table) {      // paged caches: a page is one key tile
+        if (cap % kTile != 0 || d->pool_pages < 1 || d->pool_pages > (1ll << 23)) return RKV_ERR_INVALID_ARG;
+        if (reinterpret_cast<uintptr_t>(d->block_table) & 3u) return RKV_ERR_INVALID_ARG;
+    }
     if (lay) {
         const size_t P = (size_t)d->batch * d->n_kv_heads;
         lay->cap = (int)cap;
@@ -153,6 +157,9 @@ int run(const rkv_desc_t *d, void *k_cache, void *v_cache, const void *q_window,
     p.tri = lay.tri;
     p.status = d->device_status;
     p.budgets = d->budgets;
+    p.block_table = d->block_table;
+    p.pages_per_head = lay.cap / kTile;
+    p.pool_pages = d->pool_pages;
     p.wait_cycles = d->wait_limit_cycles > 0 ? (long long)d->wait_limit_cycles : sm100_default_wait_cycles();
     p.kernel_events = d->kernel_events;
     p.dbg_counters = d->dbg_counters;
@@ -292,8 +299,8 @@ int rkv_compress_host(const rkv_desc_t *desc, void *host_k_cache, void *host_v_c
     HostLayout h;
     int rc = host_layout(desc, budget, buffer, alpha, &h);
     if (rc != RKV_OK) return rc;
-    if (!host_k_cache || !host_v_cache || !host_q_window || !host_seq_lens || !host_out_idx)
-        return RKV_ERR_INVALID_ARG;
+    if (!host_k_cache || !host_v_cache || !host_q_window || !host_seq_lens || !host_out_idx || desc->block_table)
+        return RKV_ERR_INVALID_ARG;      // (the host-buffer form takes contiguous caches only)
     if (!desc->workspace || desc->workspace_bytes < h.total) return RKV_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(desc->workspace) & 255u) return RKV_ERR_WORKSPACE;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -335,7 +342,7 @@ int rkv_append(const rkv_desc_t *d, void *k_cache, void *v_cache, const void *k_
     if (reinterpret_cast<uintptr_t>(seq_lens) & 3u) return RKV_ERR_INVALID_ARG;
     const int row_bytes = d->head_dim * (d->dtype == RKV_BF16 ? 2 : 4);
     const cudaError_t e = launch_append(k_cache, v_cache, k_new, v_new, seq_lens, d->batch, d->n_kv_heads, budget + buffer,
-                                        row_bytes, d->device_status, static_cast<cudaStream_t>(stream));
+                                        row_bytes, d->device_status, d->block_table, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? RKV_OK : cuda_fail(e, "append launch");
 }
 
@@ -389,7 +396,7 @@ int rkv_decode_attention(const rkv_desc_t *d, const void *k_cache, const void *v
     const long long wait = d->wait_limit_cycles > 0 ? (long long)d->wait_limit_cycles : sm100_default_wait_cycles();
     const cudaError_t e = launch_attend(k_cache, v_cache, q_new, seq_lens, out, static_cast<float *>(d->workspace), d->batch,
                                         d->n_kv_heads, d->n_q_heads, budget + buffer, splits, d->dtype, d->device_status,
-                                        wait, static_cast<cudaStream_t>(stream));
+                                        wait, d->block_table, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? RKV_OK : cuda_fail(e, "decode attention launch");
 }
 

@@ -38,6 +38,7 @@ struct AttendParams {
     int batch, hkv, hq, cap, splits;
     int32_t *status;
     long long wait_cycles;
+    const int32_t *block_table;  // paged caches: [P][cap / 128] page ids (a page = 128 rows), else null
 };
 
 template <typename T, int G>
@@ -69,8 +70,13 @@ __global__ void __launch_bounds__(kAttThreads, (G <= 4 && sizeof(T) == 2) ? 2 : 
     const int t_begin = (int)((long long)split * tiles_all / p.splits), t_end = (int)((long long)(split + 1) * tiles_all / p.splits);
     const int n_tiles = t_end - t_begin;
 
-    const T *K = static_cast<const T *>(p.k_cache) + (size_t)head * p.cap * kHeadDim;
-    const T *V = static_cast<const T *>(p.v_cache) + (size_t)head * p.cap * kHeadDim;
+    const T *K = static_cast<const T *>(p.k_cache), *V = static_cast<const T *>(p.v_cache);
+    // first of the rows [r, r + count) of the head in the caches' row view; with paged caches the rows must not cross a
+    // page boundary
+    auto row_at = [&](int r) -> size_t {
+        return p.block_table ? (size_t)p.block_table[(size_t)head * (p.cap / kTile) + r / kTile] * kTile + r % kTile
+                             : (size_t)head * p.cap + r;
+    };
     const ErrSink sink{p.status, nullptr, p.wait_cycles};
 
     if (threadIdx.x == 0) {
@@ -94,17 +100,24 @@ __global__ void __launch_bounds__(kAttThreads, (G <= 4 && sizeof(T) == 2) ? 2 : 
                 const int s = t % kAttStages;
                 if (!mbar_wait(smem_u32(bars + kAttStages + s), ((t / kAttStages) & 1) ^ 1, &abort_flag, sink)) break;
                 const int row0 = (t_begin + t) * kAttRows;
-                const uint32_t bytes = (uint32_t)min(kAttRows, Lc - row0) * kRowBytes;
+                const int rows = min(kAttRows, Lc - row0);
                 const uint32_t bar = smem_u32(bars + s);
-                mbar_expect_tx(bar, 2 * bytes);
-                asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                             ::"r"(smem_u32(att_smem + (size_t)s * 2 * kTileBytesT)), "l"(K + (size_t)row0 * kHeadDim), "r"(bytes),
-                               "r"(bar)
-                             : "memory");
-                asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                             ::"r"(smem_u32(att_smem + (size_t)s * 2 * kTileBytesT + kTileBytesT)), "l"(V + (size_t)row0 * kHeadDim),
-                               "r"(bytes), "r"(bar)
-                             : "memory");
+                mbar_expect_tx(bar, 2u * (uint32_t)rows * kRowBytes);
+                // one copy per operand, or two where the tile crosses a page boundary of a paged cache
+                const int first = p.block_table ? min(rows, kTile - row0 % kTile) : rows;
+                for (int part = 0; part < 2; ++part) {
+                    const int r0 = part == 0 ? 0 : first, cnt = part == 0 ? first : rows - first;
+                    if (cnt <= 0) break;
+                    const size_t src = row_at(row0 + r0) * kHeadDim;
+                    const uint32_t bytes = (uint32_t)cnt * kRowBytes, off = (uint32_t)r0 * kRowBytes;
+                    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                                 ::"r"(smem_u32(att_smem + (size_t)s * 2 * kTileBytesT) + off), "l"(K + src), "r"(bytes), "r"(bar)
+                                 : "memory");
+                    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                                 ::"r"(smem_u32(att_smem + (size_t)s * 2 * kTileBytesT + kTileBytesT) + off), "l"(V + src), "r"(bytes),
+                                   "r"(bar)
+                                 : "memory");
+                }
             }
         }
         __syncwarp();
@@ -345,7 +358,7 @@ size_t attend_partial_bytes(int heads, int splits, int G)
 
 cudaError_t launch_attend(const void *k_cache, const void *v_cache, const void *q_new, const int32_t *seq_lens, float *out,
                           float *partial, int batch, int hkv, int hq, int cap, int splits, int dtype, int32_t *status,
-                          long long wait_cycles, cudaStream_t s)
+                          long long wait_cycles, const int32_t *block_table, cudaStream_t s)
 {
     AttendParams p;
     p.k_cache = k_cache;
@@ -361,6 +374,7 @@ cudaError_t launch_attend(const void *k_cache, const void *v_cache, const void *
     p.splits = splits;
     p.status = status;
     p.wait_cycles = wait_cycles;
+    p.block_table = block_table;
     const int G = hq / hkv;
     cudaError_t e = dtype == RKV_BF16 ? launch_dtype<__nv_bfloat16>(p, G, s) : launch_dtype<float>(p, G, s);
     if (e != cudaSuccess || splits == 1) return e;

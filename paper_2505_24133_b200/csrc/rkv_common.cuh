@@ -63,6 +63,9 @@ struct Params {
     int32_t *meta;       // [2][batch]           snapshot of seq_lens (kMetaInvalid if out of range), then each
                          //                      sequence's budget (p.budget unless the caller gave per-sequence ones)
     const int32_t *budgets;   // optional [batch]: per-sequence budgets (alpha < budgets[b] <= budget), else null
+    const int32_t *block_table;   // optional [P][cap / 128]: paged caches, page (= key tile) ids into the pools, else null
+    int pages_per_head;           // cap / 128 (paged caches)
+    long long pool_pages;         // pages in the pools (paged caches)
     // zeroed by the prep stage's memset, in this order, contiguous:
     unsigned long long *counters;   // [8]       [0] = similarity tiles computed by the tcgen05 kernels, [1] = item
                                     //           ticket of the first scoring pass, [2] = entries in strag_items,
@@ -126,6 +129,18 @@ __device__ __forceinline__ int candidates_from_meta(int L, int budget, int alpha
 {
     return (L > budget) ? (L - alpha) : 0;
 }
+// Where key tile `tile` (128 rows) of head-problem `head` starts, in rows of the 2-D [rows][d] view of k_cache / v_cache:
+// head after head for contiguous caches, through the block table for paged ones (a page holds one key tile).
+__device__ __forceinline__ long long tile_row0(const Params &p, int head, int tile)
+{
+    return p.block_table ? (long long)p.block_table[(size_t)head * p.pages_per_head + tile] * kTile
+                         : (long long)head * p.cap + (long long)tile * kTile;
+}
+// ... and row r of the head.
+__device__ __forceinline__ long long row_index(const Params &p, int head, int r)
+{
+    return tile_row0(p, head, r / kTile) + (r % kTile);
+}
 // The same for sequence b as every stage after prep sees it (length and budget snapshots left by the prep stage).
 __device__ __forceinline__ int seq_budget(const Params &p, int b) { return p.meta[p.batch + b]; }
 __device__ __forceinline__ int seq_candidates(const Params &p, int b)
@@ -166,12 +181,12 @@ cudaError_t launch_scores_tri_sm100(const Params &p, cudaStream_t s);
 cudaError_t launch_select(const Params &p, cudaStream_t s);
 cudaError_t launch_gather(const Params &p, cudaStream_t s);
 cudaError_t launch_append(void *k_cache, void *v_cache, const void *k_new, const void *v_new, int32_t *seq_lens, int batch,
-                          int hkv, int cap, int row_bytes, int32_t *status, cudaStream_t s);
+                          int hkv, int cap, int row_bytes, int32_t *status, const int32_t *block_table, cudaStream_t s);
 cudaError_t launch_push_query(void *q_window, const void *q_new, int batch, int hq, int alpha, int slot, int row_bytes,
                               cudaStream_t s);
 cudaError_t launch_attend(const void *k_cache, const void *v_cache, const void *q_new, const int32_t *seq_lens, float *out,
                           float *partial, int batch, int hkv, int hq, int cap, int splits, int dtype, int32_t *status,
-                          long long wait_cycles, cudaStream_t s);
+                          long long wait_cycles, const int32_t *block_table, cudaStream_t s);
 int attend_max_group();
 int attend_splits(int heads, int cap, int sms);
 size_t attend_partial_bytes(int heads, int splits, int G);

@@ -12,7 +12,8 @@ constexpr int kDecThreads = 256;
 // k_new / v_new [batch][hkv][row_vecs] -> row seq_lens[b] of every head of sequence b
 __global__ void __launch_bounds__(kDecThreads) append_kernel(uint4 *k_cache, uint4 *v_cache, const uint4 *k_new,
                                                              const uint4 *v_new, const int32_t *seq_lens, long long total,
-                                                             int hkv, int cap, int row_vecs, int32_t *status)
+                                                             int hkv, int cap, int row_vecs, int32_t *status,
+                                                             const int32_t *block_table)
 {
     const long long t = (long long)blockIdx.x * kDecThreads + threadIdx.x;
     if (t >= total) return;
@@ -20,7 +21,10 @@ __global__ void __launch_bounds__(kDecThreads) append_kernel(uint4 *k_cache, uin
     const int head = (int)(t / row_vecs);          // b * hkv + h
     const int L = seq_lens[head / hkv];
     if (L >= 0 && L < cap) {
-        const size_t dst = ((size_t)head * cap + L) * row_vecs + vec;
+        // row L of the head: head after head, or through the block table (pages of kTile rows) for paged caches
+        const size_t row = block_table ? (size_t)block_table[(size_t)head * (cap / kTile) + L / kTile] * kTile + L % kTile
+                                       : (size_t)head * cap + L;
+        const size_t dst = row * row_vecs + vec;
         k_cache[dst] = k_new[t];
         v_cache[dst] = v_new[t];
     } else if (vec == 0 && head % hkv == 0) {
@@ -52,14 +56,14 @@ __global__ void __launch_bounds__(kDecThreads) push_query_kernel(uint4 *q_window
 }  // namespace
 
 cudaError_t launch_append(void *k_cache, void *v_cache, const void *k_new, const void *v_new, int32_t *seq_lens, int batch,
-                          int hkv, int cap, int row_bytes, int32_t *status, cudaStream_t s)
+                          int hkv, int cap, int row_bytes, int32_t *status, const int32_t *block_table, cudaStream_t s)
 {
     const int row_vecs = row_bytes / 16;
     const long long total = (long long)batch * hkv * row_vecs;
     const unsigned grid = (unsigned)((total + kDecThreads - 1) / kDecThreads);
     append_kernel<<<grid, kDecThreads, 0, s>>>(static_cast<uint4 *>(k_cache), static_cast<uint4 *>(v_cache),
                                                static_cast<const uint4 *>(k_new), static_cast<const uint4 *>(v_new),
-                                               seq_lens, total, hkv, cap, row_vecs, status);
+                                               seq_lens, total, hkv, cap, row_vecs, status, block_table);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     bump_kernel<<<(unsigned)((batch + kDecThreads - 1) / kDecThreads), kDecThreads, 0, s>>>(seq_lens, batch, cap);

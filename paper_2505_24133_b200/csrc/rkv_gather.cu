@@ -37,8 +37,8 @@ __global__ void __launch_bounds__(kGatherThreads) gather_kernel(Params p)
     if (call_aborted(p)) return;                    // a bounded wait ran out earlier in this call: caches and lengths stay as they are
     if (which == 0 && slice == 0 && head % p.hkv == 0 && threadIdx.x == 0) p.seq_lens[b] = budget_b;
 
-    uint4 *base = reinterpret_cast<uint4 *>(which ? p.v_cache : p.k_cache) + (size_t)head * p.cap * kVecPerRow +
-                  slice * kVecPerSlice;
+    // rows are addressed through row_index(): head after head, or page by page for paged caches
+    uint4 *base = reinterpret_cast<uint4 *>(which ? p.v_cache : p.k_cache) + slice * kVecPerSlice;
     const int32_t *idx = p.out_idx + (size_t)head * p.budget;
     const int lane_vec = threadIdx.x % kVecPerSlice;
     const int lane_row = threadIdx.x / kVecPerSlice;
@@ -52,13 +52,13 @@ __global__ void __launch_bounds__(kGatherThreads) gather_kernel(Params p)
         for (int q = 0; q < kVecPerThread; ++q) {
             const int j = j0 + q * kRowsPerStep + lane_row;
             src[q] = (j < j_end) ? idx[j] : -1;
-            if (src[q] >= 0 && src[q] != j) held[q] = base[(size_t)src[q] * kVecPerRow + lane_vec];
+            if (src[q] >= 0 && src[q] != j) held[q] = base[(size_t)row_index(p, head, src[q]) * kVecPerRow + lane_vec];
         }
         __syncthreads();                             // every source row of the chunk is in registers
 #pragma unroll
         for (int q = 0; q < kVecPerThread; ++q) {
             const int j = j0 + q * kRowsPerStep + lane_row;
-            if (src[q] >= 0 && src[q] != j) base[(size_t)j * kVecPerRow + lane_vec] = held[q];
+            if (src[q] >= 0 && src[q] != j) base[(size_t)row_index(p, head, j) * kVecPerRow + lane_vec] = held[q];
         }
     }
 }

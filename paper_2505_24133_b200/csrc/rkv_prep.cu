@@ -54,7 +54,7 @@ __global__ void __launch_bounds__(kPrepThreads, D <= 128 ? 5 : 2) prep_kernel(Pa
     }
     const int n = candidates_from_meta(L, budget_b, p.alpha);
 
-    const T *K = static_cast<const T *>(p.k_cache) + (size_t)head * p.cap * D;
+    const T *K_tile = static_cast<const T *>(p.k_cache) + (size_t)tile_row0(p, head, tile) * D;      // the tile's first row
     float *inv_norm = p.inv_norm + (size_t)head * p.cap_pad;
 
     const int sub = lane / kLanesPerRow;                 // which of the rows of this pass
@@ -73,7 +73,7 @@ __global__ void __launch_bounds__(kPrepThreads, D <= 128 ? 5 : 2) prep_kernel(Pa
             const uint32_t bytes = (uint32_t)rows_here * D * (uint32_t)sizeof(T);
             mbar_expect_tx(bar, bytes);
             asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                         ::"r"(smem_u32(prep_smem)), "l"(K + (size_t)tile * kTile * D), "r"(bytes), "r"(bar)
+                         ::"r"(smem_u32(prep_smem)), "l"(K_tile), "r"(bytes), "r"(bar)
                          : "memory");
         }
     }

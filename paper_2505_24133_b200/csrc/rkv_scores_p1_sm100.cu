@@ -155,7 +155,6 @@ scores_stream_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, 
                 const int n_tiles = (n + kTile - 1) / kTile;
                 const int t0 = (int)((long long)part * n_tiles / splits), t1 = (int)((long long)(part + 1) * n_tiles / splits);
                 if (t0 >= t1) continue;                                        // more parts than tiles
-                const int key_row_base = head * p.cap;                         // first row of the head in the 2-D key view
 
                 const uint32_t slot = k_item & 1;
                 if (!mbar_wait(bar(kBarSlotEmpty + slot), ((k_item >> 1) & 1) ^ 1, abort_flag, sink)) break;
@@ -176,7 +175,7 @@ scores_stream_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, 
                     tma_load_2d(qdst + half + q_rows_pad * 128, &map_hs, 64, head * 16, full);
                 }
                 if (rule_on) {
-                    const int y = key_row_base + (n_tiles - 1) * kTile;
+                    const int y = (int)tile_row0(p, head, n_tiles - 1);
                     tma_load_2d(slot_addr, &map_k, 0, y, full);
                     tma_load_2d(slot_addr + (uint32_t)pl.slot_bytes / 2, &map_k, 64, y, full);
                     // the tile's extra slice: -T / r_j of its keys in three bf16 parts
@@ -194,7 +193,7 @@ scores_stream_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, 
                         break;
                     }
                     const uint32_t dst = sbase + s * kTileBytes;
-                    const int y = key_row_base + t * kTile;
+                    const int y = (int)tile_row0(p, head, t);
                     mbar_expect_tx(bar(kBarAFull + s), kTileBytes + (rule_on ? kSliceBytes : 0));
                     tma_load_2d(dst, &map_k, 0, y, bar(kBarAFull + s));
                     tma_load_2d(dst + kHalfBytes, &map_k, 64, y, bar(kBarAFull + s));

@@ -161,7 +161,6 @@ scores_pass2_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, c
                 const int head = desc.x;
                 const int first_tile = desc.w;             // streamed tiles: first_tile .. first_tile - n_iter + 1
                 const int n_iter = desc.z >> 16;
-                const int key_row_base = head * p.cap;                         // first row of the head in the 2-D key view
                 for (int it = 0; it < n_iter; ++it) {
                     const uint32_t s = bcount % kStagesB;
                     if (!mbar_wait(bar.at(kBarBEmpty + s), ((bcount / kStagesB) & 1) ^ 1, abort_flag, sink)) {
@@ -170,7 +169,7 @@ scores_pass2_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, c
                     }
                     const uint32_t dst = sbase + kOffB + s * kTileBytes;
                     const int jt = first_tile - it;
-                    const int y = key_row_base + jt * kTile;
+                    const int y = (int)tile_row0(p, head, jt);
                     mbar_expect_tx(bar.at(kBarBFull + s), kTileBytes + kSliceBytes);
                     tma_load_2d(dst, &map_k, 0, y, bar.at(kBarBFull + s));
                     tma_load_2d(dst + kHalfBytes, &map_k, 64, y, bar.at(kBarBFull + s));
@@ -307,7 +306,7 @@ scores_pass2_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, c
                 const bool row_ok = pos[m] >= 0;
                 uint8_t *tile = smem + kOffA + (ab * 2 + m) * kTileBytes;
                 const uint4 *src = reinterpret_cast<const uint4 *>(
-                    static_cast<const __nv_bfloat16 *>(p.k_cache) + ((size_t)head * p.cap + (row_ok ? pos[m] : 0)) * kHeadDim);
+                    static_cast<const __nv_bfloat16 *>(p.k_cache) + (size_t)row_index(p, head, row_ok ? pos[m] : 0) * kHeadDim);
                 uint4 v[16];
 #pragma unroll
                 for (int c = 0; c < 16; ++c) v[c] = row_ok ? __ldg(src + c) : make_uint4(0u, 0u, 0u, 0u);
@@ -578,7 +577,7 @@ cudaError_t launch_scores_tri_sm100(const Params &p, cudaStream_t s)
     const int q_rows = p.group * p.alpha;
     const int q_rows_pad = (q_rows + 15) / 16 * 16;
     CUtensorMap map_k, map_q, map_hs, map_ns, map_ts;
-    if (!make_map(&map_k, p.k_cache, (uint64_t)p.batch * p.hkv * p.cap, kTile) ||
+    if (!make_map(&map_k, p.k_cache, key_rows_total(p), kTile) ||
         !make_map(&map_q, p.q_window, (uint64_t)p.batch * p.hq * p.alpha, (uint32_t)q_rows_pad) ||
         !make_map(&map_hs, p.head_sum_bf16, (uint64_t)p.batch * p.hkv * 16, 16u) ||
         !make_map_k16(&map_ns, p.norm_split, (uint64_t)p.batch * p.hkv * p.cap_pad) ||

@@ -17,8 +17,8 @@ namespace {
 
 constexpr int kSimtThreads = 128;
 
-// kRows rows of D elements into shared memory as fp32, rows padded to D + 1 floats (thread-per-row reads then hit
-// distinct banks); rows >= valid_rows are zero-filled.
+// kRows rows of D elements, starting at `src` (row first_row of its head), into shared memory as fp32, rows padded to
+// D + 1 floats (thread-per-row reads then hit distinct banks); rows >= valid_rows are zero-filled.
 template <typename T, int D, int kRows>
 __device__ void load_tile_rows(const T *src, int first_row, int valid_rows, float *dst /*[kRows][D + 1]*/)
 {
@@ -30,7 +30,7 @@ __device__ void load_tile_rows(const T *src, int first_row, int valid_rows, floa
         const int r = v / kVecPerRow, c = (v % kVecPerRow) * kPerVec;
         float f[kPerVec];
         if (first_row + r < valid_rows) {
-            uint4 raw = __ldg(reinterpret_cast<const uint4 *>(src + (size_t)(first_row + r) * kHeadDim + c));
+            uint4 raw = __ldg(reinterpret_cast<const uint4 *>(src + (size_t)r * kHeadDim + c));
             Elem<T>::unpack(raw, f);
         } else {
 #pragma unroll
@@ -61,7 +61,10 @@ __global__ void __launch_bounds__(kSimtThreads) scores_simt_kernel(Params p)
     const int n = seq_candidates(p, b);
     if (n == 0) return;
     const int n_tiles = (n + kTile - 1) / kTile;
-    const T *K = static_cast<const T *>(p.k_cache) + (size_t)head * p.cap * kHeadDim;
+    // first of the (at most 128, page-aligned) rows of the head starting at `first_row`
+    auto key_rows = [&](int first_row) {
+        return static_cast<const T *>(p.k_cache) + (size_t)row_index(p, head, first_row) * kHeadDim;
+    };
     const float *inv_norm = p.inv_norm + (size_t)head * p.cap_pad;
     const int t = threadIdx.x;
 
@@ -69,13 +72,13 @@ __global__ void __launch_bounds__(kSimtThreads) scores_simt_kernel(Params p)
         // ---------------- Eq. 5-6 + retention rule for rows [128 x, 128 x + 128)
         if (x >= n_tiles) return;
         const int i = x * kTile + t;
-        load_tile_rows<T, D, kTile>(K, x * kTile, n, tileA);
+        load_tile_rows<T, D, kTile>(key_rows(x * kTile), x * kTile, n, tileA);
         const float ri = (i < n) ? inv_norm[i] : 0.f;
         float total = 0.f, removed = 0.f;
         int left = p.beta;
         for (int jt = (n_tiles * kTile) / kRowsB - 1; jt >= 0; --jt) {          // descending j: "largest positions first"
             __syncthreads();
-            load_tile_rows<T, D, kRowsB>(K, jt * kRowsB, n, tileB);
+            load_tile_rows<T, D, kRowsB>(key_rows(jt * kRowsB), jt * kRowsB, n, tileB);
             if (t < kRowsB) rB[t] = (jt * kRowsB + t < n) ? inv_norm[jt * kRowsB + t] : 0.f;
             __syncthreads();
             if (i < n) {
@@ -104,7 +107,7 @@ __global__ void __launch_bounds__(kSimtThreads) scores_simt_kernel(Params p)
         float *logits = p.logits + (size_t)head * p.alpha * p.cap_pad;
         for (int jt = 0; jt < (n_tiles * kTile) / kRowsB; ++jt) {
             __syncthreads();
-            load_tile_rows<T, D, kRowsB>(K, jt * kRowsB, n, tileB);
+            load_tile_rows<T, D, kRowsB>(key_rows(jt * kRowsB), jt * kRowsB, n, tileB);
             __syncthreads();
             const int i = jt * kRowsB + t;
             if (t < kRowsB && i < n) {

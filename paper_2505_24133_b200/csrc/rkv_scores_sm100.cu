@@ -101,7 +101,6 @@ scores_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, const _
     const bool rule_on = p.beta > 0 && p.sim_threshold < 1.0f;
     const int n_iter = is_q ? n_tiles : (rule_on ? n_tiles : 0);   // streamed tiles
     const int num_m = is_q ? 1 : ((n - row0 > kTile) ? 2 : 1);     // accumulator halves in use
-    const int key_row_base = head * p.cap;                           // first row of this head in the 2-D key view
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -137,7 +136,7 @@ scores_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, const _
             } else {
                 mbar_expect_tx(bar.resident(), (uint32_t)(num_m * kTileBytes));
                 for (int m = 0; m < num_m; ++m) {
-                    const int y = key_row_base + row0 + m * kTile;
+                    const int y = (int)tile_row0(p, head, row0 / kTile + m);
                     tma_load_2d(sbase + kOffA + m * kTileBytes, &map_k, 0, y, bar.resident());
                     tma_load_2d(sbase + kOffA + m * kTileBytes + kHalfBytes, &map_k, 64, y, bar.resident());
                 }
@@ -148,7 +147,7 @@ scores_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, const _
                 if (!mbar_wait(bar.empty(s), ((t / kStages) & 1) ^ 1, abort_flag, sink)) break;
                 mbar_expect_tx(bar.full(s), kTileBytes);
                 const uint32_t dst = sbase + kOffB + s * kTileBytes;
-                const int y = key_row_base + jt * kTile;
+                const int y = (int)tile_row0(p, head, jt);
                 tma_load_2d(dst, &map_k, 0, y, bar.full(s));
                 tma_load_2d(dst + kHalfBytes, &map_k, 64, y, bar.full(s));
             }
@@ -336,7 +335,7 @@ cudaError_t launch_scores_sm100(const Params &p, cudaStream_t s)
     const int q_rows = p.group * p.alpha;
     const int q_rows_pad = (q_rows + 15) / 16 * 16;
     CUtensorMap map_k, map_q;
-    if (!make_map(&map_k, p.k_cache, (uint64_t)p.batch * p.hkv * p.cap, kTile) ||
+    if (!make_map(&map_k, p.k_cache, key_rows_total(p), kTile) ||
         !make_map(&map_q, p.q_window, (uint64_t)p.batch * p.hq * p.alpha, (uint32_t)q_rows_pad))
         return cudaErrorInvalidValue;
     cudaError_t e = cudaFuncSetAttribute(scores_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);

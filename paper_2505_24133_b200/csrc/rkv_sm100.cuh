@@ -260,6 +260,12 @@ inline EncodeTiledFn encode_fn()
     return fn;
 }
 
+// Rows of the 2-D view of k_cache: all heads' rows, or all pages of a paged pool.
+inline uint64_t key_rows_total(const Params &p)
+{
+    return p.block_table ? (uint64_t)p.pool_pages * kTile : (uint64_t)p.batch * p.hkv * p.cap;
+}
+
 // 2-D bf16 view [rows][128] of a contiguous tensor, boxes of box_rows x 64 elements, 128-byte swizzle,
 // out-of-range rows read as zero.
 inline bool make_map(CUtensorMap *map, const void *base, uint64_t rows, uint32_t box_rows)

@@ -191,3 +191,26 @@ def check_batch(k_in: torch.Tensor, v_in: torch.Tensor, q_in: torch.Tensor, seq_
                 if not np.array_equal(v_raw_out[b, h, :nb], oracle.oracle_gather(v_raw_in[b, h], gi)):
                     err(f"{tag} compacted V rows differ from the gather of the kept positions")
     return rep
+
+
+# ----------------------------------------------------------------------------- paged caches (layout only)
+def to_paged(cache: torch.Tensor, pool_pages: int, table: torch.Tensor, fill=float("nan")) -> torch.Tensor:
+    """cache [B, H, cap, d] (cap a multiple of 128) scattered into a page pool [pool_pages, 128, d]: rows
+    [128 t, 128 t + 128) of head (b, h) go to page table[b, h, t].  Pages nobody owns hold `fill`."""
+    B, H, cap, d = cache.shape
+    pool = torch.full((pool_pages, 128, d), fill, dtype=cache.dtype, device=cache.device)
+    pool[table.reshape(-1).long()] = cache.reshape(B * H * (cap // 128), 128, d)
+    return pool
+
+
+def from_paged(pool: torch.Tensor, table: torch.Tensor) -> torch.Tensor:
+    """The inverse view: [B, H, cap, d] gathered from the pool through the table."""
+    B, H, T = table.shape
+    return pool[table.reshape(-1).long()].reshape(B, H, T * 128, pool.shape[-1])
+
+
+def random_block_table(B: int, H: int, pages_per_head: int, pool_pages: int, seed: int, device="cuda") -> torch.Tensor:
+    """Distinct page ids in random order, with unused pages in between."""
+    g = torch.Generator().manual_seed(seed)
+    ids = torch.randperm(pool_pages, generator=g)[:B * H * pages_per_head]
+    return ids.reshape(B, H, pages_per_head).to(torch.int32).to(device)

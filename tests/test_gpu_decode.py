@@ -6,7 +6,7 @@ import torch
 
 import oracle
 import rkv_inputs as ri
-from parity_util import check_batch, raw_rows
+from parity_util import check_batch, from_paged, random_block_table, raw_rows, to_paged
 
 pytestmark = pytest.mark.gpu
 
@@ -195,3 +195,41 @@ def test_decode_attention_argument_checks(rkv):
     d.n_q_heads = 4
     assert rkv.rkv_decode_attention(d, 0x20000, 0x20000, 0x20000, 0x30000, 0, 256, 64, 0) == 1       # null output
     assert rkv.rkv_decode_attention(d, 0x20000, 0x20000, 0x20000, 0x30000, 0x40000, 256, 64, 0) == 3  # splits need a workspace
+
+
+# ----------------------------------------------------------------------------- paged caches in the decode-step calls
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_paged_append_and_attention(rkv, dtype):
+    """rkv_append and rkv_decode_attention through a block table: the appended rows land in the right pages (compared
+    with the oracle's append after un-paging), and the attention over the paged caches equals the oracle's over the
+    same rows (tiles of 56 rows cross the 128-row pages)."""
+    spec = ri.CacheSpec("paged_dec", 1, 4, 2, 8, 128, 256, 128, 8, 0.1, dtype, 16, 0.3, 0.05, 4, 8.0)
+    lens = [300, 127, 128, 383]
+    wl = ri.make_workload(spec, device="cuda", seed=331, seq_lens=torch.tensor(lens))
+    pages, pool_pages = spec.cap // 128, 4 * 2 * 3 + 11
+    table = random_block_table(4, 2, pages, pool_pages, seed=11)
+    kp, vp = to_paged(wl.k_cache, pool_pages, table, fill=0.0), to_paged(wl.v_cache, pool_pages, table, fill=0.0)
+    comp = rkv.Compressor(4, 2, 8, spec.budget, spec.buffer, spec.alpha, 0.1, dtype=spec.torch_dtype, block_table=table,
+                          pool_pages=pool_pages)
+    g = torch.Generator(device="cuda").manual_seed(3)
+    k_new = torch.randn(4, 2, 128, generator=g, device="cuda").to(spec.torch_dtype)
+    v_new = torch.randn(4, 2, 128, generator=g, device="cuda").to(spec.torch_dtype)
+    q_new = torch.randn(4, 8, 128, generator=g, device="cuda").to(spec.torch_dtype)
+    seq = wl.seq_lens.clone()
+    assert rkv.rkv_append(comp.desc, kp, vp, k_new, v_new, seq, spec.budget, spec.buffer) == rkv.RKV_OK
+    torch.cuda.synchronize()
+    k_ref, v_ref, s_ref = oracle.oracle_append(raw_rows(wl.k_cache), raw_rows(wl.v_cache), raw_rows(k_new), raw_rows(v_new),
+                                               np.array(lens, dtype=np.int32))
+    assert seq.tolist() == s_ref.tolist() == [301, 128, 129, 384]
+    for b, L in enumerate(s_ref.tolist()):
+        assert np.array_equal(raw_rows(from_paged(kp, table))[b, :, :L], k_ref[b, :, :L])
+        assert np.array_equal(raw_rows(from_paged(vp, table))[b, :, :L], v_ref[b, :, :L])
+    out = torch.empty(4, 8, 128, dtype=torch.float32, device="cuda")
+    assert rkv.rkv_decode_attention(comp.desc, kp, vp, q_new, seq, out, spec.budget, spec.buffer) == rkv.RKV_OK
+    torch.cuda.synchronize()
+    comp.check_status()
+    ref = oracle.oracle_decode_attention(from_paged(kp, table).float().cpu().numpy(), from_paged(vp, table).float().cpu().numpy(),
+                                         q_new.float().cpu().numpy(), seq.cpu().numpy())
+    got = out.cpu().numpy().astype(np.float64)
+    scale = np.maximum(np.abs(ref).max(axis=-1, keepdims=True), 1e-30)
+    assert (np.abs(got - ref) <= 1e-3 * scale + 1e-7).all()

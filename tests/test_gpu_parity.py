@@ -5,7 +5,7 @@ import pytest
 import torch
 
 import rkv_inputs as ri
-from parity_util import check_batch, raw_rows
+from parity_util import check_batch, from_paged, random_block_table, raw_rows, to_paged
 
 pytestmark = pytest.mark.gpu
 
@@ -331,6 +331,58 @@ def test_bounded_wait_runs_out_and_the_context_stays_usable(rkv):
     assert w[5] == 1                                        # the block reached its end
     assert rep.ok(), rep.errors
     comp.check_status()
+
+
+# ----------------------------------------------------------------------------- paged caches
+@pytest.mark.parametrize("flags,dtype", [pytest.param(0, "bf16", id="sym"), pytest.param(1, "bf16", id="simt"),
+                                         pytest.param(2, "bf16", id="rowblock"), pytest.param(0, "f32", id="f32")])
+@pytest.mark.parametrize("budget,buffer,lens", [(384, 128, [512, 500, 384, 390]), (1920, 128, [2048, 2047, 1921, 100])])
+def test_paged_caches(rkv, flags, dtype, budget, buffer, lens):
+    """Paged caches (pages of 128 rows scattered over a pool, in random order, with foreign pages full of NaN in
+    between): the step through the block table gives bit for bit what it gives on contiguous caches, the table is left
+    as it was, pages of other owners are not touched, and the result agrees with the oracle."""
+    spec = small_spec("paged", batch=4, hkv=2, hq=8, budget=budget, buffer=buffer, dtype=dtype, span=32)
+    wl = ri.make_workload(spec, device="cuda", seed=251, seq_lens=torch.tensor(lens))
+    k0, v0, q0, s0 = wl.k_cache.clone(), wl.v_cache.clone(), wl.q_window.clone(), wl.seq_lens.clone()
+    pages = spec.cap // 128
+    pool_pages = 4 * 2 * pages + 37
+    table = random_block_table(4, 2, pages, pool_pages, seed=7)
+    kp, vp = to_paged(k0, pool_pages, table), to_paged(v0, pool_pages, table)
+    kp0 = kp.clone()
+    comp = rkv.Compressor(4, 2, 8, budget, buffer, spec.alpha, spec.lam, dtype=spec.torch_dtype, flags=flags,
+                          dump_scores=True, block_table=table, pool_pages=pool_pages)
+    seq = s0.clone()
+    idx = comp.compress(kp, vp, q0, seq)
+    torch.cuda.synchronize()
+    comp.check_status()
+    assert torch.equal(comp.block_table, table)
+    k1, v1 = from_paged(kp, table), from_paged(vp, table)
+    rep = check_batch(k0, v0, q0, s0, budget=budget, alpha=spec.alpha, lam=spec.lam, gpu_idx=idx, gpu_k=k1, gpu_v=v1,
+                      gpu_seq=seq, gpu_scores=comp.scores, **DEFAULTS)
+    print(rep.summary())
+    assert rep.ok(), rep.errors
+    assert rep.compressed_heads == 2 * sum(L > budget for L in lens)
+    owned = torch.zeros(pool_pages, dtype=torch.bool, device="cuda")
+    owned[table.reshape(-1).long()] = True
+    view = torch.int16 if dtype == "bf16" else torch.int32
+    assert torch.equal(kp[~owned].view(view), kp0[~owned].view(view))          # foreign pages untouched
+    # the same call on the contiguous caches: identical index lists and rows
+    ref = rkv.Compressor(4, 2, 8, budget, buffer, spec.alpha, spec.lam, dtype=spec.torch_dtype, flags=flags)
+    ref_idx = ref.compress(wl.k_cache, wl.v_cache, wl.q_window, wl.seq_lens)
+    torch.cuda.synchronize()
+    assert torch.equal(ref_idx, idx) and torch.equal(wl.seq_lens, seq)
+    for b, L in enumerate(lens):
+        if L > budget:
+            assert torch.equal(k1[b, :, :budget].view(view), wl.k_cache[b, :, :budget].view(view))
+            assert torch.equal(v1[b, :, :budget].view(view), wl.v_cache[b, :, :budget].view(view))
+
+
+def test_paged_caches_need_whole_pages(rkv):
+    d = rkv.rkv_desc_default()
+    d.batch, d.n_kv_heads, d.n_q_heads = 2, 2, 8
+    d.block_table, d.pool_pages = 0x40000, 64
+    assert rkv.rkv_workspace_bytes(d, 256, 64, 8) == 0            # 320 rows: not a multiple of the 128-row page
+    assert rkv.rkv_workspace_bytes(d, 256, 128, 8) > 0
 
 
 # ----------------------------------------------------------------------------- other head dimensions
