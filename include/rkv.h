@@ -74,6 +74,10 @@ typedef enum { RKV_BF16 = 0, RKV_F32 = 1 } rkv_dtype_t;
                                    pooling the paper's appendix ascribes to earlier work); still taken on the scaled
                                    logits, before the one softmax.  Default is the max (Eq. 3). */
 
+#define RKV_FLAG_NO_SYMMETRIC 32u /* never take the symmetric route of the second scoring pass (by default a head in
+                                   which, after the first pass, more than 4/5 of the tokens still lack their partner is
+                                   scored by forming each pair of key tiles once; beta = 1 only).  A cross-check. */
+
 /* stage bits for rkv_compress_stages */
 #define RKV_STAGE_PREP 1u    /* key inverse norms and per-tile sums of normalised keys */
 #define RKV_STAGE_SCORES 2u  /* Eq. 2-3 pooled logits; Eq. 5 matrix + retention rule + Eq. 6 column means */

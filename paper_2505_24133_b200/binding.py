@@ -21,6 +21,7 @@ RKV_FLAG_ROWBLOCK_SCORES = 2
 RKV_FLAG_MEAN_THEN_POOL = 4
 RKV_FLAG_HEAD_MEAN = 8
 RKV_FLAG_GQA_MEAN_POOL = 16
+RKV_FLAG_NO_SYMMETRIC = 32
 RKV_STAGE_PREP, RKV_STAGE_SCORES, RKV_STAGE_SELECT, RKV_STAGE_GATHER, RKV_STAGE_ALL = 1, 2, 4, 8, 15
 
 

@@ -20,7 +20,7 @@ int cuda_fail(cudaError_t e, const char *where)
 }
 
 struct Layout {
-    size_t inv_norm, norm_split, thr_split, tile_sum, head_sum, logits, row_stat, imp, sbar, left, strag, strag_count, strag_items, self_dot, head_sum_bf16, meta, counters,
+    size_t best, dense, dense_items, inv_norm, norm_split, thr_split, tile_sum, head_sum, logits, row_stat, imp, sbar, left, strag, strag_count, strag_items, self_dot, head_sum_bf16, meta, counters,
         tile_done, zero_bytes, total;
     int cap, cap_pad, tiles, tri;
 };
@@ -76,6 +76,9 @@ int check_shapes(const rkv_desc_t *d, int budget, int buffer, int alpha, Layout 
         lay->strag = off;       off = align_up(off + tri * P * lay->cap_pad * sizeof(int32_t), 256);
         lay->strag_count = off; off = align_up(off + tri * P * sizeof(int32_t), 256);
         lay->strag_items = off; off = align_up(off + tri * P * (lay->cap_pad / 256 + 1) * sizeof(int4), 256);
+        lay->best = off;        off = align_up(off + tri * P * lay->cap_pad * sizeof(uint32_t), 256);
+        lay->dense = off;       off = align_up(off + tri * P * sizeof(int32_t), 256);
+        lay->dense_items = off; off = align_up(off + tri * P * ((lay->tiles + 1) / 2) * sizeof(int4), 256);
         lay->self_dot = off;    off = align_up(off + P * lay->cap_pad * sizeof(float), 256);
         lay->head_sum_bf16 = off; off = align_up(off + P * 16 * hd * sizeof(__nv_bfloat16), 256);
         lay->meta = off;        off = align_up(off + 2 * (size_t)d->batch * sizeof(int32_t), 256);
@@ -149,6 +152,10 @@ int run(const rkv_desc_t *d, void *k_cache, void *v_cache, const void *q_window,
     p.strag_count = reinterpret_cast<int32_t *>(ws + lay.strag_count);
     p.strag_items = reinterpret_cast<int4 *>(ws + lay.strag_items);
     p.self_dot = reinterpret_cast<float *>(ws + lay.self_dot);
+    p.best = reinterpret_cast<uint32_t *>(ws + lay.best);
+    p.dense = reinterpret_cast<int32_t *>(ws + lay.dense);
+    p.dense_items = reinterpret_cast<int4 *>(ws + lay.dense_items);
+    p.dense_ok = (d->beta == 1 && !(d->flags & RKV_FLAG_NO_SYMMETRIC)) ? 1 : 0;
     p.head_sum_bf16 = reinterpret_cast<__nv_bfloat16 *>(ws + lay.head_sum_bf16);
     p.meta = reinterpret_cast<int32_t *>(ws + lay.meta);
     p.counters = reinterpret_cast<unsigned long long *>(ws + lay.counters);
@@ -408,7 +415,10 @@ int rkv_launch_count(const rkv_desc_t *desc, uint32_t stage_mask)
     if (desc && (stage_mask & RKV_STAGE_SELECT) && (desc->flags & RKV_FLAG_HEAD_MEAN)) c += 1;   // per-sequence selection
     // the two-pass scoring path is the first pass plus up to three rounds of (listing, second pass) while the
     // retention rule is on
-    if (desc && (stage_mask & RKV_STAGE_SCORES) && use_tri(desc) && desc->beta > 0 && desc->sim_threshold < 1.0f) c += 6;
+    if (desc && (stage_mask & RKV_STAGE_SCORES) && use_tri(desc) && desc->beta > 0 && desc->sim_threshold < 1.0f) {
+        c += 6;
+        if (desc->beta == 1 && !(desc->flags & RKV_FLAG_NO_SYMMETRIC)) c += 2;      // symmetric route: scan and finish
+    }
     return c;
 }
 
@@ -419,8 +429,11 @@ int rkv_launch_count_for(const rkv_desc_t *desc, int32_t budget, int32_t buffer,
     int c = rkv_launch_count(desc, stage_mask);
     if ((stage_mask & RKV_STAGE_SELECT) && select_is_fused(lay.cap_pad, alpha)) c -= 2;
     if ((stage_mask & RKV_STAGE_SCORES) && use_tri(desc) && desc->beta > 0 && desc->sim_threshold < 1.0f)
+    {
         c -= lay.tiles < 2 ? 6                                      // one key tile: the first scoring pass has seen everything
                            : 2 * (3 - scores_pass2_rounds(lay.tiles));   // small caches take fewer rounds
+        if (desc->beta == 1 && !(desc->flags & RKV_FLAG_NO_SYMMETRIC) && !scores_dense_possible(lay.tiles, desc->beta)) c -= 2;
+    }
     return c;
 }
 

@@ -58,6 +58,10 @@ struct Params {
     int32_t *strag_count;// [P]                  tri: how many
     int4 *strag_items;   // [P * cap_pad / 256]  tri: work list of the second scoring pass: {head, first listed
                          //                      token, tokens (1..256), first streamed tile}
+    uint32_t *best;      // [P][cap_pad]         symmetric route: largest partner position + 1 found so far (0 = none)
+    int32_t *dense;      // [P]                  1: the head is scored by the symmetric route of the second pass
+    int4 *dense_items;   // [P * ceil(tiles/2)]  its work list: {head, pair of row tiles, n, -}
+    int dense_ok;        // the symmetric route may be chosen (beta = 1, not switched off)
     float *self_dot;     // [P][cap_pad]         Kbar_i . Kbar_i (1 up to rounding and eps; 0 for a zero key)
     __nv_bfloat16 *head_sum_bf16;   // [P][16][128] head_sum split into three bf16 rows (hi, mid, lo), 13 zero rows
     int32_t *meta;       // [2][batch]           snapshot of seq_lens (kMetaInvalid if out of range), then each
@@ -73,7 +77,8 @@ struct Params {
                                     //           (non-zero once a bounded wait ran out: later kernels of the call
                                     //           then leave the caches, lengths and index lists alone),
                                     //           [5] = listed-token x key-tile pairs the second pass has to form,
-                                    //           [8 + 2 r], [9 + 2 r] = work items and item ticket of its round r
+                                    //           [8 + 2 r], [9 + 2 r] = work items and item ticket of its round r,
+                                    //           [16], [17] = the same for the symmetric route
     uint32_t *tile_done;            // [P]       tiles of the head finished by the prep stage
     size_t zero_bytes;              // bytes from `counters` to the end of `tile_done`
     int tri;                        // 1: the triangle kernels score (bf16 default); 0: another kernel does
@@ -101,6 +106,7 @@ __device__ __forceinline__ void report(int32_t *status, int code)
 
 constexpr int kAbortWord = 4;       // index of the call's abort word in Params::counters
 constexpr int kPairsWord = 5;       // index of the second pass's useful-work count
+constexpr int kDenseWords = 16;     // counters[16], [17]: work items and item ticket of the symmetric route
 
 // Where a bounded wait records that it ran out: the caller's optional status word, and the call's own abort word
 // in the workspace, which the later kernels of the same call read.
@@ -192,6 +198,7 @@ int attend_splits(int heads, int cap, int sms);
 size_t attend_partial_bytes(int heads, int splits, int G);
 bool scores_sm100_available();
 long long sm100_default_wait_cycles();          // default limit of the kernels' bounded waits (about two seconds)
+bool scores_dense_possible(int tiles, int beta);   // the symmetric route of the second pass may be taken (two more launches)
 int scores_pass2_rounds(int tiles);            // list + scan rounds of the second scoring pass for caches of `tiles` key tiles
 bool select_is_fused(int cap_pad, int alpha);   // the select stage is one kernel (small caches) instead of three
 

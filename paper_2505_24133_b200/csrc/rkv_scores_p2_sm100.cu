@@ -508,6 +508,7 @@ scores_pass2_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, c
 
 // ---- before every round: list, per head, the tokens still short of partners, and cut the list into work items ----
 constexpr int kCompactThreads = 256;
+constexpr int kDenseMinTiles = 4;        // caches of fewer key tiles never take the symmetric route
 
 // `below`: key tiles under the first pass's part that earlier rounds have covered; `width`: tiles of this round's
 // window (the last round passes a width that reaches tile 0 whatever the cache size).
@@ -522,9 +523,14 @@ __global__ void __launch_bounds__(kCompactThreads) strag_compact_kernel(Params p
     int32_t *list = p.strag + (size_t)head * p.cap_pad;
     // the first pass scanned every token against the last kPass1Depth key tiles; this round starts `below` tiles
     // under that
-    const int first_tile = (n + kTile - 1) / kTile - kPass1Depth - 1 - below;
-    if (first_tile < 0 || call_aborted(p)) {     // nothing left to scan for this head (or the call has given up)
-        if (threadIdx.x == 0) p.strag_count[head] = 0;
+    const int n_tiles = (n + kTile - 1) / kTile;
+    const int first_tile = n_tiles - kPass1Depth - 1 - below;
+    if (first_tile < 0 || call_aborted(p) || (round > 0 && p.dense[head])) {
+        // nothing left to scan for this head, the call has given up, or the head went to the symmetric route
+        if (threadIdx.x == 0) {
+            p.strag_count[head] = 0;
+            if (round == 0) p.dense[head] = 0;
+        }
         return;
     }
     if (threadIdx.x == 0) running = 0;
@@ -546,6 +552,26 @@ __global__ void __launch_bounds__(kCompactThreads) strag_compact_kernel(Params p
         }
         __syncthreads();
     }
+    if (round == 0) {
+        // Most tokens still lack a partner (few pairs exceed T): the rounds would form nearly the whole matrix for this
+        // head.  It goes to the symmetric route instead, which forms each tile pair once.
+        const bool dense = p.dense_ok && n_tiles >= kDenseMinTiles && 5 * running > 4 * n;
+        if (dense) {
+            uint32_t *best = p.best + (size_t)head * p.cap_pad;
+            for (int i = threadIdx.x; i < p.cap_pad; i += kCompactThreads) best[i] = 0u;
+            if (threadIdx.x == 0) {
+                p.dense[head] = 1;
+                p.strag_count[head] = 0;
+                const int pairs_of_tiles = (n_tiles + 1) / 2;
+                const unsigned long long at = atomicAdd(&p.counters[kDenseWords], (unsigned long long)pairs_of_tiles);
+                for (int q = 0; q < pairs_of_tiles; ++q) p.dense_items[at + q] = make_int4(head, q, n, 0);   // longest first
+                // useful work: every unordered pair of the listed tokens' tiles once
+                atomicAdd(&p.counters[kPairsWord], (unsigned long long)running * (unsigned long long)(n_tiles + 1) / 2ull);
+            }
+            return;
+        }
+        if (threadIdx.x == 0) p.dense[head] = 0;
+    }
     if (threadIdx.x == 0) {
         const int count = running;
         p.strag_count[head] = count;
@@ -565,6 +591,8 @@ __global__ void __launch_bounds__(kCompactThreads) strag_compact_kernel(Params p
 }
 
 }  // namespace
+
+bool scores_dense_possible(int tiles, int beta) { return beta == 1 && tiles >= kDenseMinTiles; }
 
 int scores_pass2_rounds(int tiles)
 {
@@ -601,6 +629,7 @@ cudaError_t launch_scores_tri_sm100(const Params &p, cudaStream_t s)
     // before the long scan down to tile 0
     const int rounds = scores_pass2_rounds(p.tiles);
     static const int kRoundTiles[3] = {4, 8, 1 << 20};
+    const bool dense_possible = p.dense_ok && p.tiles >= kDenseMinTiles;
     int below = 0;
     for (int r = 0; r < rounds; ++r) {
         const int width = r == rounds - 1 ? (1 << 20) : kRoundTiles[r];
@@ -609,9 +638,12 @@ cudaError_t launch_scores_tri_sm100(const Params &p, cudaStream_t s)
         if (r == 0 && (e = mark_kernel(p, 1, s)) != cudaSuccess) return e;
         scores_pass2_sm100_kernel<<<grid2, kThreads, kSmemBytes, s>>>(p, map_k, map_ns, r);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        // the heads the first listing sent to the symmetric route (none on inputs where similar keys are common:
+        // the kernel then returns at once)
+        if (r == 0 && dense_possible && (e = launch_scores_dense_sm100(p, s, map_k, map_ns, sms)) != cudaSuccess) return e;
         below += width;
     }
-    return cudaSuccess;
+    return dense_possible ? launch_dense_finish(p, s) : cudaSuccess;
 }
 
 }  // namespace rkv

@@ -302,4 +302,8 @@ cudaError_t launch_scores_pass1_sm100(const Params &p, cudaStream_t s, const CUt
                                       const CUtensorMap &map_hs, const CUtensorMap &map_ns, const CUtensorMap &map_ts,
                                       int q_rows_pad, int sms);
 
+// symmetric route of the second pass (its own file)
+cudaError_t launch_scores_dense_sm100(const Params &p, cudaStream_t s, const CUtensorMap &map_k, const CUtensorMap &map_ns, int sms);
+cudaError_t launch_dense_finish(const Params &p, cudaStream_t s);
+
 }  // namespace rkv

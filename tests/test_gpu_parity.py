@@ -333,6 +333,34 @@ def test_bounded_wait_runs_out_and_the_context_stays_usable(rkv):
     comp.check_status()
 
 
+# ----------------------------------------------------------------------------- symmetric route of the second pass
+@pytest.mark.parametrize("T", [0.9, 0.75])
+@pytest.mark.parametrize("budget,buffer,lens", [(896, 128, [1024, 1000, 897, 513]), (520, 120, [640, 639, 600, 521])])
+def test_symmetric_route_for_heads_with_few_partners(rkv, T, budget, buffer, lens):
+    """With a high threshold nearly every token is still without a partner after the first pass, and a head is then
+    scored by forming each pair of key tiles once (row and column direction of the same product).  Checked against the
+    oracle and against the same call with that route switched off: same Sbar up to rounding, same kept sets; ragged
+    lengths (5 to 8 key tiles, odd and even counts, a ragged last tile), rows beyond the length filled with NaN."""
+    spec = small_spec("symroute", batch=4, hkv=2, hq=8, budget=budget, buffer=buffer, span=32)
+    wl_a = ri.make_workload(spec, device="cuda", seed=261, seq_lens=torch.tensor(lens))
+    wl_b = ri.make_workload(spec, device="cuda", seed=261, seq_lens=torch.tensor(lens))
+    for wl in (wl_a, wl_b):
+        for b, L in enumerate(lens):
+            wl.k_cache[b, :, L:] = float("nan")
+            wl.v_cache[b, :, L:] = float("nan")
+    rep_a, ca = run_and_check(rkv, wl_a, T=T)
+    rep_b, cb = run_and_check(rkv, wl_b, T=T, flags=rkv.RKV_FLAG_NO_SYMMETRIC)
+    print(rep_a.summary())
+    assert rep_a.ok(), rep_a.errors
+    assert rep_b.ok(), rep_b.errors
+    assert rep_a.compressed_heads == 2 * sum(L > budget for L in lens)
+    ca.check_status()
+    n_max = spec.cap - spec.alpha
+    assert torch.allclose(ca.scores[1, :, :, :n_max], cb.scores[1, :, :, :n_max], rtol=0, atol=2e-6, equal_nan=True)
+    same = (ca.out_idx == cb.out_idx).all(dim=-1).float().mean().item()
+    assert same > 0.7
+
+
 # ----------------------------------------------------------------------------- paged caches
 @pytest.mark.parametrize("flags,dtype", [pytest.param(0, "bf16", id="sym"), pytest.param(1, "bf16", id="simt"),
                                          pytest.param(2, "bf16", id="rowblock"), pytest.param(0, "f32", id="f32")])
@@ -440,7 +468,7 @@ def test_per_sequence_budget_out_of_range_is_reported(rkv):
 
 
 # ----------------------------------------------------------------------------- hard inputs at benchmark sizes
-@pytest.mark.parametrize("flags", [pytest.param(0, id="sym"), pytest.param(2, id="rowblock")])
+@pytest.mark.parametrize("flags", [pytest.param(0, id="sym"), pytest.param(32, id="rounds_only"), pytest.param(2, id="rowblock")])
 @pytest.mark.parametrize("T,beta,budget", [(0.9, 1, 2048), (0.5, 8, 2048), (1.0, 1, 2048), (0.5, 400, 2048),
                                            (0.9, 1, 4096), (0.5, 8, 4096)])
 def test_hard_retention_settings_at_benchmark_sizes(rkv, flags, T, beta, budget):
@@ -548,4 +576,4 @@ def test_kernel_events_and_executed_tile_counter(rkv):
     heads, T = spec.head_problems, -(-(spec.cap - spec.alpha) // 128)
     tiles = int(comp.counters[0].item())
     assert heads * T <= tiles <= heads * T * T
-    assert rkv.rkv_launch_count_for(comp.desc, spec.budget, spec.buffer, spec.alpha, rkv.RKV_STAGE_ALL) == 6
+    assert rkv.rkv_launch_count_for(comp.desc, spec.budget, spec.buffer, spec.alpha, rkv.RKV_STAGE_ALL) == 8
