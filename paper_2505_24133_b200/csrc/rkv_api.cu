@@ -413,10 +413,10 @@ int rkv_launch_count(const rkv_desc_t *desc, uint32_t stage_mask)
     for (uint32_t bit = 1; bit <= RKV_STAGE_GATHER; bit <<= 1) c += (stage_mask & bit) ? 1 : 0;
     if (stage_mask & RKV_STAGE_SELECT) c += 2;      // row statistics and importance run ahead of the selection kernel
     if (desc && (stage_mask & RKV_STAGE_SELECT) && (desc->flags & RKV_FLAG_HEAD_MEAN)) c += 1;   // per-sequence selection
-    // the two-pass scoring path is the first pass plus up to three rounds of (listing, second pass) while the
+    // the two-pass scoring path is the first pass plus up to two rounds of (listing, second pass) while the
     // retention rule is on
     if (desc && (stage_mask & RKV_STAGE_SCORES) && use_tri(desc) && desc->beta > 0 && desc->sim_threshold < 1.0f) {
-        c += 6;
+        c += 4;
         if (desc->beta == 1 && !(desc->flags & RKV_FLAG_NO_SYMMETRIC)) c += 2;      // symmetric route: scan and finish
     }
     return c;
@@ -430,8 +430,8 @@ int rkv_launch_count_for(const rkv_desc_t *desc, int32_t budget, int32_t buffer,
     if ((stage_mask & RKV_STAGE_SELECT) && select_is_fused(lay.cap_pad, alpha)) c -= 2;
     if ((stage_mask & RKV_STAGE_SCORES) && use_tri(desc) && desc->beta > 0 && desc->sim_threshold < 1.0f)
     {
-        c -= lay.tiles < 2 ? 6                                      // one key tile: the first scoring pass has seen everything
-                           : 2 * (3 - scores_pass2_rounds(lay.tiles));   // small caches take fewer rounds
+        c -= lay.tiles < 2 ? 4                                      // one key tile: the first scoring pass has seen everything
+                           : 2 * (2 - scores_pass2_rounds(lay.tiles));   // small caches take one round
         if (desc->beta == 1 && !(desc->flags & RKV_FLAG_NO_SYMMETRIC) && !scores_dense_possible(lay.tiles, desc->beta)) c -= 2;
     }
     return c;

@@ -12,7 +12,7 @@
 //           into two resident operand tiles by the epilogue warps; the window's key tiles stream through a ring, last
 //           to first.  The removed entries are subtracted from what the first pass stored, `left` is updated.
 //
-// A round's window is a few tiles only (kRoundTiles); the tokens that found their partners in it drop out of the next
+// The first round's window is a few tiles only (kRoundTiles); the tokens that found their partners in it drop out of the next
 // round's list, so the long scan down to tile 0 is paid only by the few tokens that have no partner at all (a
 // single-round scan would drag every listed token of a chunk along with them).  The last round's window reaches
 // tile 0.  Worst case (no pair above T): the rounds together form the whole matrix below the last tile.
@@ -597,7 +597,7 @@ bool scores_dense_possible(int tiles, int beta) { return beta == 1 && tiles >= k
 int scores_pass2_rounds(int tiles)
 {
     const int below = tiles - kPass1Depth;      // key tiles under the first pass's part, at most
-    return below <= 8 ? 1 : (below <= 16 ? 2 : 3);
+    return below <= 8 ? 1 : 2;
 }
 
 cudaError_t launch_scores_tri_sm100(const Params &p, cudaStream_t s)
@@ -628,7 +628,7 @@ cudaError_t launch_scores_tri_sm100(const Params &p, cudaStream_t s)
     // rounds of the second pass: short windows first, so that the tokens that find their partners soon drop out
     // before the long scan down to tile 0
     const int rounds = scores_pass2_rounds(p.tiles);
-    static const int kRoundTiles[3] = {4, 8, 1 << 20};
+    static const int kRoundTiles[2] = {6, 1 << 20};      // (measured: 6 + rest beats 4 + 8 + rest and 8 + rest by a little)
     const bool dense_possible = p.dense_ok && p.tiles >= kDenseMinTiles;
     int below = 0;
     for (int r = 0; r < rounds; ++r) {
