@@ -412,6 +412,8 @@ int rkv_launch_count(const rkv_desc_t *desc, uint32_t stage_mask)
     int c = 0;
     for (uint32_t bit = 1; bit <= RKV_STAGE_GATHER; bit <<= 1) c += (stage_mask & bit) ? 1 : 0;
     if (stage_mask & RKV_STAGE_SELECT) c += 2;      // row statistics and importance run ahead of the selection kernel
+    // bf16 keys of 128 dimensions: the tile sums are added up per head by a kernel of its own behind the prep kernel
+    if (desc && (stage_mask & RKV_STAGE_PREP) && desc->dtype == RKV_BF16 && (desc->head_dim == 0 || desc->head_dim == kHeadDim)) c += 1;
     if (desc && (stage_mask & RKV_STAGE_SELECT) && (desc->flags & RKV_FLAG_HEAD_MEAN)) c += 1;   // per-sequence selection
     // the two-pass scoring path is the first pass plus up to two rounds of (listing, second pass) while the
     // retention rule is on

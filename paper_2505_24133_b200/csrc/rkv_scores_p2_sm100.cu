@@ -508,7 +508,7 @@ scores_pass2_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, c
 
 // ---- before every round: list, per head, the tokens still short of partners, and cut the list into work items ----
 constexpr int kCompactThreads = 256;
-constexpr int kDenseMinTiles = 4;        // caches of fewer key tiles never take the symmetric route
+constexpr int kDenseMinTiles = 12;       // caches of fewer key tiles never take the symmetric route (two more launches)
 
 // `below`: key tiles under the first pass's part that earlier rounds have covered; `width`: tiles of this round's
 // window (the last round passes a width that reaches tile 0 whatever the cache size).

@@ -112,17 +112,16 @@ def test_rkv_compress_needs_a_current_descriptor(rkv):
     t.join()
     assert out["rc"] == 1
     assert rkv.rkv_status_string(5) == "RKV_ERR_TIMEOUT"
-    assert rkv.rkv_launch_count(_desc(rkv), rkv.RKV_STAGE_ALL) == 12     # prep, first pass + 2 x (list, scan), symmetric scan + finish, 3 select kernels, gather
-    assert rkv.rkv_launch_count(_desc(rkv, flags=rkv.RKV_FLAG_NO_SYMMETRIC), rkv.RKV_STAGE_ALL) == 10
-    assert rkv.rkv_launch_count(_desc(rkv, flags=rkv.RKV_FLAG_SIMT_SCORES), rkv.RKV_STAGE_ALL) == 6
+    assert rkv.rkv_launch_count(_desc(rkv), rkv.RKV_STAGE_ALL) == 13     # prep + head sums, first pass + 2 x (list, scan), symmetric scan + finish, 3 select kernels, gather
+    assert rkv.rkv_launch_count(_desc(rkv, flags=rkv.RKV_FLAG_NO_SYMMETRIC), rkv.RKV_STAGE_ALL) == 11
+    assert rkv.rkv_launch_count(_desc(rkv, flags=rkv.RKV_FLAG_SIMT_SCORES), rkv.RKV_STAGE_ALL) == 7
     # exact counts for given sizes: small caches run the select stage as one kernel
-    assert rkv.rkv_launch_count_for(_desc(rkv), 4096, 128, 8, rkv.RKV_STAGE_ALL) == 12
-    assert rkv.rkv_launch_count_for(_desc(rkv), 2048, 128, 8, rkv.RKV_STAGE_ALL) == 12         # 17 key tiles: two rounds as well
-    assert rkv.rkv_launch_count_for(_desc(rkv), 1024, 128, 8, rkv.RKV_STAGE_ALL) == 8
-    assert rkv.rkv_launch_count_for(_desc(rkv), 256, 64, 8, rkv.RKV_STAGE_ALL) == 6            # 3 key tiles: no symmetric route
-    assert rkv.rkv_launch_count_for(_desc(rkv), 64, 32, 8, rkv.RKV_STAGE_ALL) == 4          # one key tile: no second pass
+    assert rkv.rkv_launch_count_for(_desc(rkv), 4096, 128, 8, rkv.RKV_STAGE_ALL) == 13
+    assert rkv.rkv_launch_count_for(_desc(rkv), 2048, 128, 8, rkv.RKV_STAGE_ALL) == 13         # 17 key tiles: two rounds as well
+    assert rkv.rkv_launch_count_for(_desc(rkv), 1024, 128, 8, rkv.RKV_STAGE_ALL) == 7          # 9 key tiles: no symmetric route
+    assert rkv.rkv_launch_count_for(_desc(rkv), 64, 32, 8, rkv.RKV_STAGE_ALL) == 5          # one key tile: no second pass
     assert rkv.rkv_launch_count_for(_desc(rkv), 8, 128, 8, rkv.RKV_STAGE_ALL) == 0           # invalid sizes
-    assert rkv.rkv_launch_count_for(_desc(rkv, flags=rkv.RKV_FLAG_HEAD_MEAN), 1024, 128, 8, rkv.RKV_STAGE_ALL) == 9
+    assert rkv.rkv_launch_count_for(_desc(rkv, flags=rkv.RKV_FLAG_HEAD_MEAN), 1024, 128, 8, rkv.RKV_STAGE_ALL) == 8
 
 
 def test_product_package_does_not_touch_the_oracle():

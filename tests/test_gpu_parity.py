@@ -335,12 +335,12 @@ def test_bounded_wait_runs_out_and_the_context_stays_usable(rkv):
 
 # ----------------------------------------------------------------------------- symmetric route of the second pass
 @pytest.mark.parametrize("T", [0.9, 0.75])
-@pytest.mark.parametrize("budget,buffer,lens", [(896, 128, [1024, 1000, 897, 513]), (520, 120, [640, 639, 600, 521])])
+@pytest.mark.parametrize("budget,buffer,lens", [(1536, 128, [1664, 1640, 1537, 513]), (1500, 120, [1620, 1619, 1580, 1501])])
 def test_symmetric_route_for_heads_with_few_partners(rkv, T, budget, buffer, lens):
     """With a high threshold nearly every token is still without a partner after the first pass, and a head is then
     scored by forming each pair of key tiles once (row and column direction of the same product).  Checked against the
     oracle and against the same call with that route switched off: same Sbar up to rounding, same kept sets; ragged
-    lengths (5 to 8 key tiles, odd and even counts, a ragged last tile), rows beyond the length filled with NaN."""
+    lengths (12 and 13 key tiles, odd and even counts, ragged last tiles), rows beyond the length filled with NaN."""
     spec = small_spec("symroute", batch=4, hkv=2, hq=8, budget=budget, buffer=buffer, span=32)
     wl_a = ri.make_workload(spec, device="cuda", seed=261, seq_lens=torch.tensor(lens))
     wl_b = ri.make_workload(spec, device="cuda", seed=261, seq_lens=torch.tensor(lens))
@@ -576,4 +576,4 @@ def test_kernel_events_and_executed_tile_counter(rkv):
     heads, T = spec.head_problems, -(-(spec.cap - spec.alpha) // 128)
     tiles = int(comp.counters[0].item())
     assert heads * T <= tiles <= heads * T * T
-    assert rkv.rkv_launch_count_for(comp.desc, spec.budget, spec.buffer, spec.alpha, rkv.RKV_STAGE_ALL) == 8
+    assert rkv.rkv_launch_count_for(comp.desc, spec.budget, spec.buffer, spec.alpha, rkv.RKV_STAGE_ALL) == 7
