@@ -2,7 +2,8 @@
 
 Marshals numpy arrays into the C oracle and back; it holds no arithmetic of the
 method.  Keys and queries are handed over as float32 (bf16 widens to float32
-exactly); the C side computes in double (Eq. 1-7, Algorithm 1).
+exactly, and so does an 8-bit E4M3 cache byte, decoded by ``e4m3_to_f32`` below);
+the C side computes in double (Eq. 1-7, Algorithm 1).
 """
 from __future__ import annotations
 
@@ -183,6 +184,24 @@ def oracle_decode_attention(K, V, q_new, seq_lens) -> np.ndarray:
     if rc != 0:
         raise ValueError("rkv_oracle_decode_attention: bad arguments")
     return out
+
+
+def e4m3_to_f32(codes) -> np.ndarray:
+    """Value of every 8-bit E4M3 code (the "fn" variant of the OCP 8-bit floating point format: 1 sign bit, 4 exponent
+    bits with bias 7, 3 mantissa bits; no infinities; exponent 15 with mantissa 7 is NaN; largest finite value 448).
+    An 8-bit cache holds such codes; the method (Eq. 1-7) is defined on the values they stand for, which float32
+    represents exactly.
+
+        exponent field e = 0:   (m / 8) * 2^-6          (subnormal)
+        otherwise:              (1 + m / 8) * 2^(e - 7)
+    """
+    c = np.asarray(codes, dtype=np.uint8)
+    sign = np.where(c & 0x80, -1.0, 1.0)
+    e = ((c >> 3) & 0xF).astype(np.int32)
+    m = (c & 0x7).astype(np.float64)
+    val = np.where(e == 0, np.ldexp(m / 8.0, -6), np.ldexp(1.0 + m / 8.0, e - 7))
+    val = np.where((e == 15) & (m == 7), np.nan, val)
+    return (sign * val).astype(np.float32)
 
 
 def oracle_gather(rows: np.ndarray, idx: np.ndarray) -> np.ndarray:

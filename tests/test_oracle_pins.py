@@ -630,3 +630,40 @@ def test_per_sequence_budgets_equal_independent_calls():
     kept = res.idx[1, 0, :24]
     assert np.all(np.diff(kept) > 0) and np.array_equal(kept[-alpha:], np.arange(46, 50))    # 24 kept, observation tail
     assert np.array_equal(res.idx[2, 0, :33], np.arange(33))                                 # L = budget: the guard
+
+
+# ----------------------------------------------------------------------------- 8-bit (E4M3) cache codes
+def test_e4m3_decode_against_the_format_and_the_library_cast():
+    """An 8-bit cache holds E4M3 codes; the oracle scores the values they stand for.  The decode is pinned to the
+    format's own landmarks (1.0, the largest finite value 448, the smallest subnormal 2^-9, the smallest normal 2^-6,
+    the NaN code), to the library's cast for all 256 codes, and to the ordering of the positive codes."""
+    import torch
+    vals = oracle.e4m3_to_f32(np.arange(256, dtype=np.uint8))
+    assert vals[0x00] == 0.0 and vals[0x80] == 0.0 and np.signbit(vals[0x80])
+    assert vals[0x38] == 1.0 and vals[0xB8] == -1.0 and vals[0x40] == 2.0 and vals[0x3C] == 1.5
+    assert vals[0x7E] == 448.0 and vals[0x01] == 2.0 ** -9 and vals[0x07] == 7 * 2.0 ** -9 and vals[0x08] == 2.0 ** -6
+    assert np.isnan(vals[0x7F]) and np.isnan(vals[0xFF])
+    lib = torch.arange(256, dtype=torch.uint8).view(torch.float8_e4m3fn).to(torch.float32).numpy()
+    finite = ~np.isnan(lib)
+    assert np.array_equal(np.isnan(vals), np.isnan(lib))
+    assert np.array_equal(vals[finite].view(np.uint32), lib[finite].view(np.uint32))       # bit for bit, -0 included
+    assert np.all(np.diff(vals[:0x7F]) > 0)           # positive codes are ordered like their values
+
+
+def test_e4m3_cache_scores_are_the_scores_of_the_decoded_values():
+    """Nothing of Eq. 1-7 changes for an 8-bit cache: the head result on codes decoded by the oracle equals the
+    result on the same values given as float32 by the library's cast, and the kept rows are moved as bytes."""
+    import torch
+    rng = np.random.default_rng(77)
+    L, alpha, budget = 96, 8, 40
+    K32 = _rand(rng, L, D)
+    codes = torch.from_numpy(K32).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    Kd = oracle.e4m3_to_f32(codes)
+    Kl = torch.from_numpy(codes).view(torch.float8_e4m3fn).to(torch.float32).numpy()
+    Q = _rand(rng, 2, alpha, D)
+    a, b = _run(Kd, Q, budget=budget, alpha=alpha), _run(Kl, Q, budget=budget, alpha=alpha)
+    assert np.array_equal(a.idx, b.idx) and np.array_equal(a.Z, b.Z)
+    moved = oracle.oracle_gather(codes, a.idx)
+    assert moved.dtype == np.uint8 and np.array_equal(moved, codes[a.idx])
+    # quantisation is not a no-op on these inputs: the 8-bit values differ from the float32 ones they came from
+    assert np.abs(Kd - K32).max() > 1e-3
