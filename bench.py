@@ -373,7 +373,9 @@ def kernel_table(rkv, timed: Timed, kw, KB, peaks):
     pass2_useful = pairs2 * 2.0 * 128 * (128 + 16)     # listed tokens x keys of the streamed tiles x 2 (d + 16)
     # algorithmic work per launch: bytes a kernel has to move / flops it has to execute, nothing it merely could
     work = {
-        "prep": ("hbm", P * (n * row + spec.cap * (8 + 32))),                   # K once; r_i, Kbar_i.Kbar_i and the 32-byte slice out
+        # K once; r_i, Kbar_i.Kbar_i and the 32-byte slice out.  8-bit caches: the codes in, their bf16 copy out and in again
+        "prep": ("hbm", P * (n * row + spec.cap * (8 + 32)) if esz > 1 else
+                 P * (spec.cap * row + spec.cap * 2 * row + n * 2 * row + spec.cap * (8 + 32))),
         "scores_pass1": ("tensor", pass1_flops),
         "scores_list": ("hbm", P * n * 8),
         "scores_pass2": ("tensor", pass2_flops),
@@ -499,11 +501,15 @@ def measure_attention(rkv, dev, wl, peaks, reps=5):
     spec = wl.spec
     d = rkv.rkv_desc_default()
     d.batch, d.n_kv_heads, d.n_q_heads = spec.folded_batch, spec.n_kv_heads, spec.n_q_heads
+    d.head_dim = spec.head_dim
+    d.dtype = {"bf16": rkv.RKV_BF16, "f32": rkv.RKV_F32, "fp8": rkv.RKV_FP8_E4M3}[spec.dtype]    # the caches are read as this type
     need = rkv.rkv_decode_workspace_bytes(d, spec.budget, spec.buffer)
+    if need == 0:
+        return {"unsupported": "rkv_decode_attention does not take this cache type or shape"}
     ws = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
     d.workspace, d.workspace_bytes = ws.data_ptr(), ws.numel()
     gen = torch.Generator(device=dev).manual_seed(ri.BASE_SEED + 99)
-    q_new = torch.randn(spec.folded_batch, spec.n_q_heads, spec.head_dim, generator=gen, device=dev).to(spec.torch_dtype)
+    q_new = torch.randn(spec.folded_batch, spec.n_q_heads, spec.head_dim, generator=gen, device=dev).to(spec.query_dtype)
     out = torch.empty(spec.folded_batch, spec.n_q_heads, spec.head_dim, dtype=torch.float32, device=dev)
     stream = torch.cuda.current_stream()
     flush = torch.empty(256 * 2 ** 20, dtype=torch.uint8, device=dev)
@@ -606,7 +612,7 @@ def main():
     # ---- the other configurations, and the settings that defeat the two-pass shortcut, in the same run
     configs = {}
     if not args.no_configs and args.workload == DEFAULT_WORKLOAD and args.batch is None and args.layers is None and not kw:
-        for name, k_side in (("llama8b_b1", 20), ("llama8b_b16", 5), ("qwen7b_b64", 5), ("mha7b_b8", 5)):
+        for name, k_side in (("llama8b_b1", 20), ("llama8b_b16", 5), ("qwen7b_b64", 5), ("mha7b_b8", 5), ("llama8b_b16_fp8", 5)):
             swl = ri.make_workload(ri.SPECS[name], device=dev, seed=ri.BASE_SEED + 1000 * rank + list(ri.SPECS).index(name))
             configs[name] = side_config(rkv, rd, dev, swl, {}, k_side, 3, args.mem_gb, peaks)
             if name == "llama8b_b16":

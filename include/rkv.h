@@ -53,7 +53,16 @@ typedef enum {
     RKV_ERR_TIMEOUT = 5      /* device status only: a bounded wait inside a kernel ran out */
 } rkv_status_t;
 
-typedef enum { RKV_BF16 = 0, RKV_F32 = 1 } rkv_dtype_t;
+/* Element type of the caches.
+ *   RKV_BF16, RKV_F32: k_cache, v_cache and q_window all hold that type.
+ *   RKV_FP8_E4M3: k_cache and v_cache hold 8-bit E4M3 codes (1 sign bit, 4 exponent bits with bias 7, 3 mantissa bits,
+ *     no infinities; one byte per element, rows of head_dim bytes); q_window (and q_new of rkv_push_query) is bf16.
+ *     Eq. 1-7 are evaluated on the values the codes stand for: the keys are widened to bf16 (exactly; every E4M3 value
+ *     is a bf16 value) into the workspace, which grows by (batch * n_kv_heads * (budget + buffer) + 128) * head_dim * 2
+ *     bytes, and every scoring stage runs on that copy as for a bf16 cache.  The compaction moves the stored bytes; no
+ *     scale factor is applied or needed (cosine similarity does not see a per-tensor scale; fold a key scale into
+ *     the queries for Eq. 2).  rkv_decode_attention does not take this type (RKV_ERR_UNSUPPORTED). */
+typedef enum { RKV_BF16 = 0, RKV_F32 = 1, RKV_FP8_E4M3 = 2 } rkv_dtype_t;
 
 /* rkv_desc_t.flags */
 #define RKV_FLAG_SIMT_SCORES 1u /* score with the plain fp32 CUDA-core kernel instead of the tcgen05
@@ -98,7 +107,7 @@ typedef struct rkv_desc {
     int32_t n_q_heads;   /* query heads; G = n_q_heads / n_kv_heads must be integral (G = 1: Eq. 1) */
     int32_t head_dim;    /* d: 64, 128 or 256.  The tensor-core scoring kernels serve bf16 caches with d = 128; other
                             head dimensions are scored by the CUDA-core kernel (correct, but far slower) */
-    int32_t dtype;       /* rkv_dtype_t of k_cache, v_cache and q_window */
+    int32_t dtype;       /* rkv_dtype_t of k_cache and v_cache (and of q_window, except for 8-bit caches: bf16) */
     int32_t pool_w;      /* W of Eq. 4; 0 = no pooling.  Range [0, 64].  Default 4 (the paper prints no value) */
     int32_t beta;        /* beta of Section 3.3; 0 = rule off.  Default 1 (the paper prints no value) */
     float sim_threshold; /* T of Section 3.3, in [0, 1].  Default 0.5 (the paper prints no value) */

@@ -15,7 +15,7 @@ _LIB_PATH = os.path.join(_PKG, "librkv_b200.so")
 _lib = None
 
 RKV_OK = 0
-RKV_BF16, RKV_F32 = 0, 1
+RKV_BF16, RKV_F32, RKV_FP8_E4M3 = 0, 1, 2
 RKV_FLAG_SIMT_SCORES = 1
 RKV_FLAG_ROWBLOCK_SCORES = 2
 RKV_FLAG_MEAN_THEN_POOL = 4
@@ -212,9 +212,9 @@ class Compressor:
         d = rkv_desc_default()
         d.batch, d.n_kv_heads, d.n_q_heads = batch, n_kv_heads, n_q_heads
         d.head_dim = head_dim
-        d.dtype = RKV_BF16 if dtype == torch.bfloat16 else RKV_F32
-        if dtype not in (torch.bfloat16, torch.float32):
-            raise ValueError("dtype must be bfloat16 or float32")
+        if dtype not in (torch.bfloat16, torch.float32, torch.float8_e4m3fn):
+            raise ValueError("dtype must be bfloat16, float32 or float8_e4m3fn")
+        d.dtype = {torch.bfloat16: RKV_BF16, torch.float32: RKV_F32, torch.float8_e4m3fn: RKV_FP8_E4M3}[dtype]
         if pool_w is not None:
             d.pool_w = pool_w
         if beta is not None:

@@ -20,13 +20,18 @@ int cuda_fail(cudaError_t e, const char *where)
 }
 
 struct Layout {
-    size_t best, dense, dense_items, inv_norm, norm_split, thr_split, tile_sum, head_sum, logits, row_stat, imp, sbar, left, strag, strag_count, strag_items, self_dot, head_sum_bf16, meta, counters,
+    size_t k_wide, best, dense, dense_items, inv_norm, norm_split, thr_split, tile_sum, head_sum, logits, row_stat, imp, sbar, left, strag, strag_count, strag_items, self_dot, head_sum_bf16, meta, counters,
         tile_done, zero_bytes, total;
     int cap, cap_pad, tiles, tri;
 };
 
 // The tensor-core scoring kernels serve bf16 caches with head dimension 128; everything else (fp32 caches, head
 // dimensions 64 and 256, or on request) is scored by the CUDA-core kernel.
+// Bytes of a cache element and of a query element.  8-bit caches (E4M3 codes) are scored on a bf16 copy of their keys
+// in the workspace (every E4M3 value is a bf16 value), with bf16 queries.
+size_t cache_esz(const rkv_desc_t *d) { return d->dtype == RKV_BF16 ? 2 : d->dtype == RKV_F32 ? 4 : 1; }
+size_t query_esz(const rkv_desc_t *d) { return d->dtype == RKV_F32 ? 4 : 2; }
+
 bool use_simt(const rkv_desc_t *d)
 {
     return d->dtype == RKV_F32 || d->head_dim != kHeadDim || (d->flags & RKV_FLAG_SIMT_SCORES);
@@ -45,7 +50,7 @@ int check_shapes(const rkv_desc_t *d, int budget, int buffer, int alpha, Layout 
     if (d->pool_w < 0 || d->pool_w > 64 || d->beta < 0) return RKV_ERR_INVALID_ARG;
     if (!(d->sim_threshold >= 0.f && d->sim_threshold <= 1.f) || !(d->eps >= 0.f)) return RKV_ERR_INVALID_ARG;
     if (d->head_dim != 64 && d->head_dim != 128 && d->head_dim != 256) return RKV_ERR_UNSUPPORTED;
-    if (d->dtype != RKV_BF16 && d->dtype != RKV_F32) return RKV_ERR_UNSUPPORTED;
+    if (d->dtype != RKV_BF16 && d->dtype != RKV_F32 && d->dtype != RKV_FP8_E4M3) return RKV_ERR_UNSUPPORTED;
     const long long cap = (long long)budget + buffer;
     if (cap > RKV_MAX_CAP) return RKV_ERR_UNSUPPORTED;
     if ((long long)(d->n_q_heads / d->n_kv_heads) * alpha > RKV_MAX_GROUP_ROWS) return RKV_ERR_UNSUPPORTED;
@@ -60,6 +65,9 @@ int check_shapes(const rkv_desc_t *d, int budget, int buffer, int alpha, Layout 
         lay->tiles = (int)((cap + kTile - 1) / kTile);
         lay->cap_pad = lay->tiles * kTile;
         size_t off = 0;
+        // 8-bit caches: the keys widened to bf16, head after head, plus one tile of zero rows behind the last head
+        lay->k_wide = off;
+        if (d->dtype == RKV_FP8_E4M3) off = align_up(off + (P * lay->cap + kTile) * (size_t)d->head_dim * sizeof(__nv_bfloat16), 256);
         lay->inv_norm = off;  off = align_up(off + P * lay->cap_pad * sizeof(float), 256);
         lay->norm_split = off;  off = align_up(off + P * lay->cap_pad * 16 * sizeof(__nv_bfloat16), 256);
         lay->thr_split = off;   off = align_up(off + P * kTile * 16 * sizeof(__nv_bfloat16), 256);
@@ -129,6 +137,7 @@ int run(const rkv_desc_t *d, void *k_cache, void *v_cache, const void *q_window,
     p.buffer = buffer;
     p.alpha = alpha;
     p.dtype = d->dtype;
+    p.store_row_bytes = (int)(d->head_dim * cache_esz(d));
     p.pool_w = d->pool_w;
     p.beta = d->beta;
     p.mean_then_pool = (d->flags & RKV_FLAG_MEAN_THEN_POOL) ? 1 : 0;
@@ -182,8 +191,19 @@ int run(const rkv_desc_t *d, void *k_cache, void *v_cache, const void *q_window,
         return ev && ev[i] ? cudaEventRecord(static_cast<cudaEvent_t>(ev[i]), s) : cudaSuccess;
     };
     if ((e = mark(0)) != cudaSuccess) return cuda_fail(e, "cudaEventRecord");
+    // What the gather moves is the caller's caches as they are stored; for 8-bit caches every stage before it reads the
+    // bf16 copy of the keys (contiguous: the block table, if any, is followed once, by the widening kernel).
+    Params stored = p;
+    if (d->dtype == RKV_FP8_E4M3) {
+        p.k_cache = ws + lay.k_wide;
+        p.block_table = nullptr;
+        p.dtype = RKV_BF16;
+    }
     if (stages & RKV_STAGE_PREP) {
         if ((e = cudaMemsetAsync(p.counters, 0, p.zero_bytes, s)) != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
+        if (d->dtype == RKV_FP8_E4M3 &&
+            (e = launch_widen_keys(stored, static_cast<__nv_bfloat16 *>(p.k_cache), s)) != cudaSuccess)
+            return cuda_fail(e, "widen launch");
         if ((e = launch_prep(p, s)) != cudaSuccess) return cuda_fail(e, "prep launch");
     }
     if ((e = mark(1)) != cudaSuccess) return cuda_fail(e, "cudaEventRecord");
@@ -203,7 +223,7 @@ int run(const rkv_desc_t *d, void *k_cache, void *v_cache, const void *q_window,
         if ((e = launch_select(p, s)) != cudaSuccess) return cuda_fail(e, "select launch");
     if ((e = mark(3)) != cudaSuccess) return cuda_fail(e, "cudaEventRecord");
     if (stages & RKV_STAGE_GATHER)
-        if ((e = launch_gather(p, s)) != cudaSuccess) return cuda_fail(e, "gather launch");
+        if ((e = launch_gather(stored, s)) != cudaSuccess) return cuda_fail(e, "gather launch");
     if ((e = mark(4)) != cudaSuccess) return cuda_fail(e, "cudaEventRecord");
     return RKV_OK;
 }
@@ -218,11 +238,10 @@ int host_layout(const rkv_desc_t *d, int budget, int buffer, int alpha, HostLayo
     Layout lay;
     int rc = check_shapes(d, budget, buffer, alpha, &lay);
     if (rc != RKV_OK) return rc;
-    const size_t esz = d->dtype == RKV_BF16 ? 2 : 4;
     const size_t P = (size_t)d->batch * d->n_kv_heads;
-    h->row_bytes = (size_t)d->head_dim * esz;
+    h->row_bytes = (size_t)d->head_dim * cache_esz(d);
     h->kv_bytes = P * lay.cap * h->row_bytes;
-    h->q_bytes = (size_t)d->batch * d->n_q_heads * alpha * h->row_bytes;
+    h->q_bytes = (size_t)d->batch * d->n_q_heads * alpha * d->head_dim * query_esz(d);
     h->seq_bytes = (size_t)d->batch * sizeof(int32_t);
     h->idx_bytes = P * budget * sizeof(int32_t);
     size_t off = 0;
@@ -347,7 +366,7 @@ int rkv_append(const rkv_desc_t *d, void *k_cache, void *v_cache, const void *k_
     if (!k_cache || !v_cache || !k_new || !v_new || !seq_lens) return RKV_ERR_INVALID_ARG;
     if (!aligned16(k_cache) || !aligned16(v_cache) || !aligned16(k_new) || !aligned16(v_new)) return RKV_ERR_INVALID_ARG;
     if (reinterpret_cast<uintptr_t>(seq_lens) & 3u) return RKV_ERR_INVALID_ARG;
-    const int row_bytes = d->head_dim * (d->dtype == RKV_BF16 ? 2 : 4);
+    const int row_bytes = (int)(d->head_dim * cache_esz(d));
     const cudaError_t e = launch_append(k_cache, v_cache, k_new, v_new, seq_lens, d->batch, d->n_kv_heads, budget + buffer,
                                         row_bytes, d->device_status, d->block_table, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? RKV_OK : cuda_fail(e, "append launch");
@@ -359,7 +378,7 @@ int rkv_push_query(const rkv_desc_t *d, void *q_window, const void *q_new, int32
     int rc = check_shapes(d, alpha + 1, 1, alpha, nullptr);        // descriptor fields and alpha against the group limit
     if (rc != RKV_OK) return rc;
     if (!q_window || !q_new || !aligned16(q_window) || !aligned16(q_new)) return RKV_ERR_INVALID_ARG;
-    const int row_bytes = d->head_dim * (d->dtype == RKV_BF16 ? 2 : 4);
+    const int row_bytes = (int)(d->head_dim * query_esz(d));
     const cudaError_t e = launch_push_query(q_window, q_new, d->batch, d->n_q_heads, alpha, slot, row_bytes,
                                             static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? RKV_OK : cuda_fail(e, "push_query launch");
@@ -370,7 +389,7 @@ static int attend_plan(const rkv_desc_t *d, int32_t budget, int32_t buffer, int 
     int rc = check_shapes(d, budget, buffer, 1, nullptr);
     if (rc != RKV_OK) return rc;
     const int G = d->n_q_heads / d->n_kv_heads;
-    if (G > attend_max_group() || d->head_dim != kHeadDim) return RKV_ERR_UNSUPPORTED;
+    if (G > attend_max_group() || d->head_dim != kHeadDim || d->dtype == RKV_FP8_E4M3) return RKV_ERR_UNSUPPORTED;
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
         sms = 148;       // sizing only (no device here): the B200's count
@@ -413,7 +432,8 @@ int rkv_launch_count(const rkv_desc_t *desc, uint32_t stage_mask)
     for (uint32_t bit = 1; bit <= RKV_STAGE_GATHER; bit <<= 1) c += (stage_mask & bit) ? 1 : 0;
     if (stage_mask & RKV_STAGE_SELECT) c += 2;      // row statistics and importance run ahead of the selection kernel
     // bf16 keys of 128 dimensions: the tile sums are added up per head by a kernel of its own behind the prep kernel
-    if (desc && (stage_mask & RKV_STAGE_PREP) && desc->dtype == RKV_BF16 && (desc->head_dim == 0 || desc->head_dim == kHeadDim)) c += 1;
+    if (desc && (stage_mask & RKV_STAGE_PREP) && desc->dtype != RKV_F32 && (desc->head_dim == 0 || desc->head_dim == kHeadDim)) c += 1;
+    if (desc && (stage_mask & RKV_STAGE_PREP) && desc->dtype == RKV_FP8_E4M3) c += 1;       // 8-bit caches: the widening kernel
     if (desc && (stage_mask & RKV_STAGE_SELECT) && (desc->flags & RKV_FLAG_HEAD_MEAN)) c += 1;   // per-sequence selection
     // the two-pass scoring path is the first pass plus up to two rounds of (listing, second pass) while the
     // retention rule is on

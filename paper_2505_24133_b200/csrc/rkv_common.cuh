@@ -29,7 +29,8 @@ struct Params {
     int d;                          // head dimension: 64, 128 or 256
     int cap, cap_pad, tiles;        // cap_pad = tiles * kTile
     int budget, buffer, alpha;
-    int dtype;
+    int dtype;                      // of the keys the scoring stages read (bf16 for 8-bit caches: their widened copy)
+    int store_row_bytes;            // bytes of a row of the caches as stored (what the gather moves)
     // hyper-parameters
     int pool_w, beta;
     int head_mean;                  // Algorithm 1's aggregated selection: one kept set per sequence from the
@@ -181,6 +182,7 @@ template <> struct Elem<float> {
 
 // launchers (one per stage); each returns cudaGetLastError() of its launch
 cudaError_t launch_prep(const Params &p, cudaStream_t s);
+cudaError_t launch_widen_keys(const Params &stored, __nv_bfloat16 *wide, cudaStream_t s);
 cudaError_t launch_scores_simt(const Params &p, cudaStream_t s);
 cudaError_t launch_scores_sm100(const Params &p, cudaStream_t s);
 cudaError_t launch_scores_tri_sm100(const Params &p, cudaStream_t s);

@@ -5,7 +5,7 @@
 // One thread block owns one (head, K|V) stream (or a column slice of it) and walks it in chunks of 64 rows or more: load the chunk's source
 // rows into registers, barrier, store.  A later chunk reads only rows at or beyond its own first row, which
 // no earlier chunk writes, so one barrier per chunk is all the ordering in-place compaction needs.
-// No scratch copy, no reallocation.  HBM-bound: 16-byte loads and stores, a row is 16 (bf16) or 32 (fp32) lanes wide.
+// No scratch copy, no reallocation.  HBM-bound: 16-byte loads and stores, a row is 4 (8-bit, d = 64) to 64 (fp32, d = 256) lanes wide.
 // The block of (KV head 0, K) also stores the new length, seq_lens[b] = budget.
 #include "rkv_common.cuh"
 
@@ -76,7 +76,7 @@ cudaError_t launch_gather(const Params &p, cudaStream_t s)
     // (8 per SM): a second, partly filled wave would leave SMs idle for much of the kernel.
     const unsigned wave = 8u * (unsigned)sms;
     const int split = streams * 4u <= wave ? 4 : (streams * 2u <= wave ? 2 : (streams < wave ? 4 : 1));
-    const int vec_per_row = p.d * (p.dtype == RKV_BF16 ? 2 : 4) / 16;      // 16-byte vectors per row: 8 .. 64
+    const int vec_per_row = p.store_row_bytes / 16;      // 16-byte vectors per row: 4 .. 64
 #define RKV_GATHER_CASE(V)                                                                      \
     case V:                                                                                     \
         if (split == 4) gather_kernel<V, 4><<<streams * 4u, kGatherThreads, 0, s>>>(p);         \
@@ -84,6 +84,7 @@ cudaError_t launch_gather(const Params &p, cudaStream_t s)
         else gather_kernel<V, 1><<<streams, kGatherThreads, 0, s>>>(p);                         \
         break;
     switch (vec_per_row) {
+        RKV_GATHER_CASE(4)
         RKV_GATHER_CASE(8)
         RKV_GATHER_CASE(16)
         RKV_GATHER_CASE(32)

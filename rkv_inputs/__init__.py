@@ -32,7 +32,7 @@ class CacheSpec:
     buffer: int
     alpha: int
     lam: float
-    dtype: str                 # "bf16" | "f32"
+    dtype: str                 # "bf16" | "f32" | "fp8" (caches as 8-bit E4M3 codes, queries bf16)
     span: int                  # tokens per copied span
     copy_frac: float           # share of spans (tokens) that are noisy copies
     copy_sigma: float          # noise added to a copied span
@@ -54,7 +54,11 @@ class CacheSpec:
 
     @property
     def torch_dtype(self) -> torch.dtype:
-        return torch.bfloat16 if self.dtype == "bf16" else torch.float32
+        return {"bf16": torch.bfloat16, "f32": torch.float32, "fp8": torch.float8_e4m3fn}[self.dtype]
+
+    @property
+    def query_dtype(self) -> torch.dtype:
+        return torch.bfloat16 if self.dtype == "fp8" else self.torch_dtype
 
 
 SPECS: Dict[str, CacheSpec] = {
@@ -73,6 +77,8 @@ CONFIG_ORDER = ["tiny", "llama8b_b1", "llama8b_b16", "qwen7b_b64", "qwen14b_b32"
 # a multi-head-attention cache (G = 1, Eq. 1: every query head has its own KV head), shaped like a 7B model with 32
 # layers x 32 heads, batch 8, budget 2048: beside the five configurations above, which are all grouped-query
 SPECS["mha7b_b8"] = CacheSpec("mha7b_b8", 32, 8, 32, 32, 128, 2048, 128, 8, 0.1, "bf16", 32, 0.30, 0.05, 4, 8.0)
+# the second configuration's shape at batch 16 with the caches stored as 8-bit E4M3 codes (queries stay bf16)
+SPECS["llama8b_b16_fp8"] = CacheSpec("llama8b_b16_fp8", 32, 16, 8, 32, 128, 4096, 128, 8, 0.1, "fp8", 32, 0.30, 0.05, 4, 8.0)
 
 
 def scaled(spec: CacheSpec, *, layers: Optional[int] = None, batch: Optional[int] = None,
@@ -177,7 +183,7 @@ def make_workload(spec: CacheSpec, device="cpu", seed: Optional[int] = None,
     else:
         seq_lens = seq_lens.to(device=dev, dtype=torch.int32)
         assert seq_lens.shape == (Bf,)
-    return Workload(spec, k.to(dt).contiguous(), v.to(dt).contiguous(), q.to(dt).contiguous(), seq_lens, seed)
+    return Workload(spec, k.to(dt).contiguous(), v.to(dt).contiguous(), q.to(spec.query_dtype).contiguous(), seq_lens, seed)
 
 
 def make_stream_block(spec: CacheSpec, k_cache: torch.Tensor, v_cache: torch.Tensor, seq_lens: torch.Tensor,
@@ -213,7 +219,7 @@ def make_stream_block(spec: CacheSpec, k_cache: torch.Tensor, v_cache: torch.Ten
     k_cache[bi, :, pos, :] = new_k.to(k_cache.dtype).permute(0, 2, 1, 3)
     v_cache[bi, :, pos, :] = new_v.to(v_cache.dtype).permute(0, 2, 1, 3)
     seq_lens += nb
-    return torch.randn(Bf, spec.n_q_heads, spec.alpha, d, generator=gen, device=dev).to(k_cache.dtype)
+    return torch.randn(Bf, spec.n_q_heads, spec.alpha, d, generator=gen, device=dev).to(spec.query_dtype)
 
 
 def stream_state(spec: CacheSpec, device="cpu", seed: Optional[int] = None):

@@ -25,12 +25,23 @@ import oracle
 
 
 def to_numpy_f32(t: torch.Tensor) -> np.ndarray:
+    if t.dtype == torch.float8_e4m3fn:          # 8-bit caches: the oracle's own decode of the stored codes
+        return oracle.e4m3_to_f32(t.detach().view(torch.uint8).cpu().numpy())
     return t.detach().to("cpu", torch.float32).numpy()
 
 
+def pick(t: torch.Tensor, sel: torch.Tensor) -> torch.Tensor:
+    """t[sel] along the leading dimension (8-bit tensors are indexed through their byte view)."""
+    if t.dtype == torch.float8_e4m3fn:
+        return t.view(torch.uint8)[sel].view(torch.float8_e4m3fn)
+    return t[sel]
+
+
 def raw_rows(t: torch.Tensor) -> np.ndarray:
-    """Bit pattern view (uint16 for bf16, uint32 for fp32) on the CPU."""
+    """Bit pattern view (uint8 for E4M3 codes, uint16 for bf16, uint32 for fp32) on the CPU."""
     t = t.detach().cpu().contiguous()
+    if t.dtype == torch.float8_e4m3fn:
+        return t.view(torch.uint8).numpy()
     return t.view(torch.int16).numpy().view(np.uint16) if t.dtype == torch.bfloat16 else \
         t.view(torch.int32).numpy().view(np.uint32)
 

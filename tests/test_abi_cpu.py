@@ -135,3 +135,21 @@ def test_product_package_does_not_touch_the_oracle():
         if f.endswith((".py", ".c")):
             text = open(os.path.join(ROOT, "oracle", f)).read()
             assert "paper_2505_24133_b200" not in text and "librkv_b200" not in text
+
+
+def test_eight_bit_cache_type_sizes_and_counts(rkv):
+    """RKV_FP8_E4M3: the workspace grows by the bf16 copy of the keys, the host-buffer staging shrinks to one byte per
+    cache element (queries stay bf16), one more kernel (the widening) is launched; an unknown type is refused."""
+    P, cap, alpha = 2 * 8, 1024 + 128, 8
+    for hd in (64, 128, 256):
+        b16 = _desc(rkv, head_dim=hd)
+        f8 = _desc(rkv, head_dim=hd, dtype=rkv.RKV_FP8_E4M3)
+        w16, w8 = rkv.rkv_workspace_bytes(b16, 1024, 128, alpha), rkv.rkv_workspace_bytes(f8, 1024, 128, alpha)
+        assert w8 == w16 + (P * cap + 128) * hd * 2
+        h16, h8 = rkv.rkv_host_workspace_bytes(b16, 1024, 128, alpha), rkv.rkv_host_workspace_bytes(f8, 1024, 128, alpha)
+        assert (h16 - w16) - (h8 - w8) == 2 * P * cap * hd            # K and V staging: two bytes per element less one
+        assert rkv.rkv_launch_count_for(f8, 1024, 128, alpha, rkv.RKV_STAGE_ALL) == \
+            rkv.rkv_launch_count_for(b16, 1024, 128, alpha, rkv.RKV_STAGE_ALL) + 1
+        assert rkv.rkv_launch_count_for(f8, 1024, 128, alpha, rkv.RKV_STAGE_GATHER) == 1
+    assert rkv.rkv_workspace_bytes(_desc(rkv, dtype=3), 1024, 128, alpha) == 0
+    assert rkv.rkv_decode_workspace_bytes(_desc(rkv, dtype=rkv.RKV_FP8_E4M3), 1024, 128) == 0

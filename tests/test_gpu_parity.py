@@ -5,7 +5,7 @@ import pytest
 import torch
 
 import rkv_inputs as ri
-from parity_util import check_batch, from_paged, random_block_table, raw_rows, to_paged
+from parity_util import check_batch, from_paged, pick, random_block_table, raw_rows, to_paged
 
 pytestmark = pytest.mark.gpu
 
@@ -40,8 +40,8 @@ def run_and_check(rkv, wl, *, flags=0, W=4, beta=1, T=0.5, eps=1e-8, lam=None, c
     torch.cuda.synchronize()
     rows = list(range(spec.folded_batch)) if check_rows is None else list(check_rows)
     sel = torch.tensor(rows, device=k0.device)
-    rep = check_batch(k0[sel], v0[sel], q0[sel], s0[sel], budget=spec.budget, alpha=spec.alpha, lam=lam, W=W,
-                      beta=beta, T=T, eps=eps, gpu_idx=idx[sel], gpu_k=wl.k_cache[sel], gpu_v=wl.v_cache[sel],
+    rep = check_batch(pick(k0, sel), pick(v0, sel), q0[sel], s0[sel], budget=spec.budget, alpha=spec.alpha, lam=lam, W=W,
+                      beta=beta, T=T, eps=eps, gpu_idx=idx[sel], gpu_k=pick(wl.k_cache, sel), gpu_v=pick(wl.v_cache, sel),
                       gpu_seq=wl.seq_lens[sel], gpu_scores=comp.scores[:, sel],
                       mean_then_pool=bool(flags & 4), head_mean=bool(flags & 8), gqa_mean_pool=bool(flags & 16),
                       budgets=None if budgets is None else [budgets[r] for r in rows])
