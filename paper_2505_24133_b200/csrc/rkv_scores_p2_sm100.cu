@@ -347,7 +347,6 @@ scores_pass2_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, c
         const int quad = warp & 3;               // TMEM lane quadrant this warp may access
         const int lrow = quad * 32 + lane;       // row within the 128-row tile
         const uint32_t lane_base = tmem_base + ((uint32_t)(quad * 32) << 16);
-        const float kInf = __int_as_float(0x7f800000);
         uint32_t k_item = 0, cnt = 0;
 
         while (true) {
@@ -396,79 +395,91 @@ scores_pass2_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, c
                     const uint32_t base = lane_base + a * 256 + m * 128;
                     // a token that has its beta partners screens nothing any more
                     bool want = left > 0;
-                    if (__any_sync(0xffffffffu, want)) {
-                        // 32-column chunks, last first.  The loop is kept rolled on purpose: the warps of three roles
-                        // share the instruction cache, and one copy of this body is what fits.
-#pragma unroll 1
-                        for (int ch = 3; ch >= 0; --ch) {
-                            uint32_t g[32];
-                            tmem_ld32(base + ch * 32, g);
-                            float v[32];
-                            uint32_t hits = 0u;
-                            // The accumulator holds h = k_i . k_j - (T / r_i) (||k_j|| + eps): S[j][i] > T exactly
-                            // when h > 0, so the screening is a maximum and a sign test, with nothing to load
-                            // per column (loads of the r_j were what this epilogue's time went into: every
-                            // byte a thread receives, from TMEM or as a shared-memory broadcast, passes through
-                            // the same return path).  The listed tokens rarely have a partner in a given chunk.
-                            tmem_wait32(g);
+                    // The accumulator holds h = k_i . k_j - (T / r_i) (||k_j|| + eps): S[j][i] > T exactly when h > 0, so
+                    // the screening is a sign test, with nothing to load per column (loads of the r_j were what this
+                    // epilogue's time went into: every byte a thread receives, from TMEM or as a shared-memory
+                    // broadcast, passes through the same return path).  32-column chunks, last first; the TMEM load of
+                    // the next chunk is issued before the current one is looked at (two register sets, used alternately).
+                    auto chunk = [&](const uint32_t (&g)[32], int ch) {
+                        uint32_t colmask = 0xffffffffu;
+                        const unsigned own = (unsigned)(i - (jbase + ch * 32));           // zero diagonal (Eq. 5)
+                        if (own < 32u) colmask &= ~(1u << own);
+                        // bit c of `neg` = sign bit of entry c: one funnel shift per entry, four independent chains
+                        uint32_t n0 = 0u, n1 = 0u, n2 = 0u, n3 = 0u;
 #pragma unroll
-                            for (int c = 0; c < 32; ++c) v[c] = __uint_as_float(g[c]);
-                            float m0 = 0.f, m1 = 0.f;
+                        for (int c = 7; c >= 0; --c) {
+                            n0 = __funnelshift_l(g[c], n0, 1);
+                            n1 = __funnelshift_l(g[8 + c], n1, 1);
+                            n2 = __funnelshift_l(g[16 + c], n2, 1);
+                            n3 = __funnelshift_l(g[24 + c], n3, 1);
+                        }
+                        const uint32_t neg = (n0 | (n1 << 8)) | ((n2 << 16) | (n3 << 24));
+                        // entries with a clear sign bit (h > 0, but also +0: confirmed one by one below)
+                        uint32_t pos = want ? (~neg & colmask) : 0u;
+                        if (p.beta == 1) {
+                            // one partner at most: the candidate at the highest set bit, its value picked by a select
+                            // tree (nearly always a single turn); its r_j is fetched once, at the item's end
+                            while (pos != 0u) {
+                                const int top = 31 - __clz(pos);
+                                uint32_t t16[16], t8[8], t4[4];
 #pragma unroll
-                            for (int c = 0; c < 32; c += 4) {
-                                m0 = max3(m0, v[c], v[c + 1]);
-                                m1 = max3(m1, v[c + 2], v[c + 3]);
-                            }
-                            const float cut = want ? 0.f : kInf;
-                            if (!__any_sync(0xffffffffu, fmaxf(m0, m1) > cut)) continue;
+                                for (int c = 0; c < 16; ++c) t16[c] = (top & 16) ? g[16 + c] : g[c];
 #pragma unroll
-                            for (int c = 0; c < 32; ++c) hits |= (v[c] > cut) ? (1u << c) : 0u;
-                            const unsigned own = (unsigned)(i - (jbase + ch * 32));           // zero diagonal (Eq. 5)
-                            if (own < 32u) hits &= ~(1u << own);
-                            if (p.beta == 1) {
-                                // one partner at most: the entry at the highest set bit, picked by a select tree;
-                                // its r_j is fetched once, at the item's end
-                                if (left > 0 && hits != 0u) {
-                                    const int top = 31 - __clz(hits);
-                                    float t16[16], t8[8], t4[4];
+                                for (int c = 0; c < 8; ++c) t8[c] = (top & 8) ? t16[8 + c] : t16[c];
 #pragma unroll
-                                    for (int c = 0; c < 16; ++c) t16[c] = (top & 16) ? v[16 + c] : v[c];
-#pragma unroll
-                                    for (int c = 0; c < 8; ++c) t8[c] = (top & 8) ? t16[8 + c] : t16[c];
-#pragma unroll
-                                    for (int c = 0; c < 4; ++c) t4[c] = (top & 4) ? t8[4 + c] : t8[c];
-                                    const float u0 = (top & 2) ? t4[2] : t4[0], u1 = (top & 2) ? t4[3] : t4[1];
-                                    hit_h = (top & 1) ? u1 : u0;
+                                for (int c = 0; c < 4; ++c) t4[c] = (top & 4) ? t8[4 + c] : t8[c];
+                                const uint32_t u0 = (top & 2) ? t4[2] : t4[0], u1 = (top & 2) ? t4[3] : t4[1];
+                                const float hv = __uint_as_float((top & 1) ? u1 : u0);
+                                if (hv > 0.f) {
+                                    hit_h = hv;
                                     hit_j = jbase + ch * 32 + top;
                                     left = 0;
                                     want = false;
+                                    break;
                                 }
-                                continue;
+                                pos &= ~(1u << top);
                             }
-                            int taken = __popc(hits);
-                            for (; taken > left; --taken) hits &= hits - 1u;                   // drop the lowest positions
-                            // S = T + h r_i r_j per partner
-                            nhit += taken;
+                            return;
+                        }
+                        // several partners per token: the exact mask, cut down to the highest positions if they are more
+                        // than the token still lacks, then the sum of their h r_j (S = T + h r_i r_j per partner)
+                        if (!__any_sync(0xffffffffu, pos != 0u)) return;
+                        uint32_t hits = 0u;
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) hits |= (__uint_as_float(g[c]) > 0.f) ? (1u << c) : 0u;
+                        hits &= pos;
+                        int taken = __popc(hits);
+                        for (; taken > left; --taken) hits &= hits - 1u;                   // drop the lowest positions
+                        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+                        if (hits != 0u) {
 #pragma unroll
                             for (int q = 0; q < 8; ++q) {
                                 const float4 R = __ldg(rj4 + ch * 8 + q);
-                                v[4 * q] *= R.x;
-                                v[4 * q + 1] *= R.y;
-                                v[4 * q + 2] *= R.z;
-                                v[4 * q + 3] *= R.w;
+                                s0 += (hits >> (4 * q) & 1u) ? __uint_as_float(g[4 * q]) * R.x : 0.f;
+                                s1 += (hits >> (4 * q + 1) & 1u) ? __uint_as_float(g[4 * q + 1]) * R.y : 0.f;
+                                s2 += (hits >> (4 * q + 2) & 1u) ? __uint_as_float(g[4 * q + 2]) * R.z : 0.f;
+                                s3 += (hits >> (4 * q + 3) & 1u) ? __uint_as_float(g[4 * q + 3]) * R.w : 0.f;
                             }
-                            float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-#pragma unroll
-                            for (int c = 0; c < 32; c += 4) {
-                                s0 += (hits >> c & 1u) ? v[c] : 0.f;
-                                s1 += (hits >> (c + 1) & 1u) ? v[c + 1] : 0.f;
-                                s2 += (hits >> (c + 2) & 1u) ? v[c + 2] : 0.f;
-                                s3 += (hits >> (c + 3) & 1u) ? v[c + 3] : 0.f;
-                            }
-                            removed += (s0 + s1) + (s2 + s3);
-                            left -= taken;
-                            if (left == 0) want = false;
                         }
+                        removed += (s0 + s1) + (s2 + s3);
+                        nhit += taken;
+                        left -= taken;
+                        if (left == 0) want = false;
+                    };
+                    if (__any_sync(0xffffffffu, want)) {
+                        uint32_t ga[32], gb[32];
+                        tmem_ld32(base + 96, ga);
+                        tmem_wait32(ga);
+                        tmem_ld32(base + 64, gb);
+                        chunk(ga, 3);
+                        tmem_wait32(gb);
+                        tmem_ld32(base + 32, ga);
+                        chunk(gb, 2);
+                        tmem_wait32(ga);
+                        tmem_ld32(base, gb);
+                        chunk(ga, 1);
+                        tmem_wait32(gb);
+                        chunk(gb, 0);
                     }
                     tc_fence_before();
                     __syncwarp();
