@@ -504,8 +504,6 @@ def measure_attention(rkv, dev, wl, peaks, reps=5):
     d.head_dim = spec.head_dim
     d.dtype = {"bf16": rkv.RKV_BF16, "f32": rkv.RKV_F32, "fp8": rkv.RKV_FP8_E4M3}[spec.dtype]    # the caches are read as this type
     need = rkv.rkv_decode_workspace_bytes(d, spec.budget, spec.buffer)
-    if need == 0:
-        return {"unsupported": "rkv_decode_attention does not take this cache type or shape"}
     ws = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
     d.workspace, d.workspace_bytes = ws.data_ptr(), ws.numel()
     gen = torch.Generator(device=dev).manual_seed(ri.BASE_SEED + 99)

@@ -284,11 +284,13 @@ RKV_API int rkv_push_query(const rkv_desc_t *desc, void *q_window, const void *q
  *   seq_lens          [batch] int32 (device), read only; 0 gives a zero output row; a value outside
  *                     [0, budget + buffer] gives a zero row and RKV_ERR_INVALID_ARG in desc->device_status
  *   out               [batch][n_q_heads][head_dim] float32 (device, 16-byte aligned)
- * fp32 arithmetic throughout.  head_dim 128 and G = n_q_heads / n_kv_heads up to 8 (RKV_ERR_UNSUPPORTED otherwise).  With few
- * head-problems the rows of a head are cut into splits whose partial results go through desc->workspace:
- * rkv_decode_workspace_bytes() says how much that needs (0 for large batches; never more than a compression of the
- * same shape needs, so one workspace serves both).  Enqueues one or two kernels on `stream`; return codes as for
- * rkv_compress_ex.
+ * bf16 caches: both contractions on the tensor cores (bf16 products, fp32 accumulation, the softmax weights carried as
+ * two bf16 parts, i.e. to fp32 accuracy), softmax in fp32; fp32 caches: fp32 arithmetic throughout.  head_dim 128 and
+ * G = n_q_heads / n_kv_heads up to 8 (RKV_ERR_UNSUPPORTED otherwise).  The rows of a head are cut into splits (with
+ * few head-problems, to fill the GPU; for bf16 caches also whenever budget + buffer exceeds 1920 rows, what one block
+ * holds scores for) whose partial results go through desc->workspace: rkv_decode_workspace_bytes() says how much that
+ * needs (0 when there is a single split; never more than a compression of the same shape needs, so one workspace
+ * serves both).  Enqueues one or two kernels on `stream`; return codes as for rkv_compress_ex.
  */
 RKV_API size_t rkv_decode_workspace_bytes(const rkv_desc_t *desc, int32_t budget, int32_t buffer);
 RKV_API int rkv_decode_attention(const rkv_desc_t *desc, const void *k_cache, const void *v_cache, const void *q_new,

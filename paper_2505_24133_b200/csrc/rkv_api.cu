@@ -393,7 +393,7 @@ static int attend_plan(const rkv_desc_t *d, int32_t budget, int32_t buffer, int 
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
         sms = 148;       // sizing only (no device here): the B200's count
-    *splits = attend_splits(d->batch * d->n_kv_heads, budget + buffer, sms);
+    *splits = attend_splits(d->batch * d->n_kv_heads, budget + buffer, sms, G, d->dtype);
     *bytes = attend_partial_bytes(d->batch * d->n_kv_heads, *splits, G);
     return RKV_OK;
 }
@@ -422,7 +422,7 @@ int rkv_decode_attention(const rkv_desc_t *d, const void *k_cache, const void *v
     const long long wait = d->wait_limit_cycles > 0 ? (long long)d->wait_limit_cycles : sm100_default_wait_cycles();
     const cudaError_t e = launch_attend(k_cache, v_cache, q_new, seq_lens, out, static_cast<float *>(d->workspace), d->batch,
                                         d->n_kv_heads, d->n_q_heads, budget + buffer, splits, d->dtype, d->device_status,
-                                        wait, d->block_table, static_cast<cudaStream_t>(stream));
+                                        wait, d->block_table, d->pool_pages, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? RKV_OK : cuda_fail(e, "decode attention launch");
 }
 

@@ -1,5 +1,6 @@
-// Decode-step attention over the compressed cache (Section 3.1: between two firings of the compression the model
-// decodes against the B_budget retained tokens plus the buffer; Eq. 1 with a single query row per head):
+// Decode-step attention over the compressed cache, CUDA-core form (fp32 caches; bf16 caches take the tensor-core kernel
+// of rkv_attend_tc.cu) (Section 3.1: between two firings of the compression the model decodes against the B_budget
+// retained tokens plus the buffer; Eq. 1 with a single query row per head):
 //
 //   out[b][q] = sum_j softmax_j( q_new[b][q] . K[b][q / G][j] / sqrt(d) ) V[b][q / G][j],   j < seq_lens[b]
 //
@@ -342,9 +343,14 @@ cudaError_t launch_dtype(const AttendParams &p, int G, cudaStream_t s)
 
 int attend_max_group() { return kAttMaxG; }
 
+// bf16 caches go to the tensor-core kernel whatever the group size (it runs at the rate HBM can be read at; this kernel
+// reached 0.74 of the copy bandwidth at G = 4 and ran out of issue slots from G = 5 on); fp32 caches stay here.
+bool attend_uses_tc(int G, int dtype) { return dtype == RKV_BF16 && G >= 1; }
+
 // Splits of a head's rows: enough blocks for two waves of resident blocks (2 per SM), never finer than a tile.
-int attend_splits(int heads, int cap, int sms)
+int attend_splits(int heads, int cap, int sms, int G, int dtype)
 {
+    if (attend_uses_tc(G, dtype)) return attend_tc_splits(heads, cap, sms);
     const int tiles = (cap + kAttRows - 1) / kAttRows;
     int splits = (4 * sms + heads - 1) / heads;
     splits = splits < 1 ? 1 : splits;
@@ -358,8 +364,9 @@ size_t attend_partial_bytes(int heads, int splits, int G)
 
 cudaError_t launch_attend(const void *k_cache, const void *v_cache, const void *q_new, const int32_t *seq_lens, float *out,
                           float *partial, int batch, int hkv, int hq, int cap, int splits, int dtype, int32_t *status,
-                          long long wait_cycles, const int32_t *block_table, cudaStream_t s)
+                          long long wait_cycles, const int32_t *block_table, long long pool_pages, cudaStream_t s)
 {
+    const int G = hq / hkv;
     AttendParams p;
     p.k_cache = k_cache;
     p.v_cache = v_cache;
@@ -375,8 +382,12 @@ cudaError_t launch_attend(const void *k_cache, const void *v_cache, const void *
     p.status = status;
     p.wait_cycles = wait_cycles;
     p.block_table = block_table;
-    const int G = hq / hkv;
-    cudaError_t e = dtype == RKV_BF16 ? launch_dtype<__nv_bfloat16>(p, G, s) : launch_dtype<float>(p, G, s);
+    cudaError_t e;
+    if (attend_uses_tc(G, dtype))
+        e = launch_attend_tc(k_cache, v_cache, q_new, seq_lens, out, partial, batch, hkv, hq, cap, splits, status, wait_cycles,
+                             block_table, pool_pages, s);
+    else
+        e = launch_dtype<float>(p, G, s);
     if (e != cudaSuccess || splits == 1) return e;
     attend_merge_kernel<<<(unsigned)(batch * hkv * G), kHeadDim, 0, s>>>(p, G);
     return cudaGetLastError();

@@ -188,6 +188,71 @@ def test_decode_attention_large_batch_single_split(rkv):
     assert (np.abs(got - ref) <= 1e-3 * scale + 1e-7).all()
 
 
+@pytest.mark.parametrize("hkv,hq,batch", [(2, 10, 3), (1, 7, 40), (4, 32, 2), (1, 6, 600)])
+def test_decode_attention_tensor_core_route_large_cache(rkv, hkv, hq, batch):
+    """Query groups of 5 to 8 at the largest cache size of the configurations (33 key tiles, so every head is cut into
+    three or more splits, whatever the batch), random lengths with a full, a one-token and an empty cache among them,
+    stale rows full of NaN; checked on sampled sequences."""
+    spec = ri.CacheSpec("att_tc", 1, batch, hkv, hq, 128, 4096, 128, 8, 0.1, "bf16", 32, 0.3, 0.05, 4, 8.0)
+    lens = torch.randint(1, spec.cap + 1, (batch,), generator=torch.Generator().manual_seed(13 + hq))
+    lens[0], lens[1] = spec.cap, 1
+    if batch > 2:
+        lens[2] = 0
+    wl = ri.make_workload(spec, device="cuda", seed=341 + hq, seq_lens=lens)
+    for b in range(batch):
+        wl.k_cache[b, :, int(lens[b]):] = float("nan")
+        wl.v_cache[b, :, int(lens[b]):] = float("nan")
+    g = torch.Generator(device="cuda").manual_seed(8)
+    q_new = torch.randn(batch, hq, 128, generator=g, device="cuda").to(torch.bfloat16)
+    d = rkv.rkv_desc_default()
+    d.batch, d.n_kv_heads, d.n_q_heads = batch, hkv, hq
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    d.device_status = status.data_ptr()
+    need = rkv.rkv_decode_workspace_bytes(d, spec.budget, spec.buffer)
+    assert need > 0                                    # 33 tiles never fit one block's 15
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    d.workspace, d.workspace_bytes = ws.data_ptr(), need
+    out = torch.full((batch, hq, 128), 7.0, dtype=torch.float32, device="cuda")
+    rc = rkv.rkv_decode_attention(d, wl.k_cache, wl.v_cache, q_new, wl.seq_lens, out, spec.budget, spec.buffer)
+    assert rc == rkv.RKV_OK, rkv.rkv_status_string(rc)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    rows = sorted(set([0, 1, min(2, batch - 1), batch // 2, batch - 1]))
+    K, V = (torch.nan_to_num(t[rows].float(), nan=0.0).cpu().numpy() for t in (wl.k_cache, wl.v_cache))
+    ref = oracle.oracle_decode_attention(K, V, q_new[rows].float().cpu().numpy(), lens[rows].numpy().astype(np.int32))
+    got = out[rows].cpu().numpy().astype(np.float64)
+    assert np.isfinite(out.cpu().numpy()).all()
+    scale = np.maximum(np.abs(ref).max(axis=-1, keepdims=True), 1e-30)
+    assert (np.abs(got - ref) <= 1e-3 * scale + 1e-7).all(), float((np.abs(got - ref) / scale).max())
+    if batch > 2:
+        assert not out[2].any()
+
+
+def test_decode_attention_tensor_core_route_paged(rkv):
+    """The tensor-core kernel through a block table (G = 8)."""
+    spec = ri.CacheSpec("att_tc_paged", 1, 4, 1, 8, 128, 896, 128, 8, 0.1, "bf16", 16, 0.3, 0.05, 4, 8.0)
+    lens = [1024, 127, 129, 700]
+    wl = ri.make_workload(spec, device="cuda", seed=351, seq_lens=torch.tensor(lens))
+    pages, pool_pages = spec.cap // 128, 4 * 8 + 5
+    table = random_block_table(4, 1, pages, pool_pages, seed=12)
+    kp, vp = to_paged(wl.k_cache, pool_pages, table), to_paged(wl.v_cache, pool_pages, table)     # foreign pages: NaN
+    comp = rkv.Compressor(4, 1, 8, spec.budget, spec.buffer, spec.alpha, 0.1, block_table=table, pool_pages=pool_pages)
+    g = torch.Generator(device="cuda").manual_seed(4)
+    q_new = torch.randn(4, 8, 128, generator=g, device="cuda").to(torch.bfloat16)
+    need = rkv.rkv_decode_workspace_bytes(comp.desc, spec.budget, spec.buffer)
+    ws = torch.empty(max(need, 256), dtype=torch.uint8, device="cuda")
+    comp.desc.workspace, comp.desc.workspace_bytes = ws.data_ptr(), ws.numel()
+    out = torch.empty(4, 8, 128, dtype=torch.float32, device="cuda")
+    assert rkv.rkv_decode_attention(comp.desc, kp, vp, q_new, wl.seq_lens, out, spec.budget, spec.buffer) == rkv.RKV_OK
+    torch.cuda.synchronize()
+    comp.check_status()
+    ref = oracle.oracle_decode_attention(wl.k_cache.float().cpu().numpy(), wl.v_cache.float().cpu().numpy(),
+                                         q_new.float().cpu().numpy(), np.array(lens, dtype=np.int32))
+    got = out.cpu().numpy().astype(np.float64)
+    scale = np.maximum(np.abs(ref).max(axis=-1, keepdims=True), 1e-30)
+    assert (np.abs(got - ref) <= 1e-3 * scale + 1e-7).all(), float((np.abs(got - ref) / scale).max())
+
+
 def test_decode_attention_argument_checks(rkv):
     d = rkv.rkv_desc_default()
     d.batch, d.n_kv_heads, d.n_q_heads = 2, 1, 9           # G = 9: beyond what one block serves
