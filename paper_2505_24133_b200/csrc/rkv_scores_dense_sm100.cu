@@ -387,16 +387,21 @@ constexpr int kFinishThreads = 256;
 
 __global__ void __launch_bounds__(kFinishThreads) dense_finish_kernel(Params p)
 {
+    // work unit = (head, chunk of 256 tokens), handed out with the grid as stride: when no head took the route (the
+    // common case) a block runs through its units in a few microseconds instead of the launch paying for a block each
     const int chunks = (p.cap + kFinishThreads - 1) / kFinishThreads;
-    const int head = blockIdx.x / chunks;
-    if (!p.dense[head] || call_aborted(p)) return;
-    const int i = (blockIdx.x % chunks) * kFinishThreads + threadIdx.x;
+    const long long units = (long long)p.batch * p.hkv * chunks;
+    if (call_aborted(p)) return;
+    for (long long u = blockIdx.x; u < units; u += gridDim.x) {
+    const int head = (int)(u / chunks);
+    if (!p.dense[head]) continue;
+    const int i = (int)(u % chunks) * kFinishThreads + threadIdx.x;
     const int n = seq_candidates(p, head / p.hkv);
-    if (i >= n) return;
+    if (i >= n) continue;
     const size_t hoff = (size_t)head * p.cap_pad;
-    if (p.left[hoff + i] <= 0) return;
+    if (p.left[hoff + i] <= 0) continue;
     const uint32_t b = p.best[hoff + i];
-    if (b == 0u) return;
+    if (b == 0u) continue;
     const int j = (int)b - 1;
     const uint4 *ki = reinterpret_cast<const uint4 *>(static_cast<const __nv_bfloat16 *>(p.k_cache) + (size_t)row_index(p, head, i) * kHeadDim);
     const uint4 *kj = reinterpret_cast<const uint4 *>(static_cast<const __nv_bfloat16 *>(p.k_cache) + (size_t)row_index(p, head, j) * kHeadDim);
@@ -411,6 +416,7 @@ __global__ void __launch_bounds__(kFinishThreads) dense_finish_kernel(Params p)
     }
     p.sbar[hoff + i] -= dot * p.inv_norm[hoff + i] * p.inv_norm[hoff + j];
     p.left[hoff + i] = 0;
+    }
 }
 
 }  // namespace
@@ -425,10 +431,11 @@ cudaError_t launch_scores_dense_sm100(const Params &p, cudaStream_t s, const CUt
     return cudaGetLastError();
 }
 
-cudaError_t launch_dense_finish(const Params &p, cudaStream_t s)
+cudaError_t launch_dense_finish(const Params &p, cudaStream_t s, int sms)
 {
-    const unsigned grid = (unsigned)(p.batch * p.hkv) * (unsigned)((p.cap + kFinishThreads - 1) / kFinishThreads);
-    dense_finish_kernel<<<grid, kFinishThreads, 0, s>>>(p);
+    const unsigned long long units = (unsigned long long)(p.batch * p.hkv) * (unsigned long long)((p.cap + kFinishThreads - 1) / kFinishThreads);
+    const unsigned long long wave = 8ull * (unsigned long long)sms;             // resident blocks of this size
+    dense_finish_kernel<<<(unsigned)(units < wave ? units : wave), kFinishThreads, 0, s>>>(p);
     return cudaGetLastError();
 }
 

@@ -400,6 +400,7 @@ scores_pass2_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, c
                     // epilogue's time went into: every byte a thread receives, from TMEM or as a shared-memory
                     // broadcast, passes through the same return path).  32-column chunks, last first; the TMEM load of
                     // the next chunk is issued before the current one is looked at (two register sets, used alternately).
+                    // (beta = 1, the default: one partner per token)
                     auto chunk = [&](const uint32_t (&g)[32], int ch) {
                         uint32_t colmask = 0xffffffffu;
                         const unsigned own = (unsigned)(i - (jbase + ch * 32));           // zero diagonal (Eq. 5)
@@ -416,7 +417,7 @@ scores_pass2_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, c
                         const uint32_t neg = (n0 | (n1 << 8)) | ((n2 << 16) | (n3 << 24));
                         // entries with a clear sign bit (h > 0, but also +0: confirmed one by one below)
                         uint32_t pos = want ? (~neg & colmask) : 0u;
-                        if (p.beta == 1) {
+                        {
                             // one partner at most: the candidate at the highest set bit, its value picked by a select
                             // tree (nearly always a single turn); its r_j is fetched once, at the item's end
                             while (pos != 0u) {
@@ -439,47 +440,74 @@ scores_pass2_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, c
                                 }
                                 pos &= ~(1u << top);
                             }
-                            return;
                         }
-                        // several partners per token: the exact mask, cut down to the highest positions if they are more
-                        // than the token still lacks, then the sum of their h r_j (S = T + h r_i r_j per partner)
-                        if (!__any_sync(0xffffffffu, pos != 0u)) return;
-                        uint32_t hits = 0u;
+                    };
+                    if (p.beta == 1) {
+                        if (__any_sync(0xffffffffu, want)) {
+                            uint32_t ga[32], gb[32];
+                            tmem_ld32(base + 96, ga);
+                            tmem_wait32(ga);
+                            tmem_ld32(base + 64, gb);
+                            chunk(ga, 3);
+                            tmem_wait32(gb);
+                            tmem_ld32(base + 32, ga);
+                            chunk(gb, 2);
+                            tmem_wait32(ga);
+                            tmem_ld32(base, gb);
+                            chunk(ga, 1);
+                            tmem_wait32(gb);
+                            chunk(gb, 0);
+                        }
+                    } else if (__any_sync(0xffffffffu, want)) {
+                        // Several partners per token.  This loop is kept rolled on purpose: the warps of three roles
+                        // share the instruction cache, and one copy of this body is what fits (unrolled like the
+                        // path above it ran a third slower).
+#pragma unroll 1
+                        for (int ch = 3; ch >= 0; --ch) {
+                            uint32_t g[32];
+                            tmem_ld32(base + ch * 32, g);
+                            float v[32];
+                            uint32_t hits = 0u;
+                            tmem_wait32(g);
 #pragma unroll
-                        for (int c = 0; c < 32; ++c) hits |= (__uint_as_float(g[c]) > 0.f) ? (1u << c) : 0u;
-                        hits &= pos;
-                        int taken = __popc(hits);
-                        for (; taken > left; --taken) hits &= hits - 1u;                   // drop the lowest positions
-                        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-                        if (hits != 0u) {
+                            for (int c = 0; c < 32; ++c) v[c] = __uint_as_float(g[c]);
+                            float m0 = 0.f, m1 = 0.f;
+#pragma unroll
+                            for (int c = 0; c < 32; c += 4) {
+                                m0 = max3(m0, v[c], v[c + 1]);
+                                m1 = max3(m1, v[c + 2], v[c + 3]);
+                            }
+                            const float cut = want ? 0.f : __int_as_float(0x7f800000);
+                            if (!__any_sync(0xffffffffu, fmaxf(m0, m1) > cut)) continue;
+#pragma unroll
+                            for (int c = 0; c < 32; ++c) hits |= (v[c] > cut) ? (1u << c) : 0u;
+                            const unsigned own = (unsigned)(i - (jbase + ch * 32));           // zero diagonal (Eq. 5)
+                            if (own < 32u) hits &= ~(1u << own);
+                            // the exact mask, cut down to the highest positions if they are more than the token still
+                            // lacks, then the sum of their h r_j (S = T + h r_i r_j per partner)
+                            int taken = __popc(hits);
+                            for (; taken > left; --taken) hits &= hits - 1u;                   // drop the lowest positions
+                            nhit += taken;
 #pragma unroll
                             for (int q = 0; q < 8; ++q) {
                                 const float4 R = __ldg(rj4 + ch * 8 + q);
-                                s0 += (hits >> (4 * q) & 1u) ? __uint_as_float(g[4 * q]) * R.x : 0.f;
-                                s1 += (hits >> (4 * q + 1) & 1u) ? __uint_as_float(g[4 * q + 1]) * R.y : 0.f;
-                                s2 += (hits >> (4 * q + 2) & 1u) ? __uint_as_float(g[4 * q + 2]) * R.z : 0.f;
-                                s3 += (hits >> (4 * q + 3) & 1u) ? __uint_as_float(g[4 * q + 3]) * R.w : 0.f;
+                                v[4 * q] *= R.x;
+                                v[4 * q + 1] *= R.y;
+                                v[4 * q + 2] *= R.z;
+                                v[4 * q + 3] *= R.w;
                             }
+                            float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+                            for (int c = 0; c < 32; c += 4) {
+                                s0 += (hits >> c & 1u) ? v[c] : 0.f;
+                                s1 += (hits >> (c + 1) & 1u) ? v[c + 1] : 0.f;
+                                s2 += (hits >> (c + 2) & 1u) ? v[c + 2] : 0.f;
+                                s3 += (hits >> (c + 3) & 1u) ? v[c + 3] : 0.f;
+                            }
+                            removed += (s0 + s1) + (s2 + s3);
+                            left -= taken;
+                            if (left == 0) want = false;
                         }
-                        removed += (s0 + s1) + (s2 + s3);
-                        nhit += taken;
-                        left -= taken;
-                        if (left == 0) want = false;
-                    };
-                    if (__any_sync(0xffffffffu, want)) {
-                        uint32_t ga[32], gb[32];
-                        tmem_ld32(base + 96, ga);
-                        tmem_wait32(ga);
-                        tmem_ld32(base + 64, gb);
-                        chunk(ga, 3);
-                        tmem_wait32(gb);
-                        tmem_ld32(base + 32, ga);
-                        chunk(gb, 2);
-                        tmem_wait32(ga);
-                        tmem_ld32(base, gb);
-                        chunk(ga, 1);
-                        tmem_wait32(gb);
-                        chunk(gb, 0);
                     }
                     tc_fence_before();
                     __syncwarp();
@@ -654,7 +682,7 @@ cudaError_t launch_scores_tri_sm100(const Params &p, cudaStream_t s)
         if (r == 0 && dense_possible && (e = launch_scores_dense_sm100(p, s, map_k, map_ns, sms)) != cudaSuccess) return e;
         below += width;
     }
-    return dense_possible ? launch_dense_finish(p, s) : cudaSuccess;
+    return dense_possible ? launch_dense_finish(p, s, sms) : cudaSuccess;
 }
 
 }  // namespace rkv

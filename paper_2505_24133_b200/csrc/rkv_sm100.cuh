@@ -304,6 +304,6 @@ cudaError_t launch_scores_pass1_sm100(const Params &p, cudaStream_t s, const CUt
 
 // symmetric route of the second pass (its own file)
 cudaError_t launch_scores_dense_sm100(const Params &p, cudaStream_t s, const CUtensorMap &map_k, const CUtensorMap &map_ns, int sms);
-cudaError_t launch_dense_finish(const Params &p, cudaStream_t s);
+cudaError_t launch_dense_finish(const Params &p, cudaStream_t s, int sms);
 
 }  // namespace rkv
