@@ -61,7 +61,8 @@ typedef enum {
  *     is a bf16 value) into the workspace, which grows by (batch * n_kv_heads * (budget + buffer) + 128) * head_dim * 2
  *     bytes, and every scoring stage runs on that copy as for a bf16 cache.  The compaction moves the stored bytes; no
  *     scale factor is applied or needed (cosine similarity does not see a per-tensor scale; fold a key scale into
- *     the queries for Eq. 2).  rkv_decode_attention does not take this type (RKV_ERR_UNSUPPORTED). */
+ *     the queries for Eq. 2).  rkv_decode_attention takes this type too (q_new bf16): the codes are widened on their
+ *     way to the tensor cores, no copy is kept. */
 typedef enum { RKV_BF16 = 0, RKV_F32 = 1, RKV_FP8_E4M3 = 2 } rkv_dtype_t;
 
 /* rkv_desc_t.flags */
@@ -280,14 +281,14 @@ RKV_API int rkv_push_query(const rkv_desc_t *desc, void *q_window, const void *q
  * library:
  *   out[b][q] = sum_j softmax_j( q_new[b][q] . K[b][q / G][j] / sqrt(head_dim) ) V[b][q / G][j],  j < seq_lens[b]
  *   k_cache, v_cache  [batch][n_kv_heads][budget + buffer][head_dim] (device, desc->dtype), read only
- *   q_new             [batch][n_q_heads][head_dim] (device, desc->dtype, 16-byte aligned)
+ *   q_new             [batch][n_q_heads][head_dim] (device, desc->dtype -- bf16 for 8-bit caches --, 16-byte aligned)
  *   seq_lens          [batch] int32 (device), read only; 0 gives a zero output row; a value outside
  *                     [0, budget + buffer] gives a zero row and RKV_ERR_INVALID_ARG in desc->device_status
  *   out               [batch][n_q_heads][head_dim] float32 (device, 16-byte aligned)
- * bf16 caches: both contractions on the tensor cores (bf16 products, fp32 accumulation, the softmax weights carried as
+ * bf16 and 8-bit caches: both contractions on the tensor cores (bf16 products, fp32 accumulation, the softmax weights carried as
  * two bf16 parts, i.e. to fp32 accuracy), softmax in fp32; fp32 caches: fp32 arithmetic throughout.  head_dim 128 and
  * G = n_q_heads / n_kv_heads up to 8 (RKV_ERR_UNSUPPORTED otherwise).  The rows of a head are cut into splits (with
- * few head-problems, to fill the GPU; for bf16 caches also whenever budget + buffer exceeds 1920 rows, what one block
+ * few head-problems, to fill the GPU; for bf16 and 8-bit caches also whenever budget + buffer exceeds 1920 rows, what one block
  * holds scores for) whose partial results go through desc->workspace: rkv_decode_workspace_bytes() says how much that
  * needs (0 when there is a single split; never more than a compression of the same shape needs, so one workspace
  * serves both).  Enqueues one or two kernels on `stream`; return codes as for rkv_compress_ex.

@@ -389,7 +389,7 @@ static int attend_plan(const rkv_desc_t *d, int32_t budget, int32_t buffer, int 
     int rc = check_shapes(d, budget, buffer, 1, nullptr);
     if (rc != RKV_OK) return rc;
     const int G = d->n_q_heads / d->n_kv_heads;
-    if (G > attend_max_group() || d->head_dim != kHeadDim || d->dtype == RKV_FP8_E4M3) return RKV_ERR_UNSUPPORTED;
+    if (G > attend_max_group() || d->head_dim != kHeadDim) return RKV_ERR_UNSUPPORTED;
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
         sms = 148;       // sizing only (no device here): the B200's count

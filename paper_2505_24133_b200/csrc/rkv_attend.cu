@@ -343,9 +343,9 @@ cudaError_t launch_dtype(const AttendParams &p, int G, cudaStream_t s)
 
 int attend_max_group() { return kAttMaxG; }
 
-// bf16 caches go to the tensor-core kernel whatever the group size (it runs at the rate HBM can be read at; this kernel
+// bf16 and 8-bit caches go to the tensor-core kernel whatever the group size (it runs at the rate HBM can be read at; this kernel
 // reached 0.74 of the copy bandwidth at G = 4 and ran out of issue slots from G = 5 on); fp32 caches stay here.
-bool attend_uses_tc(int G, int dtype) { return dtype == RKV_BF16 && G >= 1; }
+bool attend_uses_tc(int G, int dtype) { return (dtype == RKV_BF16 || dtype == RKV_FP8_E4M3) && G >= 1; }
 
 // Splits of a head's rows: enough blocks for two waves of resident blocks (2 per SM), never finer than a tile.
 int attend_splits(int heads, int cap, int sms, int G, int dtype)
@@ -385,7 +385,7 @@ cudaError_t launch_attend(const void *k_cache, const void *v_cache, const void *
     cudaError_t e;
     if (attend_uses_tc(G, dtype))
         e = launch_attend_tc(k_cache, v_cache, q_new, seq_lens, out, partial, batch, hkv, hq, cap, splits, status, wait_cycles,
-                             block_table, pool_pages, s);
+                             block_table, pool_pages, dtype == RKV_FP8_E4M3, s);
     else
         e = launch_dtype<float>(p, G, s);
     if (e != cudaSuccess || splits == 1) return e;

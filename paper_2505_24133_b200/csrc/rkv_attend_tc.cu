@@ -1,5 +1,5 @@
 // Decode-step attention over the compressed cache (Section 3.1, Eq. 1 with one query row per head), tensor-core form
-// for bf16 caches with d = 128:
+// for bf16 and 8-bit caches with d = 128:
 //
 //   out[b][q] = sum_j softmax_j( q_new[b][q] . K[b][q / G][j] / sqrt(d) ) V[b][q / G][j],   j < seq_lens[b]
 //
@@ -20,7 +20,14 @@
 // weights; the sum of the weights is taken from the same parts.  Splits are merged by attend_merge_kernel.
 //
 // Warps 0..3: softmax (thread = TMEM lane = key row of a tile, later = output dimension), warp 4: TMA producer,
-// warp 5: MMA issuer and TMEM owner.  Every mbarrier wait is bounded; on expiry the block records RKV_ERR_TIMEOUT,
+// warp 5: MMA issuer and TMEM owner.
+//
+// 8-bit caches (E4M3 codes, kFp8): the tiles arrive as 128 rows of 128 bytes (a ring of two 16 KB stages) and are
+// widened into one of two bf16 operand tiles by the softmax threads, one row each, on their way to the tensor cores
+// (four raw stages and a single operand tile were measured slower: the chain widen -> product must not serialise); everything else is the same, at half the bytes per cached
+// row.  Rows beyond the length are written as zeros there.
+//
+// Every mbarrier wait is bounded; on expiry the block records RKV_ERR_TIMEOUT,
 // writes zeros and leaves through the common exit that frees TMEM.  No TMA multicast, no cluster launch.
 #include "rkv_sm100.cuh"
 
@@ -38,8 +45,13 @@ constexpr int kTcTileBytes = 2 * kTcHalf;            // 32 KB
 constexpr int kTcSmall = 16 * kHeadDim * 2;          // a [16 x 128] bf16 operand (Q^T or P): two [16 x 64] halves of 2 KB
 constexpr uint32_t kTcTmemCols = 256;                // 16 (output) + 16 per key tile
 
-constexpr int kOffRing = 0;
+constexpr int kOffRing = 0;                          // bf16 caches: kTcStages tiles.  8-bit caches: kConvBufs widened tiles,
+constexpr int kConvBufs = 2;
+constexpr int kRawStages = 2;
+constexpr int kOffRaw = kConvBufs * kTcTileBytes;    // then kRawStages raw stages of 16 KB
+constexpr int kRawBytes = kTile * kHeadDim;          // a tile of E4M3 codes
 constexpr int kOffQ = kOffRing + kTcStages * kTcTileBytes;
+static_assert(kOffRaw + kRawStages * kRawBytes <= kOffQ, "the 8-bit layout fits the room of the ring");
 constexpr int kOffP = kOffQ + kTcSmall;              // two buffers
 constexpr int kOffRed = kOffP + 2 * kTcSmall;        // [4 warps][8] floats: reductions over the softmax threads
 constexpr int kOffBars = kOffRed + 4 * 8 * 4;
@@ -51,7 +63,9 @@ enum {
     kBarPFull,                           // [2] P tile written (128 softmax threads)
     kBarPEmpty = kBarPFull + 2,          // [2] ... read by the tensor cores
     kBarOut = kBarPEmpty + 2,            // the output columns are final
-    kTcNumBars
+    kBarRawFull,                                 // [kRawStages] 8-bit caches: codes landed
+    kBarRawEmpty = kBarRawFull + kRawStages,     // [kRawStages] ... widened (128 softmax threads)
+    kTcNumBars = kBarRawEmpty + kRawStages
 };
 constexpr int kOffMisc = kOffBars + kTcNumBars * 8;  // TMEM base, abort flag
 constexpr int kTcSmem = kOffMisc + 16 + 1024;        // + slack for the 1024-byte alignment
@@ -95,7 +109,8 @@ __device__ __forceinline__ uint32_t small_off(int g, int k)
     return (uint32_t)(half * (kTcSmall / 2) + g * 128 + ((((kk >> 3) ^ (g & 7)) << 4) | ((kk & 7) << 1)));
 }
 
-template <int G>
+// With kFp8, kBarFull / kBarEmpty [0 .. kConvBufs) stand for the widened tiles (filled by the softmax threads, 128 arrivals).
+template <int G, bool kFp8>
 __global__ void __launch_bounds__(kTcThreads, 2)
 attend_tc_kernel(AttendTcParams p, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                  const __grid_constant__ CUtensorMap map_q)
@@ -141,8 +156,12 @@ attend_tc_kernel(AttendTcParams p, const __grid_constant__ CUtensorMap map_k, co
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kTcStages; ++s) {
-            mbar_init(bar(kBarFull + s), 1);
+            mbar_init(bar(kBarFull + s), kFp8 ? 128 : 1);
             mbar_init(bar(kBarEmpty + s), 1);
+        }
+        for (int s = 0; s < kRawStages; ++s) {
+            mbar_init(bar(kBarRawFull + s), 1);
+            mbar_init(bar(kBarRawEmpty + s), 128);
         }
         mbar_init(bar(kBarQ), 1);
         mbar_init(bar(kBarScores), 1);
@@ -181,14 +200,21 @@ attend_tc_kernel(AttendTcParams p, const __grid_constant__ CUtensorMap map_k, co
             tma_load_2d(sbase + kOffQ, &map_q, 0, qy, bar(kBarQ));
             tma_load_2d(sbase + kOffQ + kTcSmall / 2, &map_q, 64, qy, bar(kBarQ));
             for (int i = 0; i < 2 * T; ++i) {                // the K tiles, then the V tiles
-                const int s = i % kTcStages;
-                if (!mbar_wait(bar(kBarEmpty + s), ((i / kTcStages) & 1) ^ 1, abort_flag, sink)) break;
                 const CUtensorMap *map = i < T ? &map_k : &map_v;
                 const int y = tile_y(t0 + (i < T ? i : i - T));
-                const uint32_t dst = sbase + kOffRing + s * kTcTileBytes;
-                mbar_expect_tx(bar(kBarFull + s), kTcTileBytes);
-                tma_load_2d(dst, map, 0, y, bar(kBarFull + s));
-                tma_load_2d(dst + kTcHalf, map, 64, y, bar(kBarFull + s));
+                if (kFp8) {
+                    const int s = i % kRawStages;
+                    if (!mbar_wait(bar(kBarRawEmpty + s), ((i / kRawStages) & 1) ^ 1, abort_flag, sink)) break;
+                    mbar_expect_tx(bar(kBarRawFull + s), kRawBytes);
+                    tma_load_2d(sbase + kOffRaw + s * kRawBytes, map, 0, y, bar(kBarRawFull + s));
+                } else {
+                    const int s = i % kTcStages;
+                    if (!mbar_wait(bar(kBarEmpty + s), ((i / kTcStages) & 1) ^ 1, abort_flag, sink)) break;
+                    const uint32_t dst = sbase + kOffRing + s * kTcTileBytes;
+                    mbar_expect_tx(bar(kBarFull + s), kTcTileBytes);
+                    tma_load_2d(dst, map, 0, y, bar(kBarFull + s));
+                    tma_load_2d(dst + kTcHalf, map, 64, y, bar(kBarFull + s));
+                }
             }
         }
         __syncwarp();
@@ -197,9 +223,10 @@ attend_tc_kernel(AttendTcParams p, const __grid_constant__ CUtensorMap map_k, co
         if (lane == 0) {
             bool ok = mbar_wait(bar(kBarQ), 0, abort_flag, sink);
             const uint32_t idesc_s = instr_desc(kTile, 16);
+            constexpr int kBufs = kFp8 ? kConvBufs : kTcStages;      // operand tiles the tensor cores read from
             for (int t = 0; t < T && ok; ++t) {              // scores of key tile t into its own 16 columns
-                const int s = t % kTcStages;
-                ok = mbar_wait(bar(kBarFull + s), (t / kTcStages) & 1, abort_flag, sink);
+                const int s = t % kBufs;
+                ok = mbar_wait(bar(kBarFull + s), (t / kBufs) & 1, abort_flag, sink);
                 if (!ok) break;
                 tc_fence_after();
                 umma_tile_k128_halves(tmem + 16 + 16 * t, sbase + kOffRing + s * kTcTileBytes, kTcHalf, sbase + kOffQ,
@@ -210,8 +237,8 @@ attend_tc_kernel(AttendTcParams p, const __grid_constant__ CUtensorMap map_k, co
             // f32 accumulate, bf16 x bf16, A MN-major (bit 15), B K-major, M = 128, N = 16
             const uint32_t idesc_o = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | ((16u >> 3) << 17) | ((128u >> 4) << 24);
             for (int t = 0; t < T && ok; ++t) {              // O^T += V_t^T . P_t
-                const int i = T + t, s = i % kTcStages, pb = t & 1;
-                ok = mbar_wait(bar(kBarFull + s), (i / kTcStages) & 1, abort_flag, sink) &&
+                const int i = T + t, s = i % kBufs, pb = t & 1;
+                ok = mbar_wait(bar(kBarFull + s), (i / kBufs) & 1, abort_flag, sink) &&
                      mbar_wait(bar(kBarPFull + pb), (t >> 1) & 1, abort_flag, sink);
                 if (!ok) break;
                 tc_fence_after();
@@ -236,7 +263,35 @@ attend_tc_kernel(AttendTcParams p, const __grid_constant__ CUtensorMap map_k, co
         const int r = threadIdx.x;                                   // TMEM lane: key row of a tile, later output dimension
         const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
         const float c2 = 1.4426950408889634f * rsqrtf((float)kHeadDim);      // scores in the base-2 domain
-        bool ok = mbar_wait(bar(kBarScores), 0, abort_flag, sink);
+        // 8-bit caches: source tile i (the K tiles, then the V tiles) from its raw stage into a bf16 operand buffer, this
+        // thread's row; a row beyond the length becomes zeros
+        auto widen_tile = [&](int i) -> bool {
+            const int s = i % kRawStages, cb = i % kConvBufs;
+            if (!mbar_wait(bar(kBarRawFull + s), (i / kRawStages) & 1, abort_flag, sink)) return false;
+            if (!mbar_wait(bar(kBarEmpty + cb), ((i / kConvBufs) & 1) ^ 1, abort_flag, sink)) return false;
+            const bool row_valid = (t0 + (i < T ? i : i - T)) * kTile + r < L;
+            const uint8_t *raw = smem + kOffRaw + s * kRawBytes + r * 128;
+            uint8_t *dst = smem + kOffRing + cb * kTcTileBytes + r * 128;
+            uint4 codes[8];                                  // the whole row first: the loads must not wait for the stores
+#pragma unroll
+            for (int c = 0; c < 8; ++c) codes[c] = *reinterpret_cast<const uint4 *>(raw + ((c ^ (r & 7)) << 4));
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {                    // codes 16 c .. 16 c + 15 -> the row's bf16 chunks 2 c and 2 c + 1
+                uint4 lo = make_uint4(0u, 0u, 0u, 0u), hi = lo;
+                if (row_valid) widen16(codes[c], &lo, &hi);
+                const int half = c >> 2, pos = (2 * c) & 7;
+                *reinterpret_cast<uint4 *>(dst + half * kTcHalf + ((pos ^ (r & 7)) << 4)) = lo;
+                *reinterpret_cast<uint4 *>(dst + half * kTcHalf + (((pos + 1) ^ (r & 7)) << 4)) = hi;
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");       // generic writes -> tensor-core reads
+            mbar_arrive(bar(kBarFull + cb));
+            mbar_arrive(bar(kBarRawEmpty + s));
+            return true;
+        };
+        bool ok = true;
+        if (kFp8)
+            for (int t = 0; t < T && ok; ++t) ok = widen_tile(t);
+        if (ok) ok = mbar_wait(bar(kBarScores), 0, abort_flag, sink);
         float m[G], l[G];
 #pragma unroll
         for (int g = 0; g < G; ++g) m[g] = -INFINITY, l[g] = 0.f;
@@ -265,7 +320,8 @@ attend_tc_kernel(AttendTcParams p, const __grid_constant__ CUtensorMap map_k, co
 
         for (int t = 0; t < T && ok; ++t) {
             const int pb = t & 1;
-            ok = mbar_wait(bar(kBarPEmpty + pb), ((t >> 1) & 1) ^ 1, abort_flag, sink);
+            if (kFp8) ok = widen_tile(T + t);
+            if (ok) ok = mbar_wait(bar(kBarPEmpty + pb), ((t >> 1) & 1) ^ 1, abort_flag, sink);
             if (!ok) break;
             uint32_t acc[16];
             tmem_ld16(lane_base + 16 + 16 * t, acc);
@@ -282,7 +338,7 @@ attend_tc_kernel(AttendTcParams p, const __grid_constant__ CUtensorMap map_k, co
                 *reinterpret_cast<__nv_bfloat16 *>(pt + small_off(g, r)) = hi;
                 *reinterpret_cast<__nv_bfloat16 *>(pt + small_off(8 + g, r)) = lo;
             }
-            if (!valid) {
+            if (!kFp8 && !valid) {
                 // a row beyond the sequence's length may hold anything, and 0 x NaN would spoil the product: its V row
                 // is cleared in shared memory (only the split's last tile has such rows)
                 const int i = T + t, s = i % kTcStages;
@@ -343,14 +399,35 @@ attend_tc_kernel(AttendTcParams p, const __grid_constant__ CUtensorMap map_k, co
     }
 }
 
-template <int G>
-cudaError_t launch_tc_for(const AttendTcParams &p, const CUtensorMap &mk, const CUtensorMap &mv, const CUtensorMap &mq,
+template <int G, bool kFp8>
+cudaError_t launch_tc_one(const AttendTcParams &p, const CUtensorMap &mk, const CUtensorMap &mv, const CUtensorMap &mq,
                           cudaStream_t s)
 {
-    cudaError_t e = cudaFuncSetAttribute(attend_tc_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem);
+    cudaError_t e = cudaFuncSetAttribute(attend_tc_kernel<G, kFp8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem);
     if (e != cudaSuccess) return e;
-    attend_tc_kernel<G><<<(unsigned)(p.batch * p.hkv * p.splits), kTcThreads, kTcSmem, s>>>(p, mk, mv, mq);
+    attend_tc_kernel<G, kFp8><<<(unsigned)(p.batch * p.hkv * p.splits), kTcThreads, kTcSmem, s>>>(p, mk, mv, mq);
     return cudaGetLastError();
+}
+template <int G>
+cudaError_t launch_tc_for(const AttendTcParams &p, bool fp8, const CUtensorMap &mk, const CUtensorMap &mv, const CUtensorMap &mq,
+                          cudaStream_t s)
+{
+    return fp8 ? launch_tc_one<G, true>(p, mk, mv, mq, s) : launch_tc_one<G, false>(p, mk, mv, mq, s);
+}
+
+// 2-D view [rows][128] of a cache of E4M3 codes (128-byte rows), boxes of 128 rows, 128-byte swizzle, out-of-range
+// rows read as zero.
+bool make_map_codes(CUtensorMap *map, const void *base, uint64_t rows)
+{
+    sm100::EncodeTiledFn fn = sm100::encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)kHeadDim};
+    const cuuint32_t box[2] = {(cuuint32_t)kHeadDim, (cuuint32_t)kTile};
+    const cuuint32_t estr[2] = {1u, 1u};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 }  // namespace
@@ -368,7 +445,7 @@ int attend_tc_splits(int heads, int cap, int sms)
 
 cudaError_t launch_attend_tc(const void *k_cache, const void *v_cache, const void *q_new, const int32_t *seq_lens, float *out,
                              float *partial, int batch, int hkv, int hq, int cap, int splits, int32_t *status,
-                             long long wait_cycles, const int32_t *block_table, long long pool_pages, cudaStream_t s)
+                             long long wait_cycles, const int32_t *block_table, long long pool_pages, bool fp8, cudaStream_t s)
 {
     const int tiles = (cap + kTile - 1) / kTile;
     AttendTcParams p;
@@ -387,18 +464,18 @@ cudaError_t launch_attend_tc(const void *k_cache, const void *v_cache, const voi
     if (p.tiles_per_split > kTcMaxTiles) return cudaErrorInvalidValue;
     const uint64_t rows = block_table ? (uint64_t)pool_pages * kTile : (uint64_t)batch * hkv * cap;
     CUtensorMap mk, mv, mq;
-    if (!sm100::make_map(&mk, k_cache, rows, kTile) || !sm100::make_map(&mv, v_cache, rows, kTile) ||
-        !sm100::make_map(&mq, q_new, (uint64_t)batch * hq, 16))
-        return cudaErrorInvalidValue;
+    const bool maps_ok = fp8 ? (make_map_codes(&mk, k_cache, rows) && make_map_codes(&mv, v_cache, rows))
+                             : (sm100::make_map(&mk, k_cache, rows, kTile) && sm100::make_map(&mv, v_cache, rows, kTile));
+    if (!maps_ok || !sm100::make_map(&mq, q_new, (uint64_t)batch * hq, 16)) return cudaErrorInvalidValue;
     switch (hq / hkv) {
-        case 1: return launch_tc_for<1>(p, mk, mv, mq, s);
-        case 2: return launch_tc_for<2>(p, mk, mv, mq, s);
-        case 3: return launch_tc_for<3>(p, mk, mv, mq, s);
-        case 4: return launch_tc_for<4>(p, mk, mv, mq, s);
-        case 5: return launch_tc_for<5>(p, mk, mv, mq, s);
-        case 6: return launch_tc_for<6>(p, mk, mv, mq, s);
-        case 7: return launch_tc_for<7>(p, mk, mv, mq, s);
-        case 8: return launch_tc_for<8>(p, mk, mv, mq, s);
+        case 1: return launch_tc_for<1>(p, fp8, mk, mv, mq, s);
+        case 2: return launch_tc_for<2>(p, fp8, mk, mv, mq, s);
+        case 3: return launch_tc_for<3>(p, fp8, mk, mv, mq, s);
+        case 4: return launch_tc_for<4>(p, fp8, mk, mv, mq, s);
+        case 5: return launch_tc_for<5>(p, fp8, mk, mv, mq, s);
+        case 6: return launch_tc_for<6>(p, fp8, mk, mv, mq, s);
+        case 7: return launch_tc_for<7>(p, fp8, mk, mv, mq, s);
+        case 8: return launch_tc_for<8>(p, fp8, mk, mv, mq, s);
         default: return cudaErrorInvalidValue;
     }
 }

@@ -3,6 +3,7 @@
 #pragma once
 
 #include <cuda_bf16.h>
+#include <cuda_fp8.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -180,6 +181,28 @@ template <> struct Elem<float> {
     }
 };
 
+// 16 E4M3 codes -> 16 bf16 values (the conversion instruction goes through f16, which holds every E4M3 value too).
+// (Measured against integer / packed-bf16 decodes of the codes -- shift the low seven bits into a bf16 pattern and
+// multiply by 2^120 --: those were exact too, but slower in the kernel that widens tiles on their way to the tensor
+// cores.)
+__device__ __forceinline__ void widen16(const uint4 &codes, uint4 *lo, uint4 *hi)
+{
+    const uint32_t w[4] = {codes.x, codes.y, codes.z, codes.w};
+    uint32_t out[8];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const __half2_raw pair = __nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)((w[q] >> (16 * h)) & 0xFFFFu), __NV_E4M3);
+            const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&pair));
+            const __nv_bfloat162 b2 = __floats2bfloat162_rn(f.x, f.y);
+            out[2 * q + h] = *reinterpret_cast<const uint32_t *>(&b2);
+        }
+    }
+    *lo = make_uint4(out[0], out[1], out[2], out[3]);
+    *hi = make_uint4(out[4], out[5], out[6], out[7]);
+}
+
 // launchers (one per stage); each returns cudaGetLastError() of its launch
 cudaError_t launch_prep(const Params &p, cudaStream_t s);
 cudaError_t launch_widen_keys(const Params &stored, __nv_bfloat16 *wide, cudaStream_t s);
@@ -197,7 +220,7 @@ cudaError_t launch_attend(const void *k_cache, const void *v_cache, const void *
                           long long wait_cycles, const int32_t *block_table, long long pool_pages, cudaStream_t s);
 cudaError_t launch_attend_tc(const void *k_cache, const void *v_cache, const void *q_new, const int32_t *seq_lens, float *out,
                              float *partial, int batch, int hkv, int hq, int cap, int splits, int32_t *status,
-                             long long wait_cycles, const int32_t *block_table, long long pool_pages, cudaStream_t s);
+                             long long wait_cycles, const int32_t *block_table, long long pool_pages, bool fp8, cudaStream_t s);
 int attend_tc_splits(int heads, int cap, int sms);
 int attend_max_group();
 int attend_splits(int heads, int cap, int sms, int G, int dtype);

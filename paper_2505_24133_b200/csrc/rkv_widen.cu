@@ -8,8 +8,6 @@
 // stages that read whole 128-row tiles meet no stale bit patterns.
 //
 // HBM-bound: 1 byte read and 2 written per element, 16 elements per thread and step.
-#include <cuda_fp8.h>
-
 #include "rkv_common.cuh"
 
 namespace rkv {
@@ -17,25 +15,6 @@ namespace rkv {
 namespace {
 
 constexpr int kWidenThreads = 256;
-
-// 16 E4M3 codes -> 16 bf16 values (the conversion instruction goes through f16, which holds every E4M3 value too)
-__device__ __forceinline__ void widen16(const uint4 &codes, uint4 *lo, uint4 *hi)
-{
-    const uint32_t w[4] = {codes.x, codes.y, codes.z, codes.w};
-    uint32_t out[8];
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            const __half2_raw pair = __nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)((w[q] >> (16 * h)) & 0xFFFFu), __NV_E4M3);
-            const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&pair));
-            const __nv_bfloat162 b2 = __floats2bfloat162_rn(f.x, f.y);
-            out[2 * q + h] = *reinterpret_cast<const uint32_t *>(&b2);
-        }
-    }
-    *lo = make_uint4(out[0], out[1], out[2], out[3]);
-    *hi = make_uint4(out[4], out[5], out[6], out[7]);
-}
 
 // Block x: 128-row tile x % tiles of head-problem x / tiles.  vec_per_row = d / 16 (16-byte vectors of a stored row).
 __global__ void __launch_bounds__(kWidenThreads) widen_keys_kernel(Params p, __nv_bfloat16 *wide, int vec_per_row)

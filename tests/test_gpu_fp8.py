@@ -175,12 +175,90 @@ def test_fp8_append_push_and_host_entry_points(rkv):
     assert torch.equal(hv[:, :, :b], wl.v_cache.view(torch.uint8)[:, :, :b].cpu())
 
 
-def test_fp8_decode_attention_is_refused(rkv):
-    spec = small_spec("fp8_att", batch=2, hkv=2, hq=8, budget=256, buffer=64, dtype="fp8")
-    wl = ri.make_workload(spec, device="cuda", seed=361)
-    comp = rkv.Compressor(2, 2, 8, spec.budget, spec.buffer, spec.alpha, 0.1, dtype=FP8)
-    assert rkv.rkv_decode_workspace_bytes(comp.desc, spec.budget, spec.buffer) == 0
-    out = torch.zeros(2, 8, 128, device="cuda")
-    q_new = torch.zeros(2, 8, 128, device="cuda", dtype=torch.bfloat16)
-    rc = rkv.rkv_decode_attention(comp.desc, wl.k_cache, wl.v_cache, q_new, wl.seq_lens, out, spec.budget, spec.buffer)
-    assert rc == 2 and rkv.rkv_status_string(rc) == "RKV_ERR_UNSUPPORTED"
+@pytest.mark.parametrize("hkv,hq,budget,buffer,lens", [(2, 8, 300, 84, [384, 1, 0, 200, 129]),
+                                                       (1, 7, 4096, 128, [4224, 1, 0, 3000, 129]),
+                                                       (2, 10, 1920, 128, [2048, 2047, 1921, 100, 128])])
+def test_fp8_decode_attention_matches_the_oracle(rkv, hkv, hq, budget, buffer, lens):
+    """Section 3.1's decode step over 8-bit caches (bf16 queries): the codes are widened on their way to the tensor
+    cores, so the result is the attention over the values they stand for; ragged lengths, an empty and a one-token
+    cache, stale rows full of NaN codes, one to several splits per head."""
+    import oracle
+    spec = small_spec("fp8_att", batch=5, hkv=hkv, hq=hq, budget=budget, buffer=buffer, dtype="fp8")
+    wl = ri.make_workload(spec, device="cuda", seed=361 + hq, seq_lens=torch.tensor(lens))
+    _stale_rows_to_nan(wl, lens)
+    g = torch.Generator(device="cuda").manual_seed(7)
+    q_new = torch.randn(5, hq, 128, generator=g, device="cuda").to(torch.bfloat16)
+    comp = rkv.Compressor(5, hkv, hq, budget, buffer, spec.alpha, 0.1, dtype=FP8)
+    assert rkv.rkv_decode_workspace_bytes(comp.desc, budget, buffer) <= comp.workspace.numel()
+    out = torch.full((5, hq, 128), 7.0, dtype=torch.float32, device="cuda")
+    rc = rkv.rkv_decode_attention(comp.desc, wl.k_cache, wl.v_cache, q_new, wl.seq_lens, out, budget, buffer)
+    assert rc == rkv.RKV_OK, rkv.rkv_status_string(rc)
+    torch.cuda.synchronize()
+    comp.check_status()
+    K = np.nan_to_num(oracle.e4m3_to_f32(wl.k_cache.view(torch.uint8).cpu().numpy()), nan=0.0)
+    V = np.nan_to_num(oracle.e4m3_to_f32(wl.v_cache.view(torch.uint8).cpu().numpy()), nan=0.0)
+    ref = oracle.oracle_decode_attention(K, V, q_new.float().cpu().numpy(), np.array(lens, dtype=np.int32))
+    got = out.cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all()
+    scale = np.maximum(np.abs(ref).max(axis=-1, keepdims=True), 1e-30)
+    assert (np.abs(got - ref) <= 1e-3 * scale + 1e-7).all(), float((np.abs(got - ref) / scale).max())
+    for b, L in enumerate(lens):
+        if L == 0:
+            assert not got[b].any()                           # empty cache: zero rows
+
+
+def test_fp8_decode_attention_paged_equals_contiguous(rkv):
+    """The same call through a block table over 8-bit page pools: bit for bit the result on the contiguous caches."""
+    spec = small_spec("fp8_att_paged", batch=4, hkv=1, hq=8, budget=896, buffer=128, dtype="fp8")
+    lens = [1024, 127, 129, 700]
+    wl = ri.make_workload(spec, device="cuda", seed=371, seq_lens=torch.tensor(lens))
+    pages, pool_pages = spec.cap // 128, 4 * 8 + 5
+    table = random_block_table(4, 1, pages, pool_pages, seed=14)
+    kp = to_paged(wl.k_cache.view(torch.uint8), pool_pages, table, fill=NAN_CODE).view(FP8)
+    vp = to_paged(wl.v_cache.view(torch.uint8), pool_pages, table, fill=NAN_CODE).view(FP8)
+    g = torch.Generator(device="cuda").manual_seed(4)
+    q_new = torch.randn(4, 8, 128, generator=g, device="cuda").to(torch.bfloat16)
+    outs = []
+    for k, v, kw in ((wl.k_cache, wl.v_cache, {}), (kp, vp, dict(block_table=table, pool_pages=pool_pages))):
+        comp = rkv.Compressor(4, 1, 8, spec.budget, spec.buffer, spec.alpha, 0.1, dtype=FP8, **kw)
+        out = torch.empty(4, 8, 128, dtype=torch.float32, device="cuda")
+        assert rkv.rkv_decode_attention(comp.desc, k, v, q_new, wl.seq_lens, out, spec.budget, spec.buffer) == rkv.RKV_OK
+        torch.cuda.synchronize()
+        comp.check_status()
+        outs.append(out)
+    assert torch.equal(outs[0], outs[1])
+
+
+def test_fp8_every_code_through_the_attention_and_the_widening_kernels(rkv):
+    """All 254 finite E4M3 codes, subnormals and both zeros included, pass through the kernels' own decode exactly:
+    with a one-token cache the attention's output row IS the value row (weight 1), and a compression call on keys made
+    of every code agrees with the oracle's decode of them (the widening kernel feeds every scoring stage)."""
+    import oracle
+    codes = torch.arange(256, dtype=torch.uint8)
+    codes[0x7F], codes[0xFF] = 0x7E, 0xFE                     # the two NaN codes: replaced by the largest finite ones
+    v = torch.zeros(2, 1, 128, 128, dtype=torch.uint8)
+    v[0, 0, 0], v[1, 0, 0] = codes[:128], codes[128:]
+    k = torch.full((2, 1, 128, 128), 0x38, dtype=torch.uint8)                 # keys: all ones
+    lens = torch.tensor([1, 1], dtype=torch.int32, device="cuda")
+    d = rkv.rkv_desc_default()
+    d.batch, d.n_kv_heads, d.n_q_heads, d.dtype = 2, 1, 4, rkv.RKV_FP8_E4M3
+    q_new = torch.randn(2, 4, 128, device="cuda").to(torch.bfloat16)
+    out = torch.empty(2, 4, 128, dtype=torch.float32, device="cuda")
+    need = rkv.rkv_decode_workspace_bytes(d, 100, 28)
+    ws = torch.empty(max(need, 256), dtype=torch.uint8, device="cuda")
+    d.workspace, d.workspace_bytes = ws.data_ptr(), ws.numel()
+    rc = rkv.rkv_decode_attention(d, k.cuda().view(FP8), v.cuda().view(FP8), q_new, lens, out, 100, 28)
+    assert rc == rkv.RKV_OK
+    torch.cuda.synchronize()
+    want = oracle.e4m3_to_f32(codes.numpy())
+    got = out.cpu().numpy()
+    for g in range(4):
+        assert np.array_equal(got[0, g], want[:128]) and np.array_equal(got[1, g], want[128:])
+    # keys holding every code, through the widening kernel and a whole compression call
+    spec = small_spec("fp8_codes", batch=1, hkv=1, hq=4, budget=200, buffer=56, dtype="fp8")
+    wl = ri.make_workload(spec, device="cuda", seed=381)
+    kb = wl.k_cache.view(torch.uint8)
+    gen = torch.Generator().manual_seed(3)
+    kb[0, 0, :64] = codes[torch.randint(0, 256, (64, 128), generator=gen)].cuda()
+    rep, comp = run_and_check(rkv, wl)
+    assert rep.ok(), rep.errors
