@@ -387,11 +387,11 @@ constexpr int kFinishThreads = 256;
 
 __global__ void __launch_bounds__(kFinishThreads) dense_finish_kernel(Params p)
 {
-    // work unit = (head, chunk of 256 tokens), handed out with the grid as stride: when no head took the route (the
-    // common case) a block runs through its units in a few microseconds instead of the launch paying for a block each
+    // work unit = (head, chunk of 256 tokens), handed out with the grid as stride.  When no head took the route (the
+    // common case: no work item of the symmetric scan was ever listed) the blocks return at once.
     const int chunks = (p.cap + kFinishThreads - 1) / kFinishThreads;
     const long long units = (long long)p.batch * p.hkv * chunks;
-    if (call_aborted(p)) return;
+    if (call_aborted(p) || p.counters[kDenseWords] == 0ull) return;
     for (long long u = blockIdx.x; u < units; u += gridDim.x) {
     const int head = (int)(u / chunks);
     if (!p.dense[head]) continue;
