@@ -193,7 +193,7 @@ def stream_measure(rkv, rd, dev, rank, spec, stream_tokens):
     Appending the seeded blocks is not timed; each firing is bracketed by CUDA events on the call's stream."""
     k, v, seq, gen, scale = ri.stream_state(spec, device=dev, seed=ri.BASE_SEED + 5 + 1000 * rank)
     comp = rkv.Compressor(spec.folded_batch, spec.n_kv_heads, spec.n_q_heads, spec.budget, spec.buffer, spec.alpha,
-                          spec.lam, dtype=spec.torch_dtype, device=dev)
+                          spec.lam, dtype=spec.torch_dtype, head_dim=spec.head_dim, device=dev)
     stream = torch.cuda.current_stream()
     firings = stream_tokens // spec.buffer
     rd.barrier()
@@ -341,7 +341,7 @@ def kernel_table(rkv, timed: Timed, kw, KB, peaks):
     rate against the roofline that bounds it."""
     spec, wl, dev = timed.spec, timed.wl, timed.dev
     comp_ev = rkv.Compressor(spec.folded_batch, spec.n_kv_heads, spec.n_q_heads, spec.budget, spec.buffer, spec.alpha,
-                             spec.lam, dtype=spec.torch_dtype, device=dev, stage_events=True, **kw)
+                             spec.lam, dtype=spec.torch_dtype, head_dim=spec.head_dim, device=dev, stage_events=True, **kw)
     names = list(comp_ev.KERNEL_NAMES)
     kernel_ms = [0.0] * len(names)
     tiles_executed = pairs2 = moved_rows = 0
@@ -361,22 +361,25 @@ def kernel_table(rkv, timed: Timed, kw, KB, peaks):
     n = spec.cap - spec.alpha
     esz = wl.k_cache.element_size()
     row = spec.head_dim * esz
+    wide_row = max(spec.head_dim, 128 if spec.head_dim == 64 else 0) * 2       # a row of the bf16 scoring copy (8-bit caches, d = 64)
     P = spec.head_problems
     T = (n + 127) // 128
     q_cols = -(-(spec.n_q_heads // spec.n_kv_heads) * spec.alpha // 16) * 16 + 16
     # one tile product = 128 x 128 outputs over K = 128 + 16: the head dimension plus the one extra K = 16 step that
     # folds the threshold test into the accumulator (both scoring passes issue it for every key tile)
-    tile_flops = 2.0 * 128 * 128 * (128 + 16)
+    # (head dimension 64 runs on keys padded to 128: the padding's products are not counted as work)
+    tile_flops = 2.0 * 128 * 128 * (spec.head_dim + 16)
     rule_on = comp_ev.desc.beta > 0 and comp_ev.desc.sim_threshold < 1.0
     pass1_tiles = P * T if rule_on else 0              # every row tile meets the last key tile once
-    pass1_flops = pass1_tiles * tile_flops + P * T * 2.0 * 128 * q_cols * 128
+    pass1_flops = pass1_tiles * tile_flops + P * T * 2.0 * 128 * q_cols * spec.head_dim
     pass2_flops = max(tiles_executed - pass1_tiles, 0) * tile_flops
     pass2_useful = pairs2 * 2.0 * 128 * (128 + 16)     # listed tokens x keys of the streamed tiles x 2 (d + 16)
     # algorithmic work per launch: bytes a kernel has to move / flops it has to execute, nothing it merely could
     work = {
-        # K once; r_i, Kbar_i.Kbar_i and the 32-byte slice out.  8-bit caches: the codes in, their bf16 copy out and in again
-        "prep": ("hbm", P * (n * row + spec.cap * (8 + 32)) if esz > 1 else
-                 P * (spec.cap * row + spec.cap * 2 * row + n * 2 * row + spec.cap * (8 + 32))),
+        # K once; r_i, Kbar_i.Kbar_i and the 32-byte slice out.  8-bit caches and d = 64: the stored keys in, their bf16 /
+        # padded copy out and in again
+        "prep": ("hbm", P * (n * row + spec.cap * (8 + 32)) if (esz > 1 and spec.head_dim != 64) else
+                 P * (spec.cap * row + spec.cap * wide_row + n * wide_row + spec.cap * (8 + 32))),
         "scores_pass1": ("tensor", pass1_flops),
         "scores_list": ("hbm", P * n * 8),
         "scores_pass2": ("tensor", pass2_flops),
@@ -443,7 +446,7 @@ def measure_e2e(rkv, rd, dev, wl, kw, KE, toks):
     esz = wl.k_cache.element_size()
     row = spec.head_dim * esz
     ch = rkv.Compressor(spec.folded_batch, spec.n_kv_heads, spec.n_q_heads, spec.budget, spec.buffer, spec.alpha,
-                        spec.lam, dtype=spec.torch_dtype, device=dev, host_staging=True, **kw)
+                        spec.lam, dtype=spec.torch_dtype, head_dim=spec.head_dim, device=dev, host_staging=True, **kw)
     hk = torch.empty(wl.k_cache.shape, dtype=wl.k_cache.dtype, pin_memory=True)
     hv = torch.empty(wl.v_cache.shape, dtype=wl.v_cache.dtype, pin_memory=True)
     hq = wl.q_window.cpu().pin_memory()
@@ -535,7 +538,7 @@ def side_config(rkv, rd, dev, wl, kw, K, W, mem_gb, peaks):
     spec = wl.spec
     timed = Timed(rkv, rd, dev, wl, mem_gb, K + W)
     comp = rkv.Compressor(spec.folded_batch, spec.n_kv_heads, spec.n_q_heads, spec.budget, spec.buffer, spec.alpha,
-                          spec.lam, dtype=spec.torch_dtype, device=dev, **kw)
+                          spec.lam, dtype=spec.torch_dtype, head_dim=spec.head_dim, device=dev, **kw)
     ms_total = timed.run_timed(comp, K, W)
     toks = tokens_per_step(spec)
     value, ms_slowest = rd.whole_job_rate(toks * K, ms_total, dev)
@@ -582,7 +585,7 @@ def main():
     wl = ri.make_workload(spec, device=dev, seed=ri.BASE_SEED + 1000 * rank + list(ri.SPECS).index(args.workload))
     timed = Timed(rkv, rd, dev, wl, args.mem_gb, K + W)
     comp = rkv.Compressor(spec.folded_batch, spec.n_kv_heads, spec.n_q_heads, spec.budget, spec.buffer, spec.alpha,
-                          spec.lam, dtype=spec.torch_dtype, device=dev, **kw)
+                          spec.lam, dtype=spec.torch_dtype, head_dim=spec.head_dim, device=dev, **kw)
     launches_per_step = rkv.rkv_launch_count_for(comp.desc, spec.budget, spec.buffer, spec.alpha, rkv.RKV_STAGE_ALL)
     sampler = ClockSampler(local_rank)
     ms_total = timed.run_timed(comp, K, W, sampler)
@@ -611,7 +614,7 @@ def main():
     # ---- the other configurations, and the settings that defeat the two-pass shortcut, in the same run
     configs = {}
     if not args.no_configs and args.workload == DEFAULT_WORKLOAD and args.batch is None and args.layers is None and not kw:
-        for name, k_side in (("llama8b_b1", 20), ("llama8b_b16", 5), ("qwen7b_b64", 5), ("mha7b_b8", 5), ("llama8b_b16_fp8", 5)):
+        for name, k_side in (("llama8b_b1", 20), ("llama8b_b16", 5), ("qwen7b_b64", 5), ("mha7b_b8", 5), ("llama8b_b16_fp8", 5), ("llama1b_b64_d64", 5)):
             swl = ri.make_workload(ri.SPECS[name], device=dev, seed=ri.BASE_SEED + 1000 * rank + list(ri.SPECS).index(name))
             configs[name] = side_config(rkv, rd, dev, swl, {}, k_side, 3, args.mem_gb, peaks)
             if name == "llama8b_b16":

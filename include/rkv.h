@@ -59,7 +59,7 @@ typedef enum {
  *     no infinities; one byte per element, rows of head_dim bytes); q_window (and q_new of rkv_push_query) is bf16.
  *     Eq. 1-7 are evaluated on the values the codes stand for: the keys are widened to bf16 (exactly; every E4M3 value
  *     is a bf16 value) into the workspace, which grows by (batch * n_kv_heads * (budget + buffer) + 128) * head_dim * 2
- *     bytes, and every scoring stage runs on that copy as for a bf16 cache.  The compaction moves the stored bytes; no
+ *     bytes (nothing more for head_dim 64, whose padded copy exists anyway), and every scoring stage runs on that copy as for a bf16 cache.  The compaction moves the stored bytes; no
  *     scale factor is applied or needed (cosine similarity does not see a per-tensor scale; fold a key scale into
  *     the queries for Eq. 2).  rkv_decode_attention takes this type too (q_new bf16): the codes are widened on their
  *     way to the tensor cores, no copy is kept. */
@@ -106,8 +106,11 @@ typedef struct rkv_desc {
     int32_t batch;       /* sequences; layers that fire together are folded into this dimension */
     int32_t n_kv_heads;  /* KV heads per sequence */
     int32_t n_q_heads;   /* query heads; G = n_q_heads / n_kv_heads must be integral (G = 1: Eq. 1) */
-    int32_t head_dim;    /* d: 64, 128 or 256.  The tensor-core scoring kernels serve bf16 caches with d = 128; other
-                            head dimensions are scored by the CUDA-core kernel (correct, but far slower) */
+    int32_t head_dim;    /* d: 64, 128 or 256.  The tensor-core scoring kernels are built for bf16 keys with d = 128;
+                            bf16 and 8-bit caches with d = 64 are scored by them on a copy of the keys (and of the
+                            observation queries) padded with zeros to 128 in the workspace -- dot products and norms do
+                            not see the padding --; d = 256 and fp32 caches are scored by the CUDA-core kernel
+                            (correct, but far slower) */
     int32_t dtype;       /* rkv_dtype_t of k_cache and v_cache (and of q_window, except for 8-bit caches: bf16) */
     int32_t pool_w;      /* W of Eq. 4; 0 = no pooling.  Range [0, 64].  Default 4 (the paper prints no value) */
     int32_t beta;        /* beta of Section 3.3; 0 = rule off.  Default 1 (the paper prints no value) */

@@ -20,13 +20,14 @@ int cuda_fail(cudaError_t e, const char *where)
 }
 
 struct Layout {
-    size_t k_wide, best, dense, dense_items, inv_norm, norm_split, thr_split, tile_sum, head_sum, logits, row_stat, imp, sbar, left, strag, strag_count, strag_items, self_dot, head_sum_bf16, meta, counters,
+    size_t k_wide, q_wide, best, dense, dense_items, inv_norm, norm_split, thr_split, tile_sum, head_sum, logits, row_stat, imp, sbar, left, strag, strag_count, strag_items, self_dot, head_sum_bf16, meta, counters,
         tile_done, zero_bytes, total;
     int cap, cap_pad, tiles, tri;
 };
 
-// The tensor-core scoring kernels serve bf16 caches with head dimension 128; everything else (fp32 caches, head
-// dimensions 64 and 256, or on request) is scored by the CUDA-core kernel.
+// The tensor-core scoring kernels are built for bf16 keys of 128 dimensions.  bf16 and 8-bit caches of 128 dimensions
+// use them directly (8-bit: on a widened copy), those of 64 dimensions on a copy padded with zeros to 128 (dot products
+// and norms do not see the padding); fp32 caches, 256 dimensions, or a request for it go to the CUDA-core kernel.
 // Bytes of a cache element and of a query element.  8-bit caches (E4M3 codes) are scored on a bf16 copy of their keys
 // in the workspace (every E4M3 value is a bf16 value), with bf16 queries.
 size_t cache_esz(const rkv_desc_t *d) { return d->dtype == RKV_BF16 ? 2 : d->dtype == RKV_F32 ? 4 : 1; }
@@ -34,8 +35,14 @@ size_t query_esz(const rkv_desc_t *d) { return d->dtype == RKV_F32 ? 4 : 2; }
 
 bool use_simt(const rkv_desc_t *d)
 {
-    return d->dtype == RKV_F32 || d->head_dim != kHeadDim || (d->flags & RKV_FLAG_SIMT_SCORES);
+    return d->dtype == RKV_F32 || d->head_dim == 256 || (d->flags & RKV_FLAG_SIMT_SCORES);
 }
+// The head dimension is padded from 64 to 128 in the scoring copy (keys and observation queries).
+bool pads_dim(const rkv_desc_t *d) { return d->head_dim == 64 && !use_simt(d); }
+// The scoring stages read a copy of the keys in the workspace instead of the cache itself.
+bool needs_copy(const rkv_desc_t *d) { return d->dtype == RKV_FP8_E4M3 || pads_dim(d); }
+// Head dimension the scoring stages see.
+int scoring_dim(const rkv_desc_t *d) { return pads_dim(d) ? kHeadDim : d->head_dim; }
 
 // 1 when the triangle tensor-core kernels score (bf16 caches, unless a cross-check kernel is asked for).
 int use_tri(const rkv_desc_t *d) { return !(use_simt(d) || (d->flags & RKV_FLAG_ROWBLOCK_SCORES)); }
@@ -65,13 +72,16 @@ int check_shapes(const rkv_desc_t *d, int budget, int buffer, int alpha, Layout 
         lay->tiles = (int)((cap + kTile - 1) / kTile);
         lay->cap_pad = lay->tiles * kTile;
         size_t off = 0;
-        // 8-bit caches: the keys widened to bf16, head after head, plus one tile of zero rows behind the last head
+        // the scoring copy (8-bit caches, padded head dimension): the keys as bf16, head after head, plus one tile of zero
+        // rows behind the last head; with a padded head dimension the observation queries as well
         lay->k_wide = off;
-        if (d->dtype == RKV_FP8_E4M3) off = align_up(off + (P * lay->cap + kTile) * (size_t)d->head_dim * sizeof(__nv_bfloat16), 256);
+        if (needs_copy(d)) off = align_up(off + (P * lay->cap + kTile) * (size_t)scoring_dim(d) * sizeof(__nv_bfloat16), 256);
+        lay->q_wide = off;
+        if (pads_dim(d)) off = align_up(off + (size_t)d->batch * d->n_q_heads * alpha * kHeadDim * sizeof(__nv_bfloat16), 256);
         lay->inv_norm = off;  off = align_up(off + P * lay->cap_pad * sizeof(float), 256);
         lay->norm_split = off;  off = align_up(off + P * lay->cap_pad * 16 * sizeof(__nv_bfloat16), 256);
         lay->thr_split = off;   off = align_up(off + P * kTile * 16 * sizeof(__nv_bfloat16), 256);
-        const size_t hd = (size_t)d->head_dim;
+        const size_t hd = (size_t)scoring_dim(d);
         lay->tile_sum = off;  off = align_up(off + P * lay->tiles * hd * sizeof(float), 256);
         lay->head_sum = off;  off = align_up(off + P * hd * sizeof(float), 256);
         lay->logits = off;    off = align_up(off + P * alpha * lay->cap_pad * sizeof(float), 256);
@@ -130,6 +140,7 @@ int run(const rkv_desc_t *d, void *k_cache, void *v_cache, const void *q_window,
     p.hq = d->n_q_heads;
     p.group = d->n_q_heads / d->n_kv_heads;
     p.d = d->head_dim;
+    p.logit_scale = 1.0f / sqrtf((float)d->head_dim);
     p.cap = lay.cap;
     p.cap_pad = lay.cap_pad;
     p.tiles = lay.tiles;
@@ -194,15 +205,18 @@ int run(const rkv_desc_t *d, void *k_cache, void *v_cache, const void *q_window,
     // What the gather moves is the caller's caches as they are stored; for 8-bit caches every stage before it reads the
     // bf16 copy of the keys (contiguous: the block table, if any, is followed once, by the widening kernel).
     Params stored = p;
-    if (d->dtype == RKV_FP8_E4M3) {
+    if (needs_copy(d)) {
         p.k_cache = ws + lay.k_wide;
         p.block_table = nullptr;
         p.dtype = RKV_BF16;
+        p.d = scoring_dim(d);
+        if (pads_dim(d)) p.q_window = ws + lay.q_wide;
     }
     if (stages & RKV_STAGE_PREP) {
         if ((e = cudaMemsetAsync(p.counters, 0, p.zero_bytes, s)) != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
-        if (d->dtype == RKV_FP8_E4M3 &&
-            (e = launch_widen_keys(stored, static_cast<__nv_bfloat16 *>(p.k_cache), s)) != cudaSuccess)
+        if (needs_copy(d) &&
+            (e = launch_widen_keys(stored, static_cast<__nv_bfloat16 *>(p.k_cache), p.d, pads_dim(d) ? stored.q_window : nullptr,
+                                   pads_dim(d) ? ws + lay.q_wide : nullptr, s)) != cudaSuccess)
             return cuda_fail(e, "widen launch");
         if ((e = launch_prep(p, s)) != cudaSuccess) return cuda_fail(e, "prep launch");
     }
@@ -432,8 +446,8 @@ int rkv_launch_count(const rkv_desc_t *desc, uint32_t stage_mask)
     for (uint32_t bit = 1; bit <= RKV_STAGE_GATHER; bit <<= 1) c += (stage_mask & bit) ? 1 : 0;
     if (stage_mask & RKV_STAGE_SELECT) c += 2;      // row statistics and importance run ahead of the selection kernel
     // bf16 keys of 128 dimensions: the tile sums are added up per head by a kernel of its own behind the prep kernel
-    if (desc && (stage_mask & RKV_STAGE_PREP) && desc->dtype != RKV_F32 && (desc->head_dim == 0 || desc->head_dim == kHeadDim)) c += 1;
-    if (desc && (stage_mask & RKV_STAGE_PREP) && desc->dtype == RKV_FP8_E4M3) c += 1;       // 8-bit caches: the widening kernel
+    if (desc && (stage_mask & RKV_STAGE_PREP) && desc->dtype != RKV_F32 && (desc->head_dim == 0 || scoring_dim(desc) == kHeadDim)) c += 1;
+    if (desc && (stage_mask & RKV_STAGE_PREP) && needs_copy(desc)) c += 1;       // the kernel that writes the scoring copy
     if (desc && (stage_mask & RKV_STAGE_SELECT) && (desc->flags & RKV_FLAG_HEAD_MEAN)) c += 1;   // per-sequence selection
     // the two-pass scoring path is the first pass plus up to two rounds of (listing, second pass) while the
     // retention rule is on

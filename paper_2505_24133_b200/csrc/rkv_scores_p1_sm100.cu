@@ -269,7 +269,7 @@ scores_stream_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, 
         const int lrow = quad * 32 + lane;       // row within the 128-row tile
         const uint32_t lane_base = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)grp * 256;
         const float kInf = __int_as_float(0x7f800000);
-        const float scale = 0.08838834764831845f;             // 1 / sqrt(128)
+        const float scale = p.logit_scale;                    // 1 / sqrt(d)
         const int G = p.group;
         uint32_t k_item = 0, ccount = 0;         // ccount: tiles of the stream so far (all of them, not only this group's)
         bool ok = true;

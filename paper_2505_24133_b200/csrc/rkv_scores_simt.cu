@@ -103,7 +103,7 @@ __global__ void __launch_bounds__(kSimtThreads) scores_simt_kernel(Params p)
         const int rows = p.group * p.alpha;
         const T *Q = static_cast<const T *>(p.q_window) + ((size_t)b * p.hq + (size_t)h * p.group) * p.alpha * kHeadDim;
         load_tile_rows<T, D, kTile>(Q, 0, rows, tileA);       // query rows g * alpha + j
-        const float scale = rsqrtf((float)kHeadDim);
+        const float scale = p.logit_scale;
         float *logits = p.logits + (size_t)head * p.alpha * p.cap_pad;
         for (int jt = 0; jt < (n_tiles * kTile) / kRowsB; ++jt) {
             __syncthreads();

@@ -279,7 +279,7 @@ scores_sm100_kernel(Params p, const __grid_constant__ CUtensorMap map_k, const _
             // Eq. 2-3: thread = key, all G * alpha logits of that key in its accumulator row
             float *stage_f = reinterpret_cast<float *>(smem + kOffStage);           // [q_rows_pad][128] floats
             float *logits = p.logits + (size_t)head * p.alpha * p.cap_pad;
-            const float scale = 0.08838834764831845f;                             // 1 / sqrt(128)
+            const float scale = p.logit_scale;                                    // 1 / sqrt(d)
             for (int t = 0; t < n_iter; ++t) {
                 const int a = t & 1;
                 const int jt = n_tiles - 1 - t;

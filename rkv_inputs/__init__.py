@@ -78,6 +78,9 @@ CONFIG_ORDER = ["tiny", "llama8b_b1", "llama8b_b16", "qwen7b_b64", "qwen14b_b32"
 # layers x 32 heads, batch 8, budget 2048: beside the five configurations above, which are all grouped-query
 SPECS["mha7b_b8"] = CacheSpec("mha7b_b8", 32, 8, 32, 32, 128, 2048, 128, 8, 0.1, "bf16", 32, 0.30, 0.05, 4, 8.0)
 # the second configuration's shape at batch 16 with the caches stored as 8-bit E4M3 codes (queries stay bf16)
+# a cache with 64-dimensional heads (the shape of a 1B-parameter model of the same family: 16 layers, 8 KV heads x 4
+# query heads), batch 64, budget 2048
+SPECS["llama1b_b64_d64"] = CacheSpec("llama1b_b64_d64", 16, 64, 8, 32, 64, 2048, 128, 8, 0.1, "bf16", 32, 0.30, 0.05, 4, 8.0)
 SPECS["llama8b_b16_fp8"] = CacheSpec("llama8b_b16_fp8", 32, 16, 8, 32, 128, 4096, 128, 8, 0.1, "fp8", 32, 0.30, 0.05, 4, 8.0)
 
 

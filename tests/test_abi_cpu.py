@@ -51,7 +51,8 @@ def test_workspace_size_rules(rkv):
     # invalid shapes give 0
     assert rkv.rkv_workspace_bytes(_desc(rkv, n_q_heads=30), 1024, 128, 8) == 0      # G not integral
     assert rkv.rkv_workspace_bytes(_desc(rkv, head_dim=96), 1024, 128, 8) == 0
-    assert 0 < rkv.rkv_workspace_bytes(_desc(rkv, head_dim=64), 1024, 128, 8) < \
+    # (on the CUDA-core route; on the default route head dimension 64 carries a padded copy of the keys)
+    assert 0 < rkv.rkv_workspace_bytes(_desc(rkv, head_dim=64, flags=rkv.RKV_FLAG_SIMT_SCORES), 1024, 128, 8) < \
         rkv.rkv_workspace_bytes(_desc(rkv, head_dim=256), 1024, 128, 8)
     assert rkv.rkv_workspace_bytes(d, 8, 128, 8) == 0                                # budget <= alpha
     assert rkv.rkv_workspace_bytes(d, 8192, 128, 8) == 0                             # cap > RKV_MAX_CAP
@@ -145,12 +146,23 @@ def test_eight_bit_cache_type_sizes_and_counts(rkv):
         b16 = _desc(rkv, head_dim=hd)
         f8 = _desc(rkv, head_dim=hd, dtype=rkv.RKV_FP8_E4M3)
         w16, w8 = rkv.rkv_workspace_bytes(b16, 1024, 128, alpha), rkv.rkv_workspace_bytes(f8, 1024, 128, alpha)
-        assert w8 == w16 + (P * cap + 128) * hd * 2
+        # head dimension 64: bf16 caches are scored on a copy padded to 128 dimensions as well, so nothing is added
+        assert w8 == w16 + (0 if hd == 64 else (P * cap + 128) * hd * 2)
         h16, h8 = rkv.rkv_host_workspace_bytes(b16, 1024, 128, alpha), rkv.rkv_host_workspace_bytes(f8, 1024, 128, alpha)
         assert (h16 - w16) - (h8 - w8) == 2 * P * cap * hd            # K and V staging: two bytes per element less one
         assert rkv.rkv_launch_count_for(f8, 1024, 128, alpha, rkv.RKV_STAGE_ALL) == \
-            rkv.rkv_launch_count_for(b16, 1024, 128, alpha, rkv.RKV_STAGE_ALL) + 1
+            rkv.rkv_launch_count_for(b16, 1024, 128, alpha, rkv.RKV_STAGE_ALL) + (0 if hd == 64 else 1)
         assert rkv.rkv_launch_count_for(f8, 1024, 128, alpha, rkv.RKV_STAGE_GATHER) == 1
+    # head dimension 64 takes the kernels of head dimension 128 plus the one that writes the padded copy; on the
+    # CUDA-core route (on request) it needs neither the copy nor the extra launches
+    d64, d128 = _desc(rkv, head_dim=64), _desc(rkv)
+    assert rkv.rkv_launch_count_for(d64, 1024, 128, alpha, rkv.RKV_STAGE_ALL) == \
+        rkv.rkv_launch_count_for(d128, 1024, 128, alpha, rkv.RKV_STAGE_ALL) + 1
+    w64, w128 = rkv.rkv_workspace_bytes(d64, 1024, 128, alpha), rkv.rkv_workspace_bytes(d128, 1024, 128, alpha)
+    assert w64 == w128 + (P * cap + 128) * 128 * 2 + 2 * 32 * alpha * 128 * 2
+    s64 = _desc(rkv, head_dim=64, flags=rkv.RKV_FLAG_SIMT_SCORES)
+    assert rkv.rkv_workspace_bytes(s64, 1024, 128, alpha) < w128
+    assert rkv.rkv_launch_count_for(s64, 1024, 128, alpha, rkv.RKV_STAGE_ALL) == 4      # prep, scores, select, gather
     assert rkv.rkv_workspace_bytes(_desc(rkv, dtype=3), 1024, 128, alpha) == 0
     assert rkv.rkv_decode_workspace_bytes(_desc(rkv, dtype=rkv.RKV_FP8_E4M3), 1024, 128) == \
         rkv.rkv_decode_workspace_bytes(_desc(rkv), 1024, 128) > 0       # the attention takes 8-bit caches like bf16 ones

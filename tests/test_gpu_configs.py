@@ -48,11 +48,13 @@ def test_config2_simt_and_tcgen05_agree(rkv):
                                                        1555, 1700, 1791]),
                                        ("qwen14b_b32", [5, 200, 410, 777, 901, 1203, 1400, 1535]),
                                        ("mha7b_b8", [3, 250]),
-                                       ("llama8b_b16_fp8", [1, 77, 140, 222, 300, 399, 460, 510])])
+                                       ("llama8b_b16_fp8", [1, 77, 140, 222, 300, 399, 460, 510]),
+                                       ("llama1b_b64_d64", [0, 100, 257, 390, 512, 700, 901, 1023])])
 def test_full_size_configs_sampled(rkv, name, rows):
     """Configs 3, 4 and (one firing of) 5 at full size (about 9, 8 and 27 GB of K+V), oracle on 64 sampled
     head-problems each (sampled sequences, all their KV heads); a multi-head-attention cache (G = 1, Eq. 1) of
-    benchmark size (8192 head-problems, 9 GB); and config 3's shape with the caches stored as 8-bit E4M3 codes."""
+    benchmark size (8192 head-problems, 9 GB); config 3's shape with the caches stored as 8-bit E4M3 codes; and a cache
+    with 64-dimensional heads (tensor-core kernels on the padded copy)."""
     wl = ri.make_workload(ri.SPECS[name], device="cuda")
     rep, comp = run_and_check(rkv, wl, check_rows=rows)
     print(rep.summary())

@@ -419,7 +419,8 @@ def test_paged_caches_need_whole_pages(rkv):
 @pytest.mark.parametrize("hkv,hq,budget,buffer,lens", [(2, 8, 256, 64, [320, 300, 256]), (2, 2, 120, 17, [137, 129, 121]),
                                                        (1, 5, 1800, 128, [1928, 1900, 1801])])
 def test_head_dimensions_64_and_256(rkv, dtype, head_dim, hkv, hq, budget, buffer, lens):
-    """Head dimensions other than 128 (every stage: prep, CUDA-core scoring, both forms of the select stage, in-place
+    """Head dimensions other than 128 (every stage: prep, scoring -- bf16 keys of 64 dimensions on the tensor-core kernels
+    through a copy padded to 128, everything else on the CUDA-core kernel --, both forms of the select stage, in-place
     compaction with 128- to 1024-byte rows), grouped and multi-head (G = 1, Eq. 1) queries, ragged lengths."""
     spec = small_spec("hd", batch=3, hkv=hkv, hq=hq, budget=budget, buffer=buffer, dtype=dtype, head_dim=head_dim)
     wl = ri.make_workload(spec, device="cuda", seed=241 + head_dim, seq_lens=torch.tensor(lens))
@@ -430,6 +431,23 @@ def test_head_dimensions_64_and_256(rkv, dtype, head_dim, hkv, hq, budget, buffe
     print(rep.summary())
     assert rep.ok(), rep.errors
     assert rep.compressed_heads == hkv * sum(L > budget for L in lens)
+    comp.check_status()
+
+
+@pytest.mark.parametrize("flags", [pytest.param(1, id="simt"), pytest.param(2, id="rowblock"), pytest.param(32, id="two-pass"),
+                                   pytest.param(8, id="sym+head_mean")])
+@pytest.mark.parametrize("T,beta", [(0.5, 1), (0.9, 1), (0.5, 3)])
+def test_head_dimension_64_routes_and_settings(rkv, flags, T, beta):
+    """bf16 keys of 64 dimensions on every scoring route (the tensor-core ones through the padded copy, the CUDA-core
+    one on the cache itself) at a size where the two rounds and the symmetric route are reached; Eq. 2's scale is that
+    of the cache's own head dimension."""
+    spec = small_spec("hd64", batch=2, hkv=2, hq=8, budget=1536, buffer=128, head_dim=64, span=32)
+    lens = [spec.cap, spec.cap - 3]
+    wl = ri.make_workload(spec, device="cuda", seed=261, seq_lens=torch.tensor(lens))
+    rep, comp = run_and_check(rkv, wl, flags=flags, T=T, beta=beta)
+    print(rep.summary())
+    assert rep.ok(), rep.errors
+    assert rep.compressed_heads == 4
     comp.check_status()
 
 
