@@ -38,10 +38,10 @@ UNIT = "tokens/s"
 # workloads of that cache size; the capture has G = 4, other group sizes differ only in the few KB of queries per head).
 # None = the kernel has changed since the counters were taken.
 NCU_TRAFFIC_PER_HEAD_N4216 = {
-    "prep": 317.26e6 / 256,                   # prep kernel + the per-head key sums
-    "scores_pass1": 358.15e6 / 256, "scores_list": 4.34e6 / 256,
-    "scores_pass2": 375.90e6 / 256,           # both scans, the second listing and the symmetric route's two launches, as bench.py's interval has them
-    "row_stats": 34.61e6 / 256, "importance": 34.63e6 / 256, "select": 8.69e6 / 256, "gather": 1001.00e6 / 256,
+    "prep": 317.48e6 / 256,                   # prep kernel + the per-head key sums
+    "scores_pass1": 359.29e6 / 256, "scores_list": 4.34e6 / 256,
+    "scores_pass2": 375.66e6 / 256,           # both scans, the second listing and the symmetric route's two launches, as bench.py's interval has them
+    "row_stats": 34.61e6 / 256, "importance": 34.63e6 / 256, "select": 8.69e6 / 256, "gather": 1001.05e6 / 256,
 }
 DEFAULT_WORKLOAD = "qwen14b_b32"
 
