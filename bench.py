@@ -376,10 +376,12 @@ def kernel_table(rkv, timed: Timed, kw, KB, peaks):
     pass2_useful = pairs2 * 2.0 * 128 * (128 + 16)     # listed tokens x keys of the streamed tiles x 2 (d + 16)
     # algorithmic work per launch: bytes a kernel has to move / flops it has to execute, nothing it merely could
     work = {
-        # K once; r_i, Kbar_i.Kbar_i and the 32-byte slice out.  8-bit caches and d = 64: the stored keys in, their bf16 /
-        # padded copy out and in again
+        # K once; r_i, Kbar_i.Kbar_i and the 32-byte slice out.  8-bit caches and d = 64: the stored keys in and their bf16 /
+        # padded copy out (written by the prep kernel itself when a stored row is 128 bytes and the capacity a whole
+        # number of tiles; else by a pass of its own, and read back)
         "prep": ("hbm", P * (n * row + spec.cap * (8 + 32)) if (esz > 1 and spec.head_dim != 64) else
-                 P * (spec.cap * row + spec.cap * wide_row + n * wide_row + spec.cap * (8 + 32))),
+                 (P * (n * row + n * wide_row + spec.cap * (8 + 32)) if (row == 128 and spec.cap % 128 == 0) else
+                  P * (spec.cap * row + spec.cap * wide_row + n * wide_row + spec.cap * (8 + 32)))),
         "scores_pass1": ("tensor", pass1_flops),
         "scores_list": ("hbm", P * n * 8),
         "scores_pass2": ("tensor", pass2_flops),

@@ -43,6 +43,16 @@ bool pads_dim(const rkv_desc_t *d) { return d->head_dim == 64 && !use_simt(d); }
 bool needs_copy(const rkv_desc_t *d) { return d->dtype == RKV_FP8_E4M3 || pads_dim(d); }
 // Head dimension the scoring stages see.
 int scoring_dim(const rkv_desc_t *d) { return pads_dim(d) ? kHeadDim : d->head_dim; }
+// The prep kernel writes the copy of the keys itself (instead of a widening pass in front of it): stored rows of 128
+// bytes that become 128 bf16, in caches whose capacity is a whole number of 128-row tiles.  1: E4M3 codes, 2: bf16 of
+// 64 dimensions.
+int fuse_mode(const rkv_desc_t *d, long long cap)
+{
+    if (!needs_copy(d) || scoring_dim(d) != kHeadDim || cap % kTile != 0) return 0;
+    if (d->dtype == RKV_FP8_E4M3 && d->head_dim == kHeadDim) return 1;
+    if (d->dtype == RKV_BF16 && d->head_dim == 64) return 2;
+    return 0;
+}
 
 // 1 when the triangle tensor-core kernels score (bf16 caches, unless a cross-check kernel is asked for).
 int use_tri(const rkv_desc_t *d) { return !(use_simt(d) || (d->flags & RKV_FLAG_ROWBLOCK_SCORES)); }
@@ -211,12 +221,15 @@ int run(const rkv_desc_t *d, void *k_cache, void *v_cache, const void *q_window,
         p.dtype = RKV_BF16;
         p.d = scoring_dim(d);
         if (pads_dim(d)) p.q_window = ws + lay.q_wide;
+        p.fuse_mode = fuse_mode(d, lay.cap);
+        p.fuse_src = stored.k_cache;
+        p.fuse_table = stored.block_table;
     }
     if (stages & RKV_STAGE_PREP) {
         if ((e = cudaMemsetAsync(p.counters, 0, p.zero_bytes, s)) != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
         if (needs_copy(d) &&
             (e = launch_widen_keys(stored, static_cast<__nv_bfloat16 *>(p.k_cache), p.d, pads_dim(d) ? stored.q_window : nullptr,
-                                   pads_dim(d) ? ws + lay.q_wide : nullptr, s)) != cudaSuccess)
+                                   pads_dim(d) ? ws + lay.q_wide : nullptr, p.fuse_mode == 0, s)) != cudaSuccess)
             return cuda_fail(e, "widen launch");
         if ((e = launch_prep(p, s)) != cudaSuccess) return cuda_fail(e, "prep launch");
     }
@@ -463,6 +476,8 @@ int rkv_launch_count_for(const rkv_desc_t *desc, int32_t budget, int32_t buffer,
     Layout lay;
     if (check_shapes(desc, budget, buffer, alpha, &lay) != RKV_OK) return 0;
     int c = rkv_launch_count(desc, stage_mask);
+    // the prep kernel writes the copy of the keys itself and nothing else needs a pass of its own
+    if ((stage_mask & RKV_STAGE_PREP) && fuse_mode(desc, lay.cap) != 0 && !pads_dim(desc)) c -= 1;
     if ((stage_mask & RKV_STAGE_SELECT) && select_is_fused(lay.cap_pad, alpha)) c -= 2;
     if ((stage_mask & RKV_STAGE_SCORES) && use_tri(desc) && desc->beta > 0 && desc->sim_threshold < 1.0f)
     {

@@ -415,21 +415,6 @@ cudaError_t launch_tc_for(const AttendTcParams &p, bool fp8, const CUtensorMap &
     return fp8 ? launch_tc_one<G, true>(p, mk, mv, mq, s) : launch_tc_one<G, false>(p, mk, mv, mq, s);
 }
 
-// 2-D view [rows][128] of a cache of E4M3 codes (128-byte rows), boxes of 128 rows, 128-byte swizzle, out-of-range
-// rows read as zero.
-bool make_map_codes(CUtensorMap *map, const void *base, uint64_t rows)
-{
-    sm100::EncodeTiledFn fn = sm100::encode_fn();
-    if (!fn) return false;
-    const cuuint64_t dims[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)kHeadDim};
-    const cuuint32_t box[2] = {(cuuint32_t)kHeadDim, (cuuint32_t)kTile};
-    const cuuint32_t estr[2] = {1u, 1u};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 }  // namespace
 
 // Splits of a head's key tiles for the tensor-core kernel: enough blocks for two waves of resident blocks (2 per SM),
@@ -464,7 +449,7 @@ cudaError_t launch_attend_tc(const void *k_cache, const void *v_cache, const voi
     if (p.tiles_per_split > kTcMaxTiles) return cudaErrorInvalidValue;
     const uint64_t rows = block_table ? (uint64_t)pool_pages * kTile : (uint64_t)batch * hkv * cap;
     CUtensorMap mk, mv, mq;
-    const bool maps_ok = fp8 ? (make_map_codes(&mk, k_cache, rows) && make_map_codes(&mv, v_cache, rows))
+    const bool maps_ok = fp8 ? (sm100::make_map_row128(&mk, k_cache, rows, true) && sm100::make_map_row128(&mv, v_cache, rows, true))
                              : (sm100::make_map(&mk, k_cache, rows, kTile) && sm100::make_map(&mv, v_cache, rows, kTile));
     if (!maps_ok || !sm100::make_map(&mq, q_new, (uint64_t)batch * hq, 16)) return cudaErrorInvalidValue;
     switch (hq / hkv) {

@@ -33,6 +33,11 @@ struct Params {
     int dtype;                      // of the keys the scoring stages read (bf16 for 8-bit caches: their widened copy)
     int store_row_bytes;            // bytes of a row of the caches as stored (what the gather moves)
     float logit_scale;              // Eq. 2's 1 / sqrt(d) with the caches' own head dimension (d above may be a padded one)
+    // prep writes the scoring copy itself (k_cache above) from the stored keys: 0 = no, 1 = rows of 128 E4M3 codes,
+    // 2 = rows of 64 bf16
+    int fuse_mode;
+    const void *fuse_src;           // the stored keys
+    const int32_t *fuse_table;      // their block table (paged caches), else null
     // hyper-parameters
     int pool_w, beta;
     int head_mean;                  // Algorithm 1's aggregated selection: one kept set per sequence from the
@@ -207,7 +212,7 @@ __device__ __forceinline__ void widen16(const uint4 &codes, uint4 *lo, uint4 *hi
 // launchers (one per stage); each returns cudaGetLastError() of its launch
 cudaError_t launch_prep(const Params &p, cudaStream_t s);
 cudaError_t launch_widen_keys(const Params &stored, __nv_bfloat16 *wide, int wide_d, const void *q_src, void *q_dst,
-                              cudaStream_t s);
+                              bool keys, cudaStream_t s);
 cudaError_t launch_scores_simt(const Params &p, cudaStream_t s);
 cudaError_t launch_scores_sm100(const Params &p, cudaStream_t s);
 cudaError_t launch_scores_tri_sm100(const Params &p, cudaStream_t s);

@@ -470,6 +470,229 @@ __global__ void __launch_bounds__(kPrepTcThreads, kPrepTcBlocks) prep_tc_kernel(
     }
 }
 
+// ---- the same kernel for caches that are scored on a copy: 8-bit codes (d = 128) and bf16 keys of 64 dimensions --------
+//
+// Both store a key in 128 bytes.  The tile arrives as stored (16 KB, a ring of two stages); the thread that owns a row
+// widens / pads it into the bf16 operand tile, taking the norm on the way; the tensor cores form the key sums from that
+// tile as above, and the same tile is written out, by TMA, as the head's part of the scoring copy, which the later
+// stages read.  The stored keys are read once and the copy is not read back here: a separate widening pass in front
+// of prep_tc_kernel cost the prep stage a second sweep over keys twice the stored size.  Only for caches whose
+// capacity is a whole number of tiles (a tile's store must not reach into the next head's rows).
+constexpr int kFusedRaw = kTile * 128;                      // a stored tile: 16 KB
+constexpr int kFusedOffRaw = kPrepTcBufs * kPrepTcTile;
+constexpr int kFusedOffB = kFusedOffRaw + 2 * kFusedRaw;
+constexpr int kFusedSmem = kFusedOffB + kPrepTcB + 1024;
+constexpr int kFusedBlocks = 2;
+
+template <bool kCodes>
+__global__ void __launch_bounds__(kPrepTcThreads, kFusedBlocks)
+prep_fused_kernel(Params p, const __grid_constant__ CUtensorMap map_src, const __grid_constant__ CUtensorMap map_wide,
+                  const int32_t *src_table, int total)
+{
+    using namespace sm100;
+    constexpr int D = kHeadDim;
+    extern __shared__ uint8_t prep_tc_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(prep_tc_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t *bop = smem + kFusedOffB;
+    const uint32_t sbase = smem_u32(smem);
+    __shared__ __align__(8) unsigned long long bars[3];      // stored tile landed (per stage); product done
+    __shared__ uint32_t tmem_holder;
+    __shared__ int abort_flag;
+    const ErrSink sink = make_sink(p);
+    const int t = threadIdx.x, warp = t >> 5;
+    const uint32_t bar_raw0 = smem_u32(&bars[0]), bar_mma = smem_u32(&bars[2]);
+
+    // thread 0: the stored tile of the block's k-th list entry into stage k % 2 (an entry without candidates completes
+    // the stage's barrier phase without a copy)
+    auto issue_copy = [&](int k) {
+        const long long idx = (long long)blockIdx.x + (long long)k * gridDim.x;
+        if (idx >= total) return;
+        const PrepTile w = prep_tile_at(p, (int)idx, false);
+        const uint32_t bar = bar_raw0 + 8u * (k & 1);
+        if (w.rows_here <= 0) {
+            mbar_arrive(bar);
+            return;
+        }
+        const int y = src_table ? src_table[(size_t)w.head * (p.cap / kTile) + w.tile] * kTile : w.head * p.cap + w.tile * kTile;
+        mbar_expect_tx(bar, kFusedRaw);
+        tma_load_2d(sbase + kFusedOffRaw + (k & 1) * kFusedRaw, &map_src, 0, y, bar);
+    };
+
+    if (t == 0) {
+        abort_flag = 0;
+        mbar_init(bar_raw0, 1);
+        mbar_init(bar_raw0 + 8u, 1);
+        mbar_init(bar_mma, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        issue_copy(0);
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&tmem_holder)), "r"(kPrepTcTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    for (int x = t; x < kPrepTcB / 16; x += kPrepTcThreads) reinterpret_cast<uint4 *>(bop)[x] = make_uint4(0u, 0u, 0u, 0u);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_holder;
+    uint32_t mma_parity = 0;
+
+    int k = 0;
+    for (int idx = (int)blockIdx.x; idx < total; idx += (int)gridDim.x, ++k) {
+        const PrepTile w = prep_tile_at(p, idx, t == 0);
+        const int head = w.head, tile = w.tile, n = w.n, rows_here = w.rows_here;
+        const int buf = k & 1;
+        uint8_t *tile_smem = smem + buf * kPrepTcTile;
+        if (t == 0) {
+            // the other stage was read, by every thread, before the last barrier; and the operand tile about to be
+            // written was stored two entries ago: that store has to be through with shared memory
+            issue_copy(k + 1);
+            asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+        }
+        const bool landed = mbar_wait(bar_raw0 + 8u * buf, (uint32_t)(k >> 1) & 1u, &abort_flag, sink);
+        const bool ok = __syncthreads_and(landed);           // the block goes on as a whole, or not at all
+
+        // ---- one thread per row: the stored row into the operand tile (bf16, 128 dimensions, the layout a TMA load
+        // leaves), its norm on the way; rows that are not candidates become zeros
+        const int rt = t;
+        const int row = tile * kTile + rt;
+        float r = 0.f, sq = 0.f;
+        if (ok && rows_here > 0) {
+            uint4 out[16];
+#pragma unroll
+            for (int c = 0; c < 16; ++c) out[c] = make_uint4(0u, 0u, 0u, 0u);
+            if (rt < rows_here) {
+                const uint8_t *raw = smem + kFusedOffRaw + buf * kFusedRaw + rt * 128;
+                uint4 in[8];
+#pragma unroll
+                for (int c = 0; c < 8; ++c) in[c] = *reinterpret_cast<const uint4 *>(raw + ((c ^ (rt & 7)) << 4));
+                float2 sq2[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) sq2[e] = make_float2(0.f, 0.f);
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    if (kCodes) widen16(in[c], &out[2 * c], &out[2 * c + 1]);     // 16 codes -> bf16 chunks 2 c, 2 c + 1
+                    else out[c] = in[c];                                           // 64 dimensions: chunks 0..7, the rest zeros
+                }
+#pragma unroll
+                for (int c = 0; c < (kCodes ? 16 : 8); ++c) {
+                    float f[8];
+                    Elem<__nv_bfloat16>::unpack(out[c], f);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float2 f2 = make_float2(f[2 * e], f[2 * e + 1]);
+                        sq2[e] = __ffma2_rn(f2, f2, sq2[e]);
+                    }
+                }
+                sq = ((sq2[0].x + sq2[0].y) + (sq2[1].x + sq2[1].y)) + ((sq2[2].x + sq2[2].y) + (sq2[3].x + sq2[3].y));
+                const float nrm = sq > 0.f ? sq * rsqrtf(sq) : 0.f;
+                r = __fdividef(1.0f, nrm + p.eps);
+            }
+#pragma unroll
+            for (int c = 0; c < 16; ++c)
+                *reinterpret_cast<uint4 *>(tile_smem + (c >> 3) * (kPrepTcTile / 2) + rt * 128 + (((c & 7) ^ (rt & 7)) << 4)) = out[c];
+        }
+        if (ok) {
+            float rest = r;
+            uint32_t rp[3];
+#pragma unroll
+            for (int c = 0; c < 3; ++c) {
+                const __nv_bfloat16 h16 = __float2bfloat16_rn(rest);
+                rp[c] = (uint32_t)__bfloat16_as_ushort(h16);
+                rest -= __bfloat162float(h16);
+            }
+            const int s = rt >> 4, kk = rt & 15;
+#pragma unroll
+            for (int nn = 0; nn < 3; ++nn)
+                *reinterpret_cast<unsigned short *>(bop + s * 512 + nn * 32 + ((kk >> 3) << 4) + (kk & 7) * 2) = (unsigned short)rp[nn];
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");       // generic writes -> tensor-core and TMA reads
+        __syncthreads();
+
+        if (ok && rows_here > 0 && t == 0) {
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | ((16u >> 3) << 17) | ((128u >> 4) << 24);
+            tc_fence_after();
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+                const uint32_t a_addr = sbase + buf * kPrepTcTile + ks * 2048;
+                const uint32_t b_addr = sbase + kFusedOffB + ks * 512;
+                uint64_t da = (uint64_t)((a_addr & 0x3FFFFu) >> 4) | ((uint64_t)(16384u >> 4) << 16) | ((uint64_t)(1024u >> 4) << 32) |
+                              ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+                uint64_t db = (uint64_t)((b_addr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(256u >> 4) << 32) |
+                              ((uint64_t)1 << 46) | ((uint64_t)6 << 61);
+                asm volatile("{\n\t.reg .pred pp;\n\tsetp.ne.b32 pp, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, pp;\n\t}"
+                             ::"r"(tmem), "l"(da), "l"(db), "r"(idesc), "r"(ks) : "memory");
+            }
+            umma_commit(bar_mma);
+            // the tile, as the head's rows [128 tile, 128 tile + 128) of the scoring copy (contiguous, head after head)
+            const int yw = head * p.cap + tile * kTile;
+            asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                         ::"l"(reinterpret_cast<uint64_t>(&map_wide)), "r"(0), "r"(yw), "r"(sbase + buf * kPrepTcTile) : "memory");
+            asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                         ::"l"(reinterpret_cast<uint64_t>(&map_wide)), "r"(64), "r"(yw), "r"(sbase + buf * kPrepTcTile + kPrepTcTile / 2) : "memory");
+        }
+        if (t == 0) asm volatile("cp.async.bulk.commit_group;" ::: "memory");      // one group per entry, empty or not
+
+        if (ok) {
+            p.inv_norm[(size_t)head * p.cap_pad + row] = r;
+            p.self_dot[(size_t)head * p.cap_pad + row] = (r * r) * sq;     // Kbar_i . Kbar_i
+            if (p.tri) {
+                float rest = r > 0.f ? __fdiv_rn(1.0f, r) : 0.f;
+                uint32_t part[3];
+#pragma unroll
+                for (int c = 0; c < 3; ++c) {
+                    const __nv_bfloat16 h16 = __float2bfloat16_rn(rest);
+                    part[c] = (uint32_t)__bfloat16_as_ushort(h16);
+                    rest -= __bfloat162float(h16);
+                }
+                uint4 *dst = reinterpret_cast<uint4 *>(p.norm_split + ((size_t)head * p.cap_pad + row) * 16);
+                dst[0] = make_uint4(part[0] | (part[1] << 16), part[2] | (part[0] << 16), part[1] | (part[0] << 16), 0u);
+                dst[1] = make_uint4(0u, 0u, 0u, 0u);
+                if (tile == (n + kTile - 1) / kTile - 1) {
+                    rest = r > 0.f ? -__fdiv_rn(p.sim_threshold, r) : 0.f;
+#pragma unroll
+                    for (int c = 0; c < 3; ++c) {
+                        const __nv_bfloat16 h16 = __float2bfloat16_rn(rest);
+                        part[c] = (uint32_t)__bfloat16_as_ushort(h16);
+                        rest -= __bfloat162float(h16);
+                    }
+                    uint4 *thr = reinterpret_cast<uint4 *>(p.thr_split + ((size_t)head * kTile + rt) * 16);
+                    thr[0] = make_uint4(part[0] | (part[0] << 16), part[0] | (part[1] << 16), part[1] | (part[2] << 16), 0u);
+                    thr[1] = make_uint4(0u, 0u, 0u, 0u);
+                }
+            }
+        }
+
+        float tsum = 0.f;
+        bool done = ok;
+        if (ok && rows_here > 0) {
+            done = mbar_wait(bar_mma, mma_parity, &abort_flag, sink);
+            mma_parity ^= 1u;
+            if (done) {
+                tc_fence_after();
+                uint32_t acc[8];
+                tmem_ld8(tmem + ((uint32_t)(warp * 32) << 16), acc);      // lane = column c of the keys
+                tmem_wait8(acc);
+                tsum = (__uint_as_float(acc[0]) + __uint_as_float(acc[1])) + __uint_as_float(acc[2]);
+            }
+        }
+        tc_fence_before();
+        done = __syncthreads_and(done);
+        p.tile_sum[((size_t)head * p.tiles + tile) * D + t] = done ? tsum : 0.f;
+        if (!done) break;
+    }
+
+    if (t == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");      // the stores are through before the block leaves
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        if (abort_flag) __nanosleep(200000);       // error path only: let the copies in flight land
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kPrepTcTmemCols) : "memory");
+    }
+}
+
 // The tile sums of a head added up in tile order (a launch of its own behind prep_tc_kernel: no tickets, no fences in
 // the streaming kernel), also as three bf16 rows whose sum is s to fp32 accuracy (rows 3..15 of the 16-row block are
 // zero): appended to the query rows, they let the tensor cores form Kbar_i . s along with the logits.
@@ -508,6 +731,30 @@ static cudaError_t launch_prep_for(const Params &p, cudaStream_t s)
 cudaError_t launch_prep(const Params &p, cudaStream_t s)
 {
     const bool bf16 = p.dtype == RKV_BF16;
+    if (p.fuse_mode != 0) {                 // the tensor-core form that also writes the scoring copy
+        const uint64_t wide_rows = (uint64_t)p.batch * p.hkv * p.cap + kTile;
+        const uint64_t src_rows = p.fuse_table ? (uint64_t)p.pool_pages * kTile : (uint64_t)p.batch * p.hkv * p.cap;
+        CUtensorMap map_src, map_wide;
+        if (!sm100::make_map_row128(&map_src, p.fuse_src, src_rows, p.fuse_mode == 1) ||
+            !sm100::make_map(&map_wide, p.k_cache, wide_rows, kTile))
+            return cudaErrorInvalidValue;
+        int dev = 0, sms = 0;
+        cudaError_t e;
+        if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+        if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+        const int total = p.tiles * p.batch * p.hkv;
+        const unsigned grid = (unsigned)std::min(total, kFusedBlocks * sms);
+        if (p.fuse_mode == 1) {
+            if ((e = cudaFuncSetAttribute(prep_fused_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFusedSmem)) != cudaSuccess) return e;
+            prep_fused_kernel<true><<<grid, kPrepTcThreads, kFusedSmem, s>>>(p, map_src, map_wide, p.fuse_table, total);
+        } else {
+            if ((e = cudaFuncSetAttribute(prep_fused_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFusedSmem)) != cudaSuccess) return e;
+            prep_fused_kernel<false><<<grid, kPrepTcThreads, kFusedSmem, s>>>(p, map_src, map_wide, p.fuse_table, total);
+        }
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        head_sum_kernel<<<(unsigned)(p.batch * p.hkv), kHeadDim, 0, s>>>(p);
+        return cudaGetLastError();
+    }
     if (bf16 && p.d == kHeadDim) {          // the tensor-core form
         CUtensorMap map_k;
         if (!sm100::make_map(&map_k, p.k_cache, sm100::key_rows_total(p), kTile)) return cudaErrorInvalidValue;

@@ -281,6 +281,21 @@ inline bool make_map(CUtensorMap *map, const void *base, uint64_t rows, uint32_t
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// 2-D view [rows][128 bytes] of a cache whose rows are 128 bytes long -- E4M3 codes of 128 dimensions, or bf16 keys of 64
+// dimensions --, boxes of 128 rows, 128-byte swizzle, out-of-range rows read as zero.
+inline bool make_map_row128(CUtensorMap *map, const void *base, uint64_t rows, bool codes)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)(codes ? 128 : 64), (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {128u};
+    const cuuint32_t box[2] = {(cuuint32_t)(codes ? 128 : 64), (cuuint32_t)kTile};
+    const cuuint32_t estr[2] = {1u, 1u};
+    return fn(map, codes ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims,
+              strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // 2-D bf16 view [rows][16] (32-byte rows), boxes of 128 rows, 32-byte swizzle: the extra K = 16 slices of key rows.
 inline bool make_map_k16(CUtensorMap *map, const void *base, uint64_t rows)
 {

@@ -22,10 +22,9 @@ constexpr int kWidenThreads = 256;
 // stored row; dst_vecs: of a row of the copy (bf16; wider than the widened row when the head dimension is padded: the
 // rest of the row is zeros).  The blocks after those pad the observation queries the same way (bf16 rows only).
 __global__ void __launch_bounds__(kWidenThreads)
-widen_keys_kernel(Params p, __nv_bfloat16 *wide, int src_vecs, int dst_vecs, int codes, const uint4 *q_src, uint4 *q_dst,
+widen_keys_kernel(Params p, int key_blocks, __nv_bfloat16 *wide, int src_vecs, int dst_vecs, int codes, const uint4 *q_src, uint4 *q_dst,
                   int q_rows)
 {
-    const int key_blocks = p.tiles * p.batch * p.hkv;
     if ((int)blockIdx.x >= key_blocks) {
         // queries: rows of src_q_vecs = dst_vecs / 2 vectors (bf16, 64 dimensions) -> rows of dst_vecs, zero-padded
         const int q_vecs = dst_vecs / 2;
@@ -67,13 +66,16 @@ widen_keys_kernel(Params p, __nv_bfloat16 *wide, int src_vecs, int dst_vecs, int
 
 // stored: the caches as the caller holds them (d = stored head dimension).  wide_d: head dimension of the copy.
 // q_src / q_dst: the observation queries and their padded copy (null when the head dimension is not padded).
+// keys = false: the queries only (the prep stage writes the copy of the keys itself).
 cudaError_t launch_widen_keys(const Params &stored, __nv_bfloat16 *wide, int wide_d, const void *q_src, void *q_dst,
-                              cudaStream_t s)
+                              bool keys, cudaStream_t s)
 {
     const int codes = stored.dtype == RKV_FP8_E4M3 ? 1 : 0;
     const int q_rows = q_dst ? stored.batch * stored.hq * stored.alpha : 0;
-    const unsigned grid = (unsigned)stored.tiles * (unsigned)(stored.batch * stored.hkv) + (unsigned)((q_rows + kTile - 1) / kTile);
-    widen_keys_kernel<<<grid, kWidenThreads, 0, s>>>(stored, wide, stored.store_row_bytes / 16, wide_d * 2 / 16, codes,
+    const unsigned key_blocks = keys ? (unsigned)stored.tiles * (unsigned)(stored.batch * stored.hkv) : 0u;
+    const unsigned grid = key_blocks + (unsigned)((q_rows + kTile - 1) / kTile);
+    if (grid == 0u) return cudaSuccess;
+    widen_keys_kernel<<<grid, kWidenThreads, 0, s>>>(stored, (int)key_blocks, wide, stored.store_row_bytes / 16, wide_d * 2 / 16, codes,
                                                      static_cast<const uint4 *>(q_src), static_cast<uint4 *>(q_dst), q_rows);
     return cudaGetLastError();
 }

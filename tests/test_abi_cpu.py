@@ -151,7 +151,10 @@ def test_eight_bit_cache_type_sizes_and_counts(rkv):
         h16, h8 = rkv.rkv_host_workspace_bytes(b16, 1024, 128, alpha), rkv.rkv_host_workspace_bytes(f8, 1024, 128, alpha)
         assert (h16 - w16) - (h8 - w8) == 2 * P * cap * hd            # K and V staging: two bytes per element less one
         assert rkv.rkv_launch_count_for(f8, 1024, 128, alpha, rkv.RKV_STAGE_ALL) == \
-            rkv.rkv_launch_count_for(b16, 1024, 128, alpha, rkv.RKV_STAGE_ALL) + (0 if hd == 64 else 1)
+            rkv.rkv_launch_count_for(b16, 1024, 128, alpha, rkv.RKV_STAGE_ALL) + (1 if hd == 256 else 0)
+        # (d = 128 with a capacity of whole tiles: the prep kernel writes the widened copy itself; otherwise one more launch)
+        assert rkv.rkv_launch_count_for(f8, 1000, 100, alpha, rkv.RKV_STAGE_ALL) == \
+            rkv.rkv_launch_count_for(b16, 1000, 100, alpha, rkv.RKV_STAGE_ALL) + (0 if hd == 64 else 1)
         assert rkv.rkv_launch_count_for(f8, 1024, 128, alpha, rkv.RKV_STAGE_GATHER) == 1
     # head dimension 64 takes the kernels of head dimension 128 plus the one that writes the padded copy; on the
     # CUDA-core route (on request) it needs neither the copy nor the extra launches
