@@ -262,3 +262,36 @@ def test_fp8_every_code_through_the_attention_and_the_widening_kernels(rkv):
     kb[0, 0, :64] = codes[torch.randint(0, 256, (64, 128), generator=gen)].cuda()
     rep, comp = run_and_check(rkv, wl)
     assert rep.ok(), rep.errors
+
+
+@pytest.mark.parametrize("dtype,head_dim", [("fp8", 128), ("bf16", 64)])
+def test_scoring_copy_with_budgets_and_pages(rkv, dtype, head_dim):
+    """The prep kernel that writes the scoring copy itself (8-bit codes of 128 dimensions, bf16 keys of 64; capacity a
+    whole number of tiles), together with per-sequence budgets and a block table: the stored tiles are fetched through
+    the table, the copy is contiguous, the compaction moves the stored rows page by page."""
+    budget, buffer = 896, 128
+    lens = [1024, 1000, 600, 1024]
+    budgets = [896, 700, 896, 512]
+    spec = small_spec("copy_bp", batch=4, hkv=2, hq=8, budget=budget, buffer=buffer, dtype=dtype, head_dim=head_dim, span=32)
+    wl = ri.make_workload(spec, device="cuda", seed=391 + head_dim, seq_lens=torch.tensor(lens))
+    k0, v0, q0, s0 = wl.k_cache.clone(), wl.v_cache.clone(), wl.q_window.clone(), wl.seq_lens.clone()
+    pages, pool_pages = spec.cap // 128, 4 * 2 * 8 + 9
+    table = random_block_table(4, 2, pages, pool_pages, seed=15)
+    raw = torch.uint8 if dtype == "fp8" else torch.int16
+    fill = NAN_CODE if dtype == "fp8" else 0x7FC0                    # NaN patterns in the pages nobody owns
+    kp = to_paged(k0.view(raw), pool_pages, table, fill=fill).view(k0.dtype)
+    vp = to_paged(v0.view(raw), pool_pages, table, fill=fill).view(v0.dtype)
+    comp = rkv.Compressor(4, 2, 8, budget, buffer, spec.alpha, spec.lam, dtype=spec.torch_dtype, head_dim=head_dim,
+                          dump_scores=True, block_table=table, pool_pages=pool_pages, budgets=torch.tensor(budgets))
+    seq = s0.clone()
+    idx = comp.compress(kp, vp, q0, seq)
+    torch.cuda.synchronize()
+    comp.check_status()
+    k1 = from_paged(kp.view(raw), table).view(k0.dtype)
+    v1 = from_paged(vp.view(raw), table).view(v0.dtype)
+    rep = check_batch(k0, v0, q0, s0, budget=budget, alpha=spec.alpha, lam=spec.lam, gpu_idx=idx, gpu_k=k1, gpu_v=v1,
+                      gpu_seq=seq, gpu_scores=comp.scores, budgets=budgets, **DEFAULTS)
+    print(rep.summary())
+    assert rep.ok(), rep.errors
+    assert rep.compressed_heads == 2 * 3
+    assert seq.tolist() == [896, 700, 600, 512]
