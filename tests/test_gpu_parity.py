@@ -451,6 +451,33 @@ def test_head_dimension_64_routes_and_settings(rkv, flags, T, beta):
     comp.check_status()
 
 
+@pytest.mark.parametrize("flags", [pytest.param(0, id="sym"), pytest.param(32, id="two-pass")])
+def test_largest_supported_capacity(rkv, flags):
+    """budget + buffer = 8192 rows, the largest capacity the library takes (64 key tiles: the longest second-pass scans,
+    32 work items per head in the symmetric scan), a full cache and one a few rows short of full."""
+    spec = small_spec("maxcap", batch=2, hkv=1, hq=4, budget=8192 - 128, buffer=128, span=32)
+    lens = [8192, 8192 - 77]
+    wl = ri.make_workload(spec, device="cuda", seed=271, seq_lens=torch.tensor(lens))
+    rep, comp = run_and_check(rkv, wl, flags=flags)
+    print(rep.summary())
+    assert rep.ok(), rep.errors
+    assert rep.compressed_heads == 2
+    comp.check_status()
+
+
+@pytest.mark.parametrize("flags", [pytest.param(0, id="sym"), pytest.param(2, id="rowblock"), pytest.param(1, id="simt")])
+def test_largest_supported_query_group(rkv, flags):
+    """G * alpha = 112 query rows per KV head, the most the library takes (14 query heads per KV head with alpha = 8: the
+    first pass's product then has 128 + 112 + 16 = 256 columns, the widest a tensor-core product can be)."""
+    spec = small_spec("maxgroup", batch=2, hkv=2, hq=28, budget=1024, buffer=128, span=32)
+    wl = ri.make_workload(spec, device="cuda", seed=273, seq_lens=torch.tensor([1152, 1100]))
+    rep, comp = run_and_check(rkv, wl, flags=flags)
+    print(rep.summary())
+    assert rep.ok(), rep.errors
+    assert rep.compressed_heads == 4
+    comp.check_status()
+
+
 # ----------------------------------------------------------------------------- per-sequence budgets
 @pytest.mark.parametrize("flags", [pytest.param(1, id="simt"), pytest.param(0, id="sym"), pytest.param(2, id="rowblock"),
                                    pytest.param(8, id="sym+head_mean")])
