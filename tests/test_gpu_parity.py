@@ -451,6 +451,30 @@ def test_head_dimension_64_routes_and_settings(rkv, flags, T, beta):
     comp.check_status()
 
 
+@pytest.mark.parametrize("flags", [pytest.param(0, id="sym"), pytest.param(1, id="simt"), pytest.param(2, id="rowblock")])
+def test_degenerate_inputs(rkv, flags):
+    """The degenerate cases of the method: keys that are all zero (norm 0: Eq. 5's epsilon keeps the division finite and
+    the key similar to nothing), a whole head of zero keys, queries that are all zero (Eq. 2-3 give uniform weights),
+    and the smallest shapes the call takes (budget = alpha + 1: one candidate is kept; buffer = 1)."""
+    spec = small_spec("degen", batch=3, hkv=2, hq=8, budget=300, buffer=84)
+    wl = ri.make_workload(spec, device="cuda", seed=281)
+    wl.k_cache[0, 0, 5:40] = 0                       # a run of zero keys
+    wl.k_cache[0, 0, 383] = 0                        # the last position
+    wl.k_cache[1, 1] = 0                             # a whole head
+    wl.q_window[2] = 0                               # uniform attention for a sequence
+    rep, comp = run_and_check(rkv, wl, flags=flags)
+    print(rep.summary())
+    assert rep.ok(), rep.errors
+    assert rep.compressed_heads == 6
+    comp.check_status()
+    tiny = small_spec("degen_tiny", batch=2, hkv=2, hq=8, budget=9, buffer=1)
+    wl = ri.make_workload(tiny, device="cuda", seed=283, seq_lens=torch.tensor([10, 9]))
+    rep, comp = run_and_check(rkv, wl, flags=flags)
+    assert rep.ok(), rep.errors
+    assert rep.compressed_heads == 2 and wl.seq_lens.tolist() == [9, 9]
+    comp.check_status()
+
+
 @pytest.mark.parametrize("flags", [pytest.param(0, id="sym"), pytest.param(32, id="two-pass")])
 def test_largest_supported_capacity(rkv, flags):
     """budget + buffer = 8192 rows, the largest capacity the library takes (64 key tiles: the longest second-pass scans,
