@@ -289,8 +289,9 @@ RKV_API int rkv_push_query(const rkv_desc_t *desc, void *q_window, const void *q
  *                     [0, budget + buffer] gives a zero row and RKV_ERR_INVALID_ARG in desc->device_status
  *   out               [batch][n_q_heads][head_dim] float32 (device, 16-byte aligned)
  * bf16 and 8-bit caches: both contractions on the tensor cores (bf16 products, fp32 accumulation, the softmax weights carried as
- * two bf16 parts, i.e. to fp32 accuracy), softmax in fp32; fp32 caches: fp32 arithmetic throughout.  head_dim 128 and
- * G = n_q_heads / n_kv_heads up to 8 (RKV_ERR_UNSUPPORTED otherwise).  The rows of a head are cut into splits (with
+ * two bf16 parts, i.e. to fp32 accuracy), softmax in fp32; fp32 caches: fp32 arithmetic throughout.  head_dim 128 (any
+ * cache type) or 64 (bf16 caches: tiles padded to 128 on their way to the tensor cores), and G = n_q_heads /
+ * n_kv_heads up to 8 (RKV_ERR_UNSUPPORTED otherwise).  The rows of a head are cut into splits (with
  * few head-problems, to fill the GPU; for bf16 and 8-bit caches also whenever budget + buffer exceeds 1920 rows, what one block
  * holds scores for) whose partial results go through desc->workspace: rkv_decode_workspace_bytes() says how much that
  * needs (0 when there is a single split; never more than a compression of the same shape needs, so one workspace

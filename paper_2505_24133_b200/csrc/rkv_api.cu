@@ -416,7 +416,7 @@ static int attend_plan(const rkv_desc_t *d, int32_t budget, int32_t buffer, int 
     int rc = check_shapes(d, budget, buffer, 1, nullptr);
     if (rc != RKV_OK) return rc;
     const int G = d->n_q_heads / d->n_kv_heads;
-    if (G > attend_max_group() || d->head_dim != kHeadDim) return RKV_ERR_UNSUPPORTED;
+    if (!attend_supported(G, d->dtype, d->head_dim)) return RKV_ERR_UNSUPPORTED;
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
         sms = 148;       // sizing only (no device here): the B200's count
@@ -449,7 +449,7 @@ int rkv_decode_attention(const rkv_desc_t *d, const void *k_cache, const void *v
     const long long wait = d->wait_limit_cycles > 0 ? (long long)d->wait_limit_cycles : sm100_default_wait_cycles();
     const cudaError_t e = launch_attend(k_cache, v_cache, q_new, seq_lens, out, static_cast<float *>(d->workspace), d->batch,
                                         d->n_kv_heads, d->n_q_heads, budget + buffer, splits, d->dtype, d->device_status,
-                                        wait, d->block_table, d->pool_pages, static_cast<cudaStream_t>(stream));
+                                        wait, d->block_table, d->pool_pages, d->head_dim, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? RKV_OK : cuda_fail(e, "decode attention launch");
 }
 

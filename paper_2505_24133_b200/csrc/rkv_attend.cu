@@ -40,6 +40,7 @@ struct AttendParams {
     int32_t *status;
     long long wait_cycles;
     const int32_t *block_table;  // paged caches: [P][cap / 128] page ids (a page = 128 rows), else null
+    int d_out;                   // head dimension of the output rows (the partial results always have rows of 128 + 2)
 };
 
 template <typename T, int G>
@@ -308,7 +309,7 @@ __global__ void __launch_bounds__(kHeadDim) attend_merge_kernel(AttendParams p, 
         num = fmaf(w, part[s * stride + c], num);
         den = fmaf(w, part[s * stride + kHeadDim + 1], den);
     }
-    p.out[((size_t)b * p.hq + (size_t)h * G + g) * kHeadDim + c] = den > 0.f ? num / den : 0.f;
+    if (c < p.d_out) p.out[((size_t)b * p.hq + (size_t)h * G + g) * p.d_out + c] = den > 0.f ? num / den : 0.f;
 }
 
 template <typename T, int G>
@@ -343,6 +344,13 @@ cudaError_t launch_dtype(const AttendParams &p, int G, cudaStream_t s)
 
 int attend_max_group() { return kAttMaxG; }
 
+// Head dimension 128 for every cache type; 64 for bf16 caches (the tensor-core kernel pads the tiles to 128).
+bool attend_supported(int G, int dtype, int head_dim)
+{
+    if (G > kAttMaxG) return false;
+    return head_dim == kHeadDim || (head_dim == 64 && dtype == RKV_BF16);
+}
+
 // bf16 and 8-bit caches go to the tensor-core kernel whatever the group size (it runs at the rate HBM can be read at; this kernel
 // reached 0.74 of the copy bandwidth at G = 4 and ran out of issue slots from G = 5 on); fp32 caches stay here.
 bool attend_uses_tc(int G, int dtype) { return (dtype == RKV_BF16 || dtype == RKV_FP8_E4M3) && G >= 1; }
@@ -364,7 +372,7 @@ size_t attend_partial_bytes(int heads, int splits, int G)
 
 cudaError_t launch_attend(const void *k_cache, const void *v_cache, const void *q_new, const int32_t *seq_lens, float *out,
                           float *partial, int batch, int hkv, int hq, int cap, int splits, int dtype, int32_t *status,
-                          long long wait_cycles, const int32_t *block_table, long long pool_pages, cudaStream_t s)
+                          long long wait_cycles, const int32_t *block_table, long long pool_pages, int head_dim, cudaStream_t s)
 {
     const int G = hq / hkv;
     AttendParams p;
@@ -382,10 +390,11 @@ cudaError_t launch_attend(const void *k_cache, const void *v_cache, const void *
     p.status = status;
     p.wait_cycles = wait_cycles;
     p.block_table = block_table;
+    p.d_out = head_dim;
     cudaError_t e;
     if (attend_uses_tc(G, dtype))
         e = launch_attend_tc(k_cache, v_cache, q_new, seq_lens, out, partial, batch, hkv, hq, cap, splits, status, wait_cycles,
-                             block_table, pool_pages, dtype == RKV_FP8_E4M3, s);
+                             block_table, pool_pages, dtype == RKV_FP8_E4M3 ? 1 : (head_dim == 64 ? 2 : 0), s);
     else
         e = launch_dtype<float>(p, G, s);
     if (e != cudaSuccess || splits == 1) return e;

@@ -110,11 +110,16 @@ __device__ __forceinline__ uint32_t small_off(int g, int k)
 }
 
 // With kFp8, kBarFull / kBarEmpty [0 .. kConvBufs) stand for the widened tiles (filled by the softmax threads, 128 arrivals).
-template <int G, bool kFp8>
+// kSrc: 0 = bf16 caches of 128 dimensions (tiles go to the tensor cores as they land), 1 = E4M3 codes of 128 dimensions,
+// 2 = bf16 caches of 64 dimensions (both: rows of 128 bytes, widened / padded with zeros into bf16 operand tiles of
+// 128 dimensions; the queries of the 64-dimension case fill the first half of their operand, the rest stays zero).
+template <int G, int kSrc>
 __global__ void __launch_bounds__(kTcThreads, 2)
 attend_tc_kernel(AttendTcParams p, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                  const __grid_constant__ CUtensorMap map_q)
 {
+    constexpr bool kFp8 = kSrc != 0;            // the tiles pass through the softmax threads on their way to the tensor cores
+    constexpr int kDim = kSrc == 2 ? 64 : kHeadDim;          // head dimension of the caches, the queries and the output
     extern __shared__ uint8_t att_tc_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(att_tc_raw) + 1023) & ~(uintptr_t)1023);
     const uint32_t sbase = smem_u32(smem);
@@ -136,13 +141,13 @@ attend_tc_kernel(AttendTcParams p, const __grid_constant__ CUtensorMap map_k, co
     const int T = min(min(p.tiles_per_split, kTcMaxTiles), (L + kTile - 1) / kTile - t0);      // its tiles (<= 0: none)
     constexpr int kStride = kHeadDim + 2;
     float *part = p.partial + ((size_t)head * p.splits + split) * G * kStride;
-    float *out = p.out + ((size_t)b * p.hq + (size_t)h * G) * kHeadDim;
+    float *out = p.out + ((size_t)b * p.hq + (size_t)h * G) * kDim;
 
     if (T <= 0) {       // no cached row falls into this split (uniform for the block: nothing was allocated yet)
-        for (int x = threadIdx.x; x < G * kHeadDim; x += kTcThreads) {
-            const int g = x / kHeadDim, c = x % kHeadDim;
+        for (int x = threadIdx.x; x < G * kDim; x += kTcThreads) {
+            const int g = x / kDim, c = x % kDim;
             if (p.splits == 1) {
-                out[(size_t)g * kHeadDim + c] = 0.f;
+                out[(size_t)g * kDim + c] = 0.f;
             } else {
                 part[g * kStride + c] = 0.f;
                 if (c == 0) {
@@ -178,9 +183,10 @@ attend_tc_kernel(AttendTcParams p, const __grid_constant__ CUtensorMap map_k, co
                      ::"r"(smem_u32(tmem_holder)), "r"(kTcTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    // the P buffers start as zeros: rows of queries the group does not have are never written
-    for (int x = threadIdx.x; x < 2 * kTcSmall / 16; x += kTcThreads)
-        reinterpret_cast<uint4 *>(smem + kOffP)[x] = make_uint4(0u, 0u, 0u, 0u);
+    // the P buffers start as zeros: rows of queries the group does not have are never written (and so does the query
+    // operand: with 64 dimensions only its first half is loaded)
+    for (int x = threadIdx.x; x < 3 * kTcSmall / 16; x += kTcThreads)
+        reinterpret_cast<uint4 *>(smem + kOffQ)[x] = make_uint4(0u, 0u, 0u, 0u);
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     tc_fence_before();
     __syncthreads();
@@ -195,10 +201,10 @@ attend_tc_kernel(AttendTcParams p, const __grid_constant__ CUtensorMap map_k, co
     if (warp == 4) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            mbar_expect_tx(bar(kBarQ), kTcSmall);
+            mbar_expect_tx(bar(kBarQ), kSrc == 2 ? kTcSmall / 2 : kTcSmall);
             const int qy = b * p.hq + h * G;                 // the group's G query rows (the rows after them are not used)
             tma_load_2d(sbase + kOffQ, &map_q, 0, qy, bar(kBarQ));
-            tma_load_2d(sbase + kOffQ + kTcSmall / 2, &map_q, 64, qy, bar(kBarQ));
+            if (kSrc != 2) tma_load_2d(sbase + kOffQ + kTcSmall / 2, &map_q, 64, qy, bar(kBarQ));
             for (int i = 0; i < 2 * T; ++i) {                // the K tiles, then the V tiles
                 const CUtensorMap *map = i < T ? &map_k : &map_v;
                 const int y = tile_y(t0 + (i < T ? i : i - T));
@@ -262,7 +268,7 @@ attend_tc_kernel(AttendTcParams p, const __grid_constant__ CUtensorMap map_k, co
         // ------------------------------------------------------------------ softmax threads (warps 0..3)
         const int r = threadIdx.x;                                   // TMEM lane: key row of a tile, later output dimension
         const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
-        const float c2 = 1.4426950408889634f * rsqrtf((float)kHeadDim);      // scores in the base-2 domain
+        const float c2 = 1.4426950408889634f * rsqrtf((float)kDim);          // scores in the base-2 domain
         // 8-bit caches: source tile i (the K tiles, then the V tiles) from its raw stage into a bf16 operand buffer, this
         // thread's row; a row beyond the length becomes zeros
         auto widen_tile = [&](int i) -> bool {
@@ -277,6 +283,11 @@ attend_tc_kernel(AttendTcParams p, const __grid_constant__ CUtensorMap map_k, co
             for (int c = 0; c < 8; ++c) codes[c] = *reinterpret_cast<const uint4 *>(raw + ((c ^ (r & 7)) << 4));
 #pragma unroll
             for (int c = 0; c < 8; ++c) {                    // codes 16 c .. 16 c + 15 -> the row's bf16 chunks 2 c and 2 c + 1
+                if (kSrc == 2) {                             // 64 dimensions: the row is the first half, the second half zeros
+                    *reinterpret_cast<uint4 *>(dst + ((c ^ (r & 7)) << 4)) = row_valid ? codes[c] : make_uint4(0u, 0u, 0u, 0u);
+                    *reinterpret_cast<uint4 *>(dst + kTcHalf + ((c ^ (r & 7)) << 4)) = make_uint4(0u, 0u, 0u, 0u);
+                    continue;
+                }
                 uint4 lo = make_uint4(0u, 0u, 0u, 0u), hi = lo;
                 if (row_valid) widen16(codes[c], &lo, &hi);
                 const int half = c >> 2, pos = (2 * c) & 7;
@@ -377,8 +388,9 @@ attend_tc_kernel(AttendTcParams p, const __grid_constant__ CUtensorMap map_k, co
         for (int g = 0; g < G; ++g) {
             const float den = ok ? (red[g] + red[8 + g]) + (red[16 + g] + red[24 + g]) : 0.f;     // error path: zeros
             const float num = __uint_as_float(o[g]) + __uint_as_float(o[8 + g]);
+            if (r >= kDim) continue;                          // (64 dimensions: the padded half of the output)
             if (p.splits == 1) {
-                out[(size_t)g * kHeadDim + r] = den > 0.f ? num / den : 0.f;
+                out[(size_t)g * kDim + r] = den > 0.f ? num / den : 0.f;
             } else {
                 part[g * kStride + r] = num;
                 if (r == 0) {
@@ -399,20 +411,21 @@ attend_tc_kernel(AttendTcParams p, const __grid_constant__ CUtensorMap map_k, co
     }
 }
 
-template <int G, bool kFp8>
+template <int G, int kSrc>
 cudaError_t launch_tc_one(const AttendTcParams &p, const CUtensorMap &mk, const CUtensorMap &mv, const CUtensorMap &mq,
                           cudaStream_t s)
 {
-    cudaError_t e = cudaFuncSetAttribute(attend_tc_kernel<G, kFp8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem);
+    cudaError_t e = cudaFuncSetAttribute(attend_tc_kernel<G, kSrc>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem);
     if (e != cudaSuccess) return e;
-    attend_tc_kernel<G, kFp8><<<(unsigned)(p.batch * p.hkv * p.splits), kTcThreads, kTcSmem, s>>>(p, mk, mv, mq);
+    attend_tc_kernel<G, kSrc><<<(unsigned)(p.batch * p.hkv * p.splits), kTcThreads, kTcSmem, s>>>(p, mk, mv, mq);
     return cudaGetLastError();
 }
 template <int G>
-cudaError_t launch_tc_for(const AttendTcParams &p, bool fp8, const CUtensorMap &mk, const CUtensorMap &mv, const CUtensorMap &mq,
+cudaError_t launch_tc_for(const AttendTcParams &p, int src, const CUtensorMap &mk, const CUtensorMap &mv, const CUtensorMap &mq,
                           cudaStream_t s)
 {
-    return fp8 ? launch_tc_one<G, true>(p, mk, mv, mq, s) : launch_tc_one<G, false>(p, mk, mv, mq, s);
+    return src == 1 ? launch_tc_one<G, 1>(p, mk, mv, mq, s) : src == 2 ? launch_tc_one<G, 2>(p, mk, mv, mq, s)
+                                                                          : launch_tc_one<G, 0>(p, mk, mv, mq, s);
 }
 
 }  // namespace
@@ -430,7 +443,7 @@ int attend_tc_splits(int heads, int cap, int sms)
 
 cudaError_t launch_attend_tc(const void *k_cache, const void *v_cache, const void *q_new, const int32_t *seq_lens, float *out,
                              float *partial, int batch, int hkv, int hq, int cap, int splits, int32_t *status,
-                             long long wait_cycles, const int32_t *block_table, long long pool_pages, bool fp8, cudaStream_t s)
+                             long long wait_cycles, const int32_t *block_table, long long pool_pages, int src, cudaStream_t s)
 {
     const int tiles = (cap + kTile - 1) / kTile;
     AttendTcParams p;
@@ -449,18 +462,20 @@ cudaError_t launch_attend_tc(const void *k_cache, const void *v_cache, const voi
     if (p.tiles_per_split > kTcMaxTiles) return cudaErrorInvalidValue;
     const uint64_t rows = block_table ? (uint64_t)pool_pages * kTile : (uint64_t)batch * hkv * cap;
     CUtensorMap mk, mv, mq;
-    const bool maps_ok = fp8 ? (sm100::make_map_row128(&mk, k_cache, rows, true) && sm100::make_map_row128(&mv, v_cache, rows, true))
-                             : (sm100::make_map(&mk, k_cache, rows, kTile) && sm100::make_map(&mv, v_cache, rows, kTile));
-    if (!maps_ok || !sm100::make_map(&mq, q_new, (uint64_t)batch * hq, 16)) return cudaErrorInvalidValue;
+    // src: 0 = bf16 caches of 128 dimensions, 1 = E4M3 codes of 128 dimensions, 2 = bf16 caches of 64 dimensions
+    const bool maps_ok = src != 0 ? (sm100::make_map_row128(&mk, k_cache, rows, src == 1) && sm100::make_map_row128(&mv, v_cache, rows, src == 1))
+                                  : (sm100::make_map(&mk, k_cache, rows, kTile) && sm100::make_map(&mv, v_cache, rows, kTile));
+    const bool q_ok = src == 2 ? sm100::make_map_q64(&mq, q_new, (uint64_t)batch * hq) : sm100::make_map(&mq, q_new, (uint64_t)batch * hq, 16);
+    if (!maps_ok || !q_ok) return cudaErrorInvalidValue;
     switch (hq / hkv) {
-        case 1: return launch_tc_for<1>(p, fp8, mk, mv, mq, s);
-        case 2: return launch_tc_for<2>(p, fp8, mk, mv, mq, s);
-        case 3: return launch_tc_for<3>(p, fp8, mk, mv, mq, s);
-        case 4: return launch_tc_for<4>(p, fp8, mk, mv, mq, s);
-        case 5: return launch_tc_for<5>(p, fp8, mk, mv, mq, s);
-        case 6: return launch_tc_for<6>(p, fp8, mk, mv, mq, s);
-        case 7: return launch_tc_for<7>(p, fp8, mk, mv, mq, s);
-        case 8: return launch_tc_for<8>(p, fp8, mk, mv, mq, s);
+        case 1: return launch_tc_for<1>(p, src, mk, mv, mq, s);
+        case 2: return launch_tc_for<2>(p, src, mk, mv, mq, s);
+        case 3: return launch_tc_for<3>(p, src, mk, mv, mq, s);
+        case 4: return launch_tc_for<4>(p, src, mk, mv, mq, s);
+        case 5: return launch_tc_for<5>(p, src, mk, mv, mq, s);
+        case 6: return launch_tc_for<6>(p, src, mk, mv, mq, s);
+        case 7: return launch_tc_for<7>(p, src, mk, mv, mq, s);
+        case 8: return launch_tc_for<8>(p, src, mk, mv, mq, s);
         default: return cudaErrorInvalidValue;
     }
 }

@@ -224,13 +224,14 @@ cudaError_t launch_push_query(void *q_window, const void *q_new, int batch, int 
                               cudaStream_t s);
 cudaError_t launch_attend(const void *k_cache, const void *v_cache, const void *q_new, const int32_t *seq_lens, float *out,
                           float *partial, int batch, int hkv, int hq, int cap, int splits, int dtype, int32_t *status,
-                          long long wait_cycles, const int32_t *block_table, long long pool_pages, cudaStream_t s);
+                          long long wait_cycles, const int32_t *block_table, long long pool_pages, int head_dim, cudaStream_t s);
 cudaError_t launch_attend_tc(const void *k_cache, const void *v_cache, const void *q_new, const int32_t *seq_lens, float *out,
                              float *partial, int batch, int hkv, int hq, int cap, int splits, int32_t *status,
-                             long long wait_cycles, const int32_t *block_table, long long pool_pages, bool fp8, cudaStream_t s);
+                             long long wait_cycles, const int32_t *block_table, long long pool_pages, int src, cudaStream_t s);
 int attend_tc_splits(int heads, int cap, int sms);
 int attend_max_group();
 int attend_splits(int heads, int cap, int sms, int G, int dtype);
+bool attend_supported(int G, int dtype, int head_dim);
 size_t attend_partial_bytes(int heads, int splits, int G);
 bool scores_sm100_available();
 long long sm100_default_wait_cycles();          // default limit of the kernels' bounded waits (about two seconds)

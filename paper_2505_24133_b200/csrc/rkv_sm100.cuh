@@ -296,6 +296,20 @@ inline bool make_map_row128(CUtensorMap *map, const void *base, uint64_t rows, b
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// 2-D bf16 view [rows][64] of query rows of 64 dimensions, boxes of 16 rows, 128-byte swizzle.
+inline bool make_map_q64(CUtensorMap *map, const void *base, uint64_t rows)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {64u, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {128u};
+    const cuuint32_t box[2] = {64u, 16u};
+    const cuuint32_t estr[2] = {1u, 1u};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // 2-D bf16 view [rows][16] (32-byte rows), boxes of 128 rows, 32-byte swizzle: the extra K = 16 slices of key rows.
 inline bool make_map_k16(CUtensorMap *map, const void *base, uint64_t rows)
 {

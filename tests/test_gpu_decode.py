@@ -253,6 +253,41 @@ def test_decode_attention_tensor_core_route_paged(rkv):
     assert (np.abs(got - ref) <= 1e-3 * scale + 1e-7).all(), float((np.abs(got - ref) / scale).max())
 
 
+@pytest.mark.parametrize("hkv,hq,budget,buffer,lens", [(2, 8, 300, 84, [384, 1, 0, 200, 129]),
+                                                       (1, 7, 4096, 128, [4224, 1, 0, 3000, 129]),
+                                                       (8, 32, 1024, 128, [1152, 1151, 1000, 7, 128])])
+def test_decode_attention_head_dimension_64(rkv, hkv, hq, budget, buffer, lens):
+    """bf16 caches with 64-dimensional heads: the tensor-core kernel pads the tiles (and the queries) to 128 dimensions on
+    their way to the tensor cores; Eq. 1's scale is 1 / sqrt(64); one to several splits; stale rows full of NaN."""
+    spec = ri.CacheSpec("att64", 1, 5, hkv, hq, 64, budget, buffer, 8, 0.1, "bf16", 16, 0.3, 0.05, 4, 8.0)
+    wl = ri.make_workload(spec, device="cuda", seed=361 + hq, seq_lens=torch.tensor(lens))
+    for b, L in enumerate(lens):
+        wl.k_cache[b, :, L:] = float("nan")
+        wl.v_cache[b, :, L:] = float("nan")
+    g = torch.Generator(device="cuda").manual_seed(9)
+    q_new = torch.randn(5, hq, 64, generator=g, device="cuda").to(torch.bfloat16)
+    comp = rkv.Compressor(5, hkv, hq, budget, buffer, spec.alpha, 0.1, head_dim=64)
+    assert rkv.rkv_decode_workspace_bytes(comp.desc, budget, buffer) <= comp.workspace.numel()
+    out = torch.full((5, hq, 64), 7.0, dtype=torch.float32, device="cuda")
+    rc = rkv.rkv_decode_attention(comp.desc, wl.k_cache, wl.v_cache, q_new, wl.seq_lens, out, budget, buffer)
+    assert rc == rkv.RKV_OK, rkv.rkv_status_string(rc)
+    torch.cuda.synchronize()
+    comp.check_status()
+    K, V = (torch.nan_to_num(t.float(), nan=0.0).cpu().numpy() for t in (wl.k_cache, wl.v_cache))
+    ref = oracle.oracle_decode_attention(K, V, q_new.float().cpu().numpy(), np.array(lens, dtype=np.int32))
+    got = out.cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all()
+    scale = np.maximum(np.abs(ref).max(axis=-1, keepdims=True), 1e-30)
+    assert (np.abs(got - ref) <= 1e-3 * scale + 1e-7).all(), float((np.abs(got - ref) / scale).max())
+    for b, L in enumerate(lens):
+        if L == 0:
+            assert not got[b].any()
+    # fp32 caches of 64 dimensions are not served
+    d = rkv.rkv_desc_default()
+    d.batch, d.n_kv_heads, d.n_q_heads, d.head_dim, d.dtype = 5, hkv, hq, 64, rkv.RKV_F32
+    assert rkv.rkv_decode_attention(d, wl.k_cache, wl.v_cache, q_new, wl.seq_lens, out, budget, buffer) == 2
+
+
 def test_decode_attention_argument_checks(rkv):
     d = rkv.rkv_desc_default()
     d.batch, d.n_kv_heads, d.n_q_heads = 2, 1, 9           # G = 9: beyond what one block serves
