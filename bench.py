@@ -555,6 +555,9 @@ def side_config(rkv, rd, dev, wl, kw, K, W, mem_gb, peaks):
            "roofline_hbm": {nm: {"achieved": h["achieved"], "frac": h["frac"]} for nm, h in hbm.items()}}
     del comp
     timed.close()
+    if not kw:      # (once per workload, not for its variants): the decode step's attention over the same caches
+        att = measure_attention(rkv, dev, wl, peaks, reps=3)
+        out["decode_attention"] = {k2: att[k2] for k2 in ("ms", "gbs", "frac_of_hbm_peak", "error") if k2 in att}
     return out
 
 
